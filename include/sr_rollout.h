@@ -1,0 +1,167 @@
+/*
+ * sr_rollout.h - C ABI of the streaming-rollout frame-update library (CUDA, sm_100a).
+ *
+ * The objects are the paper's (arXiv 1806.04965):
+ *   - a network is a directed, input-connected graph N = (V, E) with 0 < |E|
+ *     (Sec. 3, Definition "network"); nodes are layers, edges are transformations;
+ *   - a rollout pattern is a map R : E -> {0, 1}; R(e) = 1 lets edge e bridge one
+ *     frame ("stream"), R(e) = 0 keeps it inside a frame (Sec. 3, Definition
+ *     "rollout pattern and window", Eq. 2); R is valid iff its rollout window is acyclic;
+ *   - the streaming rollout is R = 1 on every edge; patterns that agree with it on
+ *     all edges not leaving an input node update a whole frame in ONE step
+ *     (Theorem 1 a <=> b), i.e. in one launch group;
+ *   - a node is updated as  x_v = sigma( b_v + sum_{e in SRC_v} f_e(theta_e, x_src(e)) )
+ *     (Sec. A1.2), where the source state is taken from frame t+1-R(e) (Eq. 2);
+ *   - inference chains rollout windows of size W = 1: frame 1 of a window becomes
+ *     frame 0 of the next (Sec. 4 and Sec. 5), so two state buffers per node suffice.
+ *
+ * Conventions of every call
+ *   - returns an sr_status; never throws, never aborts; out-parameters are left
+ *     untouched on error;
+ *   - pointers named *_dev are DEVICE pointers, *_host are HOST pointers; the
+ *     caller owns every buffer it passes and keeps it alive until the work queued
+ *     on `stream` has finished;
+ *   - `stream` is a cudaStream_t passed as void* (NULL = the default stream);
+ *     reset / step / run / get_state / set_state are asynchronous on that stream;
+ *   - the library allocates no device memory: the caller provides one workspace
+ *     (sr_graph_workspace_bytes / sr_graph_bind_workspace) in which the library
+ *     places states, packed weights, biases and its launch tables;
+ *   - layouts: state / frame [B][H][W][C]; conv weight [C_out][k][k][C_in]; dense
+ *     weight [C_out][H][W][C_in] (source flattened in H, W, C order); mean-dense
+ *     weight [C_out][C_in]; bias [C];
+ *   - element type of states and input frames: float (dtype 0) or bfloat16 bit
+ *     patterns (dtype 1).  Weights and biases are always passed as float; in
+ *     bfloat16 mode weights are rounded to bfloat16 (nearest even) when stored.
+ *     Outputs (`out_dev`, `out_seq_dev`) are always float.
+ */
+#ifndef SR_ROLLOUT_H
+#define SR_ROLLOUT_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct sr_graph sr_graph;          /* opaque; owned by the library */
+
+typedef enum {
+    SR_OK = 0,
+    SR_ERR_INVALID_ARG = 1,        /* null pointer, index out of range, bad size                      */
+    SR_ERR_NOT_A_NETWORK = 2,      /* |E| = 0 or not input-connected (Sec. 3, Definition "network")   */
+    SR_ERR_INVALID_ROLLOUT = 3,    /* the rollout window of R has a cycle (Sec. 3, validity)          */
+    SR_ERR_SHAPE_MISMATCH = 4,     /* an edge does not map its source shape to its target shape       */
+    SR_ERR_UNSUPPORTED = 5,        /* a combination this library does not implement                   */
+    SR_ERR_CUDA = 6,               /* a CUDA runtime or driver call failed                            */
+    SR_ERR_TIMEOUT = 7,            /* a bounded device-side wait expired                              */
+    SR_ERR_STATE = 8               /* call order: workspace not bound, weights missing, ...           */
+} sr_status;
+
+/* A node (layer).  Dense nodes have h = w = 1.  act: 0 identity, 1 ReLU (the sigma of Sec. A1.2).
+ * Whether a node is an input is derived: it has no incoming edge (Eq. 1). */
+typedef struct { int32_t h, w, c, act; } sr_node_desc;
+
+/* An edge (transformation f_e, Sec. A1.2).
+ *   kind 0  convolution (cross-correlation) k x k, stride `stride`, zero padding (k-1)/2 on every side,
+ *           output size floor((n + 2p - k)/stride) + 1; pool = 2 appends a 2x2 stride-2 average, 0 none;
+ *   kind 1  dense over the flattened source;
+ *   kind 2  mean over h, w of the source followed by dense over channels. */
+typedef struct { int32_t src, tgt, kind, k, stride, pool; } sr_edge_desc;
+
+enum { SR_EDGE_CONV = 0, SR_EDGE_DENSE = 1, SR_EDGE_MEAN_DENSE = 2 };
+enum { SR_DTYPE_F32 = 0, SR_DTYPE_BF16 = 1 };
+
+/* Rollout-theory quantities of a compiled graph (all integers, exact). */
+typedef struct {
+    int32_t n_nodes, n_edges, n_inputs;
+    int32_t inference_factor;          /* F(R), Eq. 5 = number of launch groups per frame                */
+    int32_t n_groups;                  /* same number; kept separate for readability at call sites        */
+    int32_t streaming_parallel;        /* 1 iff R equals the streaming rollout on all edges that do not
+                                          leave an input node (Theorem 1 a), which is iff F(R) = 1        */
+    int32_t output_node;               /* the node whose state is copied to `out`: the highest-index node
+                                          without an outgoing edge to another node (else the last node)   */
+    int32_t first_response_frame;      /* first frame whose output depends on an input, windows of size 1
+                                          chained (Sec. 4); -1 if the output never depends on an input    */
+    int32_t first_response_step;       /* (first_response_frame - 1) * F(R) + level(output_node)          */
+    int32_t response_interval;         /* update steps between outputs = F(R) (Sec. 4)                    */
+    int32_t n_tensor_core_nodes;       /* nodes updated by the tcgen05 implicit-GEMM kernel               */
+    int32_t n_direct_nodes;            /* nodes updated by the CUDA-core kernels                          */
+} sr_info;
+
+/*
+ * Compile a network and a rollout pattern (Sec. 3).  Validates the graph (network definition, edge
+ * shapes) and the pattern (acyclic rollout window), computes the inference tableau of the window of
+ * size 1 (Eq. 4): level(v) = T((1, v)), and from it the launch groups of a frame: group l holds the
+ * nodes with level l, l = 1..F(R).  Pure host work; needs no GPU.
+ *   nodes, edges : host arrays, copied.      R : host array, n_edges entries, each 0 or 1.
+ *   batch        : B >= 1, or 0 for a theory-only graph (info and levels only; no device calls allowed).
+ *   dtype        : SR_DTYPE_F32 or SR_DTYPE_BF16.
+ * Errors: INVALID_ARG, NOT_A_NETWORK, SHAPE_MISMATCH, INVALID_ROLLOUT, UNSUPPORTED.
+ */
+sr_status sr_graph_create(const sr_node_desc* nodes, int n_nodes, const sr_edge_desc* edges, int n_edges,
+                          const uint8_t* R, int batch, int dtype, sr_graph** out);
+void sr_graph_destroy(sr_graph* g);
+
+sr_status sr_graph_info(const sr_graph* g, sr_info* out);
+/* level[v] = T_{R_1}((1, v)) (Eq. 4): 0 for input nodes, else the update step inside a frame. */
+sr_status sr_graph_levels(const sr_graph* g, int32_t* level_host /* n_nodes */);
+
+/* Bytes of device memory the graph needs; the caller allocates them (256-byte aligned) and binds them.
+ * Binding uploads the launch tables (synchronous copies) and zeroes the states. */
+sr_status sr_graph_workspace_bytes(const sr_graph* g, size_t* bytes);
+sr_status sr_graph_bind_workspace(sr_graph* g, void* workspace_dev, size_t bytes);
+
+/* Parameters theta_e and b_v (Sec. A1.2).  `w` holds floats in the layout given above, on the host
+ * (is_device = 0) or on the device (is_device = 1).  Synchronous.  Needs a bound workspace. */
+sr_status sr_graph_set_edge_weights(sr_graph* g, int edge, const float* w, int is_device);
+sr_status sr_graph_set_node_bias(sr_graph* g, int node, const float* bias_host);
+
+/* Options.  key 0 "engine": 0 = tensor cores where a node qualifies (default), 1 = CUDA-core kernels only.
+ *           key 1 "frames per CUDA graph" used by sr_rollout_run: 0 = plain launches, n >= 1 = graphs
+ *                  of n frames (default 0).
+ * Must be set before sr_graph_bind_workspace (engine) / before the first run (graphs). */
+sr_status sr_graph_set_option(sr_graph* g, int key, int value);
+
+/*
+ * Frame 0 (Sec. A "Training details", Eq. 3): every non-input state := 0; input node i := in0_dev[i]
+ * (one device pointer per input node, in increasing node order, each [B][H][W][C] of the graph dtype).
+ * The frame counter returns to 0.
+ */
+sr_status sr_graph_reset(sr_graph* g, const void* const* in0_dev, void* stream);
+
+/*
+ * One frame update t -> t+1 (Sec. 4: one chained window of size 1): input nodes take the caller's
+ * frame t+1; then, group by group, every node v of the group gets
+ *     x_v^{t+1} = sigma_v( b_v + sum_e f_e(theta_e, x_src(e)^{t+1-R(e)}) )
+ * and the buffers flip.  A streaming pattern runs ONE group.  If out_dev is not NULL it receives the
+ * output node's new state as float [B][C_out].
+ */
+sr_status sr_rollout_step(sr_graph* g, const void* const* in_next_dev, float* out_dev, void* stream);
+
+/*
+ * T frame updates without host round trips in between: in_seq_dev[i] points to the T frames
+ * t+1..t+T of input node i, [T][B][H][W][C]; out_seq_dev (may be NULL) receives [T][B][C_out] floats.
+ * Equivalent to T calls of sr_rollout_step.
+ */
+sr_status sr_rollout_run(sr_graph* g, const void* const* in_seq_dev, int T, float* out_seq_dev, void* stream);
+
+/* Copy the current (frame t) state of a node out of / into the graph, [B][H][W][C] of the graph dtype.
+ * Restoring all states and continuing to step resumes a rollout (Sec. 5: the next window starts
+ * from the last frame of the previous one). */
+sr_status sr_graph_get_state(const sr_graph* g, int node, void* dst_dev, void* stream);
+sr_status sr_graph_set_state(sr_graph* g, int node, const void* src_dev, void* stream);
+
+/* Frames computed since the last reset (host-side count of queued updates). */
+sr_status sr_graph_frame(const sr_graph* g, int64_t* t);
+/* Kernels launched by this graph so far (counts launches inside replayed CUDA graphs as well). */
+sr_status sr_graph_launch_count(const sr_graph* g, int64_t* n);
+/* Synchronises `stream` and reports SR_ERR_CUDA / SR_ERR_TIMEOUT if queued work failed. */
+sr_status sr_graph_sync_status(sr_graph* g, void* stream);
+
+const char* sr_status_str(sr_status s);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* SR_ROLLOUT_H */

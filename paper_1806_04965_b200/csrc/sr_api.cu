@@ -1,0 +1,526 @@
+// C ABI of the streaming-rollout library: graph objects, workspace layout, parameter upload and the
+// per-frame launch sequence (frame input, one launch group per tableau level, buffer flip).
+#include <cuda_runtime.h>
+
+#include <algorithm>
+#include <cstring>
+#include <new>
+#include <vector>
+
+#include "sr_internal.h"
+#include "sr_kernels.h"
+#include "sr_tc.h"
+
+namespace {
+
+struct GraphCache {
+    cudaStream_t capture_stream = nullptr;
+    cudaGraphExec_t exec = nullptr;
+    int frames = 0;
+    int kernels = 0;
+    bool with_out = false;
+};
+
+float round_bf16_host(float f)
+{
+    uint32_t u;
+    std::memcpy(&u, &f, 4);
+    if ((u & 0x7F800000u) == 0x7F800000u) return f;
+    u += 0x7FFFu + ((u >> 16) & 1u);
+    u &= 0xFFFF0000u;
+    std::memcpy(&f, &u, 4);
+    return f;
+}
+
+size_t node_elems(const sr_graph* g, int v)
+{
+    const sr_node_desc& d = g->nodes[v].d;
+    return (size_t)g->batch * d.h * d.w * d.c;
+}
+
+SrRegion take(size_t& off, size_t bytes)
+{
+    SrRegion r;
+    r.offset = off;
+    r.bytes = bytes;
+    off = sr_align_up(off + bytes, 256);
+    return r;
+}
+
+// Decide the engine of every node, lay out the workspace and build the block work lists.
+sr_status plan(sr_graph* g)
+{
+    if (g->batch <= 0) return SR_ERR_STATE;
+    const int n_nodes = (int)g->nodes.size(), n_edges = (int)g->edges.size();
+    for (int v = 0; v < n_nodes; ++v) {
+        SrHostNode& n = g->nodes[v];
+        n.dense_target = false;
+        if (n.is_input) continue;
+        int n_conv = 0, n_dense = 0;
+        for (int e : n.in_edges) (g->edges[e].d.kind == SR_EDGE_CONV ? n_conv : n_dense)++;
+        if (n_conv && n_dense) return SR_ERR_UNSUPPORTED;        // a node sums either convolutions or dense maps
+        n.dense_target = n_dense > 0;
+        n.use_tc = false;
+    }
+    if ((int)g->input_nodes.size() > SR_MAX_INPUTS) return SR_ERR_UNSUPPORTED;
+    if (g->opt_engine == 0 && g->dtype == SR_DTYPE_BF16) sr_tc_select_nodes(g);
+    size_t off = 0;
+    for (int v = 0; v < n_nodes; ++v) {
+        SrHostNode& n = g->nodes[v];
+        n.state[0] = take(off, node_elems(g, v) * g->elem);
+        n.state[1] = take(off, node_elems(g, v) * g->elem);
+        n.bias = take(off, (size_t)n.d.c * sizeof(float));
+    }
+    for (int e = 0; e < n_edges; ++e) {
+        SrHostEdge& he = g->edges[e];
+        const SrHostNode& t = g->nodes[he.d.tgt];
+        he.w_direct = SrRegion();
+        if (!t.use_tc) he.w_direct = take(off, (size_t)he.K * t.d.c * sizeof(float));
+    }
+    g->r_nodes = take(off, sizeof(SrDevNode) * n_nodes);
+    g->r_edges = take(off, sizeof(SrDevEdge) * n_edges);
+    g->r_ctl = take(off, sizeof(SrFrameCtl) + sizeof(int) * SR_MAX_INPUTS);
+    // work lists of the direct kernels, one contiguous range per group
+    g->items.clear();
+    g->group_item_offset.clear();
+    g->group_item_count.clear();
+    const int px = sr_direct_conv_pixels_per_block(), dco = sr_direct_dense_outputs_per_block(),
+              dsb = sr_direct_dense_samples_per_block();
+    for (size_t gi = 0; gi < g->groups.size(); ++gi) {
+        g->group_item_offset.push_back((int)g->items.size());
+        for (int v : g->groups[gi]) {
+            const SrHostNode& n = g->nodes[v];
+            if (n.use_tc) continue;
+            if (n.dense_target) {
+                for (int b0 = 0; b0 < g->batch; b0 += dsb)
+                    for (int c0 = 0; c0 < n.d.c; c0 += dco) g->items.push_back(SrDirectItem{v, b0, c0, 0});
+            } else {
+                const int HW = n.d.h * n.d.w;
+                for (int b = 0; b < g->batch; ++b)
+                    for (int p0 = 0; p0 < HW; p0 += px) g->items.push_back(SrDirectItem{v, b, p0, 0});
+            }
+        }
+        g->group_item_count.push_back((int)g->items.size() - g->group_item_offset.back());
+    }
+    g->r_items = take(off, sizeof(SrDirectItem) * std::max<size_t>(1, g->items.size()));
+    sr_status st = sr_tc_plan(g, off);
+    if (st != SR_OK) return st;
+    g->ws_bytes = off;
+    int n_tc = 0, n_direct = 0;
+    for (const SrHostNode& n : g->nodes)
+        if (!n.is_input) (n.use_tc ? n_tc : n_direct)++;
+    g->info.n_tensor_core_nodes = n_tc;
+    g->info.n_direct_nodes = n_direct;
+    return SR_OK;
+}
+
+bool cuda_ok(cudaError_t e) { return e == cudaSuccess; }
+
+sr_status ready(const sr_graph* g)
+{
+    if (!g) return SR_ERR_INVALID_ARG;
+    if (g->batch <= 0 || !g->ws) return SR_ERR_STATE;
+    for (const SrHostEdge& e : g->edges)
+        if (!e.w_set) return SR_ERR_STATE;
+    return SR_OK;
+}
+
+const int* input_list_dev(const sr_graph* g)
+{
+    return reinterpret_cast<const int*>(g->ws + g->r_ctl.offset + sizeof(SrFrameCtl));
+}
+
+// Queue the kernels of `frames` consecutive frame updates; returns the number of launches.
+int enqueue_frames(sr_graph* g, int first_off, int frames, cudaStream_t s)
+{
+    int launches = 0;
+    for (int f = first_off; f < first_off + frames; ++f) {
+        sr_launch_input(g, input_list_dev(g), f, s);
+        ++launches;
+        launches += sr_tc_stage_inputs(g, f, s);
+        for (int gi = 0; gi < (int)g->groups.size(); ++gi) {
+            if (g->group_item_count[gi] > 0) {
+                sr_launch_direct_group(g, gi, f, s);
+                ++launches;
+            }
+            launches += sr_tc_launch_group(g, gi, f, s);
+        }
+    }
+    return launches;
+}
+
+SrFrameCtl make_ctl(const sr_graph* g, const void* const* in, bool sequence, float* out)
+{
+    SrFrameCtl c{};
+    c.t = g->t;
+    c.run_t = 0;
+    for (size_t i = 0; i < g->input_nodes.size(); ++i) {
+        c.in_base[i] = in[i];
+        c.in_stride_bytes[i] = sequence ? (int64_t)(node_elems(g, g->input_nodes[i]) * g->elem) : 0;
+    }
+    c.out_base = out;
+    c.out_stride = (int64_t)g->batch * g->nodes[g->info.output_node].d.c;
+    return c;
+}
+
+}  // namespace
+
+extern "C" {
+
+sr_status sr_graph_create(const sr_node_desc* nodes, int n_nodes, const sr_edge_desc* edges, int n_edges,
+                          const uint8_t* R, int batch, int dtype, sr_graph** out)
+{
+    if (!out || batch < 0 || (dtype != SR_DTYPE_F32 && dtype != SR_DTYPE_BF16)) return SR_ERR_INVALID_ARG;
+    sr_graph* g = new (std::nothrow) sr_graph();
+    if (!g) return SR_ERR_INVALID_ARG;
+    const sr_status st = sr_compile(g, nodes, n_nodes, edges, n_edges, R);
+    if (st != SR_OK) {
+        delete g;
+        return st;
+    }
+    g->batch = batch;
+    g->dtype = dtype;
+    g->elem = dtype == SR_DTYPE_BF16 ? 2 : 4;
+    *out = g;
+    return SR_OK;
+}
+
+void sr_graph_destroy(sr_graph* g)
+{
+    if (!g) return;
+    if (g->graphs) {
+        GraphCache* c = static_cast<GraphCache*>(g->graphs);
+        if (c->exec) cudaGraphExecDestroy(c->exec);
+        if (c->capture_stream) cudaStreamDestroy(c->capture_stream);
+        delete c;
+    }
+    sr_tc_destroy(g);
+    delete g;
+}
+
+sr_status sr_graph_info(const sr_graph* g, sr_info* out)
+{
+    if (!g || !out) return SR_ERR_INVALID_ARG;
+    *out = g->info;
+    return SR_OK;
+}
+
+sr_status sr_graph_levels(const sr_graph* g, int32_t* level)
+{
+    if (!g || !level) return SR_ERR_INVALID_ARG;
+    for (size_t v = 0; v < g->nodes.size(); ++v) level[v] = g->nodes[v].level;
+    return SR_OK;
+}
+
+sr_status sr_graph_set_option(sr_graph* g, int key, int value)
+{
+    if (!g) return SR_ERR_INVALID_ARG;
+    if (key == 0) {
+        if (g->ws) return SR_ERR_STATE;
+        if (value != 0 && value != 1) return SR_ERR_INVALID_ARG;
+        g->opt_engine = value;
+        return SR_OK;
+    }
+    if (key == 1) {
+        if (value < 0 || value > 1024) return SR_ERR_INVALID_ARG;
+        g->opt_graph_frames = value;
+        return SR_OK;
+    }
+    return SR_ERR_INVALID_ARG;
+}
+
+sr_status sr_graph_workspace_bytes(const sr_graph* g, size_t* bytes)
+{
+    if (!g || !bytes) return SR_ERR_INVALID_ARG;
+    if (g->ws) {
+        *bytes = g->ws_bytes;
+        return SR_OK;
+    }
+    const sr_status st = plan(const_cast<sr_graph*>(g));
+    if (st != SR_OK) return st;
+    *bytes = g->ws_bytes;
+    return SR_OK;
+}
+
+sr_status sr_graph_bind_workspace(sr_graph* g, void* workspace_dev, size_t bytes)
+{
+    if (!g || !workspace_dev) return SR_ERR_INVALID_ARG;
+    if (g->ws) return SR_ERR_STATE;
+    if (reinterpret_cast<uintptr_t>(workspace_dev) & 255) return SR_ERR_INVALID_ARG;
+    sr_status st = plan(g);
+    if (st != SR_OK) return st;
+    if (bytes < g->ws_bytes) return SR_ERR_INVALID_ARG;
+    char* ws = static_cast<char*>(workspace_dev);
+    const int n_nodes = (int)g->nodes.size(), n_edges = (int)g->edges.size();
+    std::vector<SrDevNode> dn(n_nodes);
+    std::vector<SrDevEdge> de(n_edges);
+    int pos = 0;
+    for (int v = 0; v < n_nodes; ++v) {
+        const SrHostNode& n = g->nodes[v];
+        SrDevNode& d = dn[v];
+        d.state[0] = ws + n.state[0].offset;
+        d.state[1] = ws + n.state[1].offset;
+        d.bias = reinterpret_cast<const float*>(ws + n.bias.offset);
+        d.H = n.d.h; d.W = n.d.w; d.C = n.d.c; d.act = n.d.act;
+        d.first_edge = pos;
+        d.n_edges = (int)n.in_edges.size();
+        d.is_output = v == g->info.output_node;
+        d.input_slot = n.input_slot;
+        for (int e : n.in_edges) {
+            const SrHostEdge& he = g->edges[e];
+            const SrHostNode& s = g->nodes[he.d.src];
+            SrDevEdge& x = de[pos++];
+            x.src[0] = ws + s.state[0].offset;
+            x.src[1] = ws + s.state[1].offset;
+            x.w = reinterpret_cast<const float*>(ws + he.w_direct.offset);
+            x.Hs = s.d.h; x.Ws = s.d.w; x.Cs = s.d.c;
+            x.kind = he.d.kind; x.k = he.k_eff; x.stride = he.stride_eff; x.pad = he.pad_eff;
+            x.R = he.R; x.K = he.K; x.src_is_input = s.is_input;
+        }
+    }
+    if (!cuda_ok(cudaMemset(ws, 0, g->ws_bytes))) return SR_ERR_CUDA;
+    if (!cuda_ok(cudaMemcpy(ws + g->r_nodes.offset, dn.data(), sizeof(SrDevNode) * n_nodes, cudaMemcpyHostToDevice)))
+        return SR_ERR_CUDA;
+    if (!cuda_ok(cudaMemcpy(ws + g->r_edges.offset, de.data(), sizeof(SrDevEdge) * n_edges, cudaMemcpyHostToDevice)))
+        return SR_ERR_CUDA;
+    if (!g->items.empty() &&
+        !cuda_ok(cudaMemcpy(ws + g->r_items.offset, g->items.data(), sizeof(SrDirectItem) * g->items.size(),
+                            cudaMemcpyHostToDevice)))
+        return SR_ERR_CUDA;
+    std::vector<int> il(SR_MAX_INPUTS, 0);
+    for (size_t i = 0; i < g->input_nodes.size(); ++i) il[i] = g->input_nodes[i];
+    if (!cuda_ok(cudaMemcpy(ws + g->r_ctl.offset + sizeof(SrFrameCtl), il.data(), sizeof(int) * SR_MAX_INPUTS,
+                            cudaMemcpyHostToDevice)))
+        return SR_ERR_CUDA;
+    g->ws = ws;
+    st = sr_tc_bind(g);
+    if (st != SR_OK) {
+        g->ws = nullptr;
+        return st;
+    }
+    g->t = 0;
+    return SR_OK;
+}
+
+sr_status sr_graph_set_edge_weights(sr_graph* g, int edge, const float* w, int is_device)
+{
+    if (!g || !w || edge < 0 || edge >= (int)g->edges.size()) return SR_ERR_INVALID_ARG;
+    if (!g->ws) return SR_ERR_STATE;
+    SrHostEdge& he = g->edges[edge];
+    const SrHostNode& s = g->nodes[he.d.src];
+    const SrHostNode& t = g->nodes[he.d.tgt];
+    const int Cout = t.d.c, Cs = s.d.c;
+    const size_t n_user = (he.d.kind == SR_EDGE_CONV) ? (size_t)Cout * he.d.k * he.d.k * Cs : (size_t)Cout * he.K;
+    std::vector<float> u(n_user);
+    if (is_device) {
+        if (!cuda_ok(cudaMemcpy(u.data(), w, n_user * sizeof(float), cudaMemcpyDeviceToHost))) return SR_ERR_CUDA;
+    } else {
+        std::memcpy(u.data(), w, n_user * sizeof(float));
+    }
+    if (g->dtype == SR_DTYPE_BF16)
+        for (float& x : u) x = round_bf16_host(x);
+    // the convolution actually executed: [C_out][k'][k'][Cs]; a pooled edge gets the box-filtered kernel
+    std::vector<float> eff;
+    const int k = he.d.k, ke = he.k_eff;
+    if (he.d.kind == SR_EDGE_CONV && he.d.pool == 2) {
+        eff.assign((size_t)Cout * ke * ke * Cs, 0.f);
+        const int sh = he.d.stride;
+        for (int co = 0; co < Cout; ++co)
+            for (int dy = 0; dy < 2; ++dy)
+                for (int dx = 0; dx < 2; ++dx)
+                    for (int ky = 0; ky < k; ++ky)
+                        for (int kx = 0; kx < k; ++kx)
+                            for (int ci = 0; ci < Cs; ++ci)
+                                eff[(((size_t)co * ke + ky + dy * sh) * ke + kx + dx * sh) * Cs + ci] +=
+                                    0.25f * u[(((size_t)co * k + ky) * k + kx) * Cs + ci];
+    } else {
+        eff.swap(u);
+    }
+    if (!t.use_tc) {
+        std::vector<float> d;
+        const float* src = eff.data();
+        if (he.d.kind == SR_EDGE_CONV) {                        // [C_out][K] -> [K][C_out]
+            d.resize((size_t)he.K * Cout);
+            for (int co = 0; co < Cout; ++co)
+                for (int kk = 0; kk < he.K; ++kk) d[(size_t)kk * Cout + co] = eff[(size_t)co * he.K + kk];
+            src = d.data();
+        }
+        if (!cuda_ok(cudaMemcpy(g->ws + he.w_direct.offset, src, (size_t)he.K * Cout * sizeof(float),
+                                cudaMemcpyHostToDevice)))
+            return SR_ERR_CUDA;
+    } else {
+        const sr_status st = sr_tc_set_weights(g, edge, eff.data());
+        if (st != SR_OK) return st;
+    }
+    he.w_set = true;
+    return SR_OK;
+}
+
+sr_status sr_graph_set_node_bias(sr_graph* g, int node, const float* bias_host)
+{
+    if (!g || !bias_host || node < 0 || node >= (int)g->nodes.size()) return SR_ERR_INVALID_ARG;
+    if (!g->ws) return SR_ERR_STATE;
+    SrHostNode& n = g->nodes[node];
+    if (!cuda_ok(cudaMemcpy(g->ws + n.bias.offset, bias_host, (size_t)n.d.c * sizeof(float), cudaMemcpyHostToDevice)))
+        return SR_ERR_CUDA;
+    n.bias_set = true;
+    return SR_OK;
+}
+
+sr_status sr_graph_reset(sr_graph* g, const void* const* in0_dev, void* stream)
+{
+    if (!g || !in0_dev) return SR_ERR_INVALID_ARG;
+    if (g->batch <= 0 || !g->ws) return SR_ERR_STATE;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    for (int v = 0; v < (int)g->nodes.size(); ++v) {
+        const SrHostNode& n = g->nodes[v];
+        const size_t bytes = node_elems(g, v) * g->elem;
+        if (n.is_input) {
+            if (!in0_dev[n.input_slot]) return SR_ERR_INVALID_ARG;
+            if (!cuda_ok(cudaMemcpyAsync(g->ws + n.state[0].offset, in0_dev[n.input_slot], bytes,
+                                         cudaMemcpyDeviceToDevice, s)))
+                return SR_ERR_CUDA;
+            if (!cuda_ok(cudaMemsetAsync(g->ws + n.state[1].offset, 0, bytes, s))) return SR_ERR_CUDA;
+        } else {
+            if (!cuda_ok(cudaMemsetAsync(g->ws + n.state[0].offset, 0, bytes, s))) return SR_ERR_CUDA;
+            if (!cuda_ok(cudaMemsetAsync(g->ws + n.state[1].offset, 0, bytes, s))) return SR_ERR_CUDA;
+        }
+    }
+    g->t = 0;
+    g->launches += sr_tc_after_state_change(g, s);
+    return cuda_ok(cudaGetLastError()) ? SR_OK : SR_ERR_CUDA;
+}
+
+sr_status sr_rollout_step(sr_graph* g, const void* const* in_next_dev, float* out_dev, void* stream)
+{
+    sr_status st = ready(g);
+    if (st != SR_OK) return st;
+    if (!in_next_dev) return SR_ERR_INVALID_ARG;
+    for (size_t i = 0; i < g->input_nodes.size(); ++i)
+        if (!in_next_dev[i]) return SR_ERR_INVALID_ARG;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    sr_launch_set_ctl(g, make_ctl(g, in_next_dev, false, out_dev), s);
+    g->launches += 1 + enqueue_frames(g, 0, 1, s);
+    g->t += 1;
+    return cuda_ok(cudaGetLastError()) ? SR_OK : SR_ERR_CUDA;
+}
+
+sr_status sr_rollout_run(sr_graph* g, const void* const* in_seq_dev, int T, float* out_seq_dev, void* stream)
+{
+    sr_status st = ready(g);
+    if (st != SR_OK) return st;
+    if (!in_seq_dev || T < 0) return SR_ERR_INVALID_ARG;
+    for (size_t i = 0; i < g->input_nodes.size(); ++i)
+        if (!in_seq_dev[i]) return SR_ERR_INVALID_ARG;
+    if (T == 0) return SR_OK;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    sr_launch_set_ctl(g, make_ctl(g, in_seq_dev, true, out_seq_dev), s);
+    g->launches += 1;
+    int done = 0;
+    const int gf = g->opt_graph_frames;
+    if (gf > 0 && T >= gf) {
+        GraphCache* c = static_cast<GraphCache*>(g->graphs);
+        if (!c) {
+            c = new GraphCache();
+            g->graphs = c;
+        }
+        if (c->exec && c->frames != gf) {
+            cudaGraphExecDestroy(c->exec);
+            c->exec = nullptr;
+        }
+        if (!c->exec) {
+            if (!c->capture_stream && !cuda_ok(cudaStreamCreateWithFlags(&c->capture_stream, cudaStreamNonBlocking)))
+                return SR_ERR_CUDA;
+            cudaGraph_t graph = nullptr;
+            if (!cuda_ok(cudaStreamBeginCapture(c->capture_stream, cudaStreamCaptureModeThreadLocal))) return SR_ERR_CUDA;
+            int k = enqueue_frames(g, 0, gf, c->capture_stream);
+            sr_launch_advance(g, gf, c->capture_stream);
+            ++k;
+            if (!cuda_ok(cudaStreamEndCapture(c->capture_stream, &graph)) || !graph) return SR_ERR_CUDA;
+            const cudaError_t ie = cudaGraphInstantiate(&c->exec, graph, 0);
+            cudaGraphDestroy(graph);
+            if (!cuda_ok(ie)) return SR_ERR_CUDA;
+            c->frames = gf;
+            c->kernels = k;
+        }
+        while (T - done >= gf) {
+            if (!cuda_ok(cudaGraphLaunch(c->exec, s))) return SR_ERR_CUDA;
+            g->launches += c->kernels;
+            done += gf;
+        }
+    }
+    if (done < T) {
+        // ctl.t / ctl.run_t already stand at `done` (each graph advanced them); offsets are relative to that
+        g->launches += enqueue_frames(g, 0, T - done, s);
+        sr_launch_advance(g, T - done, s);
+        g->launches += 1;
+    }
+    g->t += T;
+    return cuda_ok(cudaGetLastError()) ? SR_OK : SR_ERR_CUDA;
+}
+
+sr_status sr_graph_get_state(const sr_graph* g, int node, void* dst_dev, void* stream)
+{
+    if (!g || !dst_dev || node < 0 || node >= (int)g->nodes.size()) return SR_ERR_INVALID_ARG;
+    if (g->batch <= 0 || !g->ws) return SR_ERR_STATE;
+    const SrHostNode& n = g->nodes[node];
+    return cuda_ok(cudaMemcpyAsync(dst_dev, g->ws + n.state[g->t & 1].offset, node_elems(g, node) * g->elem,
+                                   cudaMemcpyDeviceToDevice, static_cast<cudaStream_t>(stream)))
+               ? SR_OK : SR_ERR_CUDA;
+}
+
+sr_status sr_graph_set_state(sr_graph* g, int node, const void* src_dev, void* stream)
+{
+    if (!g || !src_dev || node < 0 || node >= (int)g->nodes.size()) return SR_ERR_INVALID_ARG;
+    if (g->batch <= 0 || !g->ws) return SR_ERR_STATE;
+    const SrHostNode& n = g->nodes[node];
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    if (!cuda_ok(cudaMemcpyAsync(g->ws + n.state[g->t & 1].offset, src_dev, node_elems(g, node) * g->elem,
+                                 cudaMemcpyDeviceToDevice, s)))
+        return SR_ERR_CUDA;
+    if (n.is_input) g->launches += sr_tc_after_state_change(g, s);
+    return SR_OK;
+}
+
+sr_status sr_graph_frame(const sr_graph* g, int64_t* t)
+{
+    if (!g || !t) return SR_ERR_INVALID_ARG;
+    *t = g->t;
+    return SR_OK;
+}
+
+sr_status sr_graph_launch_count(const sr_graph* g, int64_t* n)
+{
+    if (!g || !n) return SR_ERR_INVALID_ARG;
+    *n = g->launches;
+    return SR_OK;
+}
+
+sr_status sr_graph_sync_status(sr_graph* g, void* stream)
+{
+    if (!g) return SR_ERR_INVALID_ARG;
+    if (g->batch <= 0 || !g->ws) return SR_ERR_STATE;
+    if (!cuda_ok(cudaStreamSynchronize(static_cast<cudaStream_t>(stream)))) return SR_ERR_CUDA;
+    SrFrameCtl c;
+    if (!cuda_ok(cudaMemcpy(&c, g->ws + g->r_ctl.offset, sizeof(c), cudaMemcpyDeviceToHost))) return SR_ERR_CUDA;
+    if (c.error != 0) return SR_ERR_TIMEOUT;
+    return SR_OK;
+}
+
+const char* sr_status_str(sr_status s)
+{
+    switch (s) {
+        case SR_OK: return "ok";
+        case SR_ERR_INVALID_ARG: return "invalid argument";
+        case SR_ERR_NOT_A_NETWORK: return "not a network (no edges, or a node is not connected to an input)";
+        case SR_ERR_INVALID_ROLLOUT: return "invalid rollout pattern (its rollout window has a cycle)";
+        case SR_ERR_SHAPE_MISMATCH: return "an edge does not map its source shape to its target shape";
+        case SR_ERR_UNSUPPORTED: return "unsupported configuration";
+        case SR_ERR_CUDA: return "CUDA error";
+        case SR_ERR_TIMEOUT: return "a device-side wait expired";
+        case SR_ERR_STATE: return "call order (workspace not bound, weights not set, or graph is theory-only)";
+    }
+    return "unknown status";
+}
+
+}  // extern "C"

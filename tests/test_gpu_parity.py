@@ -1,0 +1,84 @@
+"""GPU parity: the CUDA library, called through the C ABI, against the CPU oracle on the same
+seeded inputs.  Tolerances: max-abs-diff relative to each node's output scale, 2e-2 for bfloat16
+states, 1e-4 for fp32; the dyadic worked example must match exactly."""
+import numpy as np
+import pytest
+
+from tests import parity
+from workloads import data, graphs
+
+pytestmark = pytest.mark.gpu
+
+
+def test_worked_example_exact():
+    import torch
+    from paper_1806_04965_b200 import Graph
+    g = graphs.worked_example()
+    x = torch.tensor([1, 2, 0, 3, 1], dtype=torch.float32, device="cuda:0").reshape(5, 1, 1, 1, 1)
+    w = [np.array(v, dtype=np.float32).reshape(1, 1, 1, 1) for v in (1, 0.5, 2, -1)]
+    b = [np.zeros(1, np.float32), np.array([-0.5], np.float32), np.array([0.25], np.float32)]
+    want = {"streaming": [(0.5, 0), (1.75, 0), (0.375, 3.75), (2.6875, 0)],
+            "sequential": [(1.5, 1.25), (0.25, 0.75), (2.625, 2.5), (1.8125, 2.875)],
+            "hybrid": [(1.5, 0), (0.25, 3.25), (2.625, 0), (1.8125, 4.5)]}
+    for dtype in ("fp32", "bf16"):
+        for p, R in g.patterns.items():
+            G = Graph(g.nodes, g.edges, R, batch=1, dtype=dtype)
+            G.set_weights(w, b)
+            xs = x if dtype == "fp32" else x.to(torch.bfloat16)
+            G.reset([xs[0]])
+            got = []
+            for t in range(1, 5):
+                G.step([xs[t]])
+                got.append((float(G.get_state(1).float().item()), float(G.get_state(2).float().item())))
+            assert got == [(float(a), float(c)) for (a, c) in want[p]], (dtype, p, got)
+
+
+@pytest.mark.parametrize("pattern", ["streaming", "sequential"])
+def test_c1_mlp_full_size(pattern):
+    parity.check_stepwise(graphs.build("c1"), pattern)
+    parity.check_run(graphs.build("c1"), pattern)
+    parity.check_run(graphs.build("c1"), pattern, graph_frames=4)
+
+
+@pytest.mark.parametrize("kind", ["FF", "S", "SR"])
+def test_paper_mnist_networks_fp32(kind):
+    g = graphs.mnist_net(kind, batch=3, frames=5)
+    for p in g.patterns:
+        parity.check_stepwise(g, p, zero_bias=False)
+
+
+@pytest.mark.parametrize("dtype", ["fp32", "bf16"])
+@pytest.mark.parametrize("name,kw", [
+    ("c2", dict(batch=3, frames=6)),
+    ("c3", dict(batch=2, frames=4, size=16)),
+    ("c4", dict(batch=2, frames=4, size=16)),
+    ("c5", dict(batch=2, frames=4, size=16)),
+])
+def test_configs_reduced_direct_engine(name, kw, dtype):
+    g = graphs.build(name, dtype=dtype, **kw)
+    for p in g.patterns:
+        parity.check_stepwise(g, p, engine="direct", zero_bias=False)
+
+
+def test_run_equals_steps_and_resume():
+    import torch
+    g = graphs.build("c2", batch=4, frames=8, dtype="fp32")
+    X, W, Bi = data.make_inputs(g), data.make_weights(g), data.make_biases(g, zero=False)
+    A = parity.make_graph(g, "streaming", "direct", 0, W, Bi)
+    Bg = parity.make_graph(g, "streaming", "direct", 3, W, Bi)
+    x = parity.to_device(g, X[0])
+    oa = A.rollout([x])
+    ob = Bg.rollout([x])                     # CUDA graphs of 3 frames + 2 plain frames
+    assert torch.equal(oa, ob)
+    # resume: run 4 frames, move every state into a fresh graph, run the other 4
+    C = parity.make_graph(g, "streaming", "direct", 0, W, Bi)
+    C.reset([x[0]])
+    C.run([x[1:5]])
+    D = parity.make_graph(g, "streaming", "direct", 0, W, Bi)
+    D.reset([x[4]])
+    for v in range(len(g.nodes)):
+        D.set_state(v, C.get_state(v))
+    od = torch.empty((4, g.batch, 10), dtype=torch.float32, device="cuda:0")
+    D.run([x[5:9]], od)
+    assert torch.equal(od, oa[4:])
+    assert A.launch_count() > 0
