@@ -1,11 +1,732 @@
-// Placeholder until the tcgen05 engine lands: no node is selected for the tensor cores.
+// Tensor-core engine: the node update  x_v = sigma(b_v + sum_e f_e(theta_e, x_src(e)))  (paper Sec. A1.2)
+// for all convolutional nodes of one launch group as ONE grouped implicit GEMM on tcgen05 / TMEM.
+//
+// The sum over the incoming edges of a node is one convolution over the concatenated sources
+// (paper Sec. A, "mathematically equivalent to concatenating all inputs"): the K loop of an output
+// tile simply walks the K-blocks of every incoming edge, tap by tap, into one TMEM accumulator.
+//
+//   M = 128 output pixels (a box of tb samples x th rows x tw columns), N = C_out, K-block = one
+//   filter tap x up to 64 input channels.  A-tiles come straight from the NHWC state of the source
+//   node through 4-D TMA boxes (zero fill outside the image = zero padding); a stride-s edge reads
+//   one of s*s residue-class views of the source, so every tap is again a dense box.  B-tiles come
+//   from the node's concatenated weight matrix [C_out][K] (K-major) through 2-D TMA boxes.
+//   Few-channel input edges (C_in = 1 or 3) are staged per frame into an im2col tensor with K
+//   padded to 16/32/64 so that they are ordinary K-blocks.
+//
+// Warp roles in a CTA of 192 threads: warp 0 = TMA producer, warp 1 = MMA issuer (owns TMEM),
+// warps 2..5 = epilogue (TMEM -> registers -> bias, ReLU, bf16 -> NHWC global).  Two accumulators in
+// TMEM let the epilogue of a tile overlap the main loop of the next.  CTAs are persistent and walk a
+// tile list sorted by decreasing work.  Every wait is bounded; on expiry the kernel records an error
+// in the frame control block, drains its own copies, frees TMEM and returns.
+#include <cuda.h>
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+
+#include <algorithm>
+#include <cstring>
+#include <map>
+#include <tuple>
+#include <vector>
+
 #include "sr_tc.h"
 
-void sr_tc_select_nodes(sr_graph*) {}
-sr_status sr_tc_plan(sr_graph*, size_t&) { return SR_OK; }
-sr_status sr_tc_bind(sr_graph*) { return SR_OK; }
-sr_status sr_tc_set_weights(sr_graph*, int, const float*) { return SR_ERR_UNSUPPORTED; }
-int sr_tc_stage_inputs(sr_graph*, int, cudaStream_t) { return 0; }
-int sr_tc_launch_group(sr_graph*, int, int, cudaStream_t) { return 0; }
-int sr_tc_after_state_change(sr_graph*, cudaStream_t) { return 0; }
-void sr_tc_destroy(sr_graph*) {}
+namespace {
+
+constexpr int kTileM = 128;
+constexpr int kABytes = kTileM * 128;                 // A stage: 128 rows x up to 128 bytes
+constexpr int kThreads = 192;
+constexpr int kMaxStages = 8;
+constexpr int kSmemBudget = 200 * 1024;
+constexpr long long kWaitCycles = 2000000000LL;       // about a second
+
+struct TcKBlock {
+    int32_t a_map[2];       // tensor map of the A box for source frame parity 0 / 1
+    int32_t R;              // 1: the edge reads frame t, 0: frame t+1
+    int32_t qx, qy, c0;     // box origin relative to the tile origin (columns, rows) and first channel
+    int32_t b_map;          // tensor map of the weight box
+    int32_t k_off;          // first K column in the node's weight matrix
+    int32_t n_k16;          // MMA steps (K = 16 each) in this block
+    uint32_t desc_hi;       // upper word of the shared-memory matrix descriptors (swizzle, SBO, version)
+    uint32_t tx_bytes;      // bytes both TMA boxes deliver
+    uint32_t pad_;
+};
+
+struct TcNode {
+    void* state[2];
+    const float* bias;
+    int32_t H, W, C, act;
+    int32_t tw, th, tb;
+    int32_t first_kb, n_kb;
+    uint32_t idesc;
+    int32_t pad_;
+};
+
+struct TcTile { int32_t node, b0, h0, w0; };
+
+struct TcStem {             // a few-channel input edge staged as im2col rows
+    const void* src[2];
+    void* dst[2];
+    int32_t Hs, Ws, Cs, Ho, Wo, k, stride, pad, Kp, K;
+};
+
+// ------------------------------------------------------------------------------------------ PTX helpers
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count)
+{
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes)
+{
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar)
+{
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ uint32_t mbar_try_wait(uint32_t bar, uint32_t parity)
+{
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.b32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+    return ok;
+}
+// Bounded wait.  Returns false if the limit expired or another role already gave up.
+__device__ __noinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag)
+{
+    if (mbar_try_wait(bar, parity)) return true;
+    const long long t0 = clock64();
+    for (;;) {
+#pragma unroll 1
+        for (int i = 0; i < 32; ++i)
+            if (mbar_try_wait(bar, parity)) return true;
+        if (*abort_flag) return false;
+        if (clock64() - t0 > kWaitCycles) {
+            *abort_flag = 1;
+            return false;
+        }
+    }
+}
+
+__device__ __forceinline__ void tma_load_4d(uint32_t dst, const void* map, uint32_t bar, int c0, int c1, int c2, int c3)
+{
+    asm volatile(
+        "cp.async.bulk.tensor.4d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5, %6}], [%2];"
+        ::"r"(dst), "l"(map), "r"(bar), "r"(c0), "r"(c1), "r"(c2), "r"(c3) : "memory");
+}
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const void* map, uint32_t bar, int c0, int c1)
+{
+    asm volatile(
+        "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
+        ::"r"(dst), "l"(map), "r"(bar), "r"(c0), "r"(c1) : "memory");
+}
+
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+
+__device__ __forceinline__ void tc_mma_bf16(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, uint32_t accumulate)
+{
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+        ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate) : "memory");
+}
+__device__ __forceinline__ void tc_commit(uint32_t bar)
+{
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void tc_ld32(uint32_t taddr, uint32_t (&r)[32])
+{
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+        "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+          "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]),
+          "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]),
+          "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+        : "r"(taddr) : "memory");
+}
+__device__ __forceinline__ void tc_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+
+__device__ __forceinline__ uint32_t pack_bf16(float lo, float hi)
+{
+    const __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
+    return *reinterpret_cast<const uint32_t*>(&v);
+}
+
+// ------------------------------------------------------------------------------------------ the kernel
+__global__ void __launch_bounds__(kThreads, 1)
+sr_tc_group_kernel(const CUtensorMap* __restrict__ maps, const TcNode* __restrict__ nodes,
+                   const TcKBlock* __restrict__ kbs, const TcTile* __restrict__ tiles, int n_tiles,
+                   SrFrameCtl* __restrict__ ctl, int t_off, int B, int n_stages, int stage_bytes)
+{
+    extern __shared__ uint8_t smem_raw[];
+    __shared__ uint64_t bars[2 * kMaxStages + 4];
+    __shared__ uint32_t tmem_slot;
+    __shared__ int abort_flag;
+
+    const uint32_t stage0 = (smem_u32(smem_raw) + 1023u) & ~1023u;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const uint32_t bar_full = smem_u32(&bars[0]), bar_empty = smem_u32(&bars[kMaxStages]);
+    const uint32_t bar_tfull = smem_u32(&bars[2 * kMaxStages]), bar_tempty = smem_u32(&bars[2 * kMaxStages + 2]);
+
+    if (threadIdx.x == 0) {
+        abort_flag = 0;
+        for (int s = 0; s < n_stages; ++s) {
+            mbar_init(bar_full + 8 * s, 1);
+            mbar_init(bar_empty + 8 * s, 1);
+        }
+        for (int a = 0; a < 2; ++a) {
+            mbar_init(bar_tfull + 8 * a, 1);
+            mbar_init(bar_tempty + 8 * a, 4);
+        }
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    }
+    if (warp == 1) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&tmem_slot)), "r"(512) : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = tmem_slot;
+    volatile int* abortp = &abort_flag;
+
+    const long long t = ctl->t + t_off;                     // this launch computes frame t+1 from frame t
+    const int prev = (int)(t & 1), cur = prev ^ 1;
+
+    if (warp == 0) {
+        // ---------------------------------------------------------------- TMA producer
+        if (lane == 0) {
+            uint32_t it = 0;
+            bool ok = true;
+            for (int ti = blockIdx.x; ti < n_tiles && ok; ti += gridDim.x) {
+                const TcTile tl = tiles[ti];
+                const TcNode& nd = nodes[tl.node];
+                for (int kb = 0; kb < nd.n_kb; ++kb, ++it) {
+                    const TcKBlock& k = kbs[nd.first_kb + kb];
+                    const uint32_t s = it % n_stages, ph = (it / n_stages) & 1;
+                    if (!mbar_wait(bar_empty + 8 * s, ph ^ 1, abortp)) { ok = false; break; }
+                    const uint32_t full = bar_full + 8 * s;
+                    mbar_expect_tx(full, k.tx_bytes);
+                    const uint32_t a_dst = stage0 + s * stage_bytes;
+                    tma_load_4d(a_dst, &maps[k.a_map[k.R ? prev : cur]], full, k.c0, tl.w0 + k.qx, tl.h0 + k.qy, tl.b0);
+                    tma_load_2d(a_dst + kABytes, &maps[k.b_map], full, k.k_off, 0);
+                }
+            }
+            // drain: every copy this thread started must have landed before the CTA may exit
+            const uint32_t pending = it < (uint32_t)n_stages ? it : (uint32_t)n_stages;
+            for (uint32_t j = 0; j < pending; ++j) {
+                const uint32_t i2 = it - 1 - j;
+                mbar_wait(bar_full + 8 * (i2 % n_stages), (i2 / n_stages) & 1, abortp);
+            }
+        }
+    } else if (warp == 1) {
+        // ---------------------------------------------------------------- MMA issuer
+        if (lane == 0) {
+            uint32_t it = 0, tile_it = 0;
+            bool ok = true;
+            for (int ti = blockIdx.x; ti < n_tiles && ok; ti += gridDim.x, ++tile_it) {
+                const TcTile tl = tiles[ti];
+                const TcNode& nd = nodes[tl.node];
+                const uint32_t acc = tile_it & 1, acc_ph = (tile_it >> 1) & 1;
+                if (!mbar_wait(bar_tempty + 8 * acc, acc_ph ^ 1, abortp)) { ok = false; break; }
+                tc_fence_after();
+                const uint32_t d_tmem = tmem_base + acc * 256;
+                for (int kb = 0; kb < nd.n_kb; ++kb, ++it) {
+                    const TcKBlock& k = kbs[nd.first_kb + kb];
+                    const uint32_t s = it % n_stages, ph = (it / n_stages) & 1;
+                    if (!mbar_wait(bar_full + 8 * s, ph, abortp)) { ok = false; break; }
+                    tc_fence_after();
+                    const uint32_t a_addr = stage0 + s * stage_bytes, b_addr = a_addr + kABytes;
+                    const uint64_t hi = (uint64_t)k.desc_hi << 32;
+                    for (int j = 0; j < k.n_k16; ++j) {
+                        const uint64_t a_desc = hi | (uint64_t)(((a_addr + 32 * j) >> 4) & 0x3FFFu) | (1ull << 16);
+                        const uint64_t b_desc = hi | (uint64_t)(((b_addr + 32 * j) >> 4) & 0x3FFFu) | (1ull << 16);
+                        tc_mma_bf16(d_tmem, a_desc, b_desc, nd.idesc, (kb | j) != 0);
+                    }
+                    tc_commit(bar_empty + 8 * s);           // frees the stage once these MMAs have read it
+                }
+                if (ok) tc_commit(bar_tfull + 8 * acc);     // accumulator complete
+            }
+        }
+    } else {
+        // ---------------------------------------------------------------- epilogue (warps 2..5)
+        const int quarter = warp & 3;                       // TMEM lanes 32*quarter .. +31 belong to this warp
+        const int m = quarter * 32 + lane;                  // row of the tile = output pixel
+        uint32_t tile_it = 0;
+        bool ok = true;
+        for (int ti = blockIdx.x; ti < n_tiles && ok; ti += gridDim.x, ++tile_it) {
+            const TcTile tl = tiles[ti];
+            const TcNode& nd = nodes[tl.node];
+            const uint32_t acc = tile_it & 1, acc_ph = (tile_it >> 1) & 1;
+            if (!mbar_wait(bar_tfull + 8 * acc, acc_ph, abortp)) { ok = false; break; }
+            tc_fence_after();
+            const int per = nd.tw * nd.th;
+            const int bi = m / per, rem = m - bi * per, hi = rem / nd.tw, wi = rem - hi * nd.tw;
+            const int b = tl.b0 + bi, h = tl.h0 + hi, w = tl.w0 + wi;
+            const bool valid = bi < nd.tb && b < B && h < nd.H && w < nd.W;
+            __nv_bfloat16* dst = static_cast<__nv_bfloat16*>(nd.state[cur]) + (((size_t)b * nd.H + h) * nd.W + w) * nd.C;
+            const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + acc * 256;
+            for (int c0 = 0; c0 < nd.C; c0 += 32) {
+                uint32_t r[32];
+                tc_ld32(taddr + c0, r);
+                tc_wait_ld();
+                if (valid) {
+                    uint32_t o[16];
+#pragma unroll
+                    for (int j = 0; j < 16; ++j) {
+                        float v0 = __uint_as_float(r[2 * j]) + __ldg(nd.bias + c0 + 2 * j);
+                        float v1 = __uint_as_float(r[2 * j + 1]) + __ldg(nd.bias + c0 + 2 * j + 1);
+                        if (nd.act == 1) { v0 = fmaxf(v0, 0.f); v1 = fmaxf(v1, 0.f); }
+                        o[j] = pack_bf16(v0, v1);
+                    }
+                    uint4* d4 = reinterpret_cast<uint4*>(dst + c0);
+#pragma unroll
+                    for (int j = 0; j < 4; ++j) d4[j] = make_uint4(o[4 * j], o[4 * j + 1], o[4 * j + 2], o[4 * j + 3]);
+                }
+            }
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(bar_tempty + 8 * acc);
+        }
+    }
+    __syncwarp();
+    tc_fence_before();
+    __syncthreads();
+    if (threadIdx.x == 0 && abort_flag) atomicExch(&ctl->error, 1);
+    if (warp == 1) {
+        tc_fence_after();
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(512) : "memory");
+    }
+}
+
+// Few-channel input edges: row (b, oy, ox) of the staged tensor holds the k*k*C_in receptive field
+// of that output pixel (zero outside the image, zero padded to Kp), so the edge becomes a K-block.
+__global__ void sr_tc_stage_kernel(const TcStem* __restrict__ stems, int n_stems, const SrFrameCtl* __restrict__ ctl,
+                                   int t_off, int fixed_parity, int B)
+{
+    const int cur = fixed_parity >= 0 ? fixed_parity : (int)((ctl->t + t_off + 1) & 1);
+    for (int si = 0; si < n_stems; ++si) {
+        const TcStem& st = stems[si];
+        const __nv_bfloat16* src = static_cast<const __nv_bfloat16*>(st.src[cur]);
+        __nv_bfloat16* dst = static_cast<__nv_bfloat16*>(st.dst[cur]);
+        const size_t n = (size_t)B * st.Ho * st.Wo * (st.Kp / 8);
+        for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += (size_t)gridDim.x * blockDim.x) {
+            const int chunk = (int)(i % (st.Kp / 8));
+            size_t p = i / (st.Kp / 8);
+            const int ox = (int)(p % st.Wo);
+            p /= st.Wo;
+            const int oy = (int)(p % st.Ho);
+            const int b = (int)(p / st.Ho);
+            __align__(16) __nv_bfloat16 v[8];
+#pragma unroll
+            for (int j = 0; j < 8; ++j) {
+                const int kk = chunk * 8 + j;
+                float x = 0.f;
+                if (kk < st.K) {
+                    const int ci = kk % st.Cs, tap = kk / st.Cs, kx = tap % st.k, ky = tap / st.k;
+                    const int iy = oy * st.stride + ky - st.pad, ix = ox * st.stride + kx - st.pad;
+                    if (iy >= 0 && iy < st.Hs && ix >= 0 && ix < st.Ws)
+                        x = __bfloat162float(src[(((size_t)b * st.Hs + iy) * st.Ws + ix) * st.Cs + ci]);
+                }
+                v[j] = __float2bfloat16_rn(x);
+            }
+            reinterpret_cast<uint4*>(dst)[i] = *reinterpret_cast<const uint4*>(v);
+        }
+    }
+}
+
+// ------------------------------------------------------------------------------------------ host side
+struct KbHost {
+    int edge;
+    bool stem;
+    int stem_index;
+    int ky, kx, c0, bk;
+    int k_off;
+};
+
+struct NodePlan {
+    int node;
+    int tw, th, tb;
+    int k_total;                    // columns of the concatenated weight matrix
+    std::vector<KbHost> kbs;
+    SrRegion wcat;
+    std::vector<int> edge_k_off;    // first column of each incoming edge (index parallel to in_edges)
+};
+
+struct StemPlan {
+    int edge;
+    int Kp;
+    SrRegion buf[2];
+};
+
+struct TcEngine {
+    std::vector<NodePlan> nodes;                 // tensor-core nodes
+    std::vector<int> node_of;                    // graph node -> index in nodes, or -1
+    std::vector<StemPlan> stems;
+    std::vector<int> stem_of_edge;
+    std::vector<std::vector<TcTile>> group_tiles;
+    std::vector<int> group_tile_offset, group_stage_bytes, group_stages, group_grid;
+    SrRegion r_maps, r_nodes, r_kbs, r_tiles, r_stems;
+    int n_maps = 0, n_kbs = 0, n_tiles = 0;
+    int sm_count = 148;
+};
+
+TcEngine* eng(const sr_graph* g) { return static_cast<TcEngine*>(g->tc); }
+
+int block_k(int cs) { return cs % 64 == 0 ? 64 : (cs % 32 == 0 ? 32 : 16); }
+int stem_kp(int K) { return K <= 16 ? 16 : (K <= 32 ? 32 : 64); }
+bool is_stem(const sr_graph* g, const SrHostEdge& e)
+{
+    const SrHostNode& s = g->nodes[e.d.src];
+    return s.is_input && (s.d.c % 16) != 0 && e.K <= 64;
+}
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn encode_fn()
+{
+    static EncodeTiledFn fn = nullptr;
+    if (!fn) {
+        void* p = nullptr;
+        cudaDriverEntryPointQueryResult q;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) == cudaSuccess &&
+            q == cudaDriverEntryPointSuccess)
+            fn = reinterpret_cast<EncodeTiledFn>(p);
+    }
+    return fn;
+}
+
+CUtensorMapSwizzle swizzle_of(int bk)
+{
+    return bk == 64 ? CU_TENSOR_MAP_SWIZZLE_128B : (bk == 32 ? CU_TENSOR_MAP_SWIZZLE_64B : CU_TENSOR_MAP_SWIZZLE_32B);
+}
+
+uint32_t desc_hi_of(int bk)
+{
+    const uint32_t sbo = (uint32_t)(8 * bk * 2) >> 4;                    // 8 rows of bk bf16
+    const uint32_t layout = bk == 64 ? 2u : (bk == 32 ? 4u : 6u);        // 128B / 64B / 32B swizzle
+    return sbo | (1u << 14) | (layout << 29);
+}
+
+}  // namespace
+
+// A node goes to the tensor cores if it sums convolutions only, has 32..256 output channels in
+// multiples of 32, and every incoming edge either has C_in % 16 == 0 or is a few-channel input edge.
+void sr_tc_select_nodes(sr_graph* g)
+{
+    for (size_t v = 0; v < g->nodes.size(); ++v) {
+        SrHostNode& n = g->nodes[v];
+        n.use_tc = false;
+        if (n.is_input || n.dense_target || (int)v == g->info.output_node) continue;
+        if (n.d.c % 32 != 0 || n.d.c < 32 || n.d.c > 256) continue;
+        bool ok = true;
+        int k_total = 0;
+        for (int e : n.in_edges) {
+            const SrHostEdge& he = g->edges[e];
+            const SrHostNode& s = g->nodes[he.d.src];
+            if (he.d.kind != SR_EDGE_CONV) ok = false;
+            else if (s.d.c % 16 != 0 && !is_stem(g, he)) ok = false;
+            k_total += he.K;
+        }
+        if (ok && k_total >= 64) n.use_tc = true;
+    }
+}
+
+sr_status sr_tc_plan(sr_graph* g, size_t& off)
+{
+    sr_tc_destroy(g);
+    bool any = false;
+    for (const SrHostNode& n : g->nodes) any |= n.use_tc;
+    if (!any) return SR_OK;
+    TcEngine* E = new TcEngine();
+    g->tc = E;
+    E->node_of.assign(g->nodes.size(), -1);
+    E->stem_of_edge.assign(g->edges.size(), -1);
+    auto take = [&](size_t bytes) {
+        SrRegion r;
+        r.offset = off;
+        r.bytes = bytes;
+        off = sr_align_up(off + bytes, 1024);
+        return r;
+    };
+    for (size_t v = 0; v < g->nodes.size(); ++v) {
+        const SrHostNode& n = g->nodes[v];
+        if (!n.use_tc) continue;
+        NodePlan P;
+        P.node = (int)v;
+        P.tw = std::min(n.d.w, kTileM);
+        P.th = std::min(n.d.h, kTileM / P.tw);
+        P.tb = (P.th == n.d.h && P.tw == n.d.w) ? std::max(1, std::min(g->batch, kTileM / (P.tw * P.th))) : 1;
+        int k_off = 0;
+        for (int e : n.in_edges) {
+            const SrHostEdge& he = g->edges[e];
+            const SrHostNode& s = g->nodes[he.d.src];
+            P.edge_k_off.push_back(k_off);
+            if (is_stem(g, he)) {
+                StemPlan S;
+                S.edge = e;
+                S.Kp = stem_kp(he.K);
+                const size_t bytes = (size_t)g->batch * n.d.h * n.d.w * S.Kp * 2;
+                S.buf[0] = take(bytes);
+                S.buf[1] = take(bytes);
+                E->stem_of_edge[e] = (int)E->stems.size();
+                E->stems.push_back(S);
+                P.kbs.push_back(KbHost{e, true, (int)E->stems.size() - 1, 0, 0, 0, S.Kp, k_off});
+                k_off += S.Kp;
+            } else {
+                const int bk = block_k(s.d.c);
+                for (int ky = 0; ky < he.k_eff; ++ky)
+                    for (int kx = 0; kx < he.k_eff; ++kx)
+                        for (int c0 = 0; c0 < s.d.c; c0 += bk) {
+                            P.kbs.push_back(KbHost{e, false, -1, ky, kx, c0, bk, k_off});
+                            k_off += bk;
+                        }
+            }
+        }
+        P.k_total = k_off;
+        P.wcat = take((size_t)n.d.c * P.k_total * 2);
+        E->node_of[v] = (int)E->nodes.size();
+        E->nodes.push_back(P);
+    }
+    // tiles per group, largest reduction first
+    E->group_tiles.assign(g->groups.size(), {});
+    int n_tiles = 0, n_kbs = 0;
+    for (size_t gi = 0; gi < g->groups.size(); ++gi) {
+        std::vector<std::pair<long long, TcTile>> tl;
+        int max_c = 0;
+        for (int v : g->groups[gi]) {
+            if (E->node_of[v] < 0) continue;
+            const NodePlan& P = E->nodes[E->node_of[v]];
+            const SrHostNode& n = g->nodes[v];
+            max_c = std::max(max_c, n.d.c);
+            for (int b0 = 0; b0 < g->batch; b0 += P.tb)
+                for (int h0 = 0; h0 < n.d.h; h0 += P.th)
+                    for (int w0 = 0; w0 < n.d.w; w0 += P.tw)
+                        tl.push_back({(long long)P.k_total * n.d.c, TcTile{E->node_of[v], b0, h0, w0}});
+        }
+        std::stable_sort(tl.begin(), tl.end(), [](const auto& a, const auto& b) { return a.first > b.first; });
+        for (auto& p : tl) E->group_tiles[gi].push_back(p.second);
+        E->group_tile_offset.push_back(n_tiles);
+        n_tiles += (int)tl.size();
+        const int stage_bytes = kABytes + max_c * 128;
+        E->group_stage_bytes.push_back(stage_bytes);
+        E->group_stages.push_back(std::max(2, std::min(kMaxStages, kSmemBudget / stage_bytes)));
+    }
+    for (const NodePlan& P : E->nodes) n_kbs += (int)P.kbs.size();
+    E->n_tiles = n_tiles;
+    E->n_kbs = n_kbs;
+    // upper bound on distinct tensor maps: two parities per K-block plus one weight map per (node, bk)
+    E->r_maps = take(sizeof(CUtensorMap) * (size_t)(2 * n_kbs + 3 * E->nodes.size() + 1));
+    E->r_nodes = take(sizeof(TcNode) * E->nodes.size());
+    E->r_kbs = take(sizeof(TcKBlock) * (size_t)std::max(1, n_kbs));
+    E->r_tiles = take(sizeof(TcTile) * (size_t)std::max(1, n_tiles));
+    E->r_stems = take(sizeof(TcStem) * std::max<size_t>(1, E->stems.size()));
+    return SR_OK;
+}
+
+sr_status sr_tc_bind(sr_graph* g)
+{
+    TcEngine* E = eng(g);
+    if (!E) return SR_OK;
+    EncodeTiledFn encode = encode_fn();
+    if (!encode) return SR_ERR_CUDA;
+    int dev = 0;
+    cudaGetDevice(&dev);
+    cudaDeviceGetAttribute(&E->sm_count, cudaDevAttrMultiProcessorCount, dev);
+    if (cudaFuncSetAttribute(sr_tc_group_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBudget + 1024) != cudaSuccess)
+        return SR_ERR_CUDA;
+    char* ws = g->ws;
+    std::vector<CUtensorMap> maps;
+    std::map<std::tuple<uintptr_t, int, int, int, int, int, int, int, int>, int> cache;
+    // 4-D activation view: dims (C, W', H', B), box (bk, tw, th, tb)
+    auto act_map = [&](char* base, int C, int Wv, int Hv, size_t stride_w, size_t stride_h, size_t stride_b, int bk,
+                       int tw, int th, int tb) -> int {
+        auto key = std::make_tuple((uintptr_t)base, C, Wv, Hv, (int)stride_w, bk, tw, th, tb);
+        auto it = cache.find(key);
+        if (it != cache.end()) return it->second;
+        CUtensorMap m;
+        cuuint64_t dims[4] = {(cuuint64_t)C, (cuuint64_t)Wv, (cuuint64_t)Hv, (cuuint64_t)g->batch};
+        cuuint64_t strides[3] = {(cuuint64_t)stride_w, (cuuint64_t)stride_h, (cuuint64_t)stride_b};
+        cuuint32_t box[4] = {(cuuint32_t)bk, (cuuint32_t)tw, (cuuint32_t)th, (cuuint32_t)tb};
+        cuuint32_t es[4] = {1, 1, 1, 1};
+        if (encode(&m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, base, dims, strides, box, es, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                   swizzle_of(bk), CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+            return -1;
+        maps.push_back(m);
+        cache[key] = (int)maps.size() - 1;
+        return (int)maps.size() - 1;
+    };
+    std::vector<TcNode> dn;
+    std::vector<TcKBlock> dk;
+    for (const NodePlan& P : E->nodes) {
+        const SrHostNode& n = g->nodes[P.node];
+        TcNode d{};
+        d.state[0] = ws + n.state[0].offset;
+        d.state[1] = ws + n.state[1].offset;
+        d.bias = reinterpret_cast<const float*>(ws + n.bias.offset);
+        d.H = n.d.h; d.W = n.d.w; d.C = n.d.c; d.act = n.d.act;
+        d.tw = P.tw; d.th = P.th; d.tb = P.tb;
+        d.first_kb = (int)dk.size();
+        d.n_kb = (int)P.kbs.size();
+        // instruction descriptor: D = f32, A = B = bf16, both K-major, N = C_out, M = 128
+        d.idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(n.d.c >> 3) << 17) | ((uint32_t)(kTileM >> 4) << 24);
+        std::map<int, int> wmap;                      // bk -> weight tensor map
+        for (const KbHost& kb : P.kbs) {
+            if (wmap.count(kb.bk)) continue;
+            CUtensorMap m;
+            cuuint64_t dims[2] = {(cuuint64_t)P.k_total, (cuuint64_t)n.d.c};
+            cuuint64_t strides[1] = {(cuuint64_t)P.k_total * 2};
+            cuuint32_t box[2] = {(cuuint32_t)kb.bk, (cuuint32_t)n.d.c};
+            cuuint32_t es[2] = {1, 1};
+            if (encode(&m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, ws + P.wcat.offset, dims, strides, box, es,
+                       CU_TENSOR_MAP_INTERLEAVE_NONE, swizzle_of(kb.bk), CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                       CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+                return SR_ERR_CUDA;
+            maps.push_back(m);
+            wmap[kb.bk] = (int)maps.size() - 1;
+        }
+        for (const KbHost& kb : P.kbs) {
+            const SrHostEdge& he = g->edges[kb.edge];
+            const SrHostNode& s = g->nodes[he.d.src];
+            TcKBlock k{};
+            k.R = he.R;
+            k.b_map = wmap[kb.bk];
+            k.k_off = kb.k_off;
+            k.n_k16 = kb.bk / 16;
+            k.desc_hi = desc_hi_of(kb.bk);
+            k.tx_bytes = (uint32_t)(kb.bk * 2 * (P.tw * P.th * P.tb + n.d.c));
+            if (kb.stem) {
+                const StemPlan& S = E->stems[kb.stem_index];
+                for (int par = 0; par < 2; ++par)
+                    k.a_map[par] = act_map(ws + S.buf[par].offset, S.Kp, n.d.w, n.d.h, (size_t)S.Kp * 2,
+                                           (size_t)n.d.w * S.Kp * 2, (size_t)n.d.h * n.d.w * S.Kp * 2, S.Kp, P.tw, P.th, P.tb);
+                k.qx = k.qy = k.c0 = 0;
+            } else {
+                // input pixel = stride * (output pixel + q) + r, q = floor((tap - pad) / stride), r the residue:
+                // the residue-class view of the source makes the tap a dense box starting at (w0 + qx, h0 + qy)
+                const int st = he.stride_eff, ay = kb.ky - he.pad_eff, ax = kb.kx - he.pad_eff;
+                const int qy = (ay >= 0) ? ay / st : -((-ay + st - 1) / st), ry = ay - qy * st;
+                const int qx = (ax >= 0) ? ax / st : -((-ax + st - 1) / st), rx = ax - qx * st;
+                const int Hv = (s.d.h - ry + st - 1) / st, Wv = (s.d.w - rx + st - 1) / st;
+                if (Hv <= 0 || Wv <= 0) return SR_ERR_UNSUPPORTED;
+                for (int par = 0; par < 2; ++par) {
+                    char* base = ws + s.state[par].offset + ((size_t)ry * s.d.w + rx) * s.d.c * 2;
+                    k.a_map[par] = act_map(base, s.d.c, Wv, Hv, (size_t)st * s.d.c * 2, (size_t)st * s.d.w * s.d.c * 2,
+                                           (size_t)s.d.h * s.d.w * s.d.c * 2, kb.bk, P.tw, P.th, P.tb);
+                }
+                k.qx = qx; k.qy = qy; k.c0 = kb.c0;
+            }
+            if (k.a_map[0] < 0 || k.a_map[1] < 0) return SR_ERR_CUDA;
+            dk.push_back(k);
+        }
+        dn.push_back(d);
+    }
+    if (maps.size() * sizeof(CUtensorMap) > E->r_maps.bytes) return SR_ERR_UNSUPPORTED;
+    E->n_maps = (int)maps.size();
+    std::vector<TcTile> tiles;
+    for (auto& v : E->group_tiles) tiles.insert(tiles.end(), v.begin(), v.end());
+    std::vector<TcStem> stems;
+    for (const StemPlan& S : E->stems) {
+        const SrHostEdge& he = g->edges[S.edge];
+        const SrHostNode& s = g->nodes[he.d.src];
+        const SrHostNode& t = g->nodes[he.d.tgt];
+        TcStem d{};
+        for (int par = 0; par < 2; ++par) {
+            d.src[par] = ws + s.state[par].offset;
+            d.dst[par] = ws + S.buf[par].offset;
+        }
+        d.Hs = s.d.h; d.Ws = s.d.w; d.Cs = s.d.c; d.Ho = t.d.h; d.Wo = t.d.w;
+        d.k = he.k_eff; d.stride = he.stride_eff; d.pad = he.pad_eff; d.Kp = S.Kp; d.K = he.K;
+        stems.push_back(d);
+    }
+    auto up = [&](const SrRegion& r, const void* p, size_t bytes) {
+        return bytes == 0 || cudaMemcpy(ws + r.offset, p, bytes, cudaMemcpyHostToDevice) == cudaSuccess;
+    };
+    if (!up(E->r_maps, maps.data(), maps.size() * sizeof(CUtensorMap)) || !up(E->r_nodes, dn.data(), dn.size() * sizeof(TcNode)) ||
+        !up(E->r_kbs, dk.data(), dk.size() * sizeof(TcKBlock)) || !up(E->r_tiles, tiles.data(), tiles.size() * sizeof(TcTile)) ||
+        !up(E->r_stems, stems.data(), stems.size() * sizeof(TcStem)))
+        return SR_ERR_CUDA;
+    E->group_grid.clear();
+    for (auto& v : E->group_tiles) E->group_grid.push_back((int)std::min<size_t>(v.size(), (size_t)E->sm_count));
+    return SR_OK;
+}
+
+sr_status sr_tc_set_weights(sr_graph* g, int edge, const float* w_eff)
+{
+    TcEngine* E = eng(g);
+    if (!E) return SR_ERR_STATE;
+    const SrHostEdge& he = g->edges[edge];
+    const int ni = E->node_of[he.d.tgt];
+    if (ni < 0) return SR_ERR_STATE;
+    const NodePlan& P = E->nodes[ni];
+    const SrHostNode& t = g->nodes[he.d.tgt];
+    int k_off = -1, width = he.K;
+    for (size_t i = 0; i < t.in_edges.size(); ++i)
+        if (t.in_edges[i] == edge) k_off = P.edge_k_off[i];
+    if (k_off < 0) return SR_ERR_STATE;
+    if (E->stem_of_edge[edge] >= 0) width = E->stems[E->stem_of_edge[edge]].Kp;
+    std::vector<uint16_t> h((size_t)t.d.c * width, 0);
+    for (int co = 0; co < t.d.c; ++co)
+        for (int k = 0; k < he.K; ++k) {
+            const __nv_bfloat16 b = __float2bfloat16_rn(w_eff[(size_t)co * he.K + k]);
+            std::memcpy(&h[(size_t)co * width + k], &b, 2);
+        }
+    char* dst = g->ws + P.wcat.offset + (size_t)k_off * 2;
+    if (cudaMemcpy2D(dst, (size_t)P.k_total * 2, h.data(), (size_t)width * 2, (size_t)width * 2, t.d.c,
+                     cudaMemcpyHostToDevice) != cudaSuccess)
+        return SR_ERR_CUDA;
+    return SR_OK;
+}
+
+static int launch_stage(sr_graph* g, int t_off, int fixed_parity, cudaStream_t s)
+{
+    TcEngine* E = eng(g);
+    if (!E || E->stems.empty()) return 0;
+    size_t most = 0;
+    for (const StemPlan& S : E->stems) {
+        const SrHostNode& t = g->nodes[g->edges[S.edge].d.tgt];
+        most = std::max(most, (size_t)g->batch * t.d.h * t.d.w * (S.Kp / 8));
+    }
+    const int blocks = (int)std::min<size_t>((size_t)E->sm_count * 8, (most + 255) / 256);
+    sr_tc_stage_kernel<<<blocks, 256, 0, s>>>(reinterpret_cast<const TcStem*>(g->ws + E->r_stems.offset), (int)E->stems.size(),
+                                              reinterpret_cast<const SrFrameCtl*>(g->ws + g->r_ctl.offset), t_off,
+                                              fixed_parity, g->batch);
+    return 1;
+}
+
+int sr_tc_stage_inputs(sr_graph* g, int t_off, cudaStream_t s) { return launch_stage(g, t_off, -1, s); }
+
+int sr_tc_after_state_change(sr_graph* g, cudaStream_t s) { return launch_stage(g, 0, (int)(g->t & 1), s); }
+
+int sr_tc_launch_group(sr_graph* g, int group, int t_off, cudaStream_t s)
+{
+    TcEngine* E = eng(g);
+    if (!E || E->group_tiles[group].empty()) return 0;
+    const int stages = E->group_stages[group], stage_bytes = E->group_stage_bytes[group];
+    const size_t smem = (size_t)stages * stage_bytes + 1024;
+    sr_tc_group_kernel<<<E->group_grid[group], kThreads, smem, s>>>(
+        reinterpret_cast<const CUtensorMap*>(g->ws + E->r_maps.offset), reinterpret_cast<const TcNode*>(g->ws + E->r_nodes.offset),
+        reinterpret_cast<const TcKBlock*>(g->ws + E->r_kbs.offset),
+        reinterpret_cast<const TcTile*>(g->ws + E->r_tiles.offset) + E->group_tile_offset[group],
+        (int)E->group_tiles[group].size(), reinterpret_cast<SrFrameCtl*>(g->ws + g->r_ctl.offset), t_off, g->batch, stages,
+        stage_bytes);
+    return 1;
+}
+
+void sr_tc_destroy(sr_graph* g)
+{
+    if (g && g->tc) {
+        delete eng(g);
+        g->tc = nullptr;
+    }
+}

@@ -1,0 +1,74 @@
+"""GPU parity of the tcgen05 implicit-GEMM engine against the oracle: single edges of every kind the
+engine lowers (taps, strides, channel-block widths, staged few-channel inputs, pooled edges, several
+incoming edges), ragged tiles, and the reduced benchmark graphs with the engine chosen automatically."""
+import pytest
+
+from tests import parity
+from workloads.graphs import CONV, GAP_DENSE, IDENTITY, RELU, Edge, GraphSpec, Node, check_shapes, build
+
+pytestmark = pytest.mark.gpu
+
+
+def tiny(name, nodes, edges, batch=3, frames=3, R=None):
+    g = GraphSpec(name, nodes, edges, batch=batch, frames=frames, dtype="bf16", seed=4321)
+    g.patterns = {"p": R or [1] * len(edges)}
+    check_shapes(g)
+    return g
+
+
+def run(g):
+    from paper_1806_04965_b200 import Graph
+    G = Graph(g.nodes, g.edges, g.patterns["p"], batch=g.batch, dtype="bf16")
+    assert G.info["n_tensor_core_nodes"] >= 1, G.info
+    return parity.check_stepwise(g, "p", zero_bias=False)
+
+
+@pytest.mark.parametrize("cin,cout,k,stride,size", [
+    (64, 64, 3, 1, 16), (64, 128, 3, 2, 16), (128, 256, 3, 4, 16), (64, 64, 1, 1, 16), (64, 128, 1, 2, 16),
+    (32, 64, 3, 1, 16), (16, 32, 3, 1, 16), (48, 64, 3, 1, 8), (128, 128, 3, 8, 32), (64, 32, 3, 1, 28),
+    (32, 64, 3, 2, 14), (32, 64, 3, 4, 28), (256, 256, 3, 1, 8), (64, 96, 3, 1, 7),
+])
+def test_single_conv_edge(cin, cout, k, stride, size):
+    out = size // stride
+    for R in ([0], [1]):
+        g = tiny("edge", [Node("in", size, size, cin, IDENTITY), Node("n", out, out, cout, RELU), Node("o", 1, 1, 4, IDENTITY)],
+                 [Edge(0, 1, CONV, k, stride), Edge(1, 2, GAP_DENSE)], R=R + [1])
+        run(g)
+
+
+def test_few_channel_input_edges_are_staged():
+    for cin, k in ((3, 3), (1, 3), (3, 1)):
+        g = tiny("stem", [Node("in", 16, 16, cin, IDENTITY), Node("a", 16, 16, 64), Node("b", 16, 16, 64),
+                          Node("o", 1, 1, 4, IDENTITY)],
+                 [Edge(0, 1, CONV, k, 1), Edge(1, 2, CONV, 3, 1), Edge(0, 2, CONV, k, 1), Edge(1, 1, CONV, 3, 1),
+                  Edge(2, 3, GAP_DENSE)], frames=4, R=[1, 1, 0, 1, 0])
+        run(g)
+
+
+def test_pooled_edge_and_recurrence():
+    g = tiny("pool", [Node("in", 16, 16, 64, IDENTITY), Node("a", 8, 8, 128), Node("b", 8, 8, 128), Node("o", 1, 1, 4, IDENTITY)],
+             [Edge(0, 1, CONV, 3, 1, 2), Edge(1, 1, CONV, 3, 1), Edge(1, 2, CONV, 3, 1), Edge(0, 2, CONV, 3, 2),
+              Edge(2, 3, GAP_DENSE)], frames=4)
+    run(g)
+
+
+def test_rectangular_images_and_odd_batch():
+    g = tiny("rect", [Node("in", 12, 20, 64, IDENTITY), Node("a", 12, 20, 64), Node("b", 6, 10, 64),
+                      Node("o", 1, 1, 5, IDENTITY)],
+             [Edge(0, 1, CONV, 3, 1), Edge(1, 2, CONV, 3, 2), Edge(2, 2, CONV, 3, 1), Edge(2, 3, GAP_DENSE)],
+             batch=5, frames=4)
+    run(g)
+
+
+@pytest.mark.parametrize("name,kw", [
+    ("c2", dict(batch=3, frames=6)),
+    ("c3", dict(batch=2, frames=4, size=16)),
+    ("c3", dict(batch=5, frames=3, size=32)),
+    ("c4", dict(batch=2, frames=4, size=16)),
+    ("c5", dict(batch=2, frames=4, size=16)),
+])
+def test_configs_reduced_tensor_cores(name, kw):
+    g = build(name, **kw)
+    for p in g.patterns:
+        parity.check_stepwise(g, p, engine="auto", zero_bias=False)
+        parity.check_run(g, p, engine="auto", graph_frames=2)
