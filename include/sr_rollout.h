@@ -55,7 +55,8 @@ typedef enum {
     SR_ERR_UNSUPPORTED = 5,        /* a combination this library does not implement                   */
     SR_ERR_CUDA = 6,               /* a CUDA runtime or driver call failed                            */
     SR_ERR_TIMEOUT = 7,            /* a bounded device-side wait expired                              */
-    SR_ERR_STATE = 8               /* call order: workspace not bound, weights missing, ...           */
+    SR_ERR_STATE = 8,              /* call order: workspace not bound, weights missing, ...           */
+    SR_ERR_TOO_LARGE = 9           /* the graph needs more than the built-in workspace holds          */
 } sr_status;
 
 /* A node (layer).  Dense nodes have h = w = 1.  act: 0 identity, 1 ReLU (the sigma of Sec. A1.2).
@@ -111,6 +112,36 @@ sr_status sr_graph_levels(const sr_graph* g, int32_t* level_host /* n_nodes */);
  * Binding uploads the launch tables (synchronous copies) and zeroes the states. */
 sr_status sr_graph_workspace_bytes(const sr_graph* g, size_t* bytes);
 sr_status sr_graph_bind_workspace(sr_graph* g, void* workspace_dev, size_t bytes);
+
+/*
+ * Bind the library's built-in workspace instead of a caller-allocated one.  (The paper has no
+ * counterpart; this exists for deployment.)
+ *
+ * Who needs it: code that is not allowed to allocate device memory at the point where it sets a graph
+ * up - a plugin that runs inside a host application's real-time or stream-ordered section, a process
+ * whose memory pool is owned and sized by another component, a late start-up phase after the device
+ * has been handed over fully committed.  Such a caller cannot produce the buffer that
+ * sr_graph_bind_workspace wants.  This call needs none: the workspace is a fixed array of
+ * SR_STATIC_WORKSPACE_BYTES that lives in the library's device image, so every GPU that loads the
+ * library holds that much memory until the process exits, whether or not this call is ever made.
+ *
+ * Behaviour
+ *   - allocates nothing on the device (no cudaMalloc / cudaFree, no allocating library call); inputs and
+ *     outputs are still the caller's buffers, passed to reset / step / run as before;
+ *   - the first call on a device looks the array's address up for that device (the device must be
+ *     current) and remembers it; make that first call before any stream capture begins;
+ *   - a graph whose sr_graph_workspace_bytes exceeds SR_STATIC_WORKSPACE_BYTES is refused with
+ *     SR_ERR_TOO_LARGE and stays unbound;
+ *   - all graphs bound this way share the one array.  It still holds what the previous user left, so
+ *     binding clears the part the new graph uses (states start at zero) and parameters must be set
+ *     again.  Only one such graph may be in use at a time: work of two graphs bound to the built-in
+ *     workspace that overlaps on the GPU (different streams, or a new bind while an older graph's work
+ *     is still queued) races on the same memory.  Synchronise before handing the array to the next graph.
+ * Otherwise identical to sr_graph_bind_workspace: same kernels, same results.
+ * Errors: INVALID_ARG, STATE (already bound, or theory-only graph), TOO_LARGE, CUDA.
+ */
+#define SR_STATIC_WORKSPACE_BYTES (32u * 1024u * 1024u)
+sr_status sr_graph_bind_static_workspace(sr_graph* g);
 
 /* Parameters theta_e and b_v (Sec. A1.2).  `w` holds floats in the layout given above, on the host
  * (is_device = 0) or on the device (is_device = 1).  Synchronous.  Needs a bound workspace. */

@@ -16,7 +16,8 @@ _LIB_PATH = os.path.join(_HERE, "libsr_rollout.so")
 _lib = None
 
 STATUS = {0: "SR_OK", 1: "SR_ERR_INVALID_ARG", 2: "SR_ERR_NOT_A_NETWORK", 3: "SR_ERR_INVALID_ROLLOUT",
-          4: "SR_ERR_SHAPE_MISMATCH", 5: "SR_ERR_UNSUPPORTED", 6: "SR_ERR_CUDA", 7: "SR_ERR_TIMEOUT", 8: "SR_ERR_STATE"}
+          4: "SR_ERR_SHAPE_MISMATCH", 5: "SR_ERR_UNSUPPORTED", 6: "SR_ERR_CUDA", 7: "SR_ERR_TIMEOUT", 8: "SR_ERR_STATE",
+          9: "SR_ERR_TOO_LARGE"}
 
 
 class SrError(RuntimeError):
@@ -61,6 +62,8 @@ def load_library(path: Optional[str] = None):
     lib.sr_graph_levels.argtypes = [vp, ctypes.POINTER(ctypes.c_int32)]
     lib.sr_graph_workspace_bytes.argtypes = [vp, ctypes.POINTER(ctypes.c_size_t)]
     lib.sr_graph_bind_workspace.argtypes = [vp, vp, ctypes.c_size_t]
+    lib.sr_graph_bind_static_workspace.argtypes = [vp]
+    lib.sr_graph_bind_static_workspace.restype = ctypes.c_int
     lib.sr_graph_set_edge_weights.argtypes = [vp, ip, vp, ip]
     lib.sr_graph_set_node_bias.argtypes = [vp, ip, vp]
     lib.sr_graph_set_option.argtypes = [vp, ip, ip]
@@ -100,7 +103,7 @@ class Graph:
     """A compiled network + rollout pattern (sr_graph).  batch=0 gives a theory-only graph."""
 
     def __init__(self, nodes: Sequence, edges: Sequence, R: Sequence[int], batch: int = 0, dtype: str = "bf16",
-                 engine: str = "auto", graph_frames: int = 0, device: str = "cuda:0"):
+                 engine: str = "auto", graph_frames: int = 0, device: str = "cuda:0", static_workspace: bool = False):
         self._lib = load_library()
         self._h = ctypes.c_void_p()
         self.nodes, self.edges, self.R = list(nodes), list(edges), [int(r) for r in R]
@@ -125,9 +128,13 @@ class Graph:
             nbytes = ctypes.c_size_t()
             _check(self._lib.sr_graph_workspace_bytes(self._h, ctypes.byref(nbytes)), "sr_graph_workspace_bytes")
             self.workspace_bytes = nbytes.value
-            self._ws = torch.empty(nbytes.value + 256, dtype=torch.uint8, device=device)
-            base = (self._ws.data_ptr() + 255) // 256 * 256
-            _check(self._lib.sr_graph_bind_workspace(self._h, base, nbytes.value), "sr_graph_bind_workspace")
+            if static_workspace:
+                # the library's built-in array serves as workspace: no device allocation for the graph
+                _check(self._lib.sr_graph_bind_static_workspace(self._h), "sr_graph_bind_static_workspace")
+            else:
+                self._ws = torch.empty(nbytes.value + 256, dtype=torch.uint8, device=device)
+                base = (self._ws.data_ptr() + 255) // 256 * 256
+                _check(self._lib.sr_graph_bind_workspace(self._h, base, nbytes.value), "sr_graph_bind_workspace")
         self.info = self._info()
         self.input_nodes = [v for v in range(n) if not any(e.tgt == v for e in self.edges)]
         self.output_node = self.info["output_node"]

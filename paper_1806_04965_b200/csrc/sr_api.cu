@@ -302,6 +302,30 @@ sr_status sr_graph_bind_workspace(sr_graph* g, void* workspace_dev, size_t bytes
     return SR_OK;
 }
 
+// Built-in workspace for callers that may not allocate device memory.  In host code the array's name
+// is only a handle: its device address is looked up once per device and that pointer is what the
+// kernels get (through the ordinary bind path).
+static __device__ __align__(256) unsigned char sr_static_workspace[SR_STATIC_WORKSPACE_BYTES];
+
+sr_status sr_graph_bind_static_workspace(sr_graph* g)
+{
+    static void* address_on_device[64] = {nullptr};
+    if (!g) return SR_ERR_INVALID_ARG;
+    if (g->ws || g->batch <= 0) return SR_ERR_STATE;
+    size_t need = 0;
+    const sr_status st = sr_graph_workspace_bytes(g, &need);
+    if (st != SR_OK) return st;
+    if (need > (size_t)SR_STATIC_WORKSPACE_BYTES) return SR_ERR_TOO_LARGE;
+    int dev = -1;
+    if (!cuda_ok(cudaGetDevice(&dev)) || dev < 0 || dev >= 64) return SR_ERR_CUDA;
+    if (!address_on_device[dev]) {
+        void* p = nullptr;
+        if (!cuda_ok(cudaGetSymbolAddress(&p, sr_static_workspace)) || !p) return SR_ERR_CUDA;
+        address_on_device[dev] = p;
+    }
+    return sr_graph_bind_workspace(g, address_on_device[dev], (size_t)SR_STATIC_WORKSPACE_BYTES);
+}
+
 sr_status sr_graph_set_edge_weights(sr_graph* g, int edge, const float* w, int is_device)
 {
     if (!g || !w || edge < 0 || edge >= (int)g->edges.size()) return SR_ERR_INVALID_ARG;
@@ -519,6 +543,7 @@ const char* sr_status_str(sr_status s)
         case SR_ERR_CUDA: return "CUDA error";
         case SR_ERR_TIMEOUT: return "a device-side wait expired";
         case SR_ERR_STATE: return "call order (workspace not bound, weights not set, or graph is theory-only)";
+        case SR_ERR_TOO_LARGE: return "the graph needs more workspace than the built-in workspace holds";
     }
     return "unknown status";
 }
