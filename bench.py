@@ -35,19 +35,19 @@ def frame_flops(spec) -> float:
 
 
 def frame_bytes(spec) -> float:
-    """Every source state read once per target node, every node state written once, the input frame,
-    the float output and the weights once."""
+    """Every node state read once and every non-input state written once per frame, plus the float
+    output and the weights once."""
     el = 2 if spec.dtype == "bf16" else 4
     size = lambda v: spec.batch * v.h * v.w * v.c * el
+    has_in = {e.tgt for e in spec.edges}
+    has_out = {e.src for e in spec.edges}
     total = 0
     for vi, v in enumerate(spec.nodes):
-        srcs = {e.src for e in spec.edges if e.tgt == vi}
-        if not srcs:
-            total += size(v)                                  # frame input copied in
-            continue
-        total += sum(size(spec.nodes[u]) for u in srcs) + size(v)
-    has_out = {e.src for e in spec.edges if e.src != e.tgt}
-    out = max(vi for vi in range(len(spec.nodes)) if vi not in has_out)
+        if vi in has_out:
+            total += size(v)
+        if vi in has_in:
+            total += size(v)
+    out = max(vi for vi in range(len(spec.nodes)) if vi not in {e.src for e in spec.edges if e.src != e.tgt})
     total += spec.batch * spec.nodes[out].c * 4
     for ei, e in enumerate(spec.edges):
         total += int(np.prod(data.weight_shape(spec, ei))) * el

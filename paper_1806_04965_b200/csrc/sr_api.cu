@@ -92,8 +92,20 @@ sr_status plan(sr_graph* g)
             const SrHostNode& n = g->nodes[v];
             if (n.use_tc) continue;
             if (n.dense_target) {
-                for (int b0 = 0; b0 < g->batch; b0 += dsb)
-                    for (int c0 = 0; c0 < n.d.c; c0 += dco) g->items.push_back(SrDirectItem{v, b0, c0, 0});
+                // one sample and a chunk of outputs per block, unless a mean-dense source has more channels
+                // than the block's mean buffer holds (then: one warp per output and 8 samples)
+                bool fast = true;
+                for (int e : n.in_edges)
+                    if (g->edges[e].d.kind == SR_EDGE_MEAN_DENSE && g->nodes[g->edges[e].d.src].d.c > sr_direct_head_max_channels())
+                        fast = false;
+                if (fast) {
+                    const int hco = sr_direct_head_outputs_per_block();
+                    for (int b0 = 0; b0 < g->batch; ++b0)
+                        for (int c0 = 0; c0 < n.d.c; c0 += hco) g->items.push_back(SrDirectItem{v, b0, c0, 1});
+                } else {
+                    for (int b0 = 0; b0 < g->batch; b0 += dsb)
+                        for (int c0 = 0; c0 < n.d.c; c0 += dco) g->items.push_back(SrDirectItem{v, b0, c0, 0});
+                }
             } else {
                 const int HW = n.d.h * n.d.w;
                 for (int b = 0; b < g->batch; ++b)

@@ -165,6 +165,97 @@ __device__ void dense_item(const SrDevNode& nd, const SrDevEdge* edges, const Sr
     }
 }
 
+
+constexpr int kHeadCo = 16;        // outputs per block (dense nodes, one sample per block)
+constexpr int kHeadMaxC = 1024;    // channels the mean buffer holds
+
+// Dense node, one sample and kHeadCo outputs per block.  A mean-dense edge first reduces the
+// source over its pixels into shared memory (threads run over channels: coalesced NHWC reads),
+// then every warp forms dot products with lanes striding over the reduction index and a
+// shuffle reduction at the end.  Source and weight rows are read with 16-byte loads.
+template <typename T>
+__device__ void head_item(const SrDevNode& nd, const SrDevEdge* edges, const SrDirectItem& it, int prev, int cur,
+                          float* out_f32)
+{
+    __shared__ float mean[kHeadMaxC];
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int b = it.b0;
+    float acc[kHeadCo / kWarps];
+#pragma unroll
+    for (int j = 0; j < kHeadCo / kWarps; ++j) acc[j] = 0.f;
+    for (int ei = 0; ei < nd.n_edges; ++ei) {
+        const SrDevEdge& e = edges[nd.first_edge + ei];
+        const int HW = e.Hs * e.Ws, Kx = HW * e.Cs;
+        const T* src = static_cast<const T*>(e.src[e.R ? prev : cur]) + (size_t)b * Kx;
+        if (e.kind == SR_EDGE_MEAN_DENSE) {
+            __syncthreads();
+            for (int c = threadIdx.x; c < e.Cs; c += blockDim.x) mean[c] = 0.f;
+            __syncthreads();
+            if ((e.Cs & 3) == 0 && e.Cs / 4 <= (int)blockDim.x) {
+                const int vc = e.Cs / 4, groups = blockDim.x / vc;
+                const int col = threadIdx.x % vc, grp = threadIdx.x / vc;
+                if (grp < groups) {
+                    float s4[4] = {0.f, 0.f, 0.f, 0.f};
+                    for (int p = grp; p < HW; p += groups) {
+                        float x[4];
+                        load4(src + (size_t)p * e.Cs + 4 * col, x);
+#pragma unroll
+                        for (int q = 0; q < 4; ++q) s4[q] += x[q];
+                    }
+#pragma unroll
+                    for (int q = 0; q < 4; ++q) atomicAdd(&mean[4 * col + q], s4[q]);
+                }
+            } else {
+                for (int i = threadIdx.x; i < Kx; i += blockDim.x) atomicAdd(&mean[i % e.Cs], to_f(src[i]));
+            }
+            __syncthreads();
+            const float inv = 1.f / (float)HW;
+#pragma unroll
+            for (int j = 0; j < kHeadCo / kWarps; ++j) {
+                const int co = it.p0 + warp * (kHeadCo / kWarps) + j;
+                if (co >= nd.C) continue;
+                const float* wrow = e.w + (size_t)co * e.K;
+                float part = 0.f;
+                for (int c = lane; c < e.Cs; c += 32) part = fmaf(wrow[c], mean[c], part);
+                acc[j] += part * inv;
+            }
+        } else {
+#pragma unroll
+            for (int j = 0; j < kHeadCo / kWarps; ++j) {
+                const int co = it.p0 + warp * (kHeadCo / kWarps) + j;
+                if (co >= nd.C) continue;
+                const float* wrow = e.w + (size_t)co * e.K;
+                float part = 0.f;
+                if ((Kx & 3) == 0) {
+                    for (int k = 4 * lane; k < Kx; k += 128) {
+                        float x[4];
+                        load4(src + k, x);
+                        const float4 w = *reinterpret_cast<const float4*>(wrow + k);
+                        part = fmaf(w.x, x[0], part); part = fmaf(w.y, x[1], part);
+                        part = fmaf(w.z, x[2], part); part = fmaf(w.w, x[3], part);
+                    }
+                } else {
+                    for (int k = lane; k < Kx; k += 32) part = fmaf(wrow[k], to_f(src[k]), part);
+                }
+                acc[j] += part;
+            }
+        }
+    }
+#pragma unroll
+    for (int j = 0; j < kHeadCo / kWarps; ++j) {
+        float v = acc[j];
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+        const int co = it.p0 + warp * (kHeadCo / kWarps) + j;
+        if (lane == 0 && co < nd.C) {
+            float z = v + nd.bias[co];
+            if (nd.act == 1) z = fmaxf(z, 0.f);
+            from_f(static_cast<T*>(nd.state[cur]) + (size_t)b * nd.C + co, z);
+            if (out_f32) out_f32[(size_t)b * nd.C + co] = z;
+        }
+    }
+}
+
 template <typename T>
 __global__ void __launch_bounds__(kWarps * 32)
 sr_direct_group_kernel(const SrDevNode* __restrict__ nodes, const SrDevEdge* __restrict__ edges,
@@ -176,8 +267,10 @@ sr_direct_group_kernel(const SrDevNode* __restrict__ nodes, const SrDevEdge* __r
     const int prev = (int)(t & 1), cur = prev ^ 1;
     float* out = nullptr;
     if (nd.is_output && ctl->out_base) out = ctl->out_base + (ctl->run_t + t_off) * ctl->out_stride;
-    if (nd.H == 1 && nd.W == 1 && edges[nd.first_edge].kind != SR_EDGE_CONV)
-        dense_item<T>(nd, edges, it, prev, cur, B, out);
+    if (nd.H == 1 && nd.W == 1 && edges[nd.first_edge].kind != SR_EDGE_CONV) {
+        if (it.pad_ == 1) head_item<T>(nd, edges, it, prev, cur, out);
+        else dense_item<T>(nd, edges, it, prev, cur, B, out);
+    }
     else
         conv_item<T>(nd, edges, it, prev, cur, out);
 }
@@ -261,3 +354,5 @@ void sr_launch_advance(const sr_graph* g, int n, cudaStream_t s)
 int sr_direct_conv_pixels_per_block() { return kWarps * kPix; }
 int sr_direct_dense_outputs_per_block() { return kWarps; }
 int sr_direct_dense_samples_per_block() { return kDenseB; }
+int sr_direct_head_outputs_per_block() { return kHeadCo; }
+int sr_direct_head_max_channels() { return kHeadMaxC; }

@@ -11,3 +11,5 @@ void sr_launch_advance(const sr_graph* g, int n, cudaStream_t s);
 int sr_direct_conv_pixels_per_block();
 int sr_direct_dense_outputs_per_block();
 int sr_direct_dense_samples_per_block();
+int sr_direct_head_outputs_per_block();
+int sr_direct_head_max_channels();

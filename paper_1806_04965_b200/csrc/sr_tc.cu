@@ -312,33 +312,47 @@ sr_tc_group_kernel(const CUtensorMap* __restrict__ maps, const TcNode* __restric
 __global__ void sr_tc_stage_kernel(const TcStem* __restrict__ stems, int n_stems, const SrFrameCtl* __restrict__ ctl,
                                    int t_off, int fixed_parity, int B)
 {
+    __shared__ int tap_off[64];     // offset of element kk relative to the (unpadded) window origin, -1 = padding
+    __shared__ short tap_dy[64], tap_dx[64];
     const int cur = fixed_parity >= 0 ? fixed_parity : (int)((ctl->t + t_off + 1) & 1);
     for (int si = 0; si < n_stems; ++si) {
-        const TcStem& st = stems[si];
+        const TcStem st = stems[si];
+        __syncthreads();
+        if (threadIdx.x < 64) {
+            const int kk = threadIdx.x;
+            if (kk < st.K) {
+                const int ci = kk % st.Cs, tap = kk / st.Cs, kx = tap % st.k, ky = tap / st.k;
+                tap_dy[kk] = (short)(ky - st.pad);
+                tap_dx[kk] = (short)(kx - st.pad);
+                tap_off[kk] = ((ky - st.pad) * st.Ws + (kx - st.pad)) * st.Cs + ci;
+            } else {
+                tap_dy[kk] = tap_dx[kk] = 0;
+                tap_off[kk] = -1;
+            }
+        }
+        __syncthreads();
         const __nv_bfloat16* src = static_cast<const __nv_bfloat16*>(st.src[cur]);
         __nv_bfloat16* dst = static_cast<__nv_bfloat16*>(st.dst[cur]);
-        const size_t n = (size_t)B * st.Ho * st.Wo * (st.Kp / 8);
-        for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += (size_t)gridDim.x * blockDim.x) {
-            const int chunk = (int)(i % (st.Kp / 8));
-            size_t p = i / (st.Kp / 8);
+        const int chunks = st.Kp / 8;
+        const size_t n_pix = (size_t)B * st.Ho * st.Wo;
+        for (size_t p = (size_t)blockIdx.x * blockDim.x + threadIdx.x; p < n_pix; p += (size_t)gridDim.x * blockDim.x) {
             const int ox = (int)(p % st.Wo);
-            p /= st.Wo;
-            const int oy = (int)(p % st.Ho);
-            const int b = (int)(p / st.Ho);
-            __align__(16) __nv_bfloat16 v[8];
+            const size_t r = p / st.Wo;
+            const int oy = (int)(r % st.Ho);
+            const int b = (int)(r / st.Ho);
+            const int y0 = oy * st.stride, x0 = ox * st.stride;
+            const __nv_bfloat16* base = src + (((size_t)b * st.Hs + y0) * st.Ws + x0) * st.Cs;
+            for (int c = 0; c < chunks; ++c) {
+                __align__(16) __nv_bfloat16 v[8];
 #pragma unroll
-            for (int j = 0; j < 8; ++j) {
-                const int kk = chunk * 8 + j;
-                float x = 0.f;
-                if (kk < st.K) {
-                    const int ci = kk % st.Cs, tap = kk / st.Cs, kx = tap % st.k, ky = tap / st.k;
-                    const int iy = oy * st.stride + ky - st.pad, ix = ox * st.stride + kx - st.pad;
-                    if (iy >= 0 && iy < st.Hs && ix >= 0 && ix < st.Ws)
-                        x = __bfloat162float(src[(((size_t)b * st.Hs + iy) * st.Ws + ix) * st.Cs + ci]);
+                for (int j = 0; j < 8; ++j) {
+                    const int kk = c * 8 + j;
+                    const int iy = y0 + tap_dy[kk], ix = x0 + tap_dx[kk];
+                    const bool ok = kk < st.K && iy >= 0 && iy < st.Hs && ix >= 0 && ix < st.Ws;
+                    v[j] = ok ? base[tap_off[kk]] : __float2bfloat16_rn(0.f);
                 }
-                v[j] = __float2bfloat16_rn(x);
+                reinterpret_cast<uint4*>(dst)[p * chunks + c] = *reinterpret_cast<const uint4*>(v);
             }
-            reinterpret_cast<uint4*>(dst)[i] = *reinterpret_cast<const uint4*>(v);
         }
     }
 }
@@ -438,7 +452,7 @@ void sr_tc_select_nodes(sr_graph* g)
             else if (s.d.c % 16 != 0 && !is_stem(g, he)) ok = false;
             k_total += he.K;
         }
-        if (ok && k_total >= 64) n.use_tc = true;
+        if (ok && k_total >= 1) n.use_tc = true;
     }
 }
 
@@ -695,7 +709,7 @@ static int launch_stage(sr_graph* g, int t_off, int fixed_parity, cudaStream_t s
     size_t most = 0;
     for (const StemPlan& S : E->stems) {
         const SrHostNode& t = g->nodes[g->edges[S.edge].d.tgt];
-        most = std::max(most, (size_t)g->batch * t.d.h * t.d.w * (S.Kp / 8));
+        most = std::max(most, (size_t)g->batch * t.d.h * t.d.w);
     }
     const int blocks = (int)std::min<size_t>((size_t)E->sm_count * 8, (most + 255) / 256);
     sr_tc_stage_kernel<<<blocks, 256, 0, s>>>(reinterpret_cast<const TcStem*>(g->ws + E->r_stems.offset), (int)E->stems.size(),
