@@ -12,6 +12,11 @@
 //   from the node's concatenated weight matrix [C_out][K] (K-major) through 2-D TMA boxes.
 //   Few-channel input edges (C_in = 1 or 3) are staged per frame into an im2col tensor with K
 //   padded to 16/32/64 so that they are ordinary K-blocks.
+//   A stride-1 k x k edge does not reload its activations per tap: for each filter column kx one box
+//   of th+k-1 image rows (tile width a multiple of 8 pixels, so an image row of the tile is a whole
+//   number of swizzle atoms) is loaded once, and the k taps of that column are row-shifted windows
+//   of it - the shared-memory descriptor just starts ky*tw rows further down.  A and B therefore
+//   travel through separate rings.
 //
 // Warp roles in a CTA of 192 threads: warp 0 = TMA producer, warp 1 = MMA issuer (owns TMEM),
 // warps 2..5 = epilogue (TMEM -> registers -> bias, ReLU, bf16 -> NHWC global).  Two accumulators in
@@ -35,8 +40,9 @@ namespace {
 constexpr int kTileM = 128;
 constexpr int kABytes = kTileM * 128;                 // A stage: 128 rows x up to 128 bytes
 constexpr int kThreads = 192;
-constexpr int kMaxStages = 8;
-constexpr int kSmemBudget = 200 * 1024;
+constexpr int kMaxA = 6;                              // A ring depth
+constexpr int kBUnit = 4096, kBUnits = 24;            // B ring: 24 units of 4 KiB; a weight box takes 1, 2, 4 or 8 units
+constexpr int kSmemBudget = 216 * 1024;
 constexpr long long kWaitCycles = 2000000000LL;       // about a second
 
 struct TcKBlock {
@@ -47,8 +53,11 @@ struct TcKBlock {
     int32_t k_off;          // first K column in the node's weight matrix
     int32_t n_k16;          // MMA steps (K = 16 each) in this block
     uint32_t desc_hi;       // upper word of the shared-memory matrix descriptors (swizzle, SBO, version)
-    uint32_t tx_bytes;      // bytes both TMA boxes deliver
-    uint32_t pad_;
+    uint32_t a_bytes;       // bytes of the A box this block loads into a fresh A slot; 0 = reuse the current slot
+    uint32_t b_bytes;       // bytes of the weight box
+    uint32_t a_off;         // byte offset of this block's 128 rows inside the A slot
+    uint32_t a_release;     // 1: last block that reads the current A slot
+    uint32_t pad_[2];
 };
 
 struct TcNode {
@@ -58,7 +67,7 @@ struct TcNode {
     int32_t tw, th, tb;
     int32_t first_kb, n_kb;
     uint32_t idesc;
-    int32_t pad_;
+    int32_t b_units;        // B-ring units one weight box of this node occupies (power of two)
 };
 
 struct TcTile { int32_t node, b0, h0, w0; };
@@ -95,9 +104,8 @@ __device__ __forceinline__ uint32_t mbar_try_wait(uint32_t bar, uint32_t parity)
     return ok;
 }
 // Bounded wait.  Returns false if the limit expired or another role already gave up.
-__device__ __noinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag)
+__device__ __noinline__ bool mbar_wait_slow(uint32_t bar, uint32_t parity, volatile int* abort_flag)
 {
-    if (mbar_try_wait(bar, parity)) return true;
     const long long t0 = clock64();
     for (;;) {
 #pragma unroll 1
@@ -109,6 +117,11 @@ __device__ __noinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile i
             return false;
         }
     }
+}
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag)
+{
+    if (mbar_try_wait(bar, parity)) return true;
+    return mbar_wait_slow(bar, parity, abort_flag);
 }
 
 __device__ __forceinline__ void tma_load_4d(uint32_t dst, const void* map, uint32_t bar, int c0, int c1, int c2, int c3)
@@ -163,23 +176,29 @@ __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi)
 __global__ void __launch_bounds__(kThreads, 1)
 sr_tc_group_kernel(const CUtensorMap* __restrict__ maps, const TcNode* __restrict__ nodes,
                    const TcKBlock* __restrict__ kbs, const TcTile* __restrict__ tiles, int n_tiles,
-                   SrFrameCtl* __restrict__ ctl, int t_off, int B, int n_stages, int stage_bytes)
+                   SrFrameCtl* __restrict__ ctl, int t_off, int B, int n_a, int a_slot)
 {
     extern __shared__ uint8_t smem_raw[];
-    __shared__ uint64_t bars[2 * kMaxStages + 4];
+    __shared__ uint64_t bars[2 * kMaxA + 2 * kBUnits + 4];
     __shared__ uint32_t tmem_slot;
     __shared__ int abort_flag;
 
-    const uint32_t stage0 = (smem_u32(smem_raw) + 1023u) & ~1023u;
+    const uint32_t a_ring = (smem_u32(smem_raw) + 1023u) & ~1023u;
+    const uint32_t b_ring = a_ring + (uint32_t)(n_a * a_slot);
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const uint32_t bar_full = smem_u32(&bars[0]), bar_empty = smem_u32(&bars[kMaxStages]);
-    const uint32_t bar_tfull = smem_u32(&bars[2 * kMaxStages]), bar_tempty = smem_u32(&bars[2 * kMaxStages + 2]);
+    const uint32_t bar_afull = smem_u32(&bars[0]), bar_aempty = smem_u32(&bars[kMaxA]);
+    const uint32_t bar_bfull = smem_u32(&bars[2 * kMaxA]), bar_bempty = smem_u32(&bars[2 * kMaxA + kBUnits]);
+    const uint32_t bar_tfull = smem_u32(&bars[2 * kMaxA + 2 * kBUnits]), bar_tempty = bar_tfull + 16;
 
     if (threadIdx.x == 0) {
         abort_flag = 0;
-        for (int s = 0; s < n_stages; ++s) {
-            mbar_init(bar_full + 8 * s, 1);
-            mbar_init(bar_empty + 8 * s, 1);
+        for (int s = 0; s < n_a; ++s) {
+            mbar_init(bar_afull + 8 * s, 1);
+            mbar_init(bar_aempty + 8 * s, 1);
+        }
+        for (int s = 0; s < kBUnits; ++s) {
+            mbar_init(bar_bfull + 8 * s, 1);
+            mbar_init(bar_bempty + 8 * s, 1);
         }
         for (int a = 0; a < 2; ++a) {
             mbar_init(bar_tfull + 8 * a, 1);
@@ -204,54 +223,90 @@ sr_tc_group_kernel(const CUtensorMap* __restrict__ maps, const TcNode* __restric
     if (warp == 0) {
         // ---------------------------------------------------------------- TMA producer
         if (lane == 0) {
-            uint32_t it = 0;
+            // The B ring is a ring of 4 KiB units; a weight box of a node takes b_units consecutive units
+            // starting at a multiple of b_units and is tracked by the barriers of its first unit.  Each
+            // unit's barriers flip phase only when that unit leads a box, so both sides keep a bit per
+            // unit (the MMA thread walks the identical sequence).
+            uint32_t ia = 0, bpos = 0, bphase = 0, b_used = 0;     // b_used: units that ever led a box
             bool ok = true;
+            // tables are read by value one step ahead, so that no global load sits between two waits
+            TcTile tl_next = tiles[blockIdx.x < n_tiles ? blockIdx.x : 0];
             for (int ti = blockIdx.x; ti < n_tiles && ok; ti += gridDim.x) {
-                const TcTile tl = tiles[ti];
-                const TcNode& nd = nodes[tl.node];
-                for (int kb = 0; kb < nd.n_kb; ++kb, ++it) {
-                    const TcKBlock& k = kbs[nd.first_kb + kb];
-                    const uint32_t s = it % n_stages, ph = (it / n_stages) & 1;
-                    if (!mbar_wait(bar_empty + 8 * s, ph ^ 1, abortp)) { ok = false; break; }
-                    const uint32_t full = bar_full + 8 * s;
-                    mbar_expect_tx(full, k.tx_bytes);
-                    const uint32_t a_dst = stage0 + s * stage_bytes;
-                    tma_load_4d(a_dst, &maps[k.a_map[k.R ? prev : cur]], full, k.c0, tl.w0 + k.qx, tl.h0 + k.qy, tl.b0);
-                    tma_load_2d(a_dst + kABytes, &maps[k.b_map], full, k.k_off, 0);
+                const TcTile tl = tl_next;
+                if (ti + (int)gridDim.x < n_tiles) tl_next = tiles[ti + gridDim.x];
+                const int first_kb = nodes[tl.node].first_kb, n_kb = nodes[tl.node].n_kb;
+                const uint32_t u = (uint32_t)nodes[tl.node].b_units;
+                TcKBlock k_next = kbs[first_kb];
+                for (int kb = 0; kb < n_kb; ++kb) {
+                    const TcKBlock k = k_next;
+                    if (kb + 1 < n_kb) k_next = kbs[first_kb + kb + 1];
+                    if (k.a_bytes) {
+                        const uint32_t s = ia % n_a, ph = (ia / n_a) & 1;
+                        if (!mbar_wait(bar_aempty + 8 * s, ph ^ 1, abortp)) { ok = false; break; }
+                        mbar_expect_tx(bar_afull + 8 * s, k.a_bytes);
+                        tma_load_4d(a_ring + s * a_slot, &maps[k.a_map[k.R ? prev : cur]], bar_afull + 8 * s, k.c0,
+                                    tl.w0 + k.qx, tl.h0 + k.qy, tl.b0);
+                        ++ia;
+                    }
+                    bpos = (bpos + u - 1) & ~(u - 1);
+                    if (bpos >= (uint32_t)kBUnits) bpos = 0;
+                    const uint32_t s = bpos, ph = (bphase >> s) & 1;
+                    if (!mbar_wait(bar_bempty + 8 * s, ph ^ 1, abortp)) { ok = false; break; }
+                    mbar_expect_tx(bar_bfull + 8 * s, k.b_bytes);
+                    tma_load_2d(b_ring + s * kBUnit, &maps[k.b_map], bar_bfull + 8 * s, k.k_off, 0);
+                    bphase ^= 1u << s;
+                    b_used |= 1u << s;
+                    bpos += u;
                 }
             }
             // drain: every copy this thread started must have landed before the CTA may exit
-            const uint32_t pending = it < (uint32_t)n_stages ? it : (uint32_t)n_stages;
-            for (uint32_t j = 0; j < pending; ++j) {
-                const uint32_t i2 = it - 1 - j;
-                mbar_wait(bar_full + 8 * (i2 % n_stages), (i2 / n_stages) & 1, abortp);
+            for (uint32_t j = 0; j < (uint32_t)n_a && j < ia; ++j) {
+                const uint32_t i2 = ia - 1 - j;
+                mbar_wait(bar_afull + 8 * (i2 % n_a), (i2 / n_a) & 1, abortp);
             }
+            for (uint32_t u = 0; u < (uint32_t)kBUnits; ++u)
+                if ((b_used >> u) & 1) mbar_wait(bar_bfull + 8 * u, ((bphase >> u) & 1) ^ 1, abortp);
         }
     } else if (warp == 1) {
         // ---------------------------------------------------------------- MMA issuer
         if (lane == 0) {
-            uint32_t it = 0, tile_it = 0;
+            uint32_t ia = 0, bpos = 0, bphase = 0, tile_it = 0, a_cur = 0;
             bool ok = true;
+            int node_next = tiles[blockIdx.x < n_tiles ? blockIdx.x : 0].node;
             for (int ti = blockIdx.x; ti < n_tiles && ok; ti += gridDim.x, ++tile_it) {
-                const TcTile tl = tiles[ti];
-                const TcNode& nd = nodes[tl.node];
+                const int node = node_next;
+                if (ti + (int)gridDim.x < n_tiles) node_next = tiles[ti + gridDim.x].node;
+                const int first_kb = nodes[node].first_kb, n_kb = nodes[node].n_kb;
+                const uint32_t u = (uint32_t)nodes[node].b_units, idesc = nodes[node].idesc;
+                TcKBlock k_next = kbs[first_kb];
                 const uint32_t acc = tile_it & 1, acc_ph = (tile_it >> 1) & 1;
                 if (!mbar_wait(bar_tempty + 8 * acc, acc_ph ^ 1, abortp)) { ok = false; break; }
                 tc_fence_after();
                 const uint32_t d_tmem = tmem_base + acc * 256;
-                for (int kb = 0; kb < nd.n_kb; ++kb, ++it) {
-                    const TcKBlock& k = kbs[nd.first_kb + kb];
-                    const uint32_t s = it % n_stages, ph = (it / n_stages) & 1;
-                    if (!mbar_wait(bar_full + 8 * s, ph, abortp)) { ok = false; break; }
+                for (int kb = 0; kb < n_kb; ++kb) {
+                    const TcKBlock k = k_next;
+                    if (kb + 1 < n_kb) k_next = kbs[first_kb + kb + 1];
+                    if (k.a_bytes) {
+                        a_cur = ia % n_a;
+                        if (!mbar_wait(bar_afull + 8 * a_cur, (ia / n_a) & 1, abortp)) { ok = false; break; }
+                        ++ia;
+                    }
+                    bpos = (bpos + u - 1) & ~(u - 1);
+                    if (bpos >= (uint32_t)kBUnits) bpos = 0;
+                    const uint32_t s = bpos, ph = (bphase >> s) & 1;
+                    if (!mbar_wait(bar_bfull + 8 * s, ph, abortp)) { ok = false; break; }
+                    bphase ^= 1u << s;
+                    bpos += u;
                     tc_fence_after();
-                    const uint32_t a_addr = stage0 + s * stage_bytes, b_addr = a_addr + kABytes;
+                    const uint32_t a_addr = a_ring + a_cur * a_slot + k.a_off, b_addr = b_ring + s * kBUnit;
                     const uint64_t hi = (uint64_t)k.desc_hi << 32;
                     for (int j = 0; j < k.n_k16; ++j) {
                         const uint64_t a_desc = hi | (uint64_t)(((a_addr + 32 * j) >> 4) & 0x3FFFu) | (1ull << 16);
                         const uint64_t b_desc = hi | (uint64_t)(((b_addr + 32 * j) >> 4) & 0x3FFFu) | (1ull << 16);
-                        tc_mma_bf16(d_tmem, a_desc, b_desc, nd.idesc, (kb | j) != 0);
+                        tc_mma_bf16(d_tmem, a_desc, b_desc, idesc, (kb | j) != 0);
                     }
-                    tc_commit(bar_empty + 8 * s);           // frees the stage once these MMAs have read it
+                    tc_commit(bar_bempty + 8 * s);                       // frees the B slot once these MMAs have read it
+                    if (k.a_release) tc_commit(bar_aempty + 8 * a_cur);  // last reader of the A slot
                 }
                 if (ok) tc_commit(bar_tfull + 8 * acc);     // accumulator complete
             }
@@ -264,7 +319,7 @@ sr_tc_group_kernel(const CUtensorMap* __restrict__ maps, const TcNode* __restric
         bool ok = true;
         for (int ti = blockIdx.x; ti < n_tiles && ok; ti += gridDim.x, ++tile_it) {
             const TcTile tl = tiles[ti];
-            const TcNode& nd = nodes[tl.node];
+            const TcNode nd = nodes[tl.node];
             const uint32_t acc = tile_it & 1, acc_ph = (tile_it >> 1) & 1;
             if (!mbar_wait(bar_tfull + 8 * acc, acc_ph, abortp)) { ok = false; break; }
             tc_fence_after();
@@ -364,11 +419,15 @@ struct KbHost {
     int stem_index;
     int ky, kx, c0, bk;
     int k_off;
+    int a_rows;        // image rows of the A box this block loads (0: reuses the current A slot)
+    int a_shift;       // rows by which this block's window is shifted inside the A slot
+    bool a_release;
 };
 
 struct NodePlan {
     int node;
     int tw, th, tb;
+    bool column_reuse;              // stride-1 k x k edges load one box per filter column
     int k_total;                    // columns of the concatenated weight matrix
     std::vector<KbHost> kbs;
     SrRegion wcat;
@@ -387,7 +446,7 @@ struct TcEngine {
     std::vector<StemPlan> stems;
     std::vector<int> stem_of_edge;
     std::vector<std::vector<TcTile>> group_tiles;
-    std::vector<int> group_tile_offset, group_stage_bytes, group_stages, group_grid;
+    std::vector<int> group_tile_offset, group_a_slot, group_n_a, group_grid;
     SrRegion r_maps, r_nodes, r_kbs, r_tiles, r_stems;
     int n_maps = 0, n_kbs = 0, n_tiles = 0;
     int sm_count = 148;
@@ -478,9 +537,22 @@ sr_status sr_tc_plan(sr_graph* g, size_t& off)
         if (!n.use_tc) continue;
         NodePlan P;
         P.node = (int)v;
-        P.tw = std::min(n.d.w, kTileM);
-        P.th = std::min(n.d.h, kTileM / P.tw);
-        P.tb = (P.th == n.d.h && P.tw == n.d.w) ? std::max(1, std::min(g->batch, kTileM / (P.tw * P.th))) : 1;
+        // tile shape: 8 pixels x 16 rows of one sample when a stride-1 k x k edge can reuse its boxes,
+        // else as wide as the image and as many rows (and samples) as fit in 128 pixels
+        bool wants_reuse = false;
+        for (int e : n.in_edges) {
+            const SrHostEdge& he = g->edges[e];
+            if (!is_stem(g, he) && he.stride_eff == 1 && he.k_eff >= 2) wants_reuse = true;
+        }
+        if (wants_reuse && n.d.w >= 8 && n.d.h >= 16) {
+            P.tw = 8; P.th = 16; P.tb = 1;
+            P.column_reuse = true;
+        } else {
+            P.tw = std::min(n.d.w, kTileM);
+            P.th = std::min(n.d.h, kTileM / P.tw);
+            P.tb = (P.th == n.d.h && P.tw == n.d.w) ? std::max(1, std::min(g->batch, kTileM / (P.tw * P.th))) : 1;
+            P.column_reuse = false;
+        }
         int k_off = 0;
         for (int e : n.in_edges) {
             const SrHostEdge& he = g->edges[e];
@@ -495,16 +567,25 @@ sr_status sr_tc_plan(sr_graph* g, size_t& off)
                 S.buf[1] = take(bytes);
                 E->stem_of_edge[e] = (int)E->stems.size();
                 E->stems.push_back(S);
-                P.kbs.push_back(KbHost{e, true, (int)E->stems.size() - 1, 0, 0, 0, S.Kp, k_off});
+                P.kbs.push_back(KbHost{e, true, (int)E->stems.size() - 1, 0, 0, 0, S.Kp, k_off, P.th, 0, true});
                 k_off += S.Kp;
             } else {
-                const int bk = block_k(s.d.c);
-                for (int ky = 0; ky < he.k_eff; ++ky)
-                    for (int kx = 0; kx < he.k_eff; ++kx)
-                        for (int c0 = 0; c0 < s.d.c; c0 += bk) {
-                            P.kbs.push_back(KbHost{e, false, -1, ky, kx, c0, bk, k_off});
-                            k_off += bk;
-                        }
+                const int bk = block_k(s.d.c), k = he.k_eff;
+                const int edge_off = k_off;
+                if (P.column_reuse && he.stride_eff == 1 && k >= 2) {
+                    for (int c0 = 0; c0 < s.d.c; c0 += bk)
+                        for (int kx = 0; kx < k; ++kx)
+                            for (int ky = 0; ky < k; ++ky)
+                                P.kbs.push_back(KbHost{e, false, -1, ky, kx, c0, bk, edge_off + (ky * k + kx) * s.d.c + c0,
+                                                       ky == 0 ? P.th + k - 1 : 0, ky, ky == k - 1});
+                } else {
+                    for (int ky = 0; ky < k; ++ky)
+                        for (int kx = 0; kx < k; ++kx)
+                            for (int c0 = 0; c0 < s.d.c; c0 += bk)
+                                P.kbs.push_back(KbHost{e, false, -1, ky, kx, c0, bk, edge_off + (ky * k + kx) * s.d.c + c0,
+                                                       P.th, 0, true});
+                }
+                k_off += k * k * s.d.c;
             }
         }
         P.k_total = k_off;
@@ -532,9 +613,20 @@ sr_status sr_tc_plan(sr_graph* g, size_t& off)
         for (auto& p : tl) E->group_tiles[gi].push_back(p.second);
         E->group_tile_offset.push_back(n_tiles);
         n_tiles += (int)tl.size();
-        const int stage_bytes = kABytes + max_c * 128;
-        E->group_stage_bytes.push_back(stage_bytes);
-        E->group_stages.push_back(std::max(2, std::min(kMaxStages, kSmemBudget / stage_bytes)));
+        int a_slot = kABytes;
+        for (int v : g->groups[gi]) {
+            if (E->node_of[v] < 0) continue;
+            const NodePlan& P = E->nodes[E->node_of[v]];
+            for (const KbHost& kb : P.kbs)
+                a_slot = std::max(a_slot, (int)sr_align_up((size_t)std::max(kTileM, kb.a_rows * P.tw * P.tb) * kb.bk * 2 +
+                                                           (size_t)kb.a_shift * 0, 1024));
+            if (P.column_reuse)      // the last window starts (k-1)*tw rows down and still reads 128 rows
+                for (const KbHost& kb : P.kbs)
+                    a_slot = std::max(a_slot, (int)sr_align_up((size_t)(kb.a_shift * P.tw + kTileM) * kb.bk * 2, 1024));
+        }
+        const int n_a = std::max(2, std::min(kMaxA, (kSmemBudget - kBUnits * kBUnit) / a_slot));
+        E->group_a_slot.push_back(a_slot);
+        E->group_n_a.push_back(n_a);
     }
     for (const NodePlan& P : E->nodes) n_kbs += (int)P.kbs.size();
     E->n_tiles = n_tiles;
@@ -594,6 +686,8 @@ sr_status sr_tc_bind(sr_graph* g)
         d.n_kb = (int)P.kbs.size();
         // instruction descriptor: D = f32, A = B = bf16, both K-major, N = C_out, M = 128
         d.idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(n.d.c >> 3) << 17) | ((uint32_t)(kTileM >> 4) << 24);
+        d.b_units = 1;
+        while (d.b_units * kBUnit < n.d.c * 128) d.b_units *= 2;
         std::map<int, int> wmap;                      // bk -> weight tensor map
         for (const KbHost& kb : P.kbs) {
             if (wmap.count(kb.bk)) continue;
@@ -618,13 +712,19 @@ sr_status sr_tc_bind(sr_graph* g)
             k.k_off = kb.k_off;
             k.n_k16 = kb.bk / 16;
             k.desc_hi = desc_hi_of(kb.bk);
-            k.tx_bytes = (uint32_t)(kb.bk * 2 * (P.tw * P.th * P.tb + n.d.c));
+            k.a_bytes = (uint32_t)(kb.bk * 2 * P.tw * kb.a_rows * P.tb);
+            k.b_bytes = (uint32_t)(kb.bk * 2 * n.d.c);
+            k.a_off = (uint32_t)(kb.a_shift * P.tw * kb.bk * 2);
+            k.a_release = kb.a_release ? 1u : 0u;
             if (kb.stem) {
                 const StemPlan& S = E->stems[kb.stem_index];
                 for (int par = 0; par < 2; ++par)
                     k.a_map[par] = act_map(ws + S.buf[par].offset, S.Kp, n.d.w, n.d.h, (size_t)S.Kp * 2,
                                            (size_t)n.d.w * S.Kp * 2, (size_t)n.d.h * n.d.w * S.Kp * 2, S.Kp, P.tw, P.th, P.tb);
                 k.qx = k.qy = k.c0 = 0;
+            } else if (kb.a_rows == 0) {
+                k.a_map[0] = k.a_map[1] = 0;             // reuses the box the first tap of this filter column loaded
+                k.qx = k.qy = 0; k.c0 = kb.c0;
             } else {
                 // input pixel = stride * (output pixel + q) + r, q = floor((tap - pad) / stride), r the residue:
                 // the residue-class view of the source makes the tap a dense box starting at (w0 + qx, h0 + qy)
@@ -636,7 +736,7 @@ sr_status sr_tc_bind(sr_graph* g)
                 for (int par = 0; par < 2; ++par) {
                     char* base = ws + s.state[par].offset + ((size_t)ry * s.d.w + rx) * s.d.c * 2;
                     k.a_map[par] = act_map(base, s.d.c, Wv, Hv, (size_t)st * s.d.c * 2, (size_t)st * s.d.w * s.d.c * 2,
-                                           (size_t)s.d.h * s.d.w * s.d.c * 2, kb.bk, P.tw, P.th, P.tb);
+                                           (size_t)s.d.h * s.d.w * s.d.c * 2, kb.bk, P.tw, kb.a_rows, P.tb);
                 }
                 k.qx = qx; k.qy = qy; k.c0 = kb.c0;
             }
@@ -726,14 +826,13 @@ int sr_tc_launch_group(sr_graph* g, int group, int t_off, cudaStream_t s)
 {
     TcEngine* E = eng(g);
     if (!E || E->group_tiles[group].empty()) return 0;
-    const int stages = E->group_stages[group], stage_bytes = E->group_stage_bytes[group];
-    const size_t smem = (size_t)stages * stage_bytes + 1024;
+    const int n_a = E->group_n_a[group], a_slot = E->group_a_slot[group];
+    const size_t smem = (size_t)n_a * a_slot + (size_t)kBUnits * kBUnit + 1024;
     sr_tc_group_kernel<<<E->group_grid[group], kThreads, smem, s>>>(
         reinterpret_cast<const CUtensorMap*>(g->ws + E->r_maps.offset), reinterpret_cast<const TcNode*>(g->ws + E->r_nodes.offset),
         reinterpret_cast<const TcKBlock*>(g->ws + E->r_kbs.offset),
         reinterpret_cast<const TcTile*>(g->ws + E->r_tiles.offset) + E->group_tile_offset[group],
-        (int)E->group_tiles[group].size(), reinterpret_cast<SrFrameCtl*>(g->ws + g->r_ctl.offset), t_off, g->batch, stages,
-        stage_bytes);
+        (int)E->group_tiles[group].size(), reinterpret_cast<SrFrameCtl*>(g->ws + g->r_ctl.offset), t_off, g->batch, n_a, a_slot);
     return 1;
 }
 
