@@ -46,7 +46,7 @@ constexpr int kSmemBudget = 216 * 1024;
 constexpr long long kWaitCycles = 2000000000LL;       // about a second
 
 struct TcKBlock {
-    int32_t a_map[2];       // tensor map of the A box for source frame parity 0 / 1
+    int32_t a_map0, a_map1; // tensor map of the A box for source frame parity 0 / 1
     int32_t R;              // 1: the edge reads frame t, 0: frame t+1
     int32_t qx, qy, c0;     // box origin relative to the tile origin (columns, rows) and first channel
     int32_t b_map;          // tensor map of the weight box
@@ -71,6 +71,13 @@ struct TcNode {
 };
 
 struct TcTile { int32_t node, b0, h0, w0; };
+
+// Work item of a CTA: one or two output tiles of the same node.  Two tiles share every weight box
+// (loaded once, multiplied twice), which halves the weight traffic per flop.
+struct TcPair {
+    int32_t node, n;
+    int32_t b0[2], h0[2], w0[2];
+};
 
 struct TcStem {             // a few-channel input edge staged as im2col rows
     const void* src[2];
@@ -175,7 +182,7 @@ __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi)
 // ------------------------------------------------------------------------------------------ the kernel
 __global__ void __launch_bounds__(kThreads, 1)
 sr_tc_group_kernel(const CUtensorMap* __restrict__ maps, const TcNode* __restrict__ nodes,
-                   const TcKBlock* __restrict__ kbs, const TcTile* __restrict__ tiles, int n_tiles,
+                   const TcKBlock* __restrict__ kbs, const TcPair* __restrict__ tiles, int n_tiles,
                    SrFrameCtl* __restrict__ ctl, int t_off, int B, int n_a, int a_slot)
 {
     extern __shared__ uint8_t smem_raw[];
@@ -230,9 +237,10 @@ sr_tc_group_kernel(const CUtensorMap* __restrict__ maps, const TcNode* __restric
             uint32_t ia = 0, bpos = 0, bphase = 0, b_used = 0;     // b_used: units that ever led a box
             bool ok = true;
             // tables are read by value one step ahead, so that no global load sits between two waits
-            TcTile tl_next = tiles[blockIdx.x < n_tiles ? blockIdx.x : 0];
+            const uint32_t a_half = (uint32_t)a_slot >> 1;
+            TcPair tl_next = tiles[blockIdx.x < n_tiles ? blockIdx.x : 0];
             for (int ti = blockIdx.x; ti < n_tiles && ok; ti += gridDim.x) {
-                const TcTile tl = tl_next;
+                const TcPair tl = tl_next;
                 if (ti + (int)gridDim.x < n_tiles) tl_next = tiles[ti + gridDim.x];
                 const int first_kb = nodes[tl.node].first_kb, n_kb = nodes[tl.node].n_kb;
                 const uint32_t u = (uint32_t)nodes[tl.node].b_units;
@@ -243,9 +251,13 @@ sr_tc_group_kernel(const CUtensorMap* __restrict__ maps, const TcNode* __restric
                     if (k.a_bytes) {
                         const uint32_t s = ia % n_a, ph = (ia / n_a) & 1;
                         if (!mbar_wait(bar_aempty + 8 * s, ph ^ 1, abortp)) { ok = false; break; }
-                        mbar_expect_tx(bar_afull + 8 * s, k.a_bytes);
-                        tma_load_4d(a_ring + s * a_slot, &maps[k.a_map[k.R ? prev : cur]], bar_afull + 8 * s, k.c0,
-                                    tl.w0 + k.qx, tl.h0 + k.qy, tl.b0);
+                        mbar_expect_tx(bar_afull + 8 * s, k.a_bytes * (uint32_t)tl.n);
+                        const int par = k.R ? prev : cur;
+                        const CUtensorMap* am = &maps[par ? k.a_map1 : k.a_map0];
+                        tma_load_4d(a_ring + s * a_slot, am, bar_afull + 8 * s, k.c0, tl.w0[0] + k.qx, tl.h0[0] + k.qy, tl.b0[0]);
+                        if (tl.n == 2)
+                            tma_load_4d(a_ring + s * a_slot + a_half, am, bar_afull + 8 * s, k.c0, tl.w0[1] + k.qx,
+                                        tl.h0[1] + k.qy, tl.b0[1]);
                         ++ia;
                     }
                     bpos = (bpos + u - 1) & ~(u - 1);
@@ -272,12 +284,16 @@ sr_tc_group_kernel(const CUtensorMap* __restrict__ maps, const TcNode* __restric
         if (lane == 0) {
             uint32_t ia = 0, bpos = 0, bphase = 0, tile_it = 0, a_cur = 0;
             bool ok = true;
-            int node_next = tiles[blockIdx.x < n_tiles ? blockIdx.x : 0].node;
+            const uint32_t a_half = (uint32_t)a_slot >> 1;
+            int node_next = tiles[blockIdx.x < n_tiles ? blockIdx.x : 0].node, n_next = tiles[blockIdx.x < n_tiles ? blockIdx.x : 0].n;
             for (int ti = blockIdx.x; ti < n_tiles && ok; ti += gridDim.x, ++tile_it) {
-                const int node = node_next;
-                if (ti + (int)gridDim.x < n_tiles) node_next = tiles[ti + gridDim.x].node;
+                const int node = node_next, two = n_next == 2;
+                if (ti + (int)gridDim.x < n_tiles) {
+                    node_next = tiles[ti + gridDim.x].node;
+                    n_next = tiles[ti + gridDim.x].n;
+                }
                 const int first_kb = nodes[node].first_kb, n_kb = nodes[node].n_kb;
-                const uint32_t u = (uint32_t)nodes[node].b_units, idesc = nodes[node].idesc;
+                const uint32_t u = (uint32_t)nodes[node].b_units, idesc = nodes[node].idesc, ncol = (uint32_t)nodes[node].C;
                 TcKBlock k_next = kbs[first_kb];
                 const uint32_t acc = tile_it & 1, acc_ph = (tile_it >> 1) & 1;
                 if (!mbar_wait(bar_tempty + 8 * acc, acc_ph ^ 1, abortp)) { ok = false; break; }
@@ -304,11 +320,15 @@ sr_tc_group_kernel(const CUtensorMap* __restrict__ maps, const TcNode* __restric
                         const uint64_t a_desc = hi | (uint64_t)(((a_addr + 32 * j) >> 4) & 0x3FFFu) | (1ull << 16);
                         const uint64_t b_desc = hi | (uint64_t)(((b_addr + 32 * j) >> 4) & 0x3FFFu) | (1ull << 16);
                         tc_mma_bf16(d_tmem, a_desc, b_desc, idesc, (kb | j) != 0);
+                        if (two) {
+                            const uint64_t a2 = hi | (uint64_t)(((a_addr + a_half + 32 * j) >> 4) & 0x3FFFu) | (1ull << 16);
+                            tc_mma_bf16(d_tmem + ncol, a2, b_desc, idesc, (kb | j) != 0);
+                        }
                     }
                     tc_commit(bar_bempty + 8 * s);                       // frees the B slot once these MMAs have read it
                     if (k.a_release) tc_commit(bar_aempty + 8 * a_cur);  // last reader of the A slot
                 }
-                if (ok) tc_commit(bar_tfull + 8 * acc);     // accumulator complete
+                if (ok) tc_commit(bar_tfull + 8 * acc);     // accumulators complete
             }
         }
     } else {
@@ -318,33 +338,36 @@ sr_tc_group_kernel(const CUtensorMap* __restrict__ maps, const TcNode* __restric
         uint32_t tile_it = 0;
         bool ok = true;
         for (int ti = blockIdx.x; ti < n_tiles && ok; ti += gridDim.x, ++tile_it) {
-            const TcTile tl = tiles[ti];
+            const TcPair tl = tiles[ti];
             const TcNode nd = nodes[tl.node];
             const uint32_t acc = tile_it & 1, acc_ph = (tile_it >> 1) & 1;
             if (!mbar_wait(bar_tfull + 8 * acc, acc_ph, abortp)) { ok = false; break; }
             tc_fence_after();
             const int per = nd.tw * nd.th;
             const int bi = m / per, rem = m - bi * per, hi = rem / nd.tw, wi = rem - hi * nd.tw;
-            const int b = tl.b0 + bi, h = tl.h0 + hi, w = tl.w0 + wi;
-            const bool valid = bi < nd.tb && b < B && h < nd.H && w < nd.W;
-            __nv_bfloat16* dst = static_cast<__nv_bfloat16*>(nd.state[cur]) + (((size_t)b * nd.H + h) * nd.W + w) * nd.C;
-            const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + acc * 256;
-            for (int c0 = 0; c0 < nd.C; c0 += 32) {
-                uint32_t r[32];
-                tc_ld32(taddr + c0, r);
-                tc_wait_ld();
-                if (valid) {
-                    uint32_t o[16];
+            for (int half = 0; half < tl.n; ++half) {
+                const int b = (half ? tl.b0[1] : tl.b0[0]) + bi, h = (half ? tl.h0[1] : tl.h0[0]) + hi,
+                          w = (half ? tl.w0[1] : tl.w0[0]) + wi;
+                const bool valid = bi < nd.tb && b < B && h < nd.H && w < nd.W;
+                __nv_bfloat16* dst = static_cast<__nv_bfloat16*>(nd.state[cur]) + (((size_t)b * nd.H + h) * nd.W + w) * nd.C;
+                const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + acc * 256 + half * nd.C;
+                for (int c0 = 0; c0 < nd.C; c0 += 32) {
+                    uint32_t r[32];
+                    tc_ld32(taddr + c0, r);
+                    tc_wait_ld();
+                    if (valid) {
+                        uint32_t o[16];
 #pragma unroll
-                    for (int j = 0; j < 16; ++j) {
-                        float v0 = __uint_as_float(r[2 * j]) + __ldg(nd.bias + c0 + 2 * j);
-                        float v1 = __uint_as_float(r[2 * j + 1]) + __ldg(nd.bias + c0 + 2 * j + 1);
-                        if (nd.act == 1) { v0 = fmaxf(v0, 0.f); v1 = fmaxf(v1, 0.f); }
-                        o[j] = pack_bf16(v0, v1);
+                        for (int j = 0; j < 16; ++j) {
+                            float v0 = __uint_as_float(r[2 * j]) + __ldg(nd.bias + c0 + 2 * j);
+                            float v1 = __uint_as_float(r[2 * j + 1]) + __ldg(nd.bias + c0 + 2 * j + 1);
+                            if (nd.act == 1) { v0 = fmaxf(v0, 0.f); v1 = fmaxf(v1, 0.f); }
+                            o[j] = pack_bf16(v0, v1);
+                        }
+                        uint4* d4 = reinterpret_cast<uint4*>(dst + c0);
+#pragma unroll
+                        for (int j = 0; j < 4; ++j) d4[j] = make_uint4(o[4 * j], o[4 * j + 1], o[4 * j + 2], o[4 * j + 3]);
                     }
-                    uint4* d4 = reinterpret_cast<uint4*>(dst + c0);
-#pragma unroll
-                    for (int j = 0; j < 4; ++j) d4[j] = make_uint4(o[4 * j], o[4 * j + 1], o[4 * j + 2], o[4 * j + 3]);
                 }
             }
             tc_fence_before();
@@ -445,7 +468,7 @@ struct TcEngine {
     std::vector<int> node_of;                    // graph node -> index in nodes, or -1
     std::vector<StemPlan> stems;
     std::vector<int> stem_of_edge;
-    std::vector<std::vector<TcTile>> group_tiles;
+    std::vector<std::vector<TcPair>> group_tiles;
     std::vector<int> group_tile_offset, group_a_slot, group_n_a, group_grid;
     SrRegion r_maps, r_nodes, r_kbs, r_tiles, r_stems;
     int n_maps = 0, n_kbs = 0, n_tiles = 0;
@@ -610,9 +633,23 @@ sr_status sr_tc_plan(sr_graph* g, size_t& off)
                         tl.push_back({(long long)P.k_total * n.d.c, TcTile{E->node_of[v], b0, h0, w0}});
         }
         std::stable_sort(tl.begin(), tl.end(), [](const auto& a, const auto& b) { return a.first > b.first; });
-        for (auto& p : tl) E->group_tiles[gi].push_back(p.second);
+        // pair neighbouring tiles of a node when both accumulators fit twice into TMEM (C_out <= 128)
+        for (size_t i = 0; i < tl.size();) {
+            const TcTile& a = tl[i].second;
+            TcPair pr{};
+            pr.node = a.node; pr.n = 1;
+            pr.b0[0] = a.b0; pr.h0[0] = a.h0; pr.w0[0] = a.w0;
+            const bool can_pair = g->nodes[E->nodes[a.node].node].d.c <= 128 && i + 1 < tl.size() && tl[i + 1].second.node == a.node;
+            if (can_pair) {
+                const TcTile& b = tl[i + 1].second;
+                pr.n = 2;
+                pr.b0[1] = b.b0; pr.h0[1] = b.h0; pr.w0[1] = b.w0;
+            }
+            E->group_tiles[gi].push_back(pr);
+            i += pr.n;
+        }
         E->group_tile_offset.push_back(n_tiles);
-        n_tiles += (int)tl.size();
+        n_tiles += (int)E->group_tiles[gi].size();
         int a_slot = kABytes;
         for (int v : g->groups[gi]) {
             if (E->node_of[v] < 0) continue;
@@ -624,6 +661,7 @@ sr_status sr_tc_plan(sr_graph* g, size_t& off)
                 for (const KbHost& kb : P.kbs)
                     a_slot = std::max(a_slot, (int)sr_align_up((size_t)(kb.a_shift * P.tw + kTileM) * kb.bk * 2, 1024));
         }
+        a_slot *= 2;                                  // room for the boxes of both tiles of a pair
         const int n_a = std::max(2, std::min(kMaxA, (kSmemBudget - kBUnits * kBUnit) / a_slot));
         E->group_a_slot.push_back(a_slot);
         E->group_n_a.push_back(n_a);
@@ -635,7 +673,7 @@ sr_status sr_tc_plan(sr_graph* g, size_t& off)
     E->r_maps = take(sizeof(CUtensorMap) * (size_t)(2 * n_kbs + 3 * E->nodes.size() + 1));
     E->r_nodes = take(sizeof(TcNode) * E->nodes.size());
     E->r_kbs = take(sizeof(TcKBlock) * (size_t)std::max(1, n_kbs));
-    E->r_tiles = take(sizeof(TcTile) * (size_t)std::max(1, n_tiles));
+    E->r_tiles = take(sizeof(TcPair) * (size_t)std::max(1, n_tiles));
     E->r_stems = take(sizeof(TcStem) * std::max<size_t>(1, E->stems.size()));
     return SR_OK;
 }
@@ -719,11 +757,11 @@ sr_status sr_tc_bind(sr_graph* g)
             if (kb.stem) {
                 const StemPlan& S = E->stems[kb.stem_index];
                 for (int par = 0; par < 2; ++par)
-                    k.a_map[par] = act_map(ws + S.buf[par].offset, S.Kp, n.d.w, n.d.h, (size_t)S.Kp * 2,
+                    (par ? k.a_map1 : k.a_map0) = act_map(ws + S.buf[par].offset, S.Kp, n.d.w, n.d.h, (size_t)S.Kp * 2,
                                            (size_t)n.d.w * S.Kp * 2, (size_t)n.d.h * n.d.w * S.Kp * 2, S.Kp, P.tw, P.th, P.tb);
                 k.qx = k.qy = k.c0 = 0;
             } else if (kb.a_rows == 0) {
-                k.a_map[0] = k.a_map[1] = 0;             // reuses the box the first tap of this filter column loaded
+                k.a_map0 = k.a_map1 = 0;             // reuses the box the first tap of this filter column loaded
                 k.qx = k.qy = 0; k.c0 = kb.c0;
             } else {
                 // input pixel = stride * (output pixel + q) + r, q = floor((tap - pad) / stride), r the residue:
@@ -735,19 +773,19 @@ sr_status sr_tc_bind(sr_graph* g)
                 if (Hv <= 0 || Wv <= 0) return SR_ERR_UNSUPPORTED;
                 for (int par = 0; par < 2; ++par) {
                     char* base = ws + s.state[par].offset + ((size_t)ry * s.d.w + rx) * s.d.c * 2;
-                    k.a_map[par] = act_map(base, s.d.c, Wv, Hv, (size_t)st * s.d.c * 2, (size_t)st * s.d.w * s.d.c * 2,
+                    (par ? k.a_map1 : k.a_map0) = act_map(base, s.d.c, Wv, Hv, (size_t)st * s.d.c * 2, (size_t)st * s.d.w * s.d.c * 2,
                                            (size_t)s.d.h * s.d.w * s.d.c * 2, kb.bk, P.tw, kb.a_rows, P.tb);
                 }
                 k.qx = qx; k.qy = qy; k.c0 = kb.c0;
             }
-            if (k.a_map[0] < 0 || k.a_map[1] < 0) return SR_ERR_CUDA;
+            if (k.a_map0 < 0 || k.a_map1 < 0) return SR_ERR_CUDA;
             dk.push_back(k);
         }
         dn.push_back(d);
     }
     if (maps.size() * sizeof(CUtensorMap) > E->r_maps.bytes) return SR_ERR_UNSUPPORTED;
     E->n_maps = (int)maps.size();
-    std::vector<TcTile> tiles;
+    std::vector<TcPair> tiles;
     for (auto& v : E->group_tiles) tiles.insert(tiles.end(), v.begin(), v.end());
     std::vector<TcStem> stems;
     for (const StemPlan& S : E->stems) {
@@ -767,7 +805,7 @@ sr_status sr_tc_bind(sr_graph* g)
         return bytes == 0 || cudaMemcpy(ws + r.offset, p, bytes, cudaMemcpyHostToDevice) == cudaSuccess;
     };
     if (!up(E->r_maps, maps.data(), maps.size() * sizeof(CUtensorMap)) || !up(E->r_nodes, dn.data(), dn.size() * sizeof(TcNode)) ||
-        !up(E->r_kbs, dk.data(), dk.size() * sizeof(TcKBlock)) || !up(E->r_tiles, tiles.data(), tiles.size() * sizeof(TcTile)) ||
+        !up(E->r_kbs, dk.data(), dk.size() * sizeof(TcKBlock)) || !up(E->r_tiles, tiles.data(), tiles.size() * sizeof(TcPair)) ||
         !up(E->r_stems, stems.data(), stems.size() * sizeof(TcStem)))
         return SR_ERR_CUDA;
     E->group_grid.clear();
@@ -831,7 +869,7 @@ int sr_tc_launch_group(sr_graph* g, int group, int t_off, cudaStream_t s)
     sr_tc_group_kernel<<<E->group_grid[group], kThreads, smem, s>>>(
         reinterpret_cast<const CUtensorMap*>(g->ws + E->r_maps.offset), reinterpret_cast<const TcNode*>(g->ws + E->r_nodes.offset),
         reinterpret_cast<const TcKBlock*>(g->ws + E->r_kbs.offset),
-        reinterpret_cast<const TcTile*>(g->ws + E->r_tiles.offset) + E->group_tile_offset[group],
+        reinterpret_cast<const TcPair*>(g->ws + E->r_tiles.offset) + E->group_tile_offset[group],
         (int)E->group_tiles[group].size(), reinterpret_cast<SrFrameCtl*>(g->ws + g->r_ctl.offset), t_off, g->batch, n_a, a_slot);
     return 1;
 }
