@@ -151,7 +151,12 @@ sr_status sr_graph_set_node_bias(sr_graph* g, int node, const float* bias_host);
 /* Options.  key 0 "engine": 0 = tensor cores where a node qualifies (default), 1 = CUDA-core kernels only.
  *           key 1 "frames per CUDA graph" used by sr_rollout_run: 0 = plain launches, n >= 1 = graphs
  *                  of n frames (default 0).
- * Must be set before sr_graph_bind_workspace (engine) / before the first run (graphs). */
+ *           key 2 "weight ring": 4 KiB units of shared memory the tensor-core kernel gives to weight tiles
+ *                  (8, 16, 24 or 32; 0 = default); the rest of the shared memory holds activation tiles.
+ *           key 3 "tile width": width in pixels (8, 16 or 32; 0 = default) of the 128-pixel output tiles of
+ *                  nodes that have a stride-1 k x k incoming edge (narrow tiles reload less halo, wide
+ *                  tiles read longer contiguous runs).
+ * Must be set before sr_graph_bind_workspace (engine, weight ring, tile width) / before the first run (graphs). */
 sr_status sr_graph_set_option(sr_graph* g, int key, int value);
 
 /*

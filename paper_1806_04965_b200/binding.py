@@ -103,7 +103,7 @@ class Graph:
     """A compiled network + rollout pattern (sr_graph).  batch=0 gives a theory-only graph."""
 
     def __init__(self, nodes: Sequence, edges: Sequence, R: Sequence[int], batch: int = 0, dtype: str = "bf16",
-                 engine: str = "auto", graph_frames: int = 0, device: str = "cuda:0", static_workspace: bool = False):
+                 engine: str = "auto", graph_frames: int = 0, device: str = "cuda:0", static_workspace: bool = False, weight_ring_units: int = 0, tile_width: int = 0):
         self._lib = load_library()
         self._h = ctypes.c_void_p()
         self.nodes, self.edges, self.R = list(nodes), list(edges), [int(r) for r in R]
@@ -125,6 +125,8 @@ class Graph:
             self.tdtype = torch.bfloat16 if dtype == "bf16" else torch.float32
             _check(self._lib.sr_graph_set_option(self._h, 0, {"auto": 0, "direct": 1}[engine]), "sr_graph_set_option")
             _check(self._lib.sr_graph_set_option(self._h, 1, int(graph_frames)), "sr_graph_set_option")
+            _check(self._lib.sr_graph_set_option(self._h, 2, int(weight_ring_units)), "sr_graph_set_option")
+            _check(self._lib.sr_graph_set_option(self._h, 3, int(tile_width)), "sr_graph_set_option")
             nbytes = ctypes.c_size_t()
             _check(self._lib.sr_graph_workspace_bytes(self._h, ctypes.byref(nbytes)), "sr_graph_workspace_bytes")
             self.workspace_bytes = nbytes.value

@@ -238,6 +238,18 @@ sr_status sr_graph_set_option(sr_graph* g, int key, int value)
         g->opt_graph_frames = value;
         return SR_OK;
     }
+    if (key == 3) {
+        if (g->ws) return SR_ERR_STATE;
+        if (value != 0 && value != 8 && value != 16 && value != 32) return SR_ERR_INVALID_ARG;
+        g->opt_tile_w = value;
+        return SR_OK;
+    }
+    if (key == 2) {
+        if (g->ws) return SR_ERR_STATE;
+        if (value < 0 || value > 32) return SR_ERR_INVALID_ARG;
+        g->opt_b_units = value;
+        return SR_OK;
+    }
     return SR_ERR_INVALID_ARG;
 }
 

@@ -41,24 +41,29 @@ constexpr int kTileM = 128;
 constexpr int kABytes = kTileM * 128;                 // A stage: 128 rows x up to 128 bytes
 constexpr int kThreads = 192;
 constexpr int kMaxA = 6;                              // A ring depth
-constexpr int kBUnit = 4096, kBUnits = 24;            // B ring: 24 units of 4 KiB; a weight box takes 1, 2, 4 or 8 units
-constexpr int kSmemBudget = 216 * 1024;
+constexpr int kBUnit = 4096, kMaxBUnits = 32;         // B ring: up to 32 units of 4 KiB; a weight box takes 1, 2, 4 or 8 units
+constexpr int kSmemBudget = 212 * 1024;
 constexpr long long kWaitCycles = 2000000000LL;       // about a second
 
+// One K-block of a node's reduction: 32 bytes, staged into shared memory per node so that the two
+// single-thread roles never wait on global memory between barrier waits.
 struct TcKBlock {
-    int32_t a_map0, a_map1; // tensor map of the A box for source frame parity 0 / 1
-    int32_t R;              // 1: the edge reads frame t, 0: frame t+1
-    int32_t qx, qy, c0;     // box origin relative to the tile origin (columns, rows) and first channel
-    int32_t b_map;          // tensor map of the weight box
-    int32_t k_off;          // first K column in the node's weight matrix
-    int32_t n_k16;          // MMA steps (K = 16 each) in this block
+    uint32_t k_off;         // first K column in the node's weight matrix
     uint32_t desc_hi;       // upper word of the shared-memory matrix descriptors (swizzle, SBO, version)
-    uint32_t a_bytes;       // bytes of the A box this block loads into a fresh A slot; 0 = reuse the current slot
-    uint32_t b_bytes;       // bytes of the weight box
-    uint32_t a_off;         // byte offset of this block's 128 rows inside the A slot
-    uint32_t a_release;     // 1: last block that reads the current A slot
-    uint32_t pad_[2];
+    uint16_t a_map0, a_map1;// tensor map of the A box for source frame parity 0 / 1
+    uint16_t b_map;         // tensor map of the weight box
+    int8_t qx, qy;          // box origin relative to the tile origin (columns, rows)
+    uint16_t c0;            // first channel of the box
+    uint16_t a_off16;       // (byte offset of this block's 128 rows inside the A slot) / 16
+    uint16_t a_bytes16;     // (bytes of the A box this block loads into a fresh A slot) / 16; 0 = reuse the current slot
+    uint16_t b_bytes16;     // (bytes of the weight box) / 16
+    uint8_t n_k16;          // MMA steps (K = 16 each) in this block
+    uint8_t flags;          // bit 0: the edge reads frame t (R = 1), else frame t+1; bit 1: last reader of the A slot
+    uint16_t pad_;
+    uint32_t pad2_;
 };
+static_assert(sizeof(TcKBlock) == 32, "K-block table entries are copied as two 16-byte words");
+constexpr int kMaxNodeKb = 128;                       // K-blocks per node the shared-memory table holds
 
 struct TcNode {
     void* state[2];
@@ -183,19 +188,20 @@ __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi)
 __global__ void __launch_bounds__(kThreads, 1)
 sr_tc_group_kernel(const CUtensorMap* __restrict__ maps, const TcNode* __restrict__ nodes,
                    const TcKBlock* __restrict__ kbs, const TcPair* __restrict__ tiles, int n_tiles,
-                   SrFrameCtl* __restrict__ ctl, int t_off, int B, int n_a, int a_slot)
+                   SrFrameCtl* __restrict__ ctl, int t_off, int B, int n_a, int a_slot, int n_bu)
 {
     extern __shared__ uint8_t smem_raw[];
-    __shared__ uint64_t bars[2 * kMaxA + 2 * kBUnits + 4];
+    __shared__ uint64_t bars[2 * kMaxA + 2 * kMaxBUnits + 4];
     __shared__ uint32_t tmem_slot;
     __shared__ int abort_flag;
+    __shared__ uint4 kb_tab[2][2 * kMaxNodeKb];            // K-block tables of the producer's and the issuer's current node
 
     const uint32_t a_ring = (smem_u32(smem_raw) + 1023u) & ~1023u;
     const uint32_t b_ring = a_ring + (uint32_t)(n_a * a_slot);
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const uint32_t bar_afull = smem_u32(&bars[0]), bar_aempty = smem_u32(&bars[kMaxA]);
-    const uint32_t bar_bfull = smem_u32(&bars[2 * kMaxA]), bar_bempty = smem_u32(&bars[2 * kMaxA + kBUnits]);
-    const uint32_t bar_tfull = smem_u32(&bars[2 * kMaxA + 2 * kBUnits]), bar_tempty = bar_tfull + 16;
+    const uint32_t bar_bfull = smem_u32(&bars[2 * kMaxA]), bar_bempty = smem_u32(&bars[2 * kMaxA + kMaxBUnits]);
+    const uint32_t bar_tfull = smem_u32(&bars[2 * kMaxA + 2 * kMaxBUnits]), bar_tempty = bar_tfull + 16;
 
     if (threadIdx.x == 0) {
         abort_flag = 0;
@@ -203,7 +209,7 @@ sr_tc_group_kernel(const CUtensorMap* __restrict__ maps, const TcNode* __restric
             mbar_init(bar_afull + 8 * s, 1);
             mbar_init(bar_aempty + 8 * s, 1);
         }
-        for (int s = 0; s < kBUnits; ++s) {
+        for (int s = 0; s < n_bu; ++s) {
             mbar_init(bar_bfull + 8 * s, 1);
             mbar_init(bar_bempty + 8 * s, 1);
         }
@@ -227,109 +233,108 @@ sr_tc_group_kernel(const CUtensorMap* __restrict__ maps, const TcNode* __restric
     const long long t = ctl->t + t_off;                     // this launch computes frame t+1 from frame t
     const int prev = (int)(t & 1), cur = prev ^ 1;
 
-    if (warp == 0) {
-        // ---------------------------------------------------------------- TMA producer
-        if (lane == 0) {
-            // The B ring is a ring of 4 KiB units; a weight box of a node takes b_units consecutive units
-            // starting at a multiple of b_units and is tracked by the barriers of its first unit.  Each
-            // unit's barriers flip phase only when that unit leads a box, so both sides keep a bit per
-            // unit (the MMA thread walks the identical sequence).
-            uint32_t ia = 0, bpos = 0, bphase = 0, b_used = 0;     // b_used: units that ever led a box
-            bool ok = true;
-            // tables are read by value one step ahead, so that no global load sits between two waits
-            const uint32_t a_half = (uint32_t)a_slot >> 1;
-            TcPair tl_next = tiles[blockIdx.x < n_tiles ? blockIdx.x : 0];
-            for (int ti = blockIdx.x; ti < n_tiles && ok; ti += gridDim.x) {
-                const TcPair tl = tl_next;
-                if (ti + (int)gridDim.x < n_tiles) tl_next = tiles[ti + gridDim.x];
-                const int first_kb = nodes[tl.node].first_kb, n_kb = nodes[tl.node].n_kb;
-                const uint32_t u = (uint32_t)nodes[tl.node].b_units;
-                TcKBlock k_next = kbs[first_kb];
-                for (int kb = 0; kb < n_kb; ++kb) {
-                    const TcKBlock k = k_next;
-                    if (kb + 1 < n_kb) k_next = kbs[first_kb + kb + 1];
-                    if (k.a_bytes) {
-                        const uint32_t s = ia % n_a, ph = (ia / n_a) & 1;
-                        if (!mbar_wait(bar_aempty + 8 * s, ph ^ 1, abortp)) { ok = false; break; }
-                        mbar_expect_tx(bar_afull + 8 * s, k.a_bytes * (uint32_t)tl.n);
-                        const int par = k.R ? prev : cur;
-                        const CUtensorMap* am = &maps[par ? k.a_map1 : k.a_map0];
-                        tma_load_4d(a_ring + s * a_slot, am, bar_afull + 8 * s, k.c0, tl.w0[0] + k.qx, tl.h0[0] + k.qy, tl.b0[0]);
-                        if (tl.n == 2)
-                            tma_load_4d(a_ring + s * a_slot + a_half, am, bar_afull + 8 * s, k.c0, tl.w0[1] + k.qx,
-                                        tl.h0[1] + k.qy, tl.b0[1]);
-                        ++ia;
+    if (warp <= 1) {
+        // Both single-thread roles walk the same tile list.  At every change of node the whole warp
+        // copies the node's K-block table into its own shared-memory buffer; lane 0 then runs the
+        // block loop out of shared memory.
+        uint4* my_tab = kb_tab[warp];
+        int cached_node = -1;
+        uint32_t ia = 0, bpos = 0, bphase = 0, b_used = 0, tile_it = 0, a_cur = 0;
+        const uint32_t a_half = (uint32_t)a_slot >> 1;
+        bool ok = true;
+        for (int ti = blockIdx.x; ti < n_tiles; ti += gridDim.x, ++tile_it) {
+            const TcPair tl = tiles[ti];
+            const int first_kb = nodes[tl.node].first_kb, n_kb = nodes[tl.node].n_kb;
+            const uint32_t u = (uint32_t)nodes[tl.node].b_units, idesc = nodes[tl.node].idesc, ncol = (uint32_t)nodes[tl.node].C;
+            if (tl.node != cached_node) {
+                __syncwarp();
+                const uint4* src = reinterpret_cast<const uint4*>(kbs + first_kb);
+                for (int i = lane; i < 2 * n_kb; i += 32) my_tab[i] = src[i];
+                cached_node = tl.node;
+                __syncwarp();
+            }
+            if (lane == 0 && ok) {
+                const TcKBlock* tab = reinterpret_cast<const TcKBlock*>(my_tab);
+                if (warp == 0) {
+                    // ------------------------------------------------------ TMA producer
+                    for (int kb = 0; kb < n_kb; ++kb) {
+                        const TcKBlock k = tab[kb];
+                        if (k.a_bytes16) {
+                            const uint32_t s = ia % n_a, ph = (ia / n_a) & 1;
+                            if (!mbar_wait(bar_aempty + 8 * s, ph ^ 1, abortp)) { ok = false; break; }
+                            mbar_expect_tx(bar_afull + 8 * s, ((uint32_t)k.a_bytes16 << 4) * (uint32_t)tl.n);
+                            const int par = (k.flags & 1) ? prev : cur;
+                            const CUtensorMap* am = &maps[par ? k.a_map1 : k.a_map0];
+                            tma_load_4d(a_ring + s * a_slot, am, bar_afull + 8 * s, k.c0, tl.w0[0] + k.qx, tl.h0[0] + k.qy, tl.b0[0]);
+                            if (tl.n == 2)
+                                tma_load_4d(a_ring + s * a_slot + a_half, am, bar_afull + 8 * s, k.c0, tl.w0[1] + k.qx,
+                                            tl.h0[1] + k.qy, tl.b0[1]);
+                            ++ia;
+                        }
+                        // The B ring is a ring of 4 KiB units; a weight box of a node takes b_units consecutive
+                        // units starting at a multiple of b_units and is tracked by the barriers of its first
+                        // unit.  A unit's barriers flip phase only when it leads a box, so both roles keep one
+                        // phase bit per unit and walk the identical sequence.
+                        bpos = (bpos + u - 1) & ~(u - 1);
+                        if (bpos >= (uint32_t)n_bu) bpos = 0;
+                        const uint32_t s = bpos, ph = (bphase >> s) & 1;
+                        if (!mbar_wait(bar_bempty + 8 * s, ph ^ 1, abortp)) { ok = false; break; }
+                        mbar_expect_tx(bar_bfull + 8 * s, (uint32_t)k.b_bytes16 << 4);
+                        tma_load_2d(b_ring + s * kBUnit, &maps[k.b_map], bar_bfull + 8 * s, (int)k.k_off, 0);
+                        bphase ^= 1u << s;
+                        b_used |= 1u << s;
+                        bpos += u;
                     }
-                    bpos = (bpos + u - 1) & ~(u - 1);
-                    if (bpos >= (uint32_t)kBUnits) bpos = 0;
-                    const uint32_t s = bpos, ph = (bphase >> s) & 1;
-                    if (!mbar_wait(bar_bempty + 8 * s, ph ^ 1, abortp)) { ok = false; break; }
-                    mbar_expect_tx(bar_bfull + 8 * s, k.b_bytes);
-                    tma_load_2d(b_ring + s * kBUnit, &maps[k.b_map], bar_bfull + 8 * s, k.k_off, 0);
-                    bphase ^= 1u << s;
-                    b_used |= 1u << s;
-                    bpos += u;
+                } else {
+                    // ------------------------------------------------------ MMA issuer
+                    const bool two = tl.n == 2;
+                    const uint32_t acc = tile_it & 1, acc_ph = (tile_it >> 1) & 1;
+                    if (!mbar_wait(bar_tempty + 8 * acc, acc_ph ^ 1, abortp)) ok = false;
+                    tc_fence_after();
+                    const uint32_t d_tmem = tmem_base + acc * 256;
+                    for (int kb = 0; kb < n_kb && ok; ++kb) {
+                        const TcKBlock k = tab[kb];
+                        if (k.a_bytes16) {
+                            a_cur = ia % n_a;
+                            if (!mbar_wait(bar_afull + 8 * a_cur, (ia / n_a) & 1, abortp)) { ok = false; break; }
+                            ++ia;
+                        }
+                        bpos = (bpos + u - 1) & ~(u - 1);
+                        if (bpos >= (uint32_t)n_bu) bpos = 0;
+                        const uint32_t s = bpos, ph = (bphase >> s) & 1;
+                        if (!mbar_wait(bar_bfull + 8 * s, ph, abortp)) { ok = false; break; }
+                        bphase ^= 1u << s;
+                        bpos += u;
+                        tc_fence_after();
+                        const uint64_t hi = ((uint64_t)k.desc_hi << 32) | (1ull << 16);
+                        const uint64_t a_desc = hi | (uint64_t)((((a_ring + a_cur * a_slot) >> 4) + k.a_off16) & 0x3FFFu);
+                        const uint64_t a_desc2 = hi | (uint64_t)((((a_ring + a_cur * a_slot + a_half) >> 4) + k.a_off16) & 0x3FFFu);
+                        const uint64_t b_desc = hi | (uint64_t)(((b_ring + s * kBUnit) >> 4) & 0x3FFFu);
+                        const uint32_t first = kb != 0;
+                        // a K = 16 step moves both operands 32 bytes along K: +2 in the descriptors' address field
+                        tc_mma_bf16(d_tmem, a_desc, b_desc, idesc, first);
+                        if (two) tc_mma_bf16(d_tmem + ncol, a_desc2, b_desc, idesc, first);
+                        for (uint32_t j = 1; j < k.n_k16; ++j) {
+                            tc_mma_bf16(d_tmem, a_desc + 2 * j, b_desc + 2 * j, idesc, 1);
+                            if (two) tc_mma_bf16(d_tmem + ncol, a_desc2 + 2 * j, b_desc + 2 * j, idesc, 1);
+                        }
+                        tc_commit(bar_bempty + 8 * s);                       // frees the B slot once these MMAs have read it
+                        if (k.flags & 2) tc_commit(bar_aempty + 8 * a_cur);  // last reader of the A slot
+                    }
+                    if (ok) tc_commit(bar_tfull + 8 * acc);     // accumulators complete
                 }
             }
+            ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
+            if (!ok) break;
+        }
+        if (warp == 0 && lane == 0) {
             // drain: every copy this thread started must have landed before the CTA may exit
             for (uint32_t j = 0; j < (uint32_t)n_a && j < ia; ++j) {
                 const uint32_t i2 = ia - 1 - j;
                 mbar_wait(bar_afull + 8 * (i2 % n_a), (i2 / n_a) & 1, abortp);
             }
-            for (uint32_t u = 0; u < (uint32_t)kBUnits; ++u)
-                if ((b_used >> u) & 1) mbar_wait(bar_bfull + 8 * u, ((bphase >> u) & 1) ^ 1, abortp);
-        }
-    } else if (warp == 1) {
-        // ---------------------------------------------------------------- MMA issuer
-        if (lane == 0) {
-            uint32_t ia = 0, bpos = 0, bphase = 0, tile_it = 0, a_cur = 0;
-            bool ok = true;
-            const uint32_t a_half = (uint32_t)a_slot >> 1;
-            int node_next = tiles[blockIdx.x < n_tiles ? blockIdx.x : 0].node, n_next = tiles[blockIdx.x < n_tiles ? blockIdx.x : 0].n;
-            for (int ti = blockIdx.x; ti < n_tiles && ok; ti += gridDim.x, ++tile_it) {
-                const int node = node_next, two = n_next == 2;
-                if (ti + (int)gridDim.x < n_tiles) {
-                    node_next = tiles[ti + gridDim.x].node;
-                    n_next = tiles[ti + gridDim.x].n;
-                }
-                const int first_kb = nodes[node].first_kb, n_kb = nodes[node].n_kb;
-                const uint32_t u = (uint32_t)nodes[node].b_units, idesc = nodes[node].idesc, ncol = (uint32_t)nodes[node].C;
-                TcKBlock k_next = kbs[first_kb];
-                const uint32_t acc = tile_it & 1, acc_ph = (tile_it >> 1) & 1;
-                if (!mbar_wait(bar_tempty + 8 * acc, acc_ph ^ 1, abortp)) { ok = false; break; }
-                tc_fence_after();
-                const uint32_t d_tmem = tmem_base + acc * 256;
-                for (int kb = 0; kb < n_kb; ++kb) {
-                    const TcKBlock k = k_next;
-                    if (kb + 1 < n_kb) k_next = kbs[first_kb + kb + 1];
-                    if (k.a_bytes) {
-                        a_cur = ia % n_a;
-                        if (!mbar_wait(bar_afull + 8 * a_cur, (ia / n_a) & 1, abortp)) { ok = false; break; }
-                        ++ia;
-                    }
-                    bpos = (bpos + u - 1) & ~(u - 1);
-                    if (bpos >= (uint32_t)kBUnits) bpos = 0;
-                    const uint32_t s = bpos, ph = (bphase >> s) & 1;
-                    if (!mbar_wait(bar_bfull + 8 * s, ph, abortp)) { ok = false; break; }
-                    bphase ^= 1u << s;
-                    bpos += u;
-                    tc_fence_after();
-                    const uint32_t a_addr = a_ring + a_cur * a_slot + k.a_off, b_addr = b_ring + s * kBUnit;
-                    const uint64_t hi = (uint64_t)k.desc_hi << 32;
-                    for (int j = 0; j < k.n_k16; ++j) {
-                        const uint64_t a_desc = hi | (uint64_t)(((a_addr + 32 * j) >> 4) & 0x3FFFu) | (1ull << 16);
-                        const uint64_t b_desc = hi | (uint64_t)(((b_addr + 32 * j) >> 4) & 0x3FFFu) | (1ull << 16);
-                        tc_mma_bf16(d_tmem, a_desc, b_desc, idesc, (kb | j) != 0);
-                        if (two) {
-                            const uint64_t a2 = hi | (uint64_t)(((a_addr + a_half + 32 * j) >> 4) & 0x3FFFu) | (1ull << 16);
-                            tc_mma_bf16(d_tmem + ncol, a2, b_desc, idesc, (kb | j) != 0);
-                        }
-                    }
-                    tc_commit(bar_bempty + 8 * s);                       // frees the B slot once these MMAs have read it
-                    if (k.a_release) tc_commit(bar_aempty + 8 * a_cur);  // last reader of the A slot
-                }
-                if (ok) tc_commit(bar_tfull + 8 * acc);     // accumulators complete
-            }
+            for (uint32_t v = 0; v < (uint32_t)n_bu; ++v)
+                if ((b_used >> v) & 1) mbar_wait(bar_bfull + 8 * v, ((bphase >> v) & 1) ^ 1, abortp);
         }
     } else {
         // ---------------------------------------------------------------- epilogue (warps 2..5)
@@ -469,7 +474,7 @@ struct TcEngine {
     std::vector<StemPlan> stems;
     std::vector<int> stem_of_edge;
     std::vector<std::vector<TcPair>> group_tiles;
-    std::vector<int> group_tile_offset, group_a_slot, group_n_a, group_grid;
+    std::vector<int> group_tile_offset, group_a_slot, group_n_a, group_n_bu, group_grid;
     SrRegion r_maps, r_nodes, r_kbs, r_tiles, r_stems;
     int n_maps = 0, n_kbs = 0, n_tiles = 0;
     int sm_count = 148;
@@ -526,15 +531,15 @@ void sr_tc_select_nodes(sr_graph* g)
         if (n.is_input || n.dense_target || (int)v == g->info.output_node) continue;
         if (n.d.c % 32 != 0 || n.d.c < 32 || n.d.c > 256) continue;
         bool ok = true;
-        int k_total = 0;
+        int n_blocks = 0;
         for (int e : n.in_edges) {
             const SrHostEdge& he = g->edges[e];
             const SrHostNode& s = g->nodes[he.d.src];
             if (he.d.kind != SR_EDGE_CONV) ok = false;
             else if (s.d.c % 16 != 0 && !is_stem(g, he)) ok = false;
-            k_total += he.K;
+            else n_blocks += is_stem(g, he) ? 1 : he.k_eff * he.k_eff * (s.d.c / block_k(s.d.c));
         }
-        if (ok && k_total >= 1) n.use_tc = true;
+        if (ok && n_blocks >= 1 && n_blocks <= kMaxNodeKb) n.use_tc = true;
     }
 }
 
@@ -567,8 +572,10 @@ sr_status sr_tc_plan(sr_graph* g, size_t& off)
             const SrHostEdge& he = g->edges[e];
             if (!is_stem(g, he) && he.stride_eff == 1 && he.k_eff >= 2) wants_reuse = true;
         }
-        if (wants_reuse && n.d.w >= 8 && n.d.h >= 16) {
-            P.tw = 8; P.th = 16; P.tb = 1;
+        int rtw = g->opt_tile_w > 0 ? g->opt_tile_w : 8;
+        while (rtw > 8 && (rtw > n.d.w || kTileM / rtw > n.d.h)) rtw /= 2;
+        if (wants_reuse && n.d.w >= rtw && n.d.h >= kTileM / rtw) {
+            P.tw = rtw; P.th = kTileM / rtw; P.tb = 1;
             P.column_reuse = true;
         } else {
             P.tw = std::min(n.d.w, kTileM);
@@ -662,9 +669,12 @@ sr_status sr_tc_plan(sr_graph* g, size_t& off)
                     a_slot = std::max(a_slot, (int)sr_align_up((size_t)(kb.a_shift * P.tw + kTileM) * kb.bk * 2, 1024));
         }
         a_slot *= 2;                                  // room for the boxes of both tiles of a pair
-        const int n_a = std::max(2, std::min(kMaxA, (kSmemBudget - kBUnits * kBUnit) / a_slot));
+        int n_bu = g->opt_b_units > 0 ? g->opt_b_units : 24;
+        n_bu = std::max(8, std::min(kMaxBUnits, n_bu / 8 * 8));
+        const int n_a = std::max(2, std::min(kMaxA, (kSmemBudget - n_bu * kBUnit) / a_slot));
         E->group_a_slot.push_back(a_slot);
         E->group_n_a.push_back(n_a);
+        E->group_n_bu.push_back(n_bu);
     }
     for (const NodePlan& P : E->nodes) n_kbs += (int)P.kbs.size();
     E->n_tiles = n_tiles;
@@ -745,24 +755,24 @@ sr_status sr_tc_bind(sr_graph* g)
             const SrHostEdge& he = g->edges[kb.edge];
             const SrHostNode& s = g->nodes[he.d.src];
             TcKBlock k{};
-            k.R = he.R;
-            k.b_map = wmap[kb.bk];
-            k.k_off = kb.k_off;
-            k.n_k16 = kb.bk / 16;
+            int map0 = -1, map1 = -1, qxv = 0, qyv = 0;
+            k.flags = (uint8_t)((he.R ? 1 : 0) | (kb.a_release ? 2 : 0));
+            k.b_map = (uint16_t)wmap[kb.bk];
+            k.k_off = (uint32_t)kb.k_off;
+            k.n_k16 = (uint8_t)(kb.bk / 16);
             k.desc_hi = desc_hi_of(kb.bk);
-            k.a_bytes = (uint32_t)(kb.bk * 2 * P.tw * kb.a_rows * P.tb);
-            k.b_bytes = (uint32_t)(kb.bk * 2 * n.d.c);
-            k.a_off = (uint32_t)(kb.a_shift * P.tw * kb.bk * 2);
-            k.a_release = kb.a_release ? 1u : 0u;
+            k.a_bytes16 = (uint16_t)((kb.bk * 2 * P.tw * kb.a_rows * P.tb) >> 4);
+            k.b_bytes16 = (uint16_t)((kb.bk * 2 * n.d.c) >> 4);
+            k.a_off16 = (uint16_t)((kb.a_shift * P.tw * kb.bk * 2) >> 4);
             if (kb.stem) {
                 const StemPlan& S = E->stems[kb.stem_index];
                 for (int par = 0; par < 2; ++par)
-                    (par ? k.a_map1 : k.a_map0) = act_map(ws + S.buf[par].offset, S.Kp, n.d.w, n.d.h, (size_t)S.Kp * 2,
+                    (par ? map1 : map0) = act_map(ws + S.buf[par].offset, S.Kp, n.d.w, n.d.h, (size_t)S.Kp * 2,
                                            (size_t)n.d.w * S.Kp * 2, (size_t)n.d.h * n.d.w * S.Kp * 2, S.Kp, P.tw, P.th, P.tb);
-                k.qx = k.qy = k.c0 = 0;
+                k.c0 = 0;
             } else if (kb.a_rows == 0) {
-                k.a_map0 = k.a_map1 = 0;             // reuses the box the first tap of this filter column loaded
-                k.qx = k.qy = 0; k.c0 = kb.c0;
+                map0 = map1 = 0;                         // reuses the box the first tap of this filter column loaded
+                k.c0 = (uint16_t)kb.c0;
             } else {
                 // input pixel = stride * (output pixel + q) + r, q = floor((tap - pad) / stride), r the residue:
                 // the residue-class view of the source makes the tap a dense box starting at (w0 + qx, h0 + qy)
@@ -773,12 +783,15 @@ sr_status sr_tc_bind(sr_graph* g)
                 if (Hv <= 0 || Wv <= 0) return SR_ERR_UNSUPPORTED;
                 for (int par = 0; par < 2; ++par) {
                     char* base = ws + s.state[par].offset + ((size_t)ry * s.d.w + rx) * s.d.c * 2;
-                    (par ? k.a_map1 : k.a_map0) = act_map(base, s.d.c, Wv, Hv, (size_t)st * s.d.c * 2, (size_t)st * s.d.w * s.d.c * 2,
+                    (par ? map1 : map0) = act_map(base, s.d.c, Wv, Hv, (size_t)st * s.d.c * 2, (size_t)st * s.d.w * s.d.c * 2,
                                            (size_t)s.d.h * s.d.w * s.d.c * 2, kb.bk, P.tw, kb.a_rows, P.tb);
                 }
-                k.qx = qx; k.qy = qy; k.c0 = kb.c0;
+                qxv = qx; qyv = qy; k.c0 = (uint16_t)kb.c0;
             }
-            if (k.a_map0 < 0 || k.a_map1 < 0) return SR_ERR_CUDA;
+            if (map0 < 0 || map1 < 0) return SR_ERR_CUDA;
+            if (map0 > 65535 || map1 > 65535 || qxv < -128 || qxv > 127 || qyv < -128 || qyv > 127) return SR_ERR_UNSUPPORTED;
+            k.a_map0 = (uint16_t)map0; k.a_map1 = (uint16_t)map1;
+            k.qx = (int8_t)qxv; k.qy = (int8_t)qyv;
             dk.push_back(k);
         }
         dn.push_back(d);
@@ -865,12 +878,13 @@ int sr_tc_launch_group(sr_graph* g, int group, int t_off, cudaStream_t s)
     TcEngine* E = eng(g);
     if (!E || E->group_tiles[group].empty()) return 0;
     const int n_a = E->group_n_a[group], a_slot = E->group_a_slot[group];
-    const size_t smem = (size_t)n_a * a_slot + (size_t)kBUnits * kBUnit + 1024;
+    const int n_bu = E->group_n_bu[group];
+    const size_t smem = (size_t)n_a * a_slot + (size_t)n_bu * kBUnit + 1024;
     sr_tc_group_kernel<<<E->group_grid[group], kThreads, smem, s>>>(
         reinterpret_cast<const CUtensorMap*>(g->ws + E->r_maps.offset), reinterpret_cast<const TcNode*>(g->ws + E->r_nodes.offset),
         reinterpret_cast<const TcKBlock*>(g->ws + E->r_kbs.offset),
         reinterpret_cast<const TcPair*>(g->ws + E->r_tiles.offset) + E->group_tile_offset[group],
-        (int)E->group_tiles[group].size(), reinterpret_cast<SrFrameCtl*>(g->ws + g->r_ctl.offset), t_off, g->batch, n_a, a_slot);
+        (int)E->group_tiles[group].size(), reinterpret_cast<SrFrameCtl*>(g->ws + g->r_ctl.offset), t_off, g->batch, n_a, a_slot, n_bu);
     return 1;
 }
 
