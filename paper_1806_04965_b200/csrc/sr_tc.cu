@@ -5,24 +5,32 @@
 // (paper Sec. A, "mathematically equivalent to concatenating all inputs"): the K loop of an output
 // tile simply walks the K-blocks of every incoming edge, tap by tap, into one TMEM accumulator.
 //
-//   M = 128 output pixels (a box of tb samples x th rows x tw columns), N = C_out, K-block = one
-//   filter tap x up to 64 input channels.  A-tiles come straight from the NHWC state of the source
-//   node through 4-D TMA boxes (zero fill outside the image = zero padding); a stride-s edge reads
-//   one of s*s residue-class views of the source, so every tap is again a dense box.  B-tiles come
-//   from the node's concatenated weight matrix [C_out][K] (K-major) through 2-D TMA boxes.
-//   Few-channel input edges (C_in = 1 or 3) are staged per frame into an im2col tensor with K
-//   padded to 16/32/64 so that they are ordinary K-blocks.
-//   A stride-1 k x k edge does not reload its activations per tap: for each filter column kx one box
-//   of th+k-1 image rows (tile width a multiple of 8 pixels, so an image row of the tile is a whole
-//   number of swizzle atoms) is loaded once, and the k taps of that column are row-shifted windows
-//   of it - the shared-memory descriptor just starts ky*tw rows further down.  A and B therefore
-//   travel through separate rings.
+// GEMM shape.  D[c_out][pixel] = sum_k W[c_out][k] * X[pixel][k]: the weights are the M operand
+// (128 rows per instruction, two halves for C_out > 128), up to 256 output pixels are the N operand.
+// Measured on B200, one tcgen05.mma of M = 128 costs about 110 cycles however small N is and 128
+// cycles at N = 256, and a tcgen05.commit is only free if about eight MMAs lie between commits; so
+// every instruction is given N = 256 pixels and weight tiles are released in groups.
+//
+// Operands.  K-block = one filter tap x up to 64 input channels.  Activation tiles come straight from
+// the NHWC state of the source node through 4-D TMA boxes (zero fill outside the image = zero
+// padding); a stride-s edge reads one of s*s residue-class views of the source, so every tap is again
+// a dense box.  Weight tiles come from the node's concatenated weight matrix [C_out][K] (K-major)
+// through 2-D TMA boxes.  Few-channel input edges (C_in = 1 or 3) are staged per frame into an im2col
+// tensor with K padded to 16/32/64 so that they are ordinary K-blocks.
+//
+// Pixel tile.  A tile is tb samples x th rows x tw columns (tw a multiple of 8, so an image row of
+// the tile is a whole number of swizzle atoms).  Every activation box holds th + sep rows per sample
+// (sep = k - 1 of the node's stride-1 k x k edges), and the N columns of the GEMM are the rows of
+// that stacked box: column n = (b * (th + sep) + r) * tw + x.  Columns with r >= th are never stored.
+// This makes the k taps of one filter column row-shifted windows of ONE box: the box is loaded once
+// per filter column and the shared-memory descriptor of tap ky just starts ky * tw rows further down.
 //
 // Warp roles in a CTA of 192 threads: warp 0 = TMA producer, warp 1 = MMA issuer (owns TMEM),
-// warps 2..5 = epilogue (TMEM -> registers -> bias, ReLU, bf16 -> NHWC global).  Two accumulators in
-// TMEM let the epilogue of a tile overlap the main loop of the next.  CTAs are persistent and walk a
-// tile list sorted by decreasing work.  Every wait is bounded; on expiry the kernel records an error
-// in the frame control block, drains its own copies, frees TMEM and returns.
+// warps 2..5 = epilogue (TMEM lane = output channel; bias, ReLU, bf16, NHWC stores in which a warp
+// writes 32 consecutive channels of one pixel).  Two accumulators in TMEM let the epilogue of a tile
+// overlap the main loop of the next when they fit.  CTAs are persistent and walk a tile list sorted
+// by decreasing work.  Every wait is bounded; on expiry the kernel records an error in the frame
+// control block, drains its own copies, frees TMEM and returns.
 #include <cuda.h>
 #include <cuda_bf16.h>
 #include <cuda_runtime.h>
@@ -37,52 +45,48 @@
 
 namespace {
 
-constexpr int kTileM = 128;
-constexpr int kABytes = kTileM * 128;                 // A stage: 128 rows x up to 128 bytes
+constexpr int kMaxCols = 256;                         // pixels (N of the MMA) per tile
 constexpr int kThreads = 192;
-constexpr int kMaxA = 6;                              // A ring depth
-constexpr int kBUnit = 4096, kMaxBUnits = 32;         // B ring: up to 32 units of 4 KiB; a weight box takes 1, 2, 4 or 8 units
-constexpr int kSmemBudget = 212 * 1024;
+constexpr int kMaxA = 4;                              // activation ring depth
+constexpr int kWUnit = 4096, kMaxWUnits = 32;         // weight ring: units of 4 KiB
+constexpr int kSmemBudget = 200 * 1024;
 constexpr long long kWaitCycles = 2000000000LL;       // about a second
+constexpr int kMaxNodeKb = 128;                       // K-blocks per node the shared-memory table holds
 
 // One K-block of a node's reduction: 32 bytes, staged into shared memory per node so that the two
 // single-thread roles never wait on global memory between barrier waits.
 struct TcKBlock {
     uint32_t k_off;         // first K column in the node's weight matrix
     uint32_t desc_hi;       // upper word of the shared-memory matrix descriptors (swizzle, SBO, version)
-    uint16_t a_map0, a_map1;// tensor map of the A box for source frame parity 0 / 1
-    uint16_t b_map;         // tensor map of the weight box
+    uint16_t x_map0, x_map1;// tensor map of the activation box for source frame parity 0 / 1
+    uint16_t w_map;         // tensor map of the weight box
     int8_t qx, qy;          // box origin relative to the tile origin (columns, rows)
     uint16_t c0;            // first channel of the box
-    uint16_t a_off16;       // (byte offset of this block's 128 rows inside the A slot) / 16
-    uint16_t a_bytes16;     // (bytes of the A box this block loads into a fresh A slot) / 16; 0 = reuse the current slot
-    uint16_t b_bytes16;     // (bytes of the weight box) / 16
+    uint16_t x_off16;       // (byte offset of this tap's window inside the activation slot) / 16
+    uint16_t x_bytes16;     // (bytes of the activation box this block loads into a fresh slot) / 16; 0 = reuse the slot
+    uint16_t w_bytes16;     // (bytes of the weight box) / 16
     uint8_t n_k16;          // MMA steps (K = 16 each) in this block
-    uint8_t flags;          // bit 0: the edge reads frame t (R = 1), else frame t+1; bit 1: last reader of the A slot
-    uint16_t pad_;
-    uint32_t pad2_;
+    uint8_t flags;          // 1: the edge reads frame t (R = 1), else frame t+1; 2: last reader of the activation
+                            // slot; 4: first box of a weight group; 8: last box of a weight group
+    uint8_t w_box;          // index of this block's weight box inside its group
+    uint8_t pad_[5];
 };
 static_assert(sizeof(TcKBlock) == 32, "K-block table entries are copied as two 16-byte words");
-constexpr int kMaxNodeKb = 128;                       // K-blocks per node the shared-memory table holds
 
 struct TcNode {
     void* state[2];
     const float* bias;
     int32_t H, W, C, act;
-    int32_t tw, th, tb;
+    int32_t tw, th, tb, sep;        // tile geometry (see the file comment)
+    int32_t n_cols;                 // N of the MMA: stacked rows of a tile, rounded up to 32
+    int32_t n_mh;                   // halves of 128 output channels
     int32_t first_kb, n_kb;
     uint32_t idesc;
-    int32_t b_units;        // B-ring units one weight box of this node occupies (power of two)
+    int32_t w_box_units, w_group_units;
+    int32_t pad_;
 };
 
 struct TcTile { int32_t node, b0, h0, w0; };
-
-// Work item of a CTA: one or two output tiles of the same node.  Two tiles share every weight box
-// (loaded once, multiplied twice), which halves the weight traffic per flop.
-struct TcPair {
-    int32_t node, n;
-    int32_t b0[2], h0[2], w0[2];
-};
 
 struct TcStem {             // a few-channel input edge staged as im2col rows
     const void* src[2];
@@ -187,21 +191,25 @@ __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi)
 // ------------------------------------------------------------------------------------------ the kernel
 __global__ void __launch_bounds__(kThreads, 1)
 sr_tc_group_kernel(const CUtensorMap* __restrict__ maps, const TcNode* __restrict__ nodes,
-                   const TcKBlock* __restrict__ kbs, const TcPair* __restrict__ tiles, int n_tiles,
-                   SrFrameCtl* __restrict__ ctl, int t_off, int B, int n_a, int a_slot, int n_bu)
+                   const TcKBlock* __restrict__ kbs, const TcTile* __restrict__ tiles, int n_tiles,
+                   SrFrameCtl* __restrict__ ctl, int t_off, int B, int n_a, int a_slot, int n_wu, int w_slot_units)
 {
     extern __shared__ uint8_t smem_raw[];
-    __shared__ uint64_t bars[2 * kMaxA + 2 * kMaxBUnits + 4];
+    __shared__ uint64_t bars[2 * kMaxA + 2 * kMaxWUnits + 4];
     __shared__ uint32_t tmem_slot;
     __shared__ int abort_flag;
     __shared__ uint4 kb_tab[2][2 * kMaxNodeKb];            // K-block tables of the producer's and the issuer's current node
+    __shared__ __align__(16) uint16_t epi_buf[4][32 * 32]; // per epilogue warp: 32 pixels x 32 channels, bf16
+    __shared__ int pix_off[kMaxCols];                      // element offset of every pixel of the current tile, -1 = not stored
 
-    const uint32_t a_ring = (smem_u32(smem_raw) + 1023u) & ~1023u;
-    const uint32_t b_ring = a_ring + (uint32_t)(n_a * a_slot);
+    // weight ring first: an M = 128 instruction on a node with fewer than 128 output channels reads
+    // rows past its weight box, which then still lie inside this allocation
+    const uint32_t w_ring = (smem_u32(smem_raw) + 1023u) & ~1023u;
+    const uint32_t a_ring = w_ring + (uint32_t)(n_wu * kWUnit);
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const uint32_t bar_afull = smem_u32(&bars[0]), bar_aempty = smem_u32(&bars[kMaxA]);
-    const uint32_t bar_bfull = smem_u32(&bars[2 * kMaxA]), bar_bempty = smem_u32(&bars[2 * kMaxA + kMaxBUnits]);
-    const uint32_t bar_tfull = smem_u32(&bars[2 * kMaxA + 2 * kMaxBUnits]), bar_tempty = bar_tfull + 16;
+    const uint32_t bar_wfull = smem_u32(&bars[2 * kMaxA]), bar_wempty = smem_u32(&bars[2 * kMaxA + kMaxWUnits]);
+    const uint32_t bar_tfull = smem_u32(&bars[2 * kMaxA + 2 * kMaxWUnits]), bar_tempty = bar_tfull + 16;
 
     if (threadIdx.x == 0) {
         abort_flag = 0;
@@ -209,9 +217,9 @@ sr_tc_group_kernel(const CUtensorMap* __restrict__ maps, const TcNode* __restric
             mbar_init(bar_afull + 8 * s, 1);
             mbar_init(bar_aempty + 8 * s, 1);
         }
-        for (int s = 0; s < n_bu; ++s) {
-            mbar_init(bar_bfull + 8 * s, 1);
-            mbar_init(bar_bempty + 8 * s, 1);
+        for (int s = 0; s < n_wu; ++s) {
+            mbar_init(bar_wfull + 8 * s, 1);
+            mbar_init(bar_wempty + 8 * s, 1);
         }
         for (int a = 0; a < 2; ++a) {
             mbar_init(bar_tfull + 8 * a, 1);
@@ -233,19 +241,30 @@ sr_tc_group_kernel(const CUtensorMap* __restrict__ maps, const TcNode* __restric
     const long long t = ctl->t + t_off;                     // this launch computes frame t+1 from frame t
     const int prev = (int)(t & 1), cur = prev ^ 1;
 
+    // Accumulator buffers: a tile whose n_mh * n_cols columns fit into 256 takes the less used of the
+    // two 256-column buffers, a wider tile takes both.  uses[] counts the tiles a buffer has served;
+    // the issuer and the epilogue warps walk the same tile list and make the same choice.
+    uint32_t uses0 = 0, uses1 = 0;
+
     if (warp <= 1) {
         // Both single-thread roles walk the same tile list.  At every change of node the whole warp
         // copies the node's K-block table into its own shared-memory buffer; lane 0 then runs the
         // block loop out of shared memory.
         uint4* my_tab = kb_tab[warp];
         int cached_node = -1;
-        uint32_t ia = 0, bpos = 0, bphase = 0, b_used = 0, tile_it = 0, a_cur = 0;
-        const uint32_t a_half = (uint32_t)a_slot >> 1;
+        // The weight ring is a ring of slots of w_slot_units 4 KiB units (the largest weight group of
+        // the launch), handed back through one "empty" barrier per slot.  Box i of a group starts at
+        // unit i * w_box_units of its slot and signals arrival on that unit's "full" barrier; which
+        // units lead a box depends on the node, and a unit's barrier flips phase only when used, so
+        // both roles keep one phase bit per unit.
+        const uint32_t n_ws = (uint32_t)(n_wu / w_slot_units);
+        uint32_t ia = 0, iw = 0, ws_cur = 0, wgrp = 0, wf_phase = 0, wf_used = 0, a_cur = 0;
         bool ok = true;
-        for (int ti = blockIdx.x; ti < n_tiles; ti += gridDim.x, ++tile_it) {
-            const TcPair tl = tiles[ti];
+        for (int ti = blockIdx.x; ti < n_tiles; ti += gridDim.x) {
+            const TcTile tl = tiles[ti];
             const int first_kb = nodes[tl.node].first_kb, n_kb = nodes[tl.node].n_kb;
-            const uint32_t u = (uint32_t)nodes[tl.node].b_units, idesc = nodes[tl.node].idesc, ncol = (uint32_t)nodes[tl.node].C;
+            const uint32_t box_u = (uint32_t)nodes[tl.node].w_box_units;
+            const uint32_t idesc = nodes[tl.node].idesc, n_cols = (uint32_t)nodes[tl.node].n_cols, n_mh = (uint32_t)nodes[tl.node].n_mh;
             if (tl.node != cached_node) {
                 __syncwarp();
                 const uint4* src = reinterpret_cast<const uint4*>(kbs + first_kb);
@@ -259,69 +278,76 @@ sr_tc_group_kernel(const CUtensorMap* __restrict__ maps, const TcNode* __restric
                     // ------------------------------------------------------ TMA producer
                     for (int kb = 0; kb < n_kb; ++kb) {
                         const TcKBlock k = tab[kb];
-                        if (k.a_bytes16) {
+                        if (k.x_bytes16) {
                             const uint32_t s = ia % n_a, ph = (ia / n_a) & 1;
                             if (!mbar_wait(bar_aempty + 8 * s, ph ^ 1, abortp)) { ok = false; break; }
-                            mbar_expect_tx(bar_afull + 8 * s, ((uint32_t)k.a_bytes16 << 4) * (uint32_t)tl.n);
+                            mbar_expect_tx(bar_afull + 8 * s, (uint32_t)k.x_bytes16 << 4);
                             const int par = (k.flags & 1) ? prev : cur;
-                            const CUtensorMap* am = &maps[par ? k.a_map1 : k.a_map0];
-                            tma_load_4d(a_ring + s * a_slot, am, bar_afull + 8 * s, k.c0, tl.w0[0] + k.qx, tl.h0[0] + k.qy, tl.b0[0]);
-                            if (tl.n == 2)
-                                tma_load_4d(a_ring + s * a_slot + a_half, am, bar_afull + 8 * s, k.c0, tl.w0[1] + k.qx,
-                                            tl.h0[1] + k.qy, tl.b0[1]);
+                            tma_load_4d(a_ring + s * a_slot, &maps[par ? k.x_map1 : k.x_map0], bar_afull + 8 * s, k.c0,
+                                        tl.w0 + k.qx, tl.h0 + k.qy, tl.b0);
                             ++ia;
                         }
-                        // The B ring is a ring of 4 KiB units; a weight box of a node takes b_units consecutive
-                        // units starting at a multiple of b_units and is tracked by the barriers of its first
-                        // unit.  A unit's barriers flip phase only when it leads a box, so both roles keep one
-                        // phase bit per unit and walk the identical sequence.
-                        bpos = (bpos + u - 1) & ~(u - 1);
-                        if (bpos >= (uint32_t)n_bu) bpos = 0;
-                        const uint32_t s = bpos, ph = (bphase >> s) & 1;
-                        if (!mbar_wait(bar_bempty + 8 * s, ph ^ 1, abortp)) { ok = false; break; }
-                        mbar_expect_tx(bar_bfull + 8 * s, (uint32_t)k.b_bytes16 << 4);
-                        tma_load_2d(b_ring + s * kBUnit, &maps[k.b_map], bar_bfull + 8 * s, (int)k.k_off, 0);
-                        bphase ^= 1u << s;
-                        b_used |= 1u << s;
-                        bpos += u;
+                        if (k.flags & 4) {
+                            ws_cur = iw % n_ws;
+                            if (!mbar_wait(bar_wempty + 8 * ws_cur, ((iw / n_ws) & 1) ^ 1, abortp)) { ok = false; break; }
+                            wgrp = ws_cur * (uint32_t)w_slot_units;
+                            ++iw;
+                        }
+                        const uint32_t unit = wgrp + k.w_box * box_u;
+                        mbar_expect_tx(bar_wfull + 8 * unit, (uint32_t)k.w_bytes16 << 4);
+                        tma_load_2d(w_ring + unit * kWUnit, &maps[k.w_map], bar_wfull + 8 * unit, (int)k.k_off, 0);
+                        wf_phase ^= 1u << unit;
+                        wf_used |= 1u << unit;
                     }
                 } else {
                     // ------------------------------------------------------ MMA issuer
-                    const bool two = tl.n == 2;
-                    const uint32_t acc = tile_it & 1, acc_ph = (tile_it >> 1) & 1;
-                    if (!mbar_wait(bar_tempty + 8 * acc, acc_ph ^ 1, abortp)) ok = false;
+                    const bool wide = n_mh * n_cols > 256;
+                    const uint32_t acc = wide ? 0u : (uses0 <= uses1 ? 0u : 1u);
+                    if (wide || acc == 0) {
+                        if (!mbar_wait(bar_tempty, (uses0 & 1) ^ 1, abortp)) ok = false;
+                    }
+                    if (ok && (wide || acc == 1)) {
+                        if (!mbar_wait(bar_tempty + 8, (uses1 & 1) ^ 1, abortp)) ok = false;
+                    }
                     tc_fence_after();
                     const uint32_t d_tmem = tmem_base + acc * 256;
                     for (int kb = 0; kb < n_kb && ok; ++kb) {
                         const TcKBlock k = tab[kb];
-                        if (k.a_bytes16) {
+                        if (k.x_bytes16) {
                             a_cur = ia % n_a;
                             if (!mbar_wait(bar_afull + 8 * a_cur, (ia / n_a) & 1, abortp)) { ok = false; break; }
                             ++ia;
                         }
-                        bpos = (bpos + u - 1) & ~(u - 1);
-                        if (bpos >= (uint32_t)n_bu) bpos = 0;
-                        const uint32_t s = bpos, ph = (bphase >> s) & 1;
-                        if (!mbar_wait(bar_bfull + 8 * s, ph, abortp)) { ok = false; break; }
-                        bphase ^= 1u << s;
-                        bpos += u;
+                        if (k.flags & 4) {
+                            ws_cur = iw % n_ws;
+                            wgrp = ws_cur * (uint32_t)w_slot_units;
+                            ++iw;
+                        }
+                        const uint32_t unit = wgrp + k.w_box * box_u;
+                        if (!mbar_wait(bar_wfull + 8 * unit, (wf_phase >> unit) & 1, abortp)) { ok = false; break; }
+                        wf_phase ^= 1u << unit;
                         tc_fence_after();
                         const uint64_t hi = ((uint64_t)k.desc_hi << 32) | (1ull << 16);
-                        const uint64_t a_desc = hi | (uint64_t)((((a_ring + a_cur * a_slot) >> 4) + k.a_off16) & 0x3FFFu);
-                        const uint64_t a_desc2 = hi | (uint64_t)((((a_ring + a_cur * a_slot + a_half) >> 4) + k.a_off16) & 0x3FFFu);
-                        const uint64_t b_desc = hi | (uint64_t)(((b_ring + s * kBUnit) >> 4) & 0x3FFFu);
+                        const uint64_t x_desc = hi | (uint64_t)((((a_ring + a_cur * a_slot) >> 4) + k.x_off16) & 0x3FFFu);
+                        uint64_t w_desc = hi | (uint64_t)(((w_ring + unit * kWUnit) >> 4) & 0x3FFFu);
                         const uint32_t first = kb != 0;
-                        // a K = 16 step moves both operands 32 bytes along K: +2 in the descriptors' address field
-                        tc_mma_bf16(d_tmem, a_desc, b_desc, idesc, first);
-                        if (two) tc_mma_bf16(d_tmem + ncol, a_desc2, b_desc, idesc, first);
-                        for (uint32_t j = 1; j < k.n_k16; ++j) {
-                            tc_mma_bf16(d_tmem, a_desc + 2 * j, b_desc + 2 * j, idesc, 1);
-                            if (two) tc_mma_bf16(d_tmem + ncol, a_desc2 + 2 * j, b_desc + 2 * j, idesc, 1);
+                        // a K = 16 step moves both operands 32 bytes along K (+2 in the address field);
+                        // the second half of the output channels starts 128 weight rows further
+                        for (uint32_t h = 0; h < n_mh; ++h) {
+                            tc_mma_bf16(d_tmem + h * n_cols, w_desc, x_desc, idesc, first);
+                            for (uint32_t j = 1; j < k.n_k16; ++j)
+                                tc_mma_bf16(d_tmem + h * n_cols, w_desc + 2 * j, x_desc + 2 * j, idesc, 1);
+                            w_desc += 256u * k.n_k16;
                         }
-                        tc_commit(bar_bempty + 8 * s);                       // frees the B slot once these MMAs have read it
-                        if (k.flags & 2) tc_commit(bar_aempty + 8 * a_cur);  // last reader of the A slot
+                        if (k.flags & 8) tc_commit(bar_wempty + 8 * ws_cur); // hands the weight slot back
+                        if (k.flags & 2) tc_commit(bar_aempty + 8 * a_cur);  // last reader of the activation slot
                     }
-                    if (ok) tc_commit(bar_tfull + 8 * acc);     // accumulators complete
+                    if (ok) {
+                        if (wide || acc == 0) tc_commit(bar_tfull);
+                        if (wide || acc == 1) tc_commit(bar_tfull + 8);
+                    }
+                    if (wide || acc == 0) ++uses0;
+                    if (wide || acc == 1) ++uses1;
                 }
             }
             ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
@@ -333,51 +359,83 @@ sr_tc_group_kernel(const CUtensorMap* __restrict__ maps, const TcNode* __restric
                 const uint32_t i2 = ia - 1 - j;
                 mbar_wait(bar_afull + 8 * (i2 % n_a), (i2 / n_a) & 1, abortp);
             }
-            for (uint32_t v = 0; v < (uint32_t)n_bu; ++v)
-                if ((b_used >> v) & 1) mbar_wait(bar_bfull + 8 * v, ((bphase >> v) & 1) ^ 1, abortp);
+            for (uint32_t v = 0; v < (uint32_t)n_wu; ++v)
+                if ((wf_used >> v) & 1) mbar_wait(bar_wfull + 8 * v, ((wf_phase >> v) & 1) ^ 1, abortp);
         }
     } else {
         // ---------------------------------------------------------------- epilogue (warps 2..5)
+        // TMEM lane = output channel, TMEM column = pixel.  A warp turns 32 channels x 32 pixels into
+        // NHWC order through a 2 KiB shared-memory buffer: every thread writes its channel of 32 pixels
+        // (bias, ReLU, bf16), then reads back 8 consecutive channels of one pixel and stores them as one
+        // 16-byte word, so a pixel's 32 channels leave the warp as one 64-byte run.  The element offset
+        // of every pixel of the tile (or -1 for the separator rows and for pixels outside the image) is
+        // tabulated once per tile.
         const int quarter = warp & 3;                       // TMEM lanes 32*quarter .. +31 belong to this warp
-        const int m = quarter * 32 + lane;                  // row of the tile = output pixel
-        uint32_t tile_it = 0;
+        const int et = threadIdx.x - 64;                    // 0..127 among the epilogue threads
+        uint16_t* tbuf = &epi_buf[warp - 2][0];
         bool ok = true;
-        for (int ti = blockIdx.x; ti < n_tiles && ok; ti += gridDim.x, ++tile_it) {
-            const TcPair tl = tiles[ti];
+        for (int ti = blockIdx.x; ti < n_tiles && ok; ti += gridDim.x) {
+            const TcTile tl = tiles[ti];
             const TcNode nd = nodes[tl.node];
-            const uint32_t acc = tile_it & 1, acc_ph = (tile_it >> 1) & 1;
-            if (!mbar_wait(bar_tfull + 8 * acc, acc_ph, abortp)) { ok = false; break; }
+            const int rows = nd.th + nd.sep;
+            for (int n = et; n < nd.n_cols; n += 128) {
+                const int x = n % nd.tw, q = n / nd.tw, r = q % rows, bi = q / rows;
+                const int b = tl.b0 + bi, y = tl.h0 + r, xx = tl.w0 + x;
+                const bool v = r < nd.th && bi < nd.tb && b < B && y < nd.H && xx < nd.W;
+                pix_off[n] = v ? (int)((((size_t)b * nd.H + y) * nd.W + xx) * nd.C) : -1;
+            }
+            const bool wide = nd.n_mh * nd.n_cols > 256;
+            const uint32_t acc = wide ? 0u : (uses0 <= uses1 ? 0u : 1u);
+            if (wide || acc == 0) {
+                if (!mbar_wait(bar_tfull, uses0 & 1, abortp)) ok = false;
+            }
+            if (ok && (wide || acc == 1)) {
+                if (!mbar_wait(bar_tfull + 8, uses1 & 1, abortp)) ok = false;
+            }
+            ok = __all_sync(0xffffffffu, ok);
+            asm volatile("bar.sync 1, 128;" ::: "memory");           // the offset table is complete
+            if (abort_flag) ok = false;
+            if (!ok) break;
             tc_fence_after();
-            const int per = nd.tw * nd.th;
-            const int bi = m / per, rem = m - bi * per, hi = rem / nd.tw, wi = rem - hi * nd.tw;
-            for (int half = 0; half < tl.n; ++half) {
-                const int b = (half ? tl.b0[1] : tl.b0[0]) + bi, h = (half ? tl.h0[1] : tl.h0[0]) + hi,
-                          w = (half ? tl.w0[1] : tl.w0[0]) + wi;
-                const bool valid = bi < nd.tb && b < B && h < nd.H && w < nd.W;
-                __nv_bfloat16* dst = static_cast<__nv_bfloat16*>(nd.state[cur]) + (((size_t)b * nd.H + h) * nd.W + w) * nd.C;
-                const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + acc * 256 + half * nd.C;
-                for (int c0 = 0; c0 < nd.C; c0 += 32) {
-                    uint32_t r[32];
-                    tc_ld32(taddr + c0, r);
+            __nv_bfloat16* out = static_cast<__nv_bfloat16*>(nd.state[cur]);
+            for (int h = 0; h < nd.n_mh; ++h) {
+                const int co_w = h * 128 + quarter * 32;                // first channel of this warp
+                const int co = co_w + lane;                             // TMEM lane = output channel
+                const float bias = co < nd.C ? __ldg(nd.bias + co) : 0.f;
+                const bool gvalid = co_w + (lane & 3) * 8 < nd.C;       // this thread's group of 8 channels exists
+                const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + acc * 256 + h * nd.n_cols;
+                for (int c0 = 0; c0 < nd.n_cols; c0 += 32) {
+                    uint32_t v[32];
+                    tc_ld32(taddr + c0, v);
                     tc_wait_ld();
-                    if (valid) {
-                        uint32_t o[16];
 #pragma unroll
-                        for (int j = 0; j < 16; ++j) {
-                            float v0 = __uint_as_float(r[2 * j]) + __ldg(nd.bias + c0 + 2 * j);
-                            float v1 = __uint_as_float(r[2 * j + 1]) + __ldg(nd.bias + c0 + 2 * j + 1);
-                            if (nd.act == 1) { v0 = fmaxf(v0, 0.f); v1 = fmaxf(v1, 0.f); }
-                            o[j] = pack_bf16(v0, v1);
-                        }
-                        uint4* d4 = reinterpret_cast<uint4*>(dst + c0);
-#pragma unroll
-                        for (int j = 0; j < 4; ++j) d4[j] = make_uint4(o[4 * j], o[4 * j + 1], o[4 * j + 2], o[4 * j + 3]);
+                    for (int j = 0; j < 32; ++j) {
+                        float z = __uint_as_float(v[j]) + bias;
+                        if (nd.act == 1) z = fmaxf(z, 0.f);
+                        const __nv_bfloat16 hz = __float2bfloat16_rn(z);
+                        tbuf[j * 32 + lane] = *reinterpret_cast<const uint16_t*>(&hz);
                     }
+                    __syncwarp();
+#pragma unroll
+                    for (int pass = 0; pass < 4; ++pass) {
+                        const int p = pass * 8 + (lane >> 2);
+                        const int o = pix_off[c0 + p];
+                        if (o >= 0 && gvalid) {
+                            const uint4 w = *reinterpret_cast<const uint4*>(tbuf + p * 32 + (lane & 3) * 8);
+                            *reinterpret_cast<uint4*>(out + (size_t)o + co_w + (lane & 3) * 8) = w;
+                        }
+                    }
+                    __syncwarp();
                 }
             }
             tc_fence_before();
-            __syncwarp();
-            if (lane == 0) mbar_arrive(bar_tempty + 8 * acc);
+            asm volatile("bar.sync 1, 128;" ::: "memory");           // everybody is done with the offset table
+            if (lane == 0) {
+                if (wide || acc == 0) mbar_arrive(bar_tempty);
+                if (wide || acc == 1) mbar_arrive(bar_tempty + 8);
+            }
+            if (wide || acc == 0) ++uses0;
+            if (wide || acc == 1) ++uses1;
         }
     }
     __syncwarp();
@@ -447,15 +505,15 @@ struct KbHost {
     int stem_index;
     int ky, kx, c0, bk;
     int k_off;
-    int a_rows;        // image rows of the A box this block loads (0: reuses the current A slot)
-    int a_shift;       // rows by which this block's window is shifted inside the A slot
-    bool a_release;
+    bool x_load;       // loads a fresh activation box (else: reuses the box of this filter column)
+    int x_shift;       // image rows by which this tap's window is shifted inside the box
+    bool x_release;
 };
 
 struct NodePlan {
     int node;
-    int tw, th, tb;
-    bool column_reuse;              // stride-1 k x k edges load one box per filter column
+    int tw, th, tb, sep, n_cols, n_mh;
+    int group;                      // weight boxes per group
     int k_total;                    // columns of the concatenated weight matrix
     std::vector<KbHost> kbs;
     SrRegion wcat;
@@ -473,8 +531,8 @@ struct TcEngine {
     std::vector<int> node_of;                    // graph node -> index in nodes, or -1
     std::vector<StemPlan> stems;
     std::vector<int> stem_of_edge;
-    std::vector<std::vector<TcPair>> group_tiles;
-    std::vector<int> group_tile_offset, group_a_slot, group_n_a, group_n_bu, group_grid;
+    std::vector<std::vector<TcTile>> group_tiles;
+    std::vector<int> group_tile_offset, group_a_slot, group_n_a, group_n_wu, group_w_slot, group_grid;
     SrRegion r_maps, r_nodes, r_kbs, r_tiles, r_stems;
     int n_maps = 0, n_kbs = 0, n_tiles = 0;
     int sm_count = 148;
@@ -489,6 +547,7 @@ bool is_stem(const sr_graph* g, const SrHostEdge& e)
     const SrHostNode& s = g->nodes[e.d.src];
     return s.is_input && (s.d.c % 16) != 0 && e.K <= 64;
 }
+bool reuses_columns(const sr_graph* g, const SrHostEdge& e) { return !is_stem(g, e) && e.stride_eff == 1 && e.k_eff >= 2; }
 
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
                                   const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
@@ -519,17 +578,41 @@ uint32_t desc_hi_of(int bk)
     return sbo | (1u << 14) | (layout << 29);
 }
 
+// Pick the pixel tile of a node: tw in {8, 16, 32} columns, th rows, tb samples, such that the stacked
+// rows N = tb * (th + sep) * tw - sep * tw fit 256 MMA columns.  The cost of a tile is the time of its
+// MMAs (about max(110, N/2) cycles each); the best shape computes the image with the least total cost.
+void choose_tile(int H, int W, int B, int sep, int forced_tw, NodePlan& P)
+{
+    double best = 1e30;
+    for (int tw = 8; tw <= 32; tw *= 2) {
+        if (forced_tw > 0 && tw != forced_tw && !(forced_tw > 8 && tw == 8 && forced_tw > (W + 7) / 8 * 8)) continue;
+        if (tw > 8 && tw > (W + 7) / 8 * 8) continue;
+        const int th = std::min(H, kMaxCols / tw);
+        int tb = 1;
+        if (th == H) tb = std::max(1, std::min(B, (kMaxCols + sep * tw) / ((th + sep) * tw)));
+        const int n = tb * (th + sep) * tw - sep * tw;
+        const int n_cols = (n + 31) / 32 * 32;
+        if (n_cols > kMaxCols) continue;
+        const double tiles = (double)((W + tw - 1) / tw) * ((H + th - 1) / th) * ((B + tb - 1) / tb);
+        const double cost = tiles * std::max(110.0, n_cols / 2.0) + tiles * 1e-3 * tw;      // tie: narrower tile, less halo
+        if (cost < best) {
+            best = cost;
+            P.tw = tw; P.th = th; P.tb = tb; P.n_cols = n_cols;
+        }
+    }
+}
+
 }  // namespace
 
-// A node goes to the tensor cores if it sums convolutions only, has 32..256 output channels in
-// multiples of 32, and every incoming edge either has C_in % 16 == 0 or is a few-channel input edge.
+// A node goes to the tensor cores if it sums convolutions only, has 16..256 output channels in
+// multiples of 8, and every incoming edge either has C_in % 16 == 0 or is a few-channel input edge.
 void sr_tc_select_nodes(sr_graph* g)
 {
     for (size_t v = 0; v < g->nodes.size(); ++v) {
         SrHostNode& n = g->nodes[v];
         n.use_tc = false;
         if (n.is_input || n.dense_target || (int)v == g->info.output_node) continue;
-        if (n.d.c % 32 != 0 || n.d.c < 32 || n.d.c > 256) continue;
+        if (n.d.c % 8 != 0 || n.d.c < 16 || n.d.c > 256) continue;
         bool ok = true;
         int n_blocks = 0;
         for (int e : n.in_edges) {
@@ -537,6 +620,7 @@ void sr_tc_select_nodes(sr_graph* g)
             const SrHostNode& s = g->nodes[he.d.src];
             if (he.d.kind != SR_EDGE_CONV) ok = false;
             else if (s.d.c % 16 != 0 && !is_stem(g, he)) ok = false;
+            else if (he.k_eff > 8) ok = false;
             else n_blocks += is_stem(g, he) ? 1 : he.k_eff * he.k_eff * (s.d.c / block_k(s.d.c));
         }
         if (ok && n_blocks >= 1 && n_blocks <= kMaxNodeKb) n.use_tc = true;
@@ -563,26 +647,14 @@ sr_status sr_tc_plan(sr_graph* g, size_t& off)
     for (size_t v = 0; v < g->nodes.size(); ++v) {
         const SrHostNode& n = g->nodes[v];
         if (!n.use_tc) continue;
-        NodePlan P;
+        NodePlan P{};
         P.node = (int)v;
-        // tile shape: 8 pixels x 16 rows of one sample when a stride-1 k x k edge can reuse its boxes,
-        // else as wide as the image and as many rows (and samples) as fit in 128 pixels
-        bool wants_reuse = false;
-        for (int e : n.in_edges) {
-            const SrHostEdge& he = g->edges[e];
-            if (!is_stem(g, he) && he.stride_eff == 1 && he.k_eff >= 2) wants_reuse = true;
-        }
-        int rtw = g->opt_tile_w > 0 ? g->opt_tile_w : 8;
-        while (rtw > 8 && (rtw > n.d.w || kTileM / rtw > n.d.h)) rtw /= 2;
-        if (wants_reuse && n.d.w >= rtw && n.d.h >= kTileM / rtw) {
-            P.tw = rtw; P.th = kTileM / rtw; P.tb = 1;
-            P.column_reuse = true;
-        } else {
-            P.tw = std::min(n.d.w, kTileM);
-            P.th = std::min(n.d.h, kTileM / P.tw);
-            P.tb = (P.th == n.d.h && P.tw == n.d.w) ? std::max(1, std::min(g->batch, kTileM / (P.tw * P.th))) : 1;
-            P.column_reuse = false;
-        }
+        P.sep = 0;
+        for (int e : n.in_edges)
+            if (reuses_columns(g, g->edges[e])) P.sep = std::max(P.sep, g->edges[e].k_eff - 1);
+        choose_tile(n.d.h, n.d.w, g->batch, P.sep, g->opt_tile_w, P);
+        P.n_mh = (n.d.c + 127) / 128;
+        P.group = P.n_mh >= 2 ? 1 : 3;
         int k_off = 0;
         for (int e : n.in_edges) {
             const SrHostEdge& he = g->edges[e];
@@ -597,23 +669,23 @@ sr_status sr_tc_plan(sr_graph* g, size_t& off)
                 S.buf[1] = take(bytes);
                 E->stem_of_edge[e] = (int)E->stems.size();
                 E->stems.push_back(S);
-                P.kbs.push_back(KbHost{e, true, (int)E->stems.size() - 1, 0, 0, 0, S.Kp, k_off, P.th, 0, true});
+                P.kbs.push_back(KbHost{e, true, (int)E->stems.size() - 1, 0, 0, 0, S.Kp, k_off, true, 0, true});
                 k_off += S.Kp;
             } else {
                 const int bk = block_k(s.d.c), k = he.k_eff;
                 const int edge_off = k_off;
-                if (P.column_reuse && he.stride_eff == 1 && k >= 2) {
+                if (reuses_columns(g, he)) {
                     for (int c0 = 0; c0 < s.d.c; c0 += bk)
                         for (int kx = 0; kx < k; ++kx)
                             for (int ky = 0; ky < k; ++ky)
                                 P.kbs.push_back(KbHost{e, false, -1, ky, kx, c0, bk, edge_off + (ky * k + kx) * s.d.c + c0,
-                                                       ky == 0 ? P.th + k - 1 : 0, ky, ky == k - 1});
+                                                       ky == 0, ky, ky == k - 1});
                 } else {
                     for (int ky = 0; ky < k; ++ky)
                         for (int kx = 0; kx < k; ++kx)
                             for (int c0 = 0; c0 < s.d.c; c0 += bk)
                                 P.kbs.push_back(KbHost{e, false, -1, ky, kx, c0, bk, edge_off + (ky * k + kx) * s.d.c + c0,
-                                                       P.th, 0, true});
+                                                       true, 0, true});
                 }
                 k_off += k * k * s.d.c;
             }
@@ -628,53 +700,31 @@ sr_status sr_tc_plan(sr_graph* g, size_t& off)
     int n_tiles = 0, n_kbs = 0;
     for (size_t gi = 0; gi < g->groups.size(); ++gi) {
         std::vector<std::pair<long long, TcTile>> tl;
-        int max_c = 0;
+        int a_slot = 1024, w_slot = 1;
         for (int v : g->groups[gi]) {
             if (E->node_of[v] < 0) continue;
             const NodePlan& P = E->nodes[E->node_of[v]];
             const SrHostNode& n = g->nodes[v];
-            max_c = std::max(max_c, n.d.c);
             for (int b0 = 0; b0 < g->batch; b0 += P.tb)
                 for (int h0 = 0; h0 < n.d.h; h0 += P.th)
                     for (int w0 = 0; w0 < n.d.w; w0 += P.tw)
-                        tl.push_back({(long long)P.k_total * n.d.c, TcTile{E->node_of[v], b0, h0, w0}});
+                        tl.push_back({(long long)P.kbs.size() * P.n_mh * P.n_cols, TcTile{E->node_of[v], b0, h0, w0}});
+            w_slot = std::max(w_slot, std::max(1, (n.d.c * 128 + kWUnit - 1) / kWUnit) * P.group);
+            // a window starts up to sep * tw rows into the box and the MMA reads n_cols rows from there
+            for (const KbHost& kb : P.kbs)
+                a_slot = std::max(a_slot, (int)sr_align_up((size_t)(P.sep * P.tw + P.n_cols) * kb.bk * 2, 1024));
         }
         std::stable_sort(tl.begin(), tl.end(), [](const auto& a, const auto& b) { return a.first > b.first; });
-        // pair neighbouring tiles of a node when both accumulators fit twice into TMEM (C_out <= 128)
-        for (size_t i = 0; i < tl.size();) {
-            const TcTile& a = tl[i].second;
-            TcPair pr{};
-            pr.node = a.node; pr.n = 1;
-            pr.b0[0] = a.b0; pr.h0[0] = a.h0; pr.w0[0] = a.w0;
-            const bool can_pair = g->nodes[E->nodes[a.node].node].d.c <= 128 && i + 1 < tl.size() && tl[i + 1].second.node == a.node;
-            if (can_pair) {
-                const TcTile& b = tl[i + 1].second;
-                pr.n = 2;
-                pr.b0[1] = b.b0; pr.h0[1] = b.h0; pr.w0[1] = b.w0;
-            }
-            E->group_tiles[gi].push_back(pr);
-            i += pr.n;
-        }
+        for (auto& p : tl) E->group_tiles[gi].push_back(p.second);
         E->group_tile_offset.push_back(n_tiles);
-        n_tiles += (int)E->group_tiles[gi].size();
-        int a_slot = kABytes;
-        for (int v : g->groups[gi]) {
-            if (E->node_of[v] < 0) continue;
-            const NodePlan& P = E->nodes[E->node_of[v]];
-            for (const KbHost& kb : P.kbs)
-                a_slot = std::max(a_slot, (int)sr_align_up((size_t)std::max(kTileM, kb.a_rows * P.tw * P.tb) * kb.bk * 2 +
-                                                           (size_t)kb.a_shift * 0, 1024));
-            if (P.column_reuse)      // the last window starts (k-1)*tw rows down and still reads 128 rows
-                for (const KbHost& kb : P.kbs)
-                    a_slot = std::max(a_slot, (int)sr_align_up((size_t)(kb.a_shift * P.tw + kTileM) * kb.bk * 2, 1024));
-        }
-        a_slot *= 2;                                  // room for the boxes of both tiles of a pair
-        int n_bu = g->opt_b_units > 0 ? g->opt_b_units : 24;
-        n_bu = std::max(8, std::min(kMaxBUnits, n_bu / 8 * 8));
-        const int n_a = std::max(2, std::min(kMaxA, (kSmemBudget - n_bu * kBUnit) / a_slot));
+        n_tiles += (int)tl.size();
+        int n_wu = g->opt_b_units > 0 ? g->opt_b_units : 24;
+        n_wu = std::max(2 * w_slot, std::min(kMaxWUnits, n_wu)) / w_slot * w_slot;
+        const int n_a = std::max(2, std::min(kMaxA, (kSmemBudget - n_wu * kWUnit) / a_slot));
         E->group_a_slot.push_back(a_slot);
         E->group_n_a.push_back(n_a);
-        E->group_n_bu.push_back(n_bu);
+        E->group_n_wu.push_back(n_wu);
+        E->group_w_slot.push_back(w_slot);
     }
     for (const NodePlan& P : E->nodes) n_kbs += (int)P.kbs.size();
     E->n_tiles = n_tiles;
@@ -683,7 +733,7 @@ sr_status sr_tc_plan(sr_graph* g, size_t& off)
     E->r_maps = take(sizeof(CUtensorMap) * (size_t)(2 * n_kbs + 3 * E->nodes.size() + 1));
     E->r_nodes = take(sizeof(TcNode) * E->nodes.size());
     E->r_kbs = take(sizeof(TcKBlock) * (size_t)std::max(1, n_kbs));
-    E->r_tiles = take(sizeof(TcPair) * (size_t)std::max(1, n_tiles));
+    E->r_tiles = take(sizeof(TcTile) * (size_t)std::max(1, n_tiles));
     E->r_stems = take(sizeof(TcStem) * std::max<size_t>(1, E->stems.size()));
     return SR_OK;
 }
@@ -702,16 +752,16 @@ sr_status sr_tc_bind(sr_graph* g)
     char* ws = g->ws;
     std::vector<CUtensorMap> maps;
     std::map<std::tuple<uintptr_t, int, int, int, int, int, int, int, int>, int> cache;
-    // 4-D activation view: dims (C, W', H', B), box (bk, tw, th, tb)
+    // 4-D activation view: dims (C, W', H', B), box (bk, tw, rows, tb)
     auto act_map = [&](char* base, int C, int Wv, int Hv, size_t stride_w, size_t stride_h, size_t stride_b, int bk,
-                       int tw, int th, int tb) -> int {
-        auto key = std::make_tuple((uintptr_t)base, C, Wv, Hv, (int)stride_w, bk, tw, th, tb);
+                       int tw, int rows, int tb) -> int {
+        auto key = std::make_tuple((uintptr_t)base, C, Wv, Hv, (int)stride_w, bk, tw, rows, tb);
         auto it = cache.find(key);
         if (it != cache.end()) return it->second;
         CUtensorMap m;
         cuuint64_t dims[4] = {(cuuint64_t)C, (cuuint64_t)Wv, (cuuint64_t)Hv, (cuuint64_t)g->batch};
         cuuint64_t strides[3] = {(cuuint64_t)stride_w, (cuuint64_t)stride_h, (cuuint64_t)stride_b};
-        cuuint32_t box[4] = {(cuuint32_t)bk, (cuuint32_t)tw, (cuuint32_t)th, (cuuint32_t)tb};
+        cuuint32_t box[4] = {(cuuint32_t)bk, (cuuint32_t)tw, (cuuint32_t)rows, (cuuint32_t)tb};
         cuuint32_t es[4] = {1, 1, 1, 1};
         if (encode(&m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, base, dims, strides, box, es, CU_TENSOR_MAP_INTERLEAVE_NONE,
                    swizzle_of(bk), CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
@@ -729,13 +779,15 @@ sr_status sr_tc_bind(sr_graph* g)
         d.state[1] = ws + n.state[1].offset;
         d.bias = reinterpret_cast<const float*>(ws + n.bias.offset);
         d.H = n.d.h; d.W = n.d.w; d.C = n.d.c; d.act = n.d.act;
-        d.tw = P.tw; d.th = P.th; d.tb = P.tb;
+        d.tw = P.tw; d.th = P.th; d.tb = P.tb; d.sep = P.sep;
+        d.n_cols = P.n_cols; d.n_mh = P.n_mh;
         d.first_kb = (int)dk.size();
         d.n_kb = (int)P.kbs.size();
-        // instruction descriptor: D = f32, A = B = bf16, both K-major, N = C_out, M = 128
-        d.idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(n.d.c >> 3) << 17) | ((uint32_t)(kTileM >> 4) << 24);
-        d.b_units = 1;
-        while (d.b_units * kBUnit < n.d.c * 128) d.b_units *= 2;
+        // instruction descriptor: D = f32, A = B = bf16, both K-major, M = 128 output channels, N = pixels
+        d.idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(P.n_cols >> 3) << 17) | ((uint32_t)(128 >> 4) << 24);
+        d.w_box_units = std::max(1, (n.d.c * 128 + kWUnit - 1) / kWUnit);
+        d.w_group_units = d.w_box_units * P.group;
+        const int rows = P.th + P.sep;
         std::map<int, int> wmap;                      // bk -> weight tensor map
         for (const KbHost& kb : P.kbs) {
             if (wmap.count(kb.bk)) continue;
@@ -751,26 +803,29 @@ sr_status sr_tc_bind(sr_graph* g)
             maps.push_back(m);
             wmap[kb.bk] = (int)maps.size() - 1;
         }
-        for (const KbHost& kb : P.kbs) {
+        for (size_t i = 0; i < P.kbs.size(); ++i) {
+            const KbHost& kb = P.kbs[i];
             const SrHostEdge& he = g->edges[kb.edge];
             const SrHostNode& s = g->nodes[he.d.src];
             TcKBlock k{};
             int map0 = -1, map1 = -1, qxv = 0, qyv = 0;
-            k.flags = (uint8_t)((he.R ? 1 : 0) | (kb.a_release ? 2 : 0));
-            k.b_map = (uint16_t)wmap[kb.bk];
+            const bool g_start = (int)(i % P.group) == 0, g_end = (int)(i % P.group) == P.group - 1 || i + 1 == P.kbs.size();
+            k.flags = (uint8_t)((he.R ? 1 : 0) | (kb.x_release ? 2 : 0) | (g_start ? 4 : 0) | (g_end ? 8 : 0));
+            k.w_box = (uint8_t)(i % P.group);
+            k.w_map = (uint16_t)wmap[kb.bk];
             k.k_off = (uint32_t)kb.k_off;
             k.n_k16 = (uint8_t)(kb.bk / 16);
             k.desc_hi = desc_hi_of(kb.bk);
-            k.a_bytes16 = (uint16_t)((kb.bk * 2 * P.tw * kb.a_rows * P.tb) >> 4);
-            k.b_bytes16 = (uint16_t)((kb.bk * 2 * n.d.c) >> 4);
-            k.a_off16 = (uint16_t)((kb.a_shift * P.tw * kb.bk * 2) >> 4);
+            k.x_bytes16 = kb.x_load ? (uint16_t)((kb.bk * 2 * P.tw * rows * P.tb) >> 4) : 0;
+            k.w_bytes16 = (uint16_t)((kb.bk * 2 * n.d.c) >> 4);
+            k.x_off16 = (uint16_t)((kb.x_shift * P.tw * kb.bk * 2) >> 4);
             if (kb.stem) {
                 const StemPlan& S = E->stems[kb.stem_index];
                 for (int par = 0; par < 2; ++par)
                     (par ? map1 : map0) = act_map(ws + S.buf[par].offset, S.Kp, n.d.w, n.d.h, (size_t)S.Kp * 2,
-                                           (size_t)n.d.w * S.Kp * 2, (size_t)n.d.h * n.d.w * S.Kp * 2, S.Kp, P.tw, P.th, P.tb);
+                                                  (size_t)n.d.w * S.Kp * 2, (size_t)n.d.h * n.d.w * S.Kp * 2, S.Kp, P.tw, rows, P.tb);
                 k.c0 = 0;
-            } else if (kb.a_rows == 0) {
+            } else if (!kb.x_load) {
                 map0 = map1 = 0;                         // reuses the box the first tap of this filter column loaded
                 k.c0 = (uint16_t)kb.c0;
             } else {
@@ -784,13 +839,13 @@ sr_status sr_tc_bind(sr_graph* g)
                 for (int par = 0; par < 2; ++par) {
                     char* base = ws + s.state[par].offset + ((size_t)ry * s.d.w + rx) * s.d.c * 2;
                     (par ? map1 : map0) = act_map(base, s.d.c, Wv, Hv, (size_t)st * s.d.c * 2, (size_t)st * s.d.w * s.d.c * 2,
-                                           (size_t)s.d.h * s.d.w * s.d.c * 2, kb.bk, P.tw, kb.a_rows, P.tb);
+                                                  (size_t)s.d.h * s.d.w * s.d.c * 2, kb.bk, P.tw, rows, P.tb);
                 }
                 qxv = qx; qyv = qy; k.c0 = (uint16_t)kb.c0;
             }
             if (map0 < 0 || map1 < 0) return SR_ERR_CUDA;
             if (map0 > 65535 || map1 > 65535 || qxv < -128 || qxv > 127 || qyv < -128 || qyv > 127) return SR_ERR_UNSUPPORTED;
-            k.a_map0 = (uint16_t)map0; k.a_map1 = (uint16_t)map1;
+            k.x_map0 = (uint16_t)map0; k.x_map1 = (uint16_t)map1;
             k.qx = (int8_t)qxv; k.qy = (int8_t)qyv;
             dk.push_back(k);
         }
@@ -798,7 +853,7 @@ sr_status sr_tc_bind(sr_graph* g)
     }
     if (maps.size() * sizeof(CUtensorMap) > E->r_maps.bytes) return SR_ERR_UNSUPPORTED;
     E->n_maps = (int)maps.size();
-    std::vector<TcPair> tiles;
+    std::vector<TcTile> tiles;
     for (auto& v : E->group_tiles) tiles.insert(tiles.end(), v.begin(), v.end());
     std::vector<TcStem> stems;
     for (const StemPlan& S : E->stems) {
@@ -818,7 +873,7 @@ sr_status sr_tc_bind(sr_graph* g)
         return bytes == 0 || cudaMemcpy(ws + r.offset, p, bytes, cudaMemcpyHostToDevice) == cudaSuccess;
     };
     if (!up(E->r_maps, maps.data(), maps.size() * sizeof(CUtensorMap)) || !up(E->r_nodes, dn.data(), dn.size() * sizeof(TcNode)) ||
-        !up(E->r_kbs, dk.data(), dk.size() * sizeof(TcKBlock)) || !up(E->r_tiles, tiles.data(), tiles.size() * sizeof(TcPair)) ||
+        !up(E->r_kbs, dk.data(), dk.size() * sizeof(TcKBlock)) || !up(E->r_tiles, tiles.data(), tiles.size() * sizeof(TcTile)) ||
         !up(E->r_stems, stems.data(), stems.size() * sizeof(TcStem)))
         return SR_ERR_CUDA;
     E->group_grid.clear();
@@ -877,14 +932,14 @@ int sr_tc_launch_group(sr_graph* g, int group, int t_off, cudaStream_t s)
 {
     TcEngine* E = eng(g);
     if (!E || E->group_tiles[group].empty()) return 0;
-    const int n_a = E->group_n_a[group], a_slot = E->group_a_slot[group];
-    const int n_bu = E->group_n_bu[group];
-    const size_t smem = (size_t)n_a * a_slot + (size_t)n_bu * kBUnit + 1024;
+    const int n_a = E->group_n_a[group], a_slot = E->group_a_slot[group], n_wu = E->group_n_wu[group];
+    const size_t smem = (size_t)n_a * a_slot + (size_t)n_wu * kWUnit + 1024;
     sr_tc_group_kernel<<<E->group_grid[group], kThreads, smem, s>>>(
         reinterpret_cast<const CUtensorMap*>(g->ws + E->r_maps.offset), reinterpret_cast<const TcNode*>(g->ws + E->r_nodes.offset),
         reinterpret_cast<const TcKBlock*>(g->ws + E->r_kbs.offset),
-        reinterpret_cast<const TcPair*>(g->ws + E->r_tiles.offset) + E->group_tile_offset[group],
-        (int)E->group_tiles[group].size(), reinterpret_cast<SrFrameCtl*>(g->ws + g->r_ctl.offset), t_off, g->batch, n_a, a_slot, n_bu);
+        reinterpret_cast<const TcTile*>(g->ws + E->r_tiles.offset) + E->group_tile_offset[group],
+        (int)E->group_tiles[group].size(), reinterpret_cast<SrFrameCtl*>(g->ws + g->r_ctl.offset), t_off, g->batch, n_a, a_slot,
+        n_wu, E->group_w_slot[group]);
     return 1;
 }
 
