@@ -254,11 +254,13 @@ sr_tc_group_kernel(const CUtensorMap* __restrict__ maps, const TcNode* __restric
         int cached_node = -1;
         // The weight ring is a ring of slots of w_slot_units 4 KiB units (the largest weight group of
         // the launch), handed back through one "empty" barrier per slot.  Box i of a group starts at
-        // unit i * w_box_units of its slot and signals arrival on that unit's "full" barrier; which
-        // units lead a box depends on the node, and a unit's barrier flips phase only when used, so
-        // both roles keep one phase bit per unit.
+        // unit i * w_box_units of its slot and signals arrival on that unit's "full" barrier (a full
+        // barrier per group would let the issuer wait for boxes whose activation slots it still
+        // holds).  Which units lead a box depends on the node, and a unit's barrier flips phase only
+        // when used, so both roles keep one phase bit per unit.
         const uint32_t n_ws = (uint32_t)(n_wu / w_slot_units);
-        uint32_t ia = 0, iw = 0, ws_cur = 0, wgrp = 0, wf_phase = 0, wf_used = 0, a_cur = 0;
+        uint32_t ia = 0, wf_phase = 0, wf_used = 0, ws_cur = 0, a_cur = 0;
+        uint32_t a_nxt = 0, a_ph = 0, w_nxt = 0, w_ph = 0;    // next slot of each ring and the phase of its barriers
         bool ok = true;
         for (int ti = blockIdx.x; ti < n_tiles; ti += gridDim.x) {
             const TcTile tl = tiles[ti];
@@ -279,8 +281,9 @@ sr_tc_group_kernel(const CUtensorMap* __restrict__ maps, const TcNode* __restric
                     for (int kb = 0; kb < n_kb; ++kb) {
                         const TcKBlock k = tab[kb];
                         if (k.x_bytes16) {
-                            const uint32_t s = ia % n_a, ph = (ia / n_a) & 1;
-                            if (!mbar_wait(bar_aempty + 8 * s, ph ^ 1, abortp)) { ok = false; break; }
+                            const uint32_t s = a_nxt;
+                            if (!mbar_wait(bar_aempty + 8 * s, a_ph ^ 1, abortp)) { ok = false; break; }
+                            if (++a_nxt == (uint32_t)n_a) { a_nxt = 0; a_ph ^= 1; }
                             mbar_expect_tx(bar_afull + 8 * s, (uint32_t)k.x_bytes16 << 4);
                             const int par = (k.flags & 1) ? prev : cur;
                             tma_load_4d(a_ring + s * a_slot, &maps[par ? k.x_map1 : k.x_map0], bar_afull + 8 * s, k.c0,
@@ -288,12 +291,11 @@ sr_tc_group_kernel(const CUtensorMap* __restrict__ maps, const TcNode* __restric
                             ++ia;
                         }
                         if (k.flags & 4) {
-                            ws_cur = iw % n_ws;
-                            if (!mbar_wait(bar_wempty + 8 * ws_cur, ((iw / n_ws) & 1) ^ 1, abortp)) { ok = false; break; }
-                            wgrp = ws_cur * (uint32_t)w_slot_units;
-                            ++iw;
+                            ws_cur = w_nxt;
+                            if (!mbar_wait(bar_wempty + 8 * ws_cur, w_ph ^ 1, abortp)) { ok = false; break; }
+                            if (++w_nxt == n_ws) { w_nxt = 0; w_ph ^= 1; }
                         }
-                        const uint32_t unit = wgrp + k.w_box * box_u;
+                        const uint32_t unit = ws_cur * (uint32_t)w_slot_units + k.w_box * box_u;
                         mbar_expect_tx(bar_wfull + 8 * unit, (uint32_t)k.w_bytes16 << 4);
                         tma_load_2d(w_ring + unit * kWUnit, &maps[k.w_map], bar_wfull + 8 * unit, (int)k.k_off, 0);
                         wf_phase ^= 1u << unit;
@@ -314,19 +316,17 @@ sr_tc_group_kernel(const CUtensorMap* __restrict__ maps, const TcNode* __restric
                     for (int kb = 0; kb < n_kb && ok; ++kb) {
                         const TcKBlock k = tab[kb];
                         if (k.x_bytes16) {
-                            a_cur = ia % n_a;
-                            if (!mbar_wait(bar_afull + 8 * a_cur, (ia / n_a) & 1, abortp)) { ok = false; break; }
-                            ++ia;
+                            a_cur = a_nxt;
+                            if (!mbar_wait(bar_afull + 8 * a_cur, a_ph, abortp)) { ok = false; break; }
+                            if (++a_nxt == (uint32_t)n_a) { a_nxt = 0; a_ph ^= 1; }
                         }
                         if (k.flags & 4) {
-                            ws_cur = iw % n_ws;
-                            wgrp = ws_cur * (uint32_t)w_slot_units;
-                            ++iw;
+                            ws_cur = w_nxt;
+                            if (++w_nxt == n_ws) w_nxt = 0;
                         }
-                        const uint32_t unit = wgrp + k.w_box * box_u;
+                        const uint32_t unit = ws_cur * (uint32_t)w_slot_units + k.w_box * box_u;
                         if (!mbar_wait(bar_wfull + 8 * unit, (wf_phase >> unit) & 1, abortp)) { ok = false; break; }
                         wf_phase ^= 1u << unit;
-                        tc_fence_after();
                         const uint64_t hi = ((uint64_t)k.desc_hi << 32) | (1ull << 16);
                         const uint64_t x_desc = hi | (uint64_t)((((a_ring + a_cur * a_slot) >> 4) + k.x_off16) & 0x3FFFu);
                         uint64_t w_desc = hi | (uint64_t)(((w_ring + unit * kWUnit) >> 4) & 0x3FFFu);
