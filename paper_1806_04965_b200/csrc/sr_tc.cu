@@ -119,6 +119,17 @@ __device__ __forceinline__ uint32_t mbar_try_wait(uint32_t bar, uint32_t parity)
         : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
     return ok;
 }
+// Non-blocking probe (try_wait may suspend the thread for a while; this never does).
+__device__ __forceinline__ uint32_t mbar_test_wait(uint32_t bar, uint32_t parity)
+{
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.b32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+    return ok;
+}
 // Bounded wait.  Returns false if the limit expired or another role already gave up.
 __device__ __noinline__ bool mbar_wait_slow(uint32_t bar, uint32_t parity, volatile int* abort_flag)
 {
@@ -313,34 +324,47 @@ sr_tc_group_kernel(const CUtensorMap* __restrict__ maps, const TcNode* __restric
                     }
                     tc_fence_after();
                     const uint32_t d_tmem = tmem_base + acc * 256;
+                    // Software pipeline: the table entry of the next K-block is read and its two barriers are
+                    // probed BEFORE this block's MMAs are issued, so that the probes' latency hides behind the
+                    // (blocking) MMA issue; only a failed probe turns into a real wait.
+                    TcKBlock k = tab[0];
+                    uint32_t ws_n = (k.flags & 4) ? w_nxt : ws_cur;
+                    uint32_t unit = ws_n * (uint32_t)w_slot_units + k.w_box * box_u;
+                    uint32_t got_x = k.x_bytes16 ? mbar_test_wait(bar_afull + 8 * a_nxt, a_ph) : 1u;
+                    uint32_t got_w = mbar_test_wait(bar_wfull + 8 * unit, (wf_phase >> unit) & 1);
                     for (int kb = 0; kb < n_kb && ok; ++kb) {
-                        const TcKBlock k = tab[kb];
                         if (k.x_bytes16) {
                             a_cur = a_nxt;
-                            if (!mbar_wait(bar_afull + 8 * a_cur, a_ph, abortp)) { ok = false; break; }
+                            if (!got_x && !mbar_wait(bar_afull + 8 * a_cur, a_ph, abortp)) { ok = false; break; }
                             if (++a_nxt == (uint32_t)n_a) { a_nxt = 0; a_ph ^= 1; }
                         }
                         if (k.flags & 4) {
                             ws_cur = w_nxt;
                             if (++w_nxt == n_ws) w_nxt = 0;
                         }
-                        const uint32_t unit = ws_cur * (uint32_t)w_slot_units + k.w_box * box_u;
-                        if (!mbar_wait(bar_wfull + 8 * unit, (wf_phase >> unit) & 1, abortp)) { ok = false; break; }
+                        if (!got_w && !mbar_wait(bar_wfull + 8 * unit, (wf_phase >> unit) & 1, abortp)) { ok = false; break; }
                         wf_phase ^= 1u << unit;
                         const uint64_t hi = ((uint64_t)k.desc_hi << 32) | (1ull << 16);
                         const uint64_t x_desc = hi | (uint64_t)((((a_ring + a_cur * a_slot) >> 4) + k.x_off16) & 0x3FFFu);
                         uint64_t w_desc = hi | (uint64_t)(((w_ring + unit * kWUnit) >> 4) & 0x3FFFu);
-                        const uint32_t first = kb != 0;
+                        const uint32_t first = kb != 0, n_k16 = k.n_k16, flags = k.flags, ws_done = ws_cur;
+                        if (kb + 1 < n_kb) {
+                            k = tab[kb + 1];
+                            ws_n = (k.flags & 4) ? w_nxt : ws_cur;
+                            unit = ws_n * (uint32_t)w_slot_units + k.w_box * box_u;
+                            got_x = k.x_bytes16 ? mbar_test_wait(bar_afull + 8 * a_nxt, a_ph) : 1u;
+                            got_w = mbar_test_wait(bar_wfull + 8 * unit, (wf_phase >> unit) & 1);
+                        }
                         // a K = 16 step moves both operands 32 bytes along K (+2 in the address field);
                         // the second half of the output channels starts 128 weight rows further
                         for (uint32_t h = 0; h < n_mh; ++h) {
                             tc_mma_bf16(d_tmem + h * n_cols, w_desc, x_desc, idesc, first);
-                            for (uint32_t j = 1; j < k.n_k16; ++j)
+                            for (uint32_t j = 1; j < n_k16; ++j)
                                 tc_mma_bf16(d_tmem + h * n_cols, w_desc + 2 * j, x_desc + 2 * j, idesc, 1);
-                            w_desc += 256u * k.n_k16;
+                            w_desc += 256u * n_k16;
                         }
-                        if (k.flags & 8) tc_commit(bar_wempty + 8 * ws_cur); // hands the weight slot back
-                        if (k.flags & 2) tc_commit(bar_aempty + 8 * a_cur);  // last reader of the activation slot
+                        if (flags & 8) tc_commit(bar_wempty + 8 * ws_done);  // hands the weight slot back
+                        if (flags & 2) tc_commit(bar_aempty + 8 * a_cur);    // last reader of the activation slot
                     }
                     if (ok) {
                         if (wide || acc == 0) tc_commit(bar_tfull);
