@@ -156,6 +156,9 @@ sr_status sr_graph_set_node_bias(sr_graph* g, int node, const float* bias_host);
  *           key 3 "tile width": width in pixels (8, 16 or 32; 0 = default) of the 128-pixel output tiles of
  *                  nodes that have a stride-1 k x k incoming edge (narrow tiles reload less halo, wide
  *                  tiles read longer contiguous runs).
+ *           key 4 "overlap": 1 (default) runs independent launches of a frame on a second, library-owned
+ *                  stream (the CUDA-core and the tensor-core kernel of a group; the next frame's input
+ *                  copy when no input edge has R = 0), joined before the frame ends; 0 = one stream.
  * Must be set before sr_graph_bind_workspace (engine, weight ring, tile width) / before the first run (graphs). */
 sr_status sr_graph_set_option(sr_graph* g, int key, int value);
 

@@ -21,6 +21,29 @@ struct GraphCache {
     bool with_out = false;
 };
 
+// A second stream lets independent launches of one frame overlap: the CUDA-core kernel and the
+// tensor-core kernel of a launch group, and - when no input edge stays inside the frame - the copy
+// and staging of the next input frame, which nothing of the current update reads.
+struct SideStream {
+    cudaStream_t stream = nullptr;
+    cudaEvent_t fork = nullptr, join = nullptr;
+};
+
+SideStream* side_of(sr_graph* g)
+{
+    if (!g->side) {
+        SideStream* s = new SideStream();
+        if (cudaStreamCreateWithFlags(&s->stream, cudaStreamNonBlocking) != cudaSuccess ||
+            cudaEventCreateWithFlags(&s->fork, cudaEventDisableTiming) != cudaSuccess ||
+            cudaEventCreateWithFlags(&s->join, cudaEventDisableTiming) != cudaSuccess) {
+            delete s;
+            return nullptr;
+        }
+        g->side = s;
+    }
+    return static_cast<SideStream*>(g->side);
+}
+
 float round_bf16_host(float f)
 {
     uint32_t u;
@@ -146,17 +169,47 @@ const int* input_list_dev(const sr_graph* g)
 int enqueue_frames(sr_graph* g, int first_off, int frames, cudaStream_t s)
 {
     int launches = 0;
+    SideStream* side = g->opt_overlap ? side_of(g) : nullptr;
     for (int f = first_off; f < first_off + frames; ++f) {
-        sr_launch_input(g, input_list_dev(g), f, s);
+        bool forked = false;
+        auto fork = [&]() {
+            if (!forked) {
+                cudaEventRecord(side->fork, s);
+                cudaStreamWaitEvent(side->stream, side->fork, 0);
+                forked = true;
+            }
+        };
+        auto join = [&]() {
+            if (forked) {
+                cudaEventRecord(side->join, side->stream);
+                cudaStreamWaitEvent(s, side->join, 0);
+                forked = false;
+            }
+        };
+        // frame input: on the side stream if this frame's update does not read it
+        cudaStream_t in_stream = s;
+        if (side && !g->input_feeds_same_frame) {
+            fork();
+            in_stream = side->stream;
+        }
+        sr_launch_input(g, input_list_dev(g), f, in_stream);
         ++launches;
-        launches += sr_tc_stage_inputs(g, f, s);
+        launches += sr_tc_stage_inputs(g, f, in_stream);
         for (int gi = 0; gi < (int)g->groups.size(); ++gi) {
-            if (g->group_item_count[gi] > 0) {
-                sr_launch_direct_group(g, gi, f, s);
+            const bool has_direct = g->group_item_count[gi] > 0, has_tc = sr_tc_group_has_work(g, gi);
+            if (has_direct) {
+                cudaStream_t ds = s;
+                if (side && has_tc) {
+                    fork();
+                    ds = side->stream;
+                }
+                sr_launch_direct_group(g, gi, f, ds);
                 ++launches;
             }
             launches += sr_tc_launch_group(g, gi, f, s);
+            if (gi + 1 < (int)g->groups.size()) join();       // the next group reads what this one wrote
         }
+        join();
     }
     return launches;
 }
@@ -190,6 +243,9 @@ sr_status sr_graph_create(const sr_node_desc* nodes, int n_nodes, const sr_edge_
         delete g;
         return st;
     }
+    g->input_feeds_same_frame = false;
+    for (const SrHostEdge& e : g->edges)
+        if (g->nodes[e.d.src].is_input && e.R == 0) g->input_feeds_same_frame = true;
     g->batch = batch;
     g->dtype = dtype;
     g->elem = dtype == SR_DTYPE_BF16 ? 2 : 4;
@@ -205,6 +261,13 @@ void sr_graph_destroy(sr_graph* g)
         if (c->exec) cudaGraphExecDestroy(c->exec);
         if (c->capture_stream) cudaStreamDestroy(c->capture_stream);
         delete c;
+    }
+    if (g->side) {
+        SideStream* sd = static_cast<SideStream*>(g->side);
+        cudaEventDestroy(sd->fork);
+        cudaEventDestroy(sd->join);
+        cudaStreamDestroy(sd->stream);
+        delete sd;
     }
     sr_tc_destroy(g);
     delete g;
@@ -236,6 +299,11 @@ sr_status sr_graph_set_option(sr_graph* g, int key, int value)
     if (key == 1) {
         if (value < 0 || value > 1024) return SR_ERR_INVALID_ARG;
         g->opt_graph_frames = value;
+        return SR_OK;
+    }
+    if (key == 4) {
+        if (value != 0 && value != 1) return SR_ERR_INVALID_ARG;
+        g->opt_overlap = value;
         return SR_OK;
     }
     if (key == 3) {

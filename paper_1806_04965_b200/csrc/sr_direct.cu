@@ -169,31 +169,36 @@ __device__ void dense_item(const SrDevNode& nd, const SrDevEdge* edges, const Sr
 constexpr int kHeadCo = 16;        // outputs per block (dense nodes, one sample per block)
 constexpr int kHeadMaxC = 1024;    // channels the mean buffer holds
 
-// Dense node, one sample and kHeadCo outputs per block.  A mean-dense edge first reduces the
-// source over its pixels into shared memory (threads run over channels: coalesced NHWC reads),
-// then every warp forms dot products with lanes striding over the reduction index and a
-// shuffle reduction at the end.  Source and weight rows are read with 16-byte loads.
+// Dense node, one sample and kHeadCo outputs per block.  Every thread keeps a partial sum for each of
+// the block's outputs over its own slice of the reduction index, so the weight loads of all outputs
+// are independent and in flight together (the kernel is bound by load latency, not by arithmetic);
+// a shuffle reduction and one pass through shared memory combine the slices.  A mean-dense edge first
+// reduces the source over its pixels into shared memory (threads run over channels: coalesced NHWC
+// reads).  Source and weight rows are read with 16-byte loads where the length allows it.
 template <typename T>
 __device__ void head_item(const SrDevNode& nd, const SrDevEdge* edges, const SrDirectItem& it, int prev, int cur,
                           float* out_f32)
 {
     __shared__ float mean[kHeadMaxC];
-    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int b = it.b0;
-    float acc[kHeadCo / kWarps];
+    __shared__ float red[kWarps][kHeadCo];
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, tid = threadIdx.x;
+    const int b = it.b0, co0 = it.p0;
+    const int nco = min(kHeadCo, nd.C - co0);
+    float acc[kHeadCo];
 #pragma unroll
-    for (int j = 0; j < kHeadCo / kWarps; ++j) acc[j] = 0.f;
+    for (int o = 0; o < kHeadCo; ++o) acc[o] = 0.f;
     for (int ei = 0; ei < nd.n_edges; ++ei) {
         const SrDevEdge& e = edges[nd.first_edge + ei];
         const int HW = e.Hs * e.Ws, Kx = HW * e.Cs;
         const T* src = static_cast<const T*>(e.src[e.R ? prev : cur]) + (size_t)b * Kx;
+        const float* w0 = e.w + (size_t)co0 * e.K;
         if (e.kind == SR_EDGE_MEAN_DENSE) {
             __syncthreads();
-            for (int c = threadIdx.x; c < e.Cs; c += blockDim.x) mean[c] = 0.f;
+            for (int c = tid; c < e.Cs; c += blockDim.x) mean[c] = 0.f;
             __syncthreads();
             if ((e.Cs & 3) == 0 && e.Cs / 4 <= (int)blockDim.x) {
                 const int vc = e.Cs / 4, groups = blockDim.x / vc;
-                const int col = threadIdx.x % vc, grp = threadIdx.x / vc;
+                const int col = tid % vc, grp = tid / vc;
                 if (grp < groups) {
                     float s4[4] = {0.f, 0.f, 0.f, 0.f};
                     for (int p = grp; p < HW; p += groups) {
@@ -206,53 +211,53 @@ __device__ void head_item(const SrDevNode& nd, const SrDevEdge* edges, const SrD
                     for (int q = 0; q < 4; ++q) atomicAdd(&mean[4 * col + q], s4[q]);
                 }
             } else {
-                for (int i = threadIdx.x; i < Kx; i += blockDim.x) atomicAdd(&mean[i % e.Cs], to_f(src[i]));
+                for (int i = tid; i < Kx; i += blockDim.x) atomicAdd(&mean[i % e.Cs], to_f(src[i]));
             }
             __syncthreads();
             const float inv = 1.f / (float)HW;
+            for (int c = tid; c < e.Cs; c += blockDim.x) {
+                const float m = mean[c] * inv;
 #pragma unroll
-            for (int j = 0; j < kHeadCo / kWarps; ++j) {
-                const int co = it.p0 + warp * (kHeadCo / kWarps) + j;
-                if (co >= nd.C) continue;
-                const float* wrow = e.w + (size_t)co * e.K;
-                float part = 0.f;
-                for (int c = lane; c < e.Cs; c += 32) part = fmaf(wrow[c], mean[c], part);
-                acc[j] += part * inv;
+                for (int o = 0; o < kHeadCo; ++o)
+                    if (o < nco) acc[o] = fmaf(w0[(size_t)o * e.K + c], m, acc[o]);
+            }
+        } else if ((Kx & 3) == 0) {
+            for (int k = 4 * tid; k < Kx; k += 4 * (int)blockDim.x) {
+                float x[4];
+                load4(src + k, x);
+#pragma unroll
+                for (int o = 0; o < kHeadCo; ++o) {
+                    if (o < nco) {
+                        const float4 w = *reinterpret_cast<const float4*>(w0 + (size_t)o * e.K + k);
+                        acc[o] = fmaf(w.x, x[0], acc[o]); acc[o] = fmaf(w.y, x[1], acc[o]);
+                        acc[o] = fmaf(w.z, x[2], acc[o]); acc[o] = fmaf(w.w, x[3], acc[o]);
+                    }
+                }
             }
         } else {
+            for (int k = tid; k < Kx; k += blockDim.x) {
+                const float x = to_f(src[k]);
 #pragma unroll
-            for (int j = 0; j < kHeadCo / kWarps; ++j) {
-                const int co = it.p0 + warp * (kHeadCo / kWarps) + j;
-                if (co >= nd.C) continue;
-                const float* wrow = e.w + (size_t)co * e.K;
-                float part = 0.f;
-                if ((Kx & 3) == 0) {
-                    for (int k = 4 * lane; k < Kx; k += 128) {
-                        float x[4];
-                        load4(src + k, x);
-                        const float4 w = *reinterpret_cast<const float4*>(wrow + k);
-                        part = fmaf(w.x, x[0], part); part = fmaf(w.y, x[1], part);
-                        part = fmaf(w.z, x[2], part); part = fmaf(w.w, x[3], part);
-                    }
-                } else {
-                    for (int k = lane; k < Kx; k += 32) part = fmaf(wrow[k], to_f(src[k]), part);
-                }
-                acc[j] += part;
+                for (int o = 0; o < kHeadCo; ++o)
+                    if (o < nco) acc[o] = fmaf(w0[(size_t)o * e.K + k], x, acc[o]);
             }
         }
     }
 #pragma unroll
-    for (int j = 0; j < kHeadCo / kWarps; ++j) {
-        float v = acc[j];
+    for (int o = 0; o < kHeadCo; ++o) {
+        float v = acc[o];
 #pragma unroll
-        for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
-        const int co = it.p0 + warp * (kHeadCo / kWarps) + j;
-        if (lane == 0 && co < nd.C) {
-            float z = v + nd.bias[co];
-            if (nd.act == 1) z = fmaxf(z, 0.f);
-            from_f(static_cast<T*>(nd.state[cur]) + (size_t)b * nd.C + co, z);
-            if (out_f32) out_f32[(size_t)b * nd.C + co] = z;
-        }
+        for (int d = 16; d > 0; d >>= 1) v += __shfl_xor_sync(0xffffffffu, v, d);
+        if (lane == 0) red[warp][o] = v;
+    }
+    __syncthreads();
+    if (tid < nco) {
+        float z = nd.bias[co0 + tid];
+#pragma unroll
+        for (int w = 0; w < kWarps; ++w) z += red[w][tid];
+        if (nd.act == 1) z = fmaxf(z, 0.f);
+        from_f(static_cast<T*>(nd.state[cur]) + (size_t)b * nd.C + co0 + tid, z);
+        if (out_f32) out_f32[(size_t)b * nd.C + co0 + tid] = z;
     }
 }
 

@@ -84,7 +84,7 @@ struct sr_graph {
     std::vector<int> input_nodes;
     std::vector<std::vector<int>> groups;          // groups[l-1] = nodes of level l
     // options
-    int opt_engine = 0, opt_graph_frames = 0, opt_b_units = 0, opt_tile_w = 0;
+    int opt_engine = 0, opt_graph_frames = 0, opt_b_units = 0, opt_tile_w = 0, opt_overlap = 1;
     // workspace
     size_t ws_bytes = 0;
     char* ws = nullptr;
@@ -98,6 +98,8 @@ struct sr_graph {
     int64_t launches = 0;
     void* tc = nullptr;                            // tensor-core engine state (opaque here)
     void* graphs = nullptr;                        // CUDA-graph cache (opaque here)
+    void* side = nullptr;                          // side stream and fork / join events (opaque here)
+    bool input_feeds_same_frame = false;           // some edge that leaves an input node has R = 0
 };
 
 // sr_compile.cpp

@@ -967,6 +967,12 @@ int sr_tc_launch_group(sr_graph* g, int group, int t_off, cudaStream_t s)
     return 1;
 }
 
+bool sr_tc_group_has_work(const sr_graph* g, int group)
+{
+    TcEngine* E = eng(g);
+    return E && !E->group_tiles[group].empty();
+}
+
 void sr_tc_destroy(sr_graph* g)
 {
     if (g && g->tc) {
