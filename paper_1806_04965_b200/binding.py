@@ -75,6 +75,8 @@ def load_library(path: Optional[str] = None):
     lib.sr_graph_frame.argtypes = [vp, ctypes.POINTER(ctypes.c_int64)]
     lib.sr_graph_launch_count.argtypes = [vp, ctypes.POINTER(ctypes.c_int64)]
     lib.sr_graph_sync_status.argtypes = [vp, vp]
+    lib.sr_graph_kernel_time.argtypes = [vp, ctypes.POINTER(ctypes.c_double), ctypes.POINTER(ctypes.c_int64)]
+    lib.sr_graph_kernel_time.restype = ctypes.c_int
     lib.sr_status_str.argtypes = [ip]
     lib.sr_status_str.restype = ctypes.c_char_p
     for name in ("sr_graph_create", "sr_graph_info", "sr_graph_levels", "sr_graph_workspace_bytes",
@@ -221,6 +223,15 @@ class Graph:
         v = ctypes.c_int64()
         _check(self._lib.sr_graph_launch_count(self._h, ctypes.byref(v)), "sr_graph_launch_count")
         return v.value
+
+    def set_option(self, key: int, value: int):
+        _check(self._lib.sr_graph_set_option(self._h, key, value), "sr_graph_set_option")
+
+    def kernel_time(self):
+        """(milliseconds, launches) of the event-timed tensor-core group launches since the last call."""
+        ms, n = ctypes.c_double(), ctypes.c_int64()
+        _check(self._lib.sr_graph_kernel_time(self._h, ctypes.byref(ms), ctypes.byref(n)), "sr_graph_kernel_time")
+        return ms.value, n.value
 
     def sync_status(self):
         _check(self._lib.sr_graph_sync_status(self._h, self._stream()), "sr_graph_sync_status")

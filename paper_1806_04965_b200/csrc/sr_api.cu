@@ -301,6 +301,11 @@ sr_status sr_graph_set_option(sr_graph* g, int key, int value)
         g->opt_graph_frames = value;
         return SR_OK;
     }
+    if (key == 5) {
+        if (value != 0 && value != 1) return SR_ERR_INVALID_ARG;
+        g->opt_time_tc = value;
+        return SR_OK;
+    }
     if (key == 4) {
         if (value != 0 && value != 1) return SR_ERR_INVALID_ARG;
         g->opt_overlap = value;
@@ -610,6 +615,16 @@ sr_status sr_graph_launch_count(const sr_graph* g, int64_t* n)
     if (!g || !n) return SR_ERR_INVALID_ARG;
     *n = g->launches;
     return SR_OK;
+}
+
+sr_status sr_graph_kernel_time(sr_graph* g, double* ms, int64_t* launches)
+{
+    if (!g || !ms || !launches) return SR_ERR_INVALID_ARG;
+    if (g->batch <= 0 || !g->ws) return SR_ERR_STATE;
+    long long n = 0;
+    const sr_status st = sr_tc_timing(g, ms, &n);
+    *launches = n;
+    return st;
 }
 
 sr_status sr_graph_sync_status(sr_graph* g, void* stream)

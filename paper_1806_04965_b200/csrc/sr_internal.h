@@ -84,7 +84,7 @@ struct sr_graph {
     std::vector<int> input_nodes;
     std::vector<std::vector<int>> groups;          // groups[l-1] = nodes of level l
     // options
-    int opt_engine = 0, opt_graph_frames = 0, opt_b_units = 0, opt_tile_w = 0, opt_overlap = 1;
+    int opt_engine = 0, opt_graph_frames = 0, opt_b_units = 0, opt_tile_w = 0, opt_overlap = 1, opt_time_tc = 0;
     // workspace
     size_t ws_bytes = 0;
     char* ws = nullptr;

@@ -193,11 +193,6 @@ __device__ __forceinline__ void tc_ld32(uint32_t taddr, uint32_t (&r)[32])
 }
 __device__ __forceinline__ void tc_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
 
-__device__ __forceinline__ uint32_t pack_bf16(float lo, float hi)
-{
-    const __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
-    return *reinterpret_cast<const uint32_t*>(&v);
-}
 
 // ------------------------------------------------------------------------------------------ the kernel
 __global__ void __launch_bounds__(kThreads, 1)
@@ -560,6 +555,11 @@ struct TcEngine {
     SrRegion r_maps, r_nodes, r_kbs, r_tiles, r_stems;
     int n_maps = 0, n_kbs = 0, n_tiles = 0;
     int sm_count = 148;
+    // optional timing of the group launches with CUDA events on the launching stream
+    std::vector<cudaEvent_t> ev;             // pairs: start, stop
+    size_t ev_used = 0;
+    double timed_ms = 0.0;
+    long long timed_launches = 0;
 };
 
 TcEngine* eng(const sr_graph* g) { return static_cast<TcEngine*>(g->tc); }
@@ -958,13 +958,50 @@ int sr_tc_launch_group(sr_graph* g, int group, int t_off, cudaStream_t s)
     if (!E || E->group_tiles[group].empty()) return 0;
     const int n_a = E->group_n_a[group], a_slot = E->group_a_slot[group], n_wu = E->group_n_wu[group];
     const size_t smem = (size_t)n_a * a_slot + (size_t)n_wu * kWUnit + 1024;
+    cudaStreamCaptureStatus cap = cudaStreamCaptureStatusNone;
+    bool timed = g->opt_time_tc != 0 && cudaStreamIsCapturing(s, &cap) == cudaSuccess && cap == cudaStreamCaptureStatusNone;
+    if (timed) {
+        if (E->ev_used + 2 > E->ev.size()) {
+            if (E->ev.size() >= 4096) timed = false;
+            else
+                for (int i = 0; i < 2; ++i) {
+                    cudaEvent_t e = nullptr;
+                    if (cudaEventCreate(&e) != cudaSuccess) { timed = false; break; }
+                    E->ev.push_back(e);
+                }
+        }
+        if (timed && E->ev_used + 2 <= E->ev.size()) cudaEventRecord(E->ev[E->ev_used], s);
+        else timed = false;
+    }
     sr_tc_group_kernel<<<E->group_grid[group], kThreads, smem, s>>>(
         reinterpret_cast<const CUtensorMap*>(g->ws + E->r_maps.offset), reinterpret_cast<const TcNode*>(g->ws + E->r_nodes.offset),
         reinterpret_cast<const TcKBlock*>(g->ws + E->r_kbs.offset),
         reinterpret_cast<const TcTile*>(g->ws + E->r_tiles.offset) + E->group_tile_offset[group],
         (int)E->group_tiles[group].size(), reinterpret_cast<SrFrameCtl*>(g->ws + g->r_ctl.offset), t_off, g->batch, n_a, a_slot,
         n_wu, E->group_w_slot[group]);
+    if (timed) {
+        cudaEventRecord(E->ev[E->ev_used + 1], s);
+        E->ev_used += 2;
+    }
     return 1;
+}
+
+// Sum of the event-timed durations of the tensor-core group launches since the last call (synchronises).
+sr_status sr_tc_timing(sr_graph* g, double* ms, long long* launches)
+{
+    TcEngine* E = eng(g);
+    *ms = 0.0;
+    *launches = 0;
+    if (!E) return SR_OK;
+    for (size_t i = 0; i + 1 < E->ev_used; i += 2) {
+        if (cudaEventSynchronize(E->ev[i + 1]) != cudaSuccess) return SR_ERR_CUDA;
+        float t = 0.f;
+        if (cudaEventElapsedTime(&t, E->ev[i], E->ev[i + 1]) != cudaSuccess) return SR_ERR_CUDA;
+        *ms += t;
+        *launches += 1;
+    }
+    E->ev_used = 0;
+    return SR_OK;
 }
 
 bool sr_tc_group_has_work(const sr_graph* g, int group)
@@ -976,6 +1013,7 @@ bool sr_tc_group_has_work(const sr_graph* g, int group)
 void sr_tc_destroy(sr_graph* g)
 {
     if (g && g->tc) {
+        for (cudaEvent_t e : eng(g)->ev) cudaEventDestroy(e);
         delete eng(g);
         g->tc = nullptr;
     }

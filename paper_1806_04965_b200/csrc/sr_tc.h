@@ -11,5 +11,6 @@ sr_status sr_tc_set_weights(sr_graph* g, int edge, const float* w_eff /* [C_out]
 int sr_tc_stage_inputs(sr_graph* g, int t_off, cudaStream_t s);          // returns launches queued
 int sr_tc_launch_group(sr_graph* g, int group, int t_off, cudaStream_t s);
 bool sr_tc_group_has_work(const sr_graph* g, int group);
+sr_status sr_tc_timing(sr_graph* g, double* ms, long long* launches);
 int sr_tc_after_state_change(sr_graph* g, cudaStream_t s);    // re-stage frame-t inputs after reset / set_state
 void sr_tc_destroy(sr_graph* g);
