@@ -67,6 +67,27 @@ def peaks():
     return {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0, "source": "fallback"}
 
 
+def max_over_ranks(values, dist=None, device="cpu"):
+    """Element-wise maximum of a list of floats over all ranks (the timing rule for N > 1: a job is as slow
+    as its slowest replica).  Without a process group the values come back unchanged."""
+    import torch
+    t = torch.tensor(list(values), dtype=torch.float64, device=device)
+    if dist is not None:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return [float(v) for v in t]
+
+
+def whole_job_frames_per_s(world: int, frames_per_step: int, ms_per_step: float) -> float:
+    """Replicas only: every rank rolls out its own batch of sequences, so the job's frame rate is the sum."""
+    return world * frames_per_step / ms_per_step * 1e3
+
+
+def replica_spec(args, rank: int):
+    spec = build_spec(args)
+    spec.seed += rank                                            # every rank rolls out its own sequences
+    return spec
+
+
 class ClockSampler:
     FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,clocks_event_reasons.hw_slowdown,"
               "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
@@ -211,8 +232,7 @@ def run_cuda(args):
     if world > 1:
         import torch.distributed as dist
         dist.init_process_group("nccl", device_id=torch.device("cuda", local))
-    spec = build_spec(args)
-    spec.seed += rank                                            # every rank rolls out its own sequences
+    spec = replica_spec(args, rank)
     X, W, Bi = data.make_inputs(spec), data.make_weights(spec), data.make_biases(spec)
     tdt = torch.bfloat16 if spec.dtype == "bf16" else torch.float32
     host_in = [torch.from_numpy(np.ascontiguousarray(X[v], dtype=np.float32)).to(tdt).contiguous().pin_memory()
@@ -262,10 +282,7 @@ def run_cuda(args):
             e2e_ms.append(a.elapsed_time(b))
     e2e_ms_mean = float(np.mean(e2e_ms))
     # max over ranks
-    vals = torch.tensor([main["ms_per_step"], e2e_ms_mean], dtype=torch.float64, device="cuda")
-    if dist is not None:
-        dist.all_reduce(vals, op=dist.ReduceOp.MAX)
-    ms, e2e = float(vals[0]), float(vals[1])
+    ms, e2e = max_over_ranks([main["ms_per_step"], e2e_ms_mean], dist, "cuda")
     fl, by = frame_flops(spec), frame_bytes(spec)
     intensity = fl / by
     tensor_bound = spec.dtype == "bf16" and intensity > 1e3 * pk["bf16_tflops_sustained"] / pk["hbm_gbs"]
@@ -313,7 +330,7 @@ def run_cuda(args):
     roof["peak_source"] = pk["source"]
     roof["algorithmic_flops_per_frame"] = fl
     roof["algorithmic_bytes_per_frame"] = by
-    line = {"metric": METRIC, "value": world * T / ms * 1e3, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+    line = {"metric": METRIC, "value": whole_job_frames_per_s(world, T, ms), "unit": UNIT, "n_gpus": world, "steps": args.steps,
             "warmup": args.warmup, "ms_per_step": ms, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
             "dtype": "bf16" if spec.dtype == "bf16" else "f32", "data": "synthetic",
             "config": {"workload": spec.name, "pattern": args.pattern, "batch": spec.batch, "frames_per_step": T,
@@ -322,7 +339,7 @@ def run_cuda(args):
             "us_per_frame": us_frame, "sample_frames_per_s": world * spec.batch * T / ms * 1e3,
             "patterns": {p: {k: r[k] for k in ("frames_per_s", "us_per_frame", "groups_per_frame", "launches")}
                          for p, r in results.items()},
-            "e2e": {"value": world * T / e2e * 1e3, "unit": UNIT,
+            "e2e": {"value": whole_job_frames_per_s(world, T, e2e), "unit": UNIT,
                     "h2d_bytes_per_step": int(sum(h.numel() * h.element_size() for h in host_in)),
                     "d2h_bytes_per_step": int(out_host.numel() * 4)},
             "gpu_launches": int(main["launches"]), "roofline": roof, "clocks": clocks,

@@ -1,0 +1,48 @@
+"""GPU parity at the benchmark's full sizes, in the launch configuration bench.py times (sr_rollout_run
+with CUDA graphs of 16 frames, tensor cores where they apply).  The oracle evaluates a few whole
+sequences of the batch (sequences are independent, so those samples are exact); output sequence and
+final states of every node are compared.  c5 runs fewer frames at full size (the oracle needs about
+5 G multiply-adds per sample and frame) and all 128 frames at reduced image size."""
+import pytest
+
+from tests import parity
+from workloads import graphs
+
+pytestmark = pytest.mark.gpu
+
+
+def test_c2_full_size_all_patterns():
+    g = graphs.build("c2")
+    for p in g.patterns:
+        parity.check_run(g, p, graph_frames=16, samples=[0, 31, 63])
+
+
+def test_c3_full_size_all_patterns():
+    g = graphs.build("c3")
+    for p in g.patterns:
+        parity.check_run(g, p, graph_frames=16, samples=[0, 255])
+
+
+def test_c4_full_size_streaming():
+    g = graphs.build("c4")
+    parity.check_run(g, "streaming", graph_frames=16, samples=[0, 127])
+
+
+def test_c4_full_batch_sequential_fewer_frames():
+    g = graphs.build("c4", frames=8)
+    parity.check_run(g, "sequential", graph_frames=0, samples=[64])
+
+
+def test_c5_full_size_fewer_frames():
+    g = graphs.build("c5", frames=10)
+    parity.check_run(g, "streaming", graph_frames=4, samples=[0, 31])
+    g2 = graphs.build("c5", frames=3)
+    for p in ("sequential", "hybrid0", "hybrid1", "hybrid2"):
+        parity.check_run(g2, p, graph_frames=0, samples=[17])
+
+
+def test_c5_all_128_frames_reduced_images():
+    # recurrent edges over 128 frames with states re-rounded to bf16 every frame: the drift stays in tolerance
+    g = graphs.build("c5", size=16, batch=8)
+    for p in ("streaming", "hybrid1"):
+        parity.check_run(g, p, graph_frames=16, samples=[0, 7])
