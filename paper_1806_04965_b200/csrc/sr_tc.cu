@@ -86,7 +86,7 @@ struct TcNode {
     int32_t pad_;
 };
 
-struct TcTile { int32_t node, b0, h0, w0; };
+struct TcTile { int32_t node, b0, h0, w0, m0, pad_[3]; };   // m0: first output channel of the tile (0 or 128)
 
 struct TcStem {             // a few-channel input edge staged as im2col rows
     const void* src[2];
@@ -303,7 +303,7 @@ sr_tc_group_kernel(const CUtensorMap* __restrict__ maps, const TcNode* __restric
                         }
                         const uint32_t unit = ws_cur * (uint32_t)w_slot_units + k.w_box * box_u;
                         mbar_expect_tx(bar_wfull + 8 * unit, (uint32_t)k.w_bytes16 << 4);
-                        tma_load_2d(w_ring + unit * kWUnit, &maps[k.w_map], bar_wfull + 8 * unit, (int)k.k_off, 0);
+                        tma_load_2d(w_ring + unit * kWUnit, &maps[k.w_map], bar_wfull + 8 * unit, (int)k.k_off, tl.m0);
                         wf_phase ^= 1u << unit;
                         wf_used |= 1u << unit;
                     }
@@ -418,7 +418,7 @@ sr_tc_group_kernel(const CUtensorMap* __restrict__ maps, const TcNode* __restric
             tc_fence_after();
             __nv_bfloat16* out = static_cast<__nv_bfloat16*>(nd.state[cur]);
             for (int h = 0; h < nd.n_mh; ++h) {
-                const int co_w = h * 128 + quarter * 32;                // first channel of this warp
+                const int co_w = tl.m0 + h * 128 + quarter * 32;        // first channel of this warp
                 const int co = co_w + lane;                             // TMEM lane = output channel
                 const float bias = co < nd.C ? __ldg(nd.bias + co) : 0.f;
                 const bool gvalid = co_w + (lane & 3) * 8 < nd.C;       // this thread's group of 8 channels exists
@@ -677,8 +677,8 @@ sr_status sr_tc_plan(sr_graph* g, size_t& off)
         for (int e : n.in_edges)
             if (reuses_columns(g, g->edges[e])) P.sep = std::max(P.sep, g->edges[e].k_eff - 1);
         choose_tile(n.d.h, n.d.w, g->batch, P.sep, g->opt_tile_w, P);
-        P.n_mh = (n.d.c + 127) / 128;
-        P.group = P.n_mh >= 2 ? 1 : 3;
+        P.n_mh = 1;                                   // a node with more than 128 output channels is tiled in halves
+        P.group = 3;
         int k_off = 0;
         for (int e : n.in_edges) {
             const SrHostEdge& he = g->edges[e];
@@ -732,8 +732,9 @@ sr_status sr_tc_plan(sr_graph* g, size_t& off)
             for (int b0 = 0; b0 < g->batch; b0 += P.tb)
                 for (int h0 = 0; h0 < n.d.h; h0 += P.th)
                     for (int w0 = 0; w0 < n.d.w; w0 += P.tw)
-                        tl.push_back({(long long)P.kbs.size() * P.n_mh * P.n_cols, TcTile{E->node_of[v], b0, h0, w0}});
-            w_slot = std::max(w_slot, std::max(1, (n.d.c * 128 + kWUnit - 1) / kWUnit) * P.group);
+                        for (int m0 = 0; m0 < n.d.c; m0 += 128)
+                            tl.push_back({(long long)P.kbs.size() * P.n_cols, TcTile{E->node_of[v], b0, h0, w0, m0, {0, 0, 0}}});
+            w_slot = std::max(w_slot, std::max(1, (std::min(n.d.c, 128) * 128 + kWUnit - 1) / kWUnit) * P.group);
             // a window starts up to sep * tw rows into the box and the MMA reads n_cols rows from there
             for (const KbHost& kb : P.kbs)
                 a_slot = std::max(a_slot, (int)sr_align_up((size_t)(P.sep * P.tw + P.n_cols) * kb.bk * 2, 1024));
@@ -809,7 +810,7 @@ sr_status sr_tc_bind(sr_graph* g)
         d.n_kb = (int)P.kbs.size();
         // instruction descriptor: D = f32, A = B = bf16, both K-major, M = 128 output channels, N = pixels
         d.idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(P.n_cols >> 3) << 17) | ((uint32_t)(128 >> 4) << 24);
-        d.w_box_units = std::max(1, (n.d.c * 128 + kWUnit - 1) / kWUnit);
+        d.w_box_units = std::max(1, (std::min(n.d.c, 128) * 128 + kWUnit - 1) / kWUnit);
         d.w_group_units = d.w_box_units * P.group;
         const int rows = P.th + P.sep;
         std::map<int, int> wmap;                      // bk -> weight tensor map
@@ -818,7 +819,7 @@ sr_status sr_tc_bind(sr_graph* g)
             CUtensorMap m;
             cuuint64_t dims[2] = {(cuuint64_t)P.k_total, (cuuint64_t)n.d.c};
             cuuint64_t strides[1] = {(cuuint64_t)P.k_total * 2};
-            cuuint32_t box[2] = {(cuuint32_t)kb.bk, (cuuint32_t)n.d.c};
+            cuuint32_t box[2] = {(cuuint32_t)kb.bk, (cuuint32_t)std::min(n.d.c, 128)};
             cuuint32_t es[2] = {1, 1};
             if (encode(&m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, ws + P.wcat.offset, dims, strides, box, es,
                        CU_TENSOR_MAP_INTERLEAVE_NONE, swizzle_of(kb.bk), CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
@@ -841,7 +842,7 @@ sr_status sr_tc_bind(sr_graph* g)
             k.n_k16 = (uint8_t)(kb.bk / 16);
             k.desc_hi = desc_hi_of(kb.bk);
             k.x_bytes16 = kb.x_load ? (uint16_t)((kb.bk * 2 * P.tw * rows * P.tb) >> 4) : 0;
-            k.w_bytes16 = (uint16_t)((kb.bk * 2 * n.d.c) >> 4);
+            k.w_bytes16 = (uint16_t)((kb.bk * 2 * std::min(n.d.c, 128)) >> 4);
             k.x_off16 = (uint16_t)((kb.x_shift * P.tw * kb.bk * 2) >> 4);
             if (kb.stem) {
                 const StemPlan& S = E->stems[kb.stem_index];
