@@ -46,7 +46,8 @@
 namespace {
 
 constexpr int kMaxCols = 256;                         // pixels (N of the MMA) per tile
-constexpr int kThreads = 192;
+constexpr int kThreads = 224;
+constexpr int kFifo = 16;                             // burst descriptors in flight between scout and issuer
 constexpr int kMaxA = 4;                              // activation ring depth
 constexpr int kWUnit = 4096, kMaxWUnits = 32;         // weight ring: units of 4 KiB
 constexpr int kSmemBudget = 200 * 1024;
@@ -175,6 +176,27 @@ __device__ __forceinline__ void tc_mma_bf16(uint32_t d_tmem, uint64_t a_desc, ui
         "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
         ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate) : "memory");
 }
+__device__ __forceinline__ void st_shared_v4(uint32_t addr, uint32_t x, uint32_t y, uint32_t z, uint32_t w)
+{
+    asm volatile("st.volatile.shared.v4.u32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(x), "r"(y), "r"(z), "r"(w) : "memory");
+}
+__device__ __forceinline__ uint4 ld_shared_v4(uint32_t addr)
+{
+    uint4 v;
+    asm volatile("ld.volatile.shared.v4.u32 {%0, %1, %2, %3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(addr) : "memory");
+    return v;
+}
+// Same with the descriptors given as (address word, shared upper word).
+__device__ __forceinline__ void tc_mma_bf16_lohi(uint32_t d_tmem, uint32_t a_lo, uint32_t b_lo, uint32_t hi, uint32_t idesc, uint32_t accumulate)
+{
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t.reg .b64 da, db;\n\t"
+        "setp.ne.b32 p, %5, 0;\n\t"
+        "mov.b64 da, {%1, %3};\n\t"
+        "mov.b64 db, {%2, %3};\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], da, db, %4, p;\n\t}"
+        ::"r"(d_tmem), "r"(a_lo), "r"(b_lo), "r"(hi), "r"(idesc), "r"(accumulate) : "memory");
+}
 __device__ __forceinline__ void tc_commit(uint32_t bar)
 {
     asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
@@ -207,6 +229,8 @@ sr_tc_group_kernel(const CUtensorMap* __restrict__ maps, const TcNode* __restric
     __shared__ uint4 kb_tab[2][2 * kMaxNodeKb];            // K-block tables of the producer's and the issuer's current node
     __shared__ __align__(16) uint16_t epi_buf[4][32 * 32]; // per epilogue warp: 32 pixels x 32 channels, bf16
     __shared__ int pix_off[kMaxCols];                      // element offset of every pixel of the current tile, -1 = not stored
+    __shared__ __align__(16) uint4 fifo[kFifo][2];         // burst descriptors, scout -> issuer
+    __shared__ volatile uint32_t fifo_read;                // descriptors the issuer has taken
 
     // weight ring first: an M = 128 instruction on a node with fewer than 128 output channels reads
     // rows past its weight box, which then still lie inside this allocation
@@ -217,8 +241,13 @@ sr_tc_group_kernel(const CUtensorMap* __restrict__ maps, const TcNode* __restric
     const uint32_t bar_wfull = smem_u32(&bars[2 * kMaxA]), bar_wempty = smem_u32(&bars[2 * kMaxA + kMaxWUnits]);
     const uint32_t bar_tfull = smem_u32(&bars[2 * kMaxA + 2 * kMaxWUnits]), bar_tempty = bar_tfull + 16;
 
+    if (threadIdx.x < kFifo) {
+        fifo[threadIdx.x][0] = make_uint4(0, 0, 0, 0);
+        fifo[threadIdx.x][1] = make_uint4(0, 0, 0, 0);
+    }
     if (threadIdx.x == 0) {
         abort_flag = 0;
+        fifo_read = 0;
         for (int s = 0; s < n_a; ++s) {
             mbar_init(bar_afull + 8 * s, 1);
             mbar_init(bar_aempty + 8 * s, 1);
@@ -252,11 +281,12 @@ sr_tc_group_kernel(const CUtensorMap* __restrict__ maps, const TcNode* __restric
     // the issuer and the epilogue warps walk the same tile list and make the same choice.
     uint32_t uses0 = 0, uses1 = 0;
 
-    if (warp <= 1) {
-        // Both single-thread roles walk the same tile list.  At every change of node the whole warp
+    if (warp == 0 || warp == 6) {
+        // The producer (warp 0) and the scout (warp 6) walk the same tile list.  At every change of node the whole warp
         // copies the node's K-block table into its own shared-memory buffer; lane 0 then runs the
         // block loop out of shared memory.
-        uint4* my_tab = kb_tab[warp];
+        uint4* my_tab = kb_tab[warp == 0 ? 0 : 1];
+        uint32_t n_pub = 0;                                   // bursts published so far (scout)
         int cached_node = -1;
         // The weight ring is a ring of slots of w_slot_units 4 KiB units (the largest weight group of
         // the launch), handed back through one "empty" barrier per slot.  Box i of a group starts at
@@ -272,7 +302,7 @@ sr_tc_group_kernel(const CUtensorMap* __restrict__ maps, const TcNode* __restric
             const TcTile tl = tiles[ti];
             const int first_kb = nodes[tl.node].first_kb, n_kb = nodes[tl.node].n_kb;
             const uint32_t box_u = (uint32_t)nodes[tl.node].w_box_units;
-            const uint32_t idesc = nodes[tl.node].idesc, n_cols = (uint32_t)nodes[tl.node].n_cols, n_mh = (uint32_t)nodes[tl.node].n_mh;
+            const uint32_t idesc = nodes[tl.node].idesc;
             if (tl.node != cached_node) {
                 __syncwarp();
                 const uint4* src = reinterpret_cast<const uint4*>(kbs + first_kb);
@@ -308,69 +338,74 @@ sr_tc_group_kernel(const CUtensorMap* __restrict__ maps, const TcNode* __restric
                         wf_used |= 1u << unit;
                     }
                 } else {
-                    // ------------------------------------------------------ MMA issuer
-                    const bool wide = n_mh * n_cols > 256;
-                    const uint32_t acc = wide ? 0u : (uses0 <= uses1 ? 0u : 1u);
-                    if (wide || acc == 0) {
-                        if (!mbar_wait(bar_tempty, (uses0 & 1) ^ 1, abortp)) ok = false;
-                    }
-                    if (ok && (wide || acc == 1)) {
-                        if (!mbar_wait(bar_tempty + 8, (uses1 & 1) ^ 1, abortp)) ok = false;
-                    }
-                    tc_fence_after();
-                    const uint32_t d_tmem = tmem_base + acc * 256;
-                    // Software pipeline: the table entry of the next K-block is read and its two barriers are
-                    // probed BEFORE this block's MMAs are issued, so that the probes' latency hides behind the
-                    // (blocking) MMA issue; only a failed probe turns into a real wait.
-                    TcKBlock k = tab[0];
-                    uint32_t ws_n = (k.flags & 4) ? w_nxt : ws_cur;
-                    uint32_t unit = ws_n * (uint32_t)w_slot_units + k.w_box * box_u;
-                    uint32_t got_x = k.x_bytes16 ? mbar_test_wait(bar_afull + 8 * a_nxt, a_ph) : 1u;
-                    uint32_t got_w = mbar_test_wait(bar_wfull + 8 * unit, (wf_phase >> unit) & 1);
-                    for (int kb = 0; kb < n_kb && ok; ++kb) {
-                        if (k.x_bytes16) {
-                            a_cur = a_nxt;
-                            if (!got_x && !mbar_wait(bar_afull + 8 * a_cur, a_ph, abortp)) { ok = false; break; }
-                            if (++a_nxt == (uint32_t)n_a) { a_nxt = 0; a_ph ^= 1; }
+                    // ------------------------------------------------------ scout
+                    // Measured: whatever the issuing thread executes between two tcgen05.mma costs tensor-pipe
+                    // time one for one (a probe of a ready barrier ~165 cycles, a shared-memory load ~110, a
+                    // commit ~50), except for ~200 cycles per burst of >= 8 MMAs.  So this thread does all the
+                    // waiting and address arithmetic and hands the issuer one 32-byte descriptor per weight
+                    // group (up to 3 K-blocks = 12 MMAs): descriptor address words, flags, barriers to commit.
+                    const uint32_t acc = uses0 <= uses1 ? 0u : 1u;
+                    if (!mbar_wait(bar_tempty + 8 * acc, ((acc ? uses1 : uses0) & 1) ^ 1, abortp)) ok = false;
+                    int kb = 0;
+                    while (kb < n_kb && ok) {
+                        uint32_t lo[3] = {0u, 0u, 0u}, nt = 0, act_mask = 0, n_k16 = 0, desc_hi = 0, commit_w = 0, loads = 0;
+                        const uint32_t first = kb == 0;
+                        // a burst stays inside one weight group and never holds so many fresh activation slots
+                        // that the producer could not load the next one (it would wait for this very burst)
+                        const uint32_t max_loads = n_a > 2 ? (uint32_t)n_a - 1 : 1u;
+                        while (nt < 3 && kb < n_kb) {
+                            const TcKBlock k = tab[kb];
+                            if (nt > 0 && k.x_bytes16 && loads >= max_loads) break;
+                            if (k.x_bytes16) {
+                                a_cur = a_nxt;
+                                if (!mbar_wait(bar_afull + 8 * a_cur, a_ph, abortp)) { ok = false; break; }
+                                if (++a_nxt == (uint32_t)n_a) { a_nxt = 0; a_ph ^= 1; }
+                                ++loads;
+                            }
+                            if (k.flags & 4) {
+                                ws_cur = w_nxt;
+                                if (++w_nxt == n_ws) w_nxt = 0;
+                            }
+                            const uint32_t unit = ws_cur * (uint32_t)w_slot_units + k.w_box * box_u;
+                            if (!mbar_wait(bar_wfull + 8 * unit, (wf_phase >> unit) & 1, abortp)) { ok = false; break; }
+                            wf_phase ^= 1u << unit;
+                            const uint32_t x_lo = (((a_ring + a_cur * a_slot) >> 4) + k.x_off16) & 0x3FFFu;
+                            const uint32_t w_lo = ((w_ring + unit * kWUnit) >> 4) & 0x3FFFu;
+                            lo[nt] = w_lo | (x_lo << 16);
+                            if (k.flags & 2) act_mask |= 1u << a_cur;
+                            n_k16 = k.n_k16;
+                            desc_hi = k.desc_hi;
+                            ++nt;
+                            ++kb;
+                            if (k.flags & 8) { commit_w = 1; break; }
                         }
-                        if (k.flags & 4) {
-                            ws_cur = w_nxt;
-                            if (++w_nxt == n_ws) w_nxt = 0;
+                        if (!ok) break;
+                        ++n_pub;
+                        if (n_pub - fifo_read >= (uint32_t)kFifo) {          // never overwrite a descriptor not yet taken
+                            const long long t0 = clock64();
+                            while (n_pub - fifo_read >= (uint32_t)kFifo)
+                                if (abort_flag || clock64() - t0 > kWaitCycles) { abort_flag = 1; ok = false; break; }
+                            if (!ok) break;
                         }
-                        if (!got_w && !mbar_wait(bar_wfull + 8 * unit, (wf_phase >> unit) & 1, abortp)) { ok = false; break; }
-                        wf_phase ^= 1u << unit;
-                        const uint64_t hi = ((uint64_t)k.desc_hi << 32) | (1ull << 16);
-                        const uint64_t x_desc = hi | (uint64_t)((((a_ring + a_cur * a_slot) >> 4) + k.x_off16) & 0x3FFFu);
-                        uint64_t w_desc = hi | (uint64_t)(((w_ring + unit * kWUnit) >> 4) & 0x3FFFu);
-                        const uint32_t first = kb != 0, n_k16 = k.n_k16, flags = k.flags, ws_done = ws_cur;
-                        if (kb + 1 < n_kb) {
-                            k = tab[kb + 1];
-                            ws_n = (k.flags & 4) ? w_nxt : ws_cur;
-                            unit = ws_n * (uint32_t)w_slot_units + k.w_box * box_u;
-                            got_x = k.x_bytes16 ? mbar_test_wait(bar_afull + 8 * a_nxt, a_ph) : 1u;
-                            got_w = mbar_test_wait(bar_wfull + 8 * unit, (wf_phase >> unit) & 1);
-                        }
-                        // a K = 16 step moves both operands 32 bytes along K (+2 in the address field);
-                        // the second half of the output channels starts 128 weight rows further
-                        for (uint32_t h = 0; h < n_mh; ++h) {
-                            tc_mma_bf16(d_tmem + h * n_cols, w_desc, x_desc, idesc, first);
-                            for (uint32_t j = 1; j < n_k16; ++j)
-                                tc_mma_bf16(d_tmem + h * n_cols, w_desc + 2 * j, x_desc + 2 * j, idesc, 1);
-                            w_desc += 256u * n_k16;
-                        }
-                        if (flags & 8) tc_commit(bar_wempty + 8 * ws_done);  // hands the weight slot back
-                        if (flags & 2) tc_commit(bar_aempty + 8 * a_cur);    // last reader of the activation slot
+                        const uint32_t fl = nt | (n_k16 << 2) | (first << 5) | (acc << 6) | (commit_w << 7) | (ws_cur << 8) | (act_mask << 11) |
+                                            ((kb == n_kb ? 1u : 0u) << 15);
+                        const uint32_t e = smem_u32(&fifo[n_pub & (kFifo - 1)][0]);
+                        st_shared_v4(e + 16, lo[0], lo[1], lo[2], n_pub);
+                        __threadfence_block();
+                        st_shared_v4(e, n_pub, desc_hi, idesc, fl);
                     }
-                    if (ok) {
-                        if (wide || acc == 0) tc_commit(bar_tfull);
-                        if (wide || acc == 1) tc_commit(bar_tfull + 8);
-                    }
-                    if (wide || acc == 0) ++uses0;
-                    if (wide || acc == 1) ++uses1;
+                    if (acc == 0) ++uses0; else ++uses1;
                 }
             }
             ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
             if (!ok) break;
+        }
+        if (warp == 6 && lane == 0) {
+            ++n_pub;                                                                // tell the issuer to stop
+            const uint32_t e = smem_u32(&fifo[n_pub & (kFifo - 1)][0]);
+            st_shared_v4(e + 16, 0, 0, 0, n_pub);
+            __threadfence_block();
+            st_shared_v4(e, n_pub, 0, 0, 1u << 16);
         }
         if (warp == 0 && lane == 0) {
             // drain: every copy this thread started must have landed before the CTA may exit
@@ -380,6 +415,54 @@ sr_tc_group_kernel(const CUtensorMap* __restrict__ maps, const TcNode* __restric
             }
             for (uint32_t v = 0; v < (uint32_t)n_wu; ++v)
                 if ((wf_used >> v) & 1) mbar_wait(bar_wfull + 8 * v, ((wf_phase >> v) & 1) ^ 1, abortp);
+        }
+    } else if (warp == 1) {
+        // ---------------------------------------------------------------- MMA issuer
+        // One thread; it reads burst descriptors and issues, nothing else (see the scout).
+        if (lane == 0) {
+            uint32_t n = 0;
+            for (;;) {
+                ++n;
+                const uint32_t e = smem_u32(&fifo[n & (kFifo - 1)][0]);
+                uint4 q0 = ld_shared_v4(e);
+                if (q0.x != n) {
+                    const long long t0 = clock64();
+                    bool give_up = false;
+                    while ((q0 = ld_shared_v4(e)).x != n) {
+                        if (abort_flag || clock64() - t0 > kWaitCycles) { give_up = true; break; }
+                    }
+                    if (give_up) { abort_flag = 1; break; }
+                }
+                __threadfence_block();
+                const uint4 q1 = ld_shared_v4(e + 16);
+                fifo_read = n;
+                const uint32_t fl = q0.w;
+                if (fl & (1u << 16)) break;
+                const uint32_t hi = q0.y, idesc = q0.z, nt = fl & 3u, nk = (fl >> 2) & 7u, acc = (fl >> 6) & 1u;
+                const uint32_t d_tmem = tmem_base + acc * 256;
+                if (fl & 32u) tc_fence_after();                          // first burst of a tile: the accumulator was just handed back
+                uint32_t accum = (fl & 32u) ? 0u : 1u;
+                const uint32_t los[3] = {q1.x, q1.y, q1.z};
+#pragma unroll
+                for (uint32_t t = 0; t < 3; ++t) {
+                    if (t < nt) {
+                        const uint32_t wl = (los[t] & 0x3FFFu) | 0x10000u, xl = (los[t] >> 16) | 0x10000u;
+                        // a K = 16 step moves both operands 32 bytes along K: +2 in the descriptors' address field
+                        for (uint32_t j = 0; j < nk; ++j) {
+                            tc_mma_bf16_lohi(d_tmem, wl + 2 * j, xl + 2 * j, hi, idesc, accum);
+                            accum = 1u;
+                        }
+                    }
+                }
+                if (fl & 128u) tc_commit(bar_wempty + 8 * ((fl >> 8) & 7u));   // hands the weight slot back
+                uint32_t m = (fl >> 11) & 15u;
+                while (m) {                                              // activation slots this burst read last
+                    const uint32_t sl = __ffs(m) - 1;
+                    tc_commit(bar_aempty + 8 * sl);
+                    m &= m - 1;
+                }
+                if (fl & (1u << 15)) tc_commit(bar_tfull + 8 * acc);     // accumulator complete
+            }
         }
     } else {
         // ---------------------------------------------------------------- epilogue (warps 2..5)
@@ -828,15 +911,27 @@ sr_status sr_tc_bind(sr_graph* g)
             maps.push_back(m);
             wmap[kb.bk] = (int)maps.size() - 1;
         }
+        // weight groups: up to P.group consecutive K-blocks of equal channel-block width
+        std::vector<int> box_of(P.kbs.size(), 0);
+        std::vector<char> starts(P.kbs.size(), 0), ends(P.kbs.size(), 0);
+        for (size_t i = 0, in_group = 0; i < P.kbs.size(); ++i) {
+            if (in_group == 0 || (int)in_group == P.group || P.kbs[i].bk != P.kbs[i - 1].bk) {
+                starts[i] = 1;
+                if (i > 0) ends[i - 1] = 1;
+                in_group = 0;
+            }
+            box_of[i] = (int)in_group++;
+        }
+        if (!P.kbs.empty()) ends[P.kbs.size() - 1] = 1;
         for (size_t i = 0; i < P.kbs.size(); ++i) {
             const KbHost& kb = P.kbs[i];
             const SrHostEdge& he = g->edges[kb.edge];
             const SrHostNode& s = g->nodes[he.d.src];
             TcKBlock k{};
             int map0 = -1, map1 = -1, qxv = 0, qyv = 0;
-            const bool g_start = (int)(i % P.group) == 0, g_end = (int)(i % P.group) == P.group - 1 || i + 1 == P.kbs.size();
+            const bool g_start = starts[i] != 0, g_end = ends[i] != 0;
             k.flags = (uint8_t)((he.R ? 1 : 0) | (kb.x_release ? 2 : 0) | (g_start ? 4 : 0) | (g_end ? 8 : 0));
-            k.w_box = (uint8_t)(i % P.group);
+            k.w_box = (uint8_t)box_of[i];
             k.w_map = (uint16_t)wmap[kb.bk];
             k.k_off = (uint32_t)kb.k_off;
             k.n_k16 = (uint8_t)(kb.bk / 16);
