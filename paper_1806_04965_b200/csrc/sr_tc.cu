@@ -70,7 +70,8 @@ struct TcKBlock {
     uint8_t flags;          // 1: the edge reads frame t (R = 1), else frame t+1; 2: last reader of the activation
                             // slot; 4: first box of a weight group; 8: last box of a weight group
     uint8_t w_box;          // index of this block's weight box inside its group
-    uint8_t pad_[5];
+    uint8_t x_sbo16;        // (bytes between 8-pixel groups of the activation operand) / 16: one image row of the box
+    uint8_t pad_[4];
 };
 static_assert(sizeof(TcKBlock) == 32, "K-block table entries are copied as two 16-byte words");
 
@@ -187,15 +188,16 @@ __device__ __forceinline__ uint4 ld_shared_v4(uint32_t addr)
     return v;
 }
 // Same with the descriptors given as (address word, shared upper word).
-__device__ __forceinline__ void tc_mma_bf16_lohi(uint32_t d_tmem, uint32_t a_lo, uint32_t b_lo, uint32_t hi, uint32_t idesc, uint32_t accumulate)
+__device__ __forceinline__ void tc_mma_bf16_lohi(uint32_t d_tmem, uint32_t a_lo, uint32_t a_hi, uint32_t b_lo, uint32_t b_hi, uint32_t idesc,
+                                                 uint32_t accumulate)
 {
     asm volatile(
         "{\n\t.reg .pred p;\n\t.reg .b64 da, db;\n\t"
-        "setp.ne.b32 p, %5, 0;\n\t"
-        "mov.b64 da, {%1, %3};\n\t"
-        "mov.b64 db, {%2, %3};\n\t"
-        "tcgen05.mma.cta_group::1.kind::f16 [%0], da, db, %4, p;\n\t}"
-        ::"r"(d_tmem), "r"(a_lo), "r"(b_lo), "r"(hi), "r"(idesc), "r"(accumulate) : "memory");
+        "setp.ne.b32 p, %6, 0;\n\t"
+        "mov.b64 da, {%1, %2};\n\t"
+        "mov.b64 db, {%3, %4};\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], da, db, %5, p;\n\t}"
+        ::"r"(d_tmem), "r"(a_lo), "r"(a_hi), "r"(b_lo), "r"(b_hi), "r"(idesc), "r"(accumulate) : "memory");
 }
 __device__ __forceinline__ void tc_commit(uint32_t bar)
 {
@@ -348,7 +350,7 @@ sr_tc_group_kernel(const CUtensorMap* __restrict__ maps, const TcNode* __restric
                     if (!mbar_wait(bar_tempty + 8 * acc, ((acc ? uses1 : uses0) & 1) ^ 1, abortp)) ok = false;
                     int kb = 0;
                     while (kb < n_kb && ok) {
-                        uint32_t lo[3] = {0u, 0u, 0u}, nt = 0, act_mask = 0, n_k16 = 0, desc_hi = 0, commit_w = 0, loads = 0;
+                        uint32_t lo[3] = {0u, 0u, 0u}, nt = 0, act_mask = 0, n_k16 = 0, desc_hi = 0, x_hi = 0, commit_w = 0, loads = 0;
                         const uint32_t first = kb == 0;
                         // a burst stays inside one weight group and never holds so many fresh activation slots
                         // that the producer could not load the next one (it would wait for this very burst)
@@ -375,6 +377,7 @@ sr_tc_group_kernel(const CUtensorMap* __restrict__ maps, const TcNode* __restric
                             if (k.flags & 2) act_mask |= 1u << a_cur;
                             n_k16 = k.n_k16;
                             desc_hi = k.desc_hi;
+                            x_hi = (k.desc_hi & ~0x3FFFu) | k.x_sbo16;
                             ++nt;
                             ++kb;
                             if (k.flags & 8) { commit_w = 1; break; }
@@ -390,7 +393,7 @@ sr_tc_group_kernel(const CUtensorMap* __restrict__ maps, const TcNode* __restric
                         const uint32_t fl = nt | (n_k16 << 2) | (first << 5) | (acc << 6) | (commit_w << 7) | (ws_cur << 8) | (act_mask << 11) |
                                             ((kb == n_kb ? 1u : 0u) << 15);
                         const uint32_t e = smem_u32(&fifo[n_pub & (kFifo - 1)][0]);
-                        st_shared_v4(e + 16, lo[0], lo[1], lo[2], n_pub);
+                        st_shared_v4(e + 16, lo[0], lo[1], lo[2], x_hi);
                         __threadfence_block();
                         st_shared_v4(e, n_pub, desc_hi, idesc, fl);
                     }
@@ -438,7 +441,7 @@ sr_tc_group_kernel(const CUtensorMap* __restrict__ maps, const TcNode* __restric
                 fifo_read = n;
                 const uint32_t fl = q0.w;
                 if (fl & (1u << 16)) break;
-                const uint32_t hi = q0.y, idesc = q0.z, nt = fl & 3u, nk = (fl >> 2) & 7u, acc = (fl >> 6) & 1u;
+                const uint32_t w_hi = q0.y, x_hi = q1.w, idesc = q0.z, nt = fl & 3u, nk = (fl >> 2) & 7u, acc = (fl >> 6) & 1u;
                 const uint32_t d_tmem = tmem_base + acc * 256;
                 if (fl & 32u) tc_fence_after();                          // first burst of a tile: the accumulator was just handed back
                 uint32_t accum = (fl & 32u) ? 0u : 1u;
@@ -449,7 +452,7 @@ sr_tc_group_kernel(const CUtensorMap* __restrict__ maps, const TcNode* __restric
                         const uint32_t wl = (los[t] & 0x3FFFu) | 0x10000u, xl = (los[t] >> 16) | 0x10000u;
                         // a K = 16 step moves both operands 32 bytes along K: +2 in the descriptors' address field
                         for (uint32_t j = 0; j < nk; ++j) {
-                            tc_mma_bf16_lohi(d_tmem, wl + 2 * j, xl + 2 * j, hi, idesc, accum);
+                            tc_mma_bf16_lohi(d_tmem, wl + 2 * j, w_hi, xl + 2 * j, x_hi, idesc, accum);
                             accum = 1u;
                         }
                     }
@@ -607,14 +610,16 @@ struct KbHost {
     int stem_index;
     int ky, kx, c0, bk;
     int k_off;
-    bool x_load;       // loads a fresh activation box (else: reuses the box of this filter column)
-    int x_shift;       // image rows by which this tap's window is shifted inside the box
+    bool x_load;       // loads a fresh activation box (else: reuses the box loaded earlier for this channel block)
+    int x_shift;       // pixels by which this tap's window is shifted inside the box
+    int x_width;       // pixels per image row of the box (tile width, plus k-1 when the box serves all filter columns)
     bool x_release;
 };
 
 struct NodePlan {
     int node;
     int tw, th, tb, sep, n_cols, n_mh;
+    bool one_box;                   // tw == 8: one activation box per channel block serves all k x k taps
     int group;                      // weight boxes per group
     int k_total;                    // columns of the concatenated weight matrix
     std::vector<KbHost> kbs;
@@ -760,6 +765,7 @@ sr_status sr_tc_plan(sr_graph* g, size_t& off)
         for (int e : n.in_edges)
             if (reuses_columns(g, g->edges[e])) P.sep = std::max(P.sep, g->edges[e].k_eff - 1);
         choose_tile(n.d.h, n.d.w, g->batch, P.sep, g->opt_tile_w, P);
+        P.one_box = P.tw == 8 && P.sep > 0;
         P.n_mh = 1;                                   // a node with more than 128 output channels is tiled in halves
         P.group = 3;
         int k_off = 0;
@@ -776,23 +782,33 @@ sr_status sr_tc_plan(sr_graph* g, size_t& off)
                 S.buf[1] = take(bytes);
                 E->stem_of_edge[e] = (int)E->stems.size();
                 E->stems.push_back(S);
-                P.kbs.push_back(KbHost{e, true, (int)E->stems.size() - 1, 0, 0, 0, S.Kp, k_off, true, 0, true});
+                P.kbs.push_back(KbHost{e, true, (int)E->stems.size() - 1, 0, 0, 0, S.Kp, k_off, true, 0, P.tw, true});
                 k_off += S.Kp;
             } else {
                 const int bk = block_k(s.d.c), k = he.k_eff;
                 const int edge_off = k_off;
-                if (reuses_columns(g, he)) {
+                if (reuses_columns(g, he) && P.one_box) {
+                    // one box of (tw + k - 1) x (th + sep) pixels per channel block; tap (ky, kx) is the window that
+                    // starts ky image rows and kx pixels into it (the 8-pixel groups of the operand are one image
+                    // row of the box apart, whatever the row length)
+                    const int bw = P.tw + k - 1;
+                    for (int c0 = 0; c0 < s.d.c; c0 += bk)
+                        for (int ky = 0; ky < k; ++ky)
+                            for (int kx = 0; kx < k; ++kx)
+                                P.kbs.push_back(KbHost{e, false, -1, ky, kx, c0, bk, edge_off + (ky * k + kx) * s.d.c + c0,
+                                                       ky == 0 && kx == 0, ky * bw + kx, bw, ky == k - 1 && kx == k - 1});
+                } else if (reuses_columns(g, he)) {
                     for (int c0 = 0; c0 < s.d.c; c0 += bk)
                         for (int kx = 0; kx < k; ++kx)
                             for (int ky = 0; ky < k; ++ky)
                                 P.kbs.push_back(KbHost{e, false, -1, ky, kx, c0, bk, edge_off + (ky * k + kx) * s.d.c + c0,
-                                                       ky == 0, ky, ky == k - 1});
+                                                       ky == 0, ky * P.tw, P.tw, ky == k - 1});
                 } else {
                     for (int ky = 0; ky < k; ++ky)
                         for (int kx = 0; kx < k; ++kx)
                             for (int c0 = 0; c0 < s.d.c; c0 += bk)
                                 P.kbs.push_back(KbHost{e, false, -1, ky, kx, c0, bk, edge_off + (ky * k + kx) * s.d.c + c0,
-                                                       true, 0, true});
+                                                       true, 0, P.tw, true});
                 }
                 k_off += k * k * s.d.c;
             }
@@ -819,8 +835,12 @@ sr_status sr_tc_plan(sr_graph* g, size_t& off)
                             tl.push_back({(long long)P.kbs.size() * P.n_cols, TcTile{E->node_of[v], b0, h0, w0, m0, {0, 0, 0}}});
             w_slot = std::max(w_slot, std::max(1, (std::min(n.d.c, 128) * 128 + kWUnit - 1) / kWUnit) * P.group);
             // a window starts up to sep * tw rows into the box and the MMA reads n_cols rows from there
-            for (const KbHost& kb : P.kbs)
-                a_slot = std::max(a_slot, (int)sr_align_up((size_t)(P.sep * P.tw + P.n_cols) * kb.bk * 2, 1024));
+            for (const KbHost& kb : P.kbs) {
+                const size_t box_px = (size_t)kb.x_width * (P.th + P.sep) * P.tb;
+                // the last 8-pixel group a window reads: shift + (n_cols / 8 - 1) rows of the box + 8 pixels
+                const size_t reach_px = (size_t)(P.sep * kb.x_width + P.sep) + (size_t)(P.n_cols / 8 - 1) * (kb.x_width * 8 / P.tw) + 8;
+                a_slot = std::max(a_slot, (int)sr_align_up(std::max(box_px, reach_px) * kb.bk * 2, 1024));
+            }
         }
         std::stable_sort(tl.begin(), tl.end(), [](const auto& a, const auto& b) { return a.first > b.first; });
         for (auto& p : tl) E->group_tiles[gi].push_back(p.second);
@@ -915,7 +935,7 @@ sr_status sr_tc_bind(sr_graph* g)
         std::vector<int> box_of(P.kbs.size(), 0);
         std::vector<char> starts(P.kbs.size(), 0), ends(P.kbs.size(), 0);
         for (size_t i = 0, in_group = 0; i < P.kbs.size(); ++i) {
-            if (in_group == 0 || (int)in_group == P.group || P.kbs[i].bk != P.kbs[i - 1].bk) {
+            if (in_group == 0 || (int)in_group == P.group || P.kbs[i].bk != P.kbs[i - 1].bk || P.kbs[i].x_width != P.kbs[i - 1].x_width) {
                 starts[i] = 1;
                 if (i > 0) ends[i - 1] = 1;
                 in_group = 0;
@@ -936,9 +956,10 @@ sr_status sr_tc_bind(sr_graph* g)
             k.k_off = (uint32_t)kb.k_off;
             k.n_k16 = (uint8_t)(kb.bk / 16);
             k.desc_hi = desc_hi_of(kb.bk);
-            k.x_bytes16 = kb.x_load ? (uint16_t)((kb.bk * 2 * P.tw * rows * P.tb) >> 4) : 0;
+            k.x_bytes16 = kb.x_load ? (uint16_t)((kb.bk * 2 * kb.x_width * rows * P.tb) >> 4) : 0;
+            k.x_sbo16 = (uint8_t)((kb.x_width * 8 / P.tw * kb.bk * 2) >> 4);
             k.w_bytes16 = (uint16_t)((kb.bk * 2 * std::min(n.d.c, 128)) >> 4);
-            k.x_off16 = (uint16_t)((kb.x_shift * P.tw * kb.bk * 2) >> 4);
+            k.x_off16 = (uint16_t)((kb.x_shift * kb.bk * 2) >> 4);
             if (kb.stem) {
                 const StemPlan& S = E->stems[kb.stem_index];
                 for (int par = 0; par < 2; ++par)
@@ -959,7 +980,7 @@ sr_status sr_tc_bind(sr_graph* g)
                 for (int par = 0; par < 2; ++par) {
                     char* base = ws + s.state[par].offset + ((size_t)ry * s.d.w + rx) * s.d.c * 2;
                     (par ? map1 : map0) = act_map(base, s.d.c, Wv, Hv, (size_t)st * s.d.c * 2, (size_t)st * s.d.w * s.d.c * 2,
-                                                  (size_t)s.d.h * s.d.w * s.d.c * 2, kb.bk, P.tw, rows, P.tb);
+                                                  (size_t)s.d.h * s.d.w * s.d.c * 2, kb.bk, kb.x_width, rows, P.tb);
                 }
                 qxv = qx; qyv = qy; k.c0 = (uint16_t)kb.c0;
             }
