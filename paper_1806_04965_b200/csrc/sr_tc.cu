@@ -222,7 +222,7 @@ __device__ __forceinline__ void tc_wait_ld() { asm volatile("tcgen05.wait::ld.sy
 __global__ void __launch_bounds__(kThreads, 1)
 sr_tc_group_kernel(const CUtensorMap* __restrict__ maps, const TcNode* __restrict__ nodes,
                    const TcKBlock* __restrict__ kbs, const TcTile* __restrict__ tiles, int n_tiles,
-                   SrFrameCtl* __restrict__ ctl, int t_off, int B, int n_a, int a_slot, int n_wu, int w_slot_units)
+                   SrFrameCtl* __restrict__ ctl, int t_off, int B, int n_a, int a_slot, int n_wu, int w_slot_units, int tmem_cols)
 {
     extern __shared__ uint8_t smem_raw[];
     __shared__ uint64_t bars[2 * kMaxA + 2 * kMaxWUnits + 4];
@@ -266,7 +266,7 @@ sr_tc_group_kernel(const CUtensorMap* __restrict__ maps, const TcNode* __restric
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
     }
     if (warp == 1) {
-        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&tmem_slot)), "r"(512) : "memory");
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&tmem_slot)), "r"(tmem_cols) : "memory");
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
     }
     tc_fence_before();
@@ -346,7 +346,7 @@ sr_tc_group_kernel(const CUtensorMap* __restrict__ maps, const TcNode* __restric
                     // commit ~50), except for ~200 cycles per burst of >= 8 MMAs.  So this thread does all the
                     // waiting and address arithmetic and hands the issuer one 32-byte descriptor per weight
                     // group (up to 3 K-blocks = 12 MMAs): descriptor address words, flags, barriers to commit.
-                    const uint32_t acc = uses0 <= uses1 ? 0u : 1u;
+                    const uint32_t acc = (tmem_cols >= 512 && uses0 > uses1) ? 1u : 0u;   // 256 columns: one accumulator
                     if (!mbar_wait(bar_tempty + 8 * acc, ((acc ? uses1 : uses0) & 1) ^ 1, abortp)) ok = false;
                     int kb = 0;
                     while (kb < n_kb && ok) {
@@ -490,7 +490,7 @@ sr_tc_group_kernel(const CUtensorMap* __restrict__ maps, const TcNode* __restric
                 pix_off[n] = v ? (int)((((size_t)b * nd.H + y) * nd.W + xx) * nd.C) : -1;
             }
             const bool wide = nd.n_mh * nd.n_cols > 256;
-            const uint32_t acc = wide ? 0u : (uses0 <= uses1 ? 0u : 1u);
+            const uint32_t acc = (!wide && tmem_cols >= 512 && uses0 > uses1) ? 1u : 0u;
             if (wide || acc == 0) {
                 if (!mbar_wait(bar_tfull, uses0 & 1, abortp)) ok = false;
             }
@@ -549,7 +549,7 @@ sr_tc_group_kernel(const CUtensorMap* __restrict__ maps, const TcNode* __restric
     if (threadIdx.x == 0 && abort_flag) atomicExch(&ctl->error, 1);
     if (warp == 1) {
         tc_fence_after();
-        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(512) : "memory");
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(tmem_cols) : "memory");
     }
 }
 
@@ -639,7 +639,7 @@ struct TcEngine {
     std::vector<StemPlan> stems;
     std::vector<int> stem_of_edge;
     std::vector<std::vector<TcTile>> group_tiles;
-    std::vector<int> group_tile_offset, group_a_slot, group_n_a, group_n_wu, group_w_slot, group_grid;
+    std::vector<int> group_tile_offset, group_a_slot, group_n_a, group_n_wu, group_w_slot, group_grid, group_ctas_per_sm;
     SrRegion r_maps, r_nodes, r_kbs, r_tiles, r_stems;
     int n_maps = 0, n_kbs = 0, n_tiles = 0;
     int sm_count = 148;
@@ -848,7 +848,16 @@ sr_status sr_tc_plan(sr_graph* g, size_t& off)
         n_tiles += (int)tl.size();
         int n_wu = g->opt_b_units > 0 ? g->opt_b_units : 24;
         n_wu = std::max(2 * w_slot, std::min(kMaxWUnits, n_wu)) / w_slot * w_slot;
-        const int n_a = std::max(2, std::min(kMaxA, (kSmemBudget - n_wu * kWUnit) / a_slot));
+        int n_a = std::max(2, std::min(kMaxA, (kSmemBudget - n_wu * kWUnit) / a_slot));
+        // Small launches (a few tiles per SM) are bound by the latency of one tile, not by throughput: give every
+        // CTA the smallest rings and one accumulator, so that two CTAs share an SM and twice as many tiles are in flight.
+        int per_sm = 1;
+        if ((int)tl.size() <= 4 * 148 && 2 * w_slot * kWUnit + 2 * a_slot <= 88 * 1024) {
+            per_sm = 2;
+            n_wu = 2 * w_slot;
+            n_a = 2;
+        }
+        E->group_ctas_per_sm.push_back(per_sm);
         E->group_a_slot.push_back(a_slot);
         E->group_n_a.push_back(n_a);
         E->group_n_wu.push_back(n_wu);
@@ -1018,7 +1027,8 @@ sr_status sr_tc_bind(sr_graph* g)
         !up(E->r_stems, stems.data(), stems.size() * sizeof(TcStem)))
         return SR_ERR_CUDA;
     E->group_grid.clear();
-    for (auto& v : E->group_tiles) E->group_grid.push_back((int)std::min<size_t>(v.size(), (size_t)E->sm_count));
+    for (size_t gi = 0; gi < E->group_tiles.size(); ++gi)
+        E->group_grid.push_back((int)std::min<size_t>(E->group_tiles[gi].size(), (size_t)E->sm_count * E->group_ctas_per_sm[gi]));
     return SR_OK;
 }
 
@@ -1095,7 +1105,7 @@ int sr_tc_launch_group(sr_graph* g, int group, int t_off, cudaStream_t s)
         reinterpret_cast<const TcKBlock*>(g->ws + E->r_kbs.offset),
         reinterpret_cast<const TcTile*>(g->ws + E->r_tiles.offset) + E->group_tile_offset[group],
         (int)E->group_tiles[group].size(), reinterpret_cast<SrFrameCtl*>(g->ws + g->r_ctl.offset), t_off, g->batch, n_a, a_slot,
-        n_wu, E->group_w_slot[group]);
+        n_wu, E->group_w_slot[group], E->group_ctas_per_sm[group] > 1 ? 256 : 512);
     if (timed) {
         cudaEventRecord(E->ev[E->ev_used + 1], s);
         E->ev_used += 2;
