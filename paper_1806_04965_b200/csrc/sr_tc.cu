@@ -612,8 +612,9 @@ struct KbHost {
     int k_off;
     bool x_load;       // loads a fresh activation box (else: reuses the box loaded earlier for this channel block)
     int x_shift;       // pixels by which this tap's window is shifted inside the box
-    int x_width;       // pixels per image row of the box (tile width, plus k-1 when the box serves all filter columns)
+    int x_width;       // pixels per image row of the box (tile width, plus the pixel range of the taps it serves)
     bool x_release;
+    int box_qy = 0, box_qx = 0, box_ry = 0, box_rx = 0;   // origin and residue class of the box (loading block)
 };
 
 struct NodePlan {
@@ -659,7 +660,6 @@ bool is_stem(const sr_graph* g, const SrHostEdge& e)
     const SrHostNode& s = g->nodes[e.d.src];
     return s.is_input && (s.d.c % 16) != 0 && e.K <= 64;
 }
-bool reuses_columns(const sr_graph* g, const SrHostEdge& e) { return !is_stem(g, e) && e.stride_eff == 1 && e.k_eff >= 2; }
 
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
                                   const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
@@ -761,11 +761,28 @@ sr_status sr_tc_plan(sr_graph* g, size_t& off)
         if (!n.use_tc) continue;
         NodePlan P{};
         P.node = (int)v;
+        // sep: how many image rows the taps that share one activation box are apart at most
+        auto tap_q = [](int tap, int pad, int st, int& q, int& r) {
+            const int a = tap - pad;
+            q = (a >= 0) ? a / st : -((-a + st - 1) / st);
+            r = a - q * st;
+        };
         P.sep = 0;
-        for (int e : n.in_edges)
-            if (reuses_columns(g, g->edges[e])) P.sep = std::max(P.sep, g->edges[e].k_eff - 1);
+        for (int e : n.in_edges) {
+            const SrHostEdge& he = g->edges[e];
+            if (is_stem(g, he)) continue;
+            for (int r0 = 0; r0 < he.stride_eff; ++r0) {
+                int lo = 1 << 20, hi = -(1 << 20);
+                for (int t = 0; t < he.k_eff; ++t) {
+                    int q, r;
+                    tap_q(t, he.pad_eff, he.stride_eff, q, r);
+                    if (r == r0) { lo = std::min(lo, q); hi = std::max(hi, q); }
+                }
+                if (hi >= lo) P.sep = std::max(P.sep, hi - lo);
+            }
+        }
         choose_tile(n.d.h, n.d.w, g->batch, P.sep, g->opt_tile_w, P);
-        P.one_box = P.tw == 8 && P.sep > 0;
+        P.one_box = P.tw == 8;
         P.n_mh = 1;                                   // a node with more than 128 output channels is tiled in halves
         P.group = 3;
         int k_off = 0;
@@ -785,31 +802,39 @@ sr_status sr_tc_plan(sr_graph* g, size_t& off)
                 P.kbs.push_back(KbHost{e, true, (int)E->stems.size() - 1, 0, 0, 0, S.Kp, k_off, true, 0, P.tw, true});
                 k_off += S.Kp;
             } else {
-                const int bk = block_k(s.d.c), k = he.k_eff;
+                // Taps whose input pixels fall into the same residue class of the stride read the same view of the
+                // source, shifted by whole pixels: they share ONE activation box and differ only in where their window
+                // starts inside it (rows always; pixels too when the tile is 8 wide, because then the 8-pixel groups of
+                // the operand are simply one box row apart, whatever the row length).
+                const int bk = block_k(s.d.c), k = he.k_eff, st = he.stride_eff;
                 const int edge_off = k_off;
-                if (reuses_columns(g, he) && P.one_box) {
-                    // one box of (tw + k - 1) x (th + sep) pixels per channel block; tap (ky, kx) is the window that
-                    // starts ky image rows and kx pixels into it (the 8-pixel groups of the operand are one image
-                    // row of the box apart, whatever the row length)
-                    const int bw = P.tw + k - 1;
-                    for (int c0 = 0; c0 < s.d.c; c0 += bk)
-                        for (int ky = 0; ky < k; ++ky)
-                            for (int kx = 0; kx < k; ++kx)
-                                P.kbs.push_back(KbHost{e, false, -1, ky, kx, c0, bk, edge_off + (ky * k + kx) * s.d.c + c0,
-                                                       ky == 0 && kx == 0, ky * bw + kx, bw, ky == k - 1 && kx == k - 1});
-                } else if (reuses_columns(g, he)) {
-                    for (int c0 = 0; c0 < s.d.c; c0 += bk)
-                        for (int kx = 0; kx < k; ++kx)
-                            for (int ky = 0; ky < k; ++ky)
-                                P.kbs.push_back(KbHost{e, false, -1, ky, kx, c0, bk, edge_off + (ky * k + kx) * s.d.c + c0,
-                                                       ky == 0, ky * P.tw, P.tw, ky == k - 1});
-                } else {
-                    for (int ky = 0; ky < k; ++ky)
-                        for (int kx = 0; kx < k; ++kx)
-                            for (int c0 = 0; c0 < s.d.c; c0 += bk)
-                                P.kbs.push_back(KbHost{e, false, -1, ky, kx, c0, bk, edge_off + (ky * k + kx) * s.d.c + c0,
-                                                       true, 0, P.tw, true});
-                }
+                struct Tap { int ky, kx, qy, qx; };
+                std::map<std::tuple<int, int, int>, std::vector<Tap>> classes;      // (ry, rx, qx or 0) -> taps
+                for (int ky = 0; ky < k; ++ky)
+                    for (int kx = 0; kx < k; ++kx) {
+                        int qy, ry, qx, rx;
+                        tap_q(ky, he.pad_eff, st, qy, ry);
+                        tap_q(kx, he.pad_eff, st, qx, rx);
+                        classes[std::make_tuple(ry, rx, P.one_box ? 0 : qx)].push_back(Tap{ky, kx, qy, qx});
+                    }
+                for (int c0 = 0; c0 < s.d.c; c0 += bk)
+                    for (auto& cl : classes) {
+                        const std::vector<Tap>& taps = cl.second;
+                        int qy0 = 1 << 20, qx0 = 1 << 20, qx1 = -(1 << 20);
+                        for (const Tap& t : taps) { qy0 = std::min(qy0, t.qy); qx0 = std::min(qx0, t.qx); qx1 = std::max(qx1, t.qx); }
+                        const int bw = P.tw + (qx1 - qx0);
+                        for (size_t i = 0; i < taps.size(); ++i) {
+                            const Tap& t = taps[i];
+                            // the first tap of the class carries the box origin (qy0, qx0) through its ky / kx fields
+                            KbHost kb{e, false, -1, t.ky, t.kx, c0, bk, edge_off + (t.ky * k + t.kx) * s.d.c + c0,
+                                      i == 0, (t.qy - qy0) * bw + (t.qx - qx0), bw, i + 1 == taps.size()};
+                            kb.box_qy = qy0;
+                            kb.box_qx = qx0;
+                            kb.box_ry = std::get<0>(cl.first);
+                            kb.box_rx = std::get<1>(cl.first);
+                            P.kbs.push_back(kb);
+                        }
+                    }
                 k_off += k * k * s.d.c;
             }
         }
@@ -838,7 +863,7 @@ sr_status sr_tc_plan(sr_graph* g, size_t& off)
             for (const KbHost& kb : P.kbs) {
                 const size_t box_px = (size_t)kb.x_width * (P.th + P.sep) * P.tb;
                 // the last 8-pixel group a window reads: shift + (n_cols / 8 - 1) rows of the box + 8 pixels
-                const size_t reach_px = (size_t)(P.sep * kb.x_width + P.sep) + (size_t)(P.n_cols / 8 - 1) * (kb.x_width * 8 / P.tw) + 8;
+                const size_t reach_px = (size_t)kb.x_shift + (size_t)(P.n_cols / 8 - 1) * (kb.x_width * 8 / P.tw) + 8;
                 a_slot = std::max(a_slot, (int)sr_align_up(std::max(box_px, reach_px) * kb.bk * 2, 1024));
             }
         }
@@ -981,9 +1006,8 @@ sr_status sr_tc_bind(sr_graph* g)
             } else {
                 // input pixel = stride * (output pixel + q) + r, q = floor((tap - pad) / stride), r the residue:
                 // the residue-class view of the source makes the tap a dense box starting at (w0 + qx, h0 + qy)
-                const int st = he.stride_eff, ay = kb.ky - he.pad_eff, ax = kb.kx - he.pad_eff;
-                const int qy = (ay >= 0) ? ay / st : -((-ay + st - 1) / st), ry = ay - qy * st;
-                const int qx = (ax >= 0) ? ax / st : -((-ax + st - 1) / st), rx = ax - qx * st;
+                const int st = he.stride_eff;
+                const int qy = kb.box_qy, ry = kb.box_ry, qx = kb.box_qx, rx = kb.box_rx;
                 const int Hv = (s.d.h - ry + st - 1) / st, Wv = (s.d.w - rx + st - 1) / st;
                 if (Hv <= 0 || Wv <= 0) return SR_ERR_UNSUPPORTED;
                 for (int par = 0; par < 2; ++par) {
