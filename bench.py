@@ -27,7 +27,7 @@ from workloads import data, graphs  # noqa: E402
 
 # dram__bytes_read.sum + dram__bytes_write.sum of one tensor-core group launch from the ncu captures summarised under
 # profiles/ (null where no capture of the current kernel exists)
-TRAFFIC = {"c2": 5.77e6, "c3": 262.5e6, "c5": 613.0e6}
+TRAFFIC = {"c2": 5.78e6, "c3": 264.1e6, "c4": 157.5e6, "c5": 612.4e6}
 
 METRIC = "streaming_rollout_frames_per_sec"
 UNIT = "frames/s"
