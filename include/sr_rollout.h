@@ -88,6 +88,8 @@ typedef struct {
     int32_t response_interval;         /* update steps between outputs = F(R) (Sec. 4)                    */
     int32_t n_tensor_core_nodes;       /* nodes updated by the tcgen05 implicit-GEMM kernel               */
     int32_t n_direct_nodes;            /* nodes updated by the CUDA-core kernels                          */
+    int32_t resident_cluster;          /* CTAs per sequence of the shared-memory-resident kernel that
+                                          sr_rollout_run uses for this graph; 0 = it does not apply       */
 } sr_info;
 
 /*
@@ -161,7 +163,15 @@ sr_status sr_graph_set_node_bias(sr_graph* g, int node, const float* bias_host);
  *                  copy when no input edge has R = 0), joined before the frame ends; 0 = one stream.
  *           key 5 "kernel timing": 1 brackets every tensor-core group launch with CUDA events on the launching
  *                  stream (plain launches only, not inside CUDA graphs); read with sr_graph_kernel_time.
- * Must be set before sr_graph_bind_workspace (engine, weight ring, tile width) / before the first run (graphs). */
+ *           key 6 "resident": 1 (default) lets sr_rollout_run use the resident kernel when the network qualifies
+ *                  (bfloat16; per-sequence states and convolution weights fit in the shared memory of a
+ *                  thread-block cluster): one cluster per sequence walks all T frames in one launch with
+ *                  the states on chip; 0 = always the per-frame launch path.  sr_rollout_step always uses
+ *                  the launch path.
+ *           key 7 "resident cluster size": CTAs per sequence, 1, 2 or 4; 0 (default) = chosen by the library.
+ *           key 8 "resident warps": warps per CTA of the resident kernel, 4..16; 0 = default.
+ * Must be set before sr_graph_workspace_bytes / sr_graph_bind_workspace (engine, weight ring, tile width,
+ * resident keys) / before the first run (graphs). */
 sr_status sr_graph_set_option(sr_graph* g, int key, int value);
 
 /*

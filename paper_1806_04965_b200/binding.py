@@ -40,7 +40,7 @@ class _Info(ctypes.Structure):
     _fields_ = [(n, ctypes.c_int32) for n in
                 ("n_nodes", "n_edges", "n_inputs", "inference_factor", "n_groups", "streaming_parallel",
                  "output_node", "first_response_frame", "first_response_step", "response_interval",
-                 "n_tensor_core_nodes", "n_direct_nodes")]
+                 "n_tensor_core_nodes", "n_direct_nodes", "resident_cluster")]
 
 
 def load_library(path: Optional[str] = None):
@@ -105,7 +105,8 @@ class Graph:
     """A compiled network + rollout pattern (sr_graph).  batch=0 gives a theory-only graph."""
 
     def __init__(self, nodes: Sequence, edges: Sequence, R: Sequence[int], batch: int = 0, dtype: str = "bf16",
-                 engine: str = "auto", graph_frames: int = 0, device: str = "cuda:0", static_workspace: bool = False, weight_ring_units: int = 0, tile_width: int = 0):
+                 engine: str = "auto", graph_frames: int = 0, device: str = "cuda:0", static_workspace: bool = False, weight_ring_units: int = 0, tile_width: int = 0,
+                 resident: bool = True, resident_cluster: int = 0, resident_warps: int = 0):
         self._lib = load_library()
         self._h = ctypes.c_void_p()
         self.nodes, self.edges, self.R = list(nodes), list(edges), [int(r) for r in R]
@@ -129,6 +130,9 @@ class Graph:
             _check(self._lib.sr_graph_set_option(self._h, 1, int(graph_frames)), "sr_graph_set_option")
             _check(self._lib.sr_graph_set_option(self._h, 2, int(weight_ring_units)), "sr_graph_set_option")
             _check(self._lib.sr_graph_set_option(self._h, 3, int(tile_width)), "sr_graph_set_option")
+            _check(self._lib.sr_graph_set_option(self._h, 6, 1 if resident else 0), "sr_graph_set_option")
+            _check(self._lib.sr_graph_set_option(self._h, 7, int(resident_cluster)), "sr_graph_set_option")
+            _check(self._lib.sr_graph_set_option(self._h, 8, int(resident_warps)), "sr_graph_set_option")
             nbytes = ctypes.c_size_t()
             _check(self._lib.sr_graph_workspace_bytes(self._h, ctypes.byref(nbytes)), "sr_graph_workspace_bytes")
             self.workspace_bytes = nbytes.value

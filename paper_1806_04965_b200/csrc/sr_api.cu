@@ -9,6 +9,7 @@
 
 #include "sr_internal.h"
 #include "sr_kernels.h"
+#include "sr_resident.h"
 #include "sr_tc.h"
 
 namespace {
@@ -140,12 +141,16 @@ sr_status plan(sr_graph* g)
     g->r_items = take(off, sizeof(SrDirectItem) * std::max<size_t>(1, g->items.size()));
     sr_status st = sr_tc_plan(g, off);
     if (st != SR_OK) return st;
+    st = sr_rs_plan(g, off);
+    if (st != SR_OK) return st;
     g->ws_bytes = off;
     int n_tc = 0, n_direct = 0;
     for (const SrHostNode& n : g->nodes)
         if (!n.is_input) (n.use_tc ? n_tc : n_direct)++;
     g->info.n_tensor_core_nodes = n_tc;
     g->info.n_direct_nodes = n_direct;
+    int rs_warps = 0, rs_smem = 0;
+    sr_rs_describe(g, &g->info.resident_cluster, &rs_warps, &rs_smem);
     return SR_OK;
 }
 
@@ -270,6 +275,7 @@ void sr_graph_destroy(sr_graph* g)
         delete sd;
     }
     sr_tc_destroy(g);
+    sr_rs_destroy(g);
     delete g;
 }
 
@@ -321,6 +327,24 @@ sr_status sr_graph_set_option(sr_graph* g, int key, int value)
         if (g->ws) return SR_ERR_STATE;
         if (value < 0 || value > 32) return SR_ERR_INVALID_ARG;
         g->opt_b_units = value;
+        return SR_OK;
+    }
+    if (key == 6) {
+        if (g->ws) return SR_ERR_STATE;
+        if (value != 0 && value != 1) return SR_ERR_INVALID_ARG;
+        g->opt_resident = value;
+        return SR_OK;
+    }
+    if (key == 7) {
+        if (g->ws) return SR_ERR_STATE;
+        if (value != 0 && value != 1 && value != 2 && value != 4) return SR_ERR_INVALID_ARG;
+        g->opt_rs_cluster = value;
+        return SR_OK;
+    }
+    if (key == 8) {
+        if (g->ws) return SR_ERR_STATE;
+        if (value != 0 && (value < 4 || value > 16)) return SR_ERR_INVALID_ARG;
+        g->opt_rs_warps = value;
         return SR_OK;
     }
     return SR_ERR_INVALID_ARG;
@@ -391,6 +415,7 @@ sr_status sr_graph_bind_workspace(sr_graph* g, void* workspace_dev, size_t bytes
         return SR_ERR_CUDA;
     g->ws = ws;
     st = sr_tc_bind(g);
+    if (st == SR_OK) st = sr_rs_bind(g);
     if (st != SR_OK) {
         g->ws = nullptr;
         return st;
@@ -473,6 +498,10 @@ sr_status sr_graph_set_edge_weights(sr_graph* g, int edge, const float* w, int i
         const sr_status st = sr_tc_set_weights(g, edge, eff.data());
         if (st != SR_OK) return st;
     }
+    {
+        const sr_status st = sr_rs_set_weights(g, edge, eff.data());
+        if (st != SR_OK) return st;
+    }
     he.w_set = true;
     return SR_OK;
 }
@@ -537,6 +566,22 @@ sr_status sr_rollout_run(sr_graph* g, const void* const* in_seq_dev, int T, floa
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     sr_launch_set_ctl(g, make_ctl(g, in_seq_dev, true, out_seq_dev), s);
     g->launches += 1;
+    if (sr_rs_available(g)) {
+        bool aligned = true;                                     // the resident kernel fetches input rows in 4-byte words
+        for (size_t i = 0; i < g->input_nodes.size(); ++i)
+            if (reinterpret_cast<uintptr_t>(in_seq_dev[i]) & 3) aligned = false;
+        if (aligned) {
+            // one launch walks all T frames with the states in shared memory, then the frame counter
+            // advances and whatever the launch path derives from the input state is refreshed
+            st = sr_rs_launch(g, T, s);
+            if (st != SR_OK) return st;
+            sr_launch_advance(g, T, s);
+            g->launches += 2;
+            g->t += T;
+            g->launches += sr_tc_after_state_change(g, s);
+            return cuda_ok(cudaGetLastError()) ? SR_OK : SR_ERR_CUDA;
+        }
+    }
     int done = 0;
     const int gf = g->opt_graph_frames;
     if (gf > 0 && T >= gf) {

@@ -85,6 +85,7 @@ struct sr_graph {
     std::vector<std::vector<int>> groups;          // groups[l-1] = nodes of level l
     // options
     int opt_engine = 0, opt_graph_frames = 0, opt_b_units = 0, opt_tile_w = 0, opt_overlap = 1, opt_time_tc = 0;
+    int opt_resident = 1, opt_rs_cluster = 0, opt_rs_warps = 0;
     // workspace
     size_t ws_bytes = 0;
     char* ws = nullptr;
@@ -97,6 +98,7 @@ struct sr_graph {
     int64_t t = 0;
     int64_t launches = 0;
     void* tc = nullptr;                            // tensor-core engine state (opaque here)
+    void* rs = nullptr;                            // resident engine state (opaque here)
     void* graphs = nullptr;                        // CUDA-graph cache (opaque here)
     void* side = nullptr;                          // side stream and fork / join events (opaque here)
     bool input_feeds_same_frame = false;           // some edge that leaves an input node has R = 0

@@ -1,0 +1,1169 @@
+// Resident engine of the frame update
+//     x_v^{t+1} = sigma_v( b_v + sum_e f_e(theta_e, x_src(e)^{t+1-R(e)}) )        (paper Sec. A1.2, Eq. 2)
+// for networks whose per-sample state fits in shared memory.
+//
+// The sequences of a batch are independent (the paper's rollouts couple nodes and frames, never
+// samples), so ONE thread-block cluster owns ONE sequence and walks all T frames of a run with every
+// node state, every convolution weight and the rollout tables resident in shared memory.  Nothing but
+// the next input frame and the output crosses HBM per frame, and no launch or device-wide barrier
+// separates frames: a frame ends at a cluster barrier (a block barrier for a cluster of one).
+//   * The CTAs of a cluster split every node by image rows; a CTA keeps its own rows plus the halo
+//     rows its convolutions read, and the owner of a row writes it into the neighbour's halo through
+//     distributed shared memory as part of its epilogue.
+//   * A frame of a streaming rollout is one level: all (node, 16-pixel, 32-channel) units of the CTA
+//     are spread over its warps by estimated cost once, on the host.  Sequential and hybrid patterns
+//     run their F(R) tableau levels (Eq. 4, Eq. 5) with a barrier after each.
+//   * A unit is an implicit GEMM on mma.sync m16n8k16 (bf16 in, fp32 accumulate): the A rows are
+//     gathered by ldmatrix straight from the NHWC state (one row address per lane = one pixel of one
+//     filter tap; out-of-image taps point at a zero line), the B fragments come from weights packed
+//     per k-step in ldmatrix order.  The sum over incoming edges is one accumulator walked over the
+//     k-steps of all edges (the concatenated-convolution view of Sec. A).  Tiles of 16 pixels of ONE
+//     sample are far below the size the tcgen05 pipe needs to pay off (an instruction with M = 128
+//     costs >= 110 cycles however few columns it has), which is why this engine uses the warp-level
+//     tensor path and the batch-tiled tcgen05 kernel serves the large networks.
+//   * Few-channel edges (C_in * k * k <= 64, the first layer of an image network) build their A
+//     fragments from scalar shared-memory loads through a small per-edge lookup table.
+//   * Dense and mean-dense heads run on CUDA cores: every warp reduces a slice of the flattened
+//     source into a slot, slots of all CTAs are summed in a fixed order after the barrier.
+// State layout in shared memory: [row][col][C] bf16 in 16-byte chunks, chunk q stored at
+// (q & ~7) | ((q ^ (q >> 3)) & 7) so that the eight row addresses of an ldmatrix phase fall into
+// different bank groups for unit-stride and stride-2 taps.
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+
+#include <algorithm>
+#include <cstring>
+#include <vector>
+
+#include "sr_internal.h"
+#include "sr_resident.h"
+
+namespace {
+
+constexpr int kRsMaxCluster = 4;
+constexpr int kRsSmemMax = 232448;            // 227 KiB of dynamic shared memory per CTA
+constexpr int kRsMaxThreads = 512;
+constexpr int kRsDenseUnitChunks = 64;        // 16-byte chunks of the source per dense unit
+constexpr int kRsMaxDenseC = 64;
+
+enum { RS_INPUT = 0, RS_CONV = 1, RS_DENSE = 2 };
+enum { RS_E_MMA = 0, RS_E_GATHER = 1, RS_E_DENSE = 2, RS_E_MEAN = 3 };
+enum { RS_U_CONV = 0, RS_U_DENSE = 1 };
+
+struct RsNode {
+    int32_t kind, H, W, C;
+    int32_t act, level, lo, hi;              // level: 0-based tableau level; [lo, hi) rows owned by this CTA
+    int32_t slo, shi, is_output, input_slot; // [slo, shi) rows stored (own + halo)
+    int32_t buf[3], bias_off;                // byte offsets in shared memory (inputs rotate over three buffers)
+    int32_t w_off, first_edge, n_edges, buf_bytes;
+    int32_t up_lo, up_hi, up_slo, dn_lo;     // own rows that the previous / next CTA of the cluster also stores
+    int32_t dn_hi, dn_slo, slot_off, n_slots;
+    int32_t has_consumers, pix_off, pad1, pad2;   // pix_off: table of (row << 16 | col) of the CTA's own pixels
+    char* gstate[2];                         // the node's two state buffers in global memory
+};
+
+struct RsEdge {
+    int32_t src, type, k, stride;
+    int32_t pad, R, ksteps, lut_off;
+    int32_t Kreal, wd_off, wd_ld, n_chunks;  // dense: weights in shared memory at wd_off (row pitch wd_ld elements) or < 0
+    int32_t x_chunk0, wchunk_mod;            // dense: first source chunk of this CTA's slice; mean-dense: chunks per pixel
+    float scale;
+    int32_t pad_;
+    const char* wd_global;                   // dense weights in global memory, already at this CTA's slice
+    int64_t wd_gld;                          // row pitch there, in elements
+};
+
+struct RsUnit { int32_t kind, node, a, b, c, d; };
+struct RsCopy { const char* src; int32_t dst, bytes; };
+
+struct RsHeader {
+    int32_t n_nodes, n_edges, n_levels, n_warps;
+    int32_t off_nodes, off_edges, off_units, off_ubegin;
+    int32_t off_copies, n_copies, zero_off, smem_bytes;
+    int32_t dense_level_mask, sync_after_finalize, blob_bytes, pad_;
+};
+
+// ------------------------------------------------------------------------------------------------ device helpers
+__device__ __forceinline__ uint32_t rs_smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+__device__ __forceinline__ uint32_t rs_swz(uint32_t q) { return (q & ~7u) | ((q ^ (q >> 3)) & 7u); }
+
+__device__ __forceinline__ void rs_ldsm4(uint32_t (&r)[4], uint32_t addr)
+{
+    asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0,%1,%2,%3}, [%4];\n"
+                 : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]) : "r"(addr));
+}
+
+__device__ __forceinline__ void rs_mma(float (&d)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1)
+{
+    asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};\n"
+                 : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
+                 : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
+}
+
+__device__ __forceinline__ uint32_t rs_cluster_rank()
+{
+    uint32_t r;
+    asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+    return r;
+}
+
+__device__ __forceinline__ uint32_t rs_mapa(uint32_t addr, uint32_t rank)
+{
+    uint32_t r;
+    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(addr), "r"(rank));
+    return r;
+}
+
+__device__ __forceinline__ void rs_st_cluster_u32(uint32_t addr, uint32_t v)
+{
+    asm volatile("st.shared::cluster.u32 [%0], %1;" ::"r"(addr), "r"(v) : "memory");
+}
+
+__device__ __forceinline__ void rs_st_cluster_v4(uint32_t addr, const uint32_t (&v)[4])
+{
+    asm volatile("st.shared::cluster.v4.u32 [%0], {%1,%2,%3,%4};" ::"r"(addr), "r"(v[0]), "r"(v[1]), "r"(v[2]), "r"(v[3]) : "memory");
+}
+
+__device__ __forceinline__ void rs_cp_async4(uint32_t dst, const void* src)
+{
+    asm volatile("cp.async.ca.shared.global [%0], [%1], 4;" ::"r"(dst), "l"(src) : "memory");
+}
+
+__device__ __forceinline__ void rs_cp_async16(uint32_t dst, const void* src)
+{
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst), "l"(src) : "memory");
+}
+
+__device__ __forceinline__ void rs_cp_async_wait_all() { asm volatile("cp.async.wait_all;" ::: "memory"); }
+
+// End of a level: every warp of every CTA of the cluster has finished its units; their shared-memory
+// writes (local and remote) are visible afterwards.
+__device__ __forceinline__ void rs_level_barrier(int cs)
+{
+    if (cs > 1) {
+        __syncwarp();
+        asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
+    } else {
+        __syncthreads();
+    }
+}
+
+__device__ __forceinline__ uint32_t rs_pack_bf16(float lo, float hi)
+{
+    const __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
+    return *reinterpret_cast<const uint32_t*>(&v);
+}
+
+struct RsCtx {
+    unsigned char* smem;
+    uint32_t sbase;
+    const RsHeader* H;
+    const RsNode* nodes;
+    const RsEdge* edges;
+    uint32_t rank;
+    int cs, lane;
+};
+
+template <int NK>
+__device__ __forceinline__ void rs_mma_steps(float (&acc)[4][4], const uint32_t (&aaddr)[NK], uint32_t waddr, uint32_t wstride)
+{
+    uint32_t a[NK][4], bq[NK][2][4];
+#pragma unroll
+    for (int i = 0; i < NK; ++i) {
+        rs_ldsm4(a[i], aaddr[i]);
+        rs_ldsm4(bq[i][0], waddr + i * wstride);
+        rs_ldsm4(bq[i][1], waddr + i * wstride + 512);
+    }
+#pragma unroll
+    for (int i = 0; i < NK; ++i)
+#pragma unroll
+        for (int nt = 0; nt < 4; ++nt) rs_mma(acc[nt], a[i], bq[i][nt >> 1][(nt & 1) * 2], bq[i][nt >> 1][(nt & 1) * 2 + 1]);
+}
+
+// One (16 pixels x 32 channels) tile of a convolutional node: all k-steps of all incoming edges into one
+// accumulator, then bias, activation, bf16 cast and the stores into the next frame's buffer (own copy and,
+// for halo rows, the neighbour's).  `f` is the frame index relative to the start of the run: the update
+// computes relative frame f + 1.
+__device__ __forceinline__ void rs_conv_unit(const RsCtx& cx, const RsNode& nd, int j0, int n0, int f)
+{
+    const int lane = cx.lane;
+    const int W = nd.W, npix = (nd.hi - nd.lo) * W;
+    const uint32_t zaddr = cx.sbase + cx.H->zero_off;
+    float acc[4][4];
+#pragma unroll
+    for (int i = 0; i < 4; ++i)
+#pragma unroll
+        for (int j = 0; j < 4; ++j) acc[i][j] = 0.f;
+    // the pixel whose row address this lane supplies to ldmatrix, and the 8-channel half it points at
+    // (the table is padded to a multiple of 16 pixels with 0xFFFFFFFF)
+    const uint32_t* pix = reinterpret_cast<const uint32_t*>(cx.smem + nd.pix_off);
+    const uint32_t tl = pix[j0 + (lane & 15)];
+    const bool vl = tl != 0xFFFFFFFFu;
+    const int oyl = (int)(tl >> 16), oxl = (int)(tl & 0xFFFFu);
+    const int khalf = lane >> 4;
+    // the two pixels whose accumulator rows this lane holds
+    const int g = lane >> 2, tq = lane & 3;
+    int oy[2], ox[2];
+    bool pv[2];
+#pragma unroll
+    for (int r = 0; r < 2; ++r) {
+        const uint32_t t = pix[j0 + g + 8 * r];
+        pv[r] = t != 0xFFFFFFFFu;
+        oy[r] = (int)(t >> 16);
+        ox[r] = (int)(t & 0xFFFFu);
+    }
+    (void)npix;
+    const uint32_t wstride = (uint32_t)(nd.C >> 5) * 1024u;
+    uint32_t waddr = cx.sbase + nd.w_off + (uint32_t)(n0 >> 5) * 1024u + lane * 16;
+    for (int ei = 0; ei < nd.n_edges; ++ei) {
+        const RsEdge& e = cx.edges[nd.first_edge + ei];
+        const RsNode& sn = cx.nodes[e.src];
+        const int fb = f + 1 - e.R;                                   // relative frame of the source state (Eq. 2)
+        const int sbuf = sn.kind == RS_INPUT ? sn.buf[fb % 3] : sn.buf[fb & 1];
+        const int Hs = sn.H, Ws = sn.W;
+        if (e.type == RS_E_MMA) {
+            const uint32_t sb = cx.sbase + sbuf;
+            const int nch = sn.C >> 3, nc16 = sn.C >> 4;
+            const int iy0 = oyl * e.stride - e.pad, ix0 = oxl * e.stride - e.pad;
+            for (int ky = 0; ky < e.k; ++ky) {
+                const int iy = iy0 + ky;
+                const bool rowok = vl && iy >= sn.slo && iy < sn.shi;   // stored rows cover every in-image row a tile reads
+                const int rowq = (iy - sn.slo) * Ws * nch + khalf;
+                for (int kx = 0; kx < e.k; ++kx) {
+                    const int ix = ix0 + kx;
+                    const bool ok = rowok && (unsigned)ix < (unsigned)Ws;
+                    if (!__any_sync(0xffffffffu, ok)) {
+                        waddr += nc16 * wstride;
+                        continue;
+                    }
+                    const uint32_t q0 = (uint32_t)(rowq + ix * nch);
+                    int c = 0;
+                    for (; c + 2 <= nc16; c += 2) {
+                        uint32_t aa[2];
+                        aa[0] = ok ? sb + rs_swz(q0 + 2 * c) * 16 : zaddr;
+                        aa[1] = ok ? sb + rs_swz(q0 + 2 * c + 2) * 16 : zaddr;
+                        rs_mma_steps<2>(acc, aa, waddr, wstride);
+                        waddr += 2 * wstride;
+                    }
+                    if (c < nc16) {
+                        uint32_t aa[1];
+                        aa[0] = ok ? sb + rs_swz(q0 + 2 * c) * 16 : zaddr;
+                        rs_mma_steps<1>(acc, aa, waddr, wstride);
+                        waddr += wstride;
+                    }
+                }
+            }
+        } else {
+            // few-channel edge: A fragments from scalar loads; the table gives (ky, kx, channel) of every k index
+            const uint16_t* src = reinterpret_cast<const uint16_t*>(cx.smem + sbuf);
+            const uint32_t* lut = reinterpret_cast<const uint32_t*>(cx.smem + e.lut_off);
+            const int Cs = sn.C;
+            int iy0[2], ix0[2];
+#pragma unroll
+            for (int r = 0; r < 2; ++r) {
+                iy0[r] = oy[r] * e.stride - e.pad;
+                ix0[r] = ox[r] * e.stride - e.pad;
+            }
+            for (int ks = 0; ks < e.ksteps; ++ks) {
+                uint32_t a[4];
+#pragma unroll
+                for (int h = 0; h < 2; ++h) {
+                    const uint2 L = *reinterpret_cast<const uint2*>(lut + ks * 16 + h * 8 + 2 * tq);
+#pragma unroll
+                    for (int r = 0; r < 2; ++r) {
+                        uint32_t v[2];
+#pragma unroll
+                        for (int z = 0; z < 2; ++z) {
+                            const uint32_t t = z ? L.y : L.x;
+                            const int iy = iy0[r] + (int)(t & 15u), ix = ix0[r] + (int)((t >> 4) & 15u);
+                            const bool ok = pv[r] && (t >> 31) && iy >= sn.slo && iy < sn.shi && ix >= 0 && ix < Ws;
+                            v[z] = ok ? (uint32_t)src[((iy - sn.slo) * Ws + ix) * Cs + (int)((t >> 8) & 255u)] : 0u;
+                        }
+                        a[h * 2 + r] = v[0] | (v[1] << 16);
+                    }
+                }
+                uint32_t b0[4], b1[4];
+                rs_ldsm4(b0, waddr);
+                rs_ldsm4(b1, waddr + 512);
+                rs_mma(acc[0], a, b0[0], b0[1]);
+                rs_mma(acc[1], a, b0[2], b0[3]);
+                rs_mma(acc[2], a, b1[0], b1[1]);
+                rs_mma(acc[3], a, b1[2], b1[3]);
+                waddr += wstride;
+            }
+            (void)Hs;
+        }
+    }
+    // epilogue.  Column c of n-tile nt holds output channel n0 + (c >> 1) * 8 + nt * 2 + (c & 1) (the host packs
+    // the weights that way), so this lane's eight accumulator columns are the consecutive channels
+    // n0 + tq * 8 .. + 7: one 16-byte chunk per pixel.
+    const float* bias = reinterpret_cast<const float*>(cx.smem + nd.bias_off) + n0 + tq * 8;
+    const float4 bl = *reinterpret_cast<const float4*>(bias), bh = *reinterpret_cast<const float4*>(bias + 4);
+    const float bb[8] = {bl.x, bl.y, bl.z, bl.w, bh.x, bh.y, bh.z, bh.w};
+    const uint32_t nchd = (uint32_t)(nd.C >> 3), ch = (uint32_t)((n0 >> 3) + tq);
+    const uint32_t dbuf = (uint32_t)nd.buf[(f + 1) & 1];
+    const bool relu = nd.act == 1;
+#pragma unroll
+    for (int r = 0; r < 2; ++r) {
+        if (!pv[r]) continue;
+        const int y = oy[r], x = ox[r];
+        uint32_t pk[4];
+#pragma unroll
+        for (int nt = 0; nt < 4; ++nt) {
+            float v0 = acc[nt][2 * r] + bb[2 * nt], v1 = acc[nt][2 * r + 1] + bb[2 * nt + 1];
+            if (relu) {
+                v0 = fmaxf(v0, 0.f);
+                v1 = fmaxf(v1, 0.f);
+            }
+            pk[nt] = rs_pack_bf16(v0, v1);
+        }
+        const uint32_t off = rs_swz((uint32_t)((y - nd.slo) * W + x) * nchd + ch) * 16u;
+        if (off < (uint32_t)nd.buf_bytes) *reinterpret_cast<uint4*>(cx.smem + dbuf + off) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
+        if (cx.rank > 0 && y >= nd.up_lo && y < nd.up_hi) {
+            const uint32_t o2 = rs_swz((uint32_t)((y - nd.up_slo) * W + x) * nchd + ch) * 16u;
+            if (o2 < (uint32_t)nd.buf_bytes) rs_st_cluster_v4(rs_mapa(cx.sbase + dbuf + o2, cx.rank - 1), pk);
+        }
+        if ((int)cx.rank + 1 < cx.cs && y >= nd.dn_lo && y < nd.dn_hi) {
+            const uint32_t o2 = rs_swz((uint32_t)((y - nd.dn_slo) * W + x) * nchd + ch) * 16u;
+            if (o2 < (uint32_t)nd.buf_bytes) rs_st_cluster_v4(rs_mapa(cx.sbase + dbuf + o2, cx.rank + 1), pk);
+        }
+    }
+}
+
+__device__ __forceinline__ void rs_unpack8(const uint4& q, float (&v)[8])
+{
+    v[0] = __uint_as_float(q.x << 16); v[1] = __uint_as_float(q.x & 0xFFFF0000u);
+    v[2] = __uint_as_float(q.y << 16); v[3] = __uint_as_float(q.y & 0xFFFF0000u);
+    v[4] = __uint_as_float(q.z << 16); v[5] = __uint_as_float(q.z & 0xFFFF0000u);
+    v[6] = __uint_as_float(q.w << 16); v[7] = __uint_as_float(q.w & 0xFFFF0000u);
+}
+
+// A slice of a dense / mean-dense edge: this warp's partial dot products of the 16-byte chunks
+// [c_begin, c_end) of the CTA's part of the source with the matching weight columns, for every output,
+// written to slot `slot` of the target node in every CTA of the cluster.
+__device__ __forceinline__ void rs_dense_unit(const RsCtx& cx, const RsNode& nd, const RsEdge& e, int c_begin, int c_end,
+                                              int slot, int f)
+{
+    const int lane = cx.lane;
+    const RsNode& sn = cx.nodes[e.src];
+    const int fb = f + 1 - e.R;
+    const unsigned char* xb = cx.smem + sn.buf[fb & 1];
+    const bool swz = sn.kind == RS_CONV;
+    const char* wb = e.wd_off >= 0 ? reinterpret_cast<const char*>(cx.smem + e.wd_off) : e.wd_global;
+    const long long ld = e.wd_off >= 0 ? (long long)e.wd_ld : (long long)e.wd_gld;
+    const uint32_t slot_base = (uint32_t)nd.slot_off + (uint32_t)((((f + 1) & 1) * nd.n_slots + slot) * nd.C) * 4u;
+    for (int ob = 0; ob < nd.C; ob += 8) {
+        float acc[8];
+#pragma unroll
+        for (int j = 0; j < 8; ++j) acc[j] = 0.f;
+        for (int cl = c_begin + lane; cl < c_end; cl += 32) {
+            const uint32_t q = (uint32_t)(e.x_chunk0 + cl);
+            const uint4 xq = *reinterpret_cast<const uint4*>(xb + (swz ? rs_swz(q) : q) * 16u);
+            float x[8];
+            rs_unpack8(xq, x);
+            const int wc = e.wchunk_mod ? cl % e.wchunk_mod : cl;
+#pragma unroll
+            for (int j = 0; j < 8; ++j) {
+                if (ob + j < nd.C) {
+                    const uint4 wq = *reinterpret_cast<const uint4*>(wb + ((long long)(ob + j) * ld + (long long)wc * 8) * 2);
+                    float w[8];
+                    rs_unpack8(wq, w);
+#pragma unroll
+                    for (int i = 0; i < 8; ++i) acc[j] = fmaf(w[i], x[i], acc[j]);
+                }
+            }
+        }
+#pragma unroll
+        for (int j = 0; j < 8; ++j) {
+#pragma unroll
+            for (int s = 16; s >= 1; s >>= 1) acc[j] += __shfl_xor_sync(0xffffffffu, acc[j], s);
+        }
+        if (lane < 8 && ob + lane < nd.C) {
+            float v = 0.f;
+#pragma unroll
+            for (int j = 0; j < 8; ++j)
+                if (j == lane) v = acc[j];
+            v *= e.scale;
+            const uint32_t a = cx.sbase + slot_base + (uint32_t)(ob + lane) * 4u;
+            if (cx.cs > 1) {
+                for (int r = 0; r < cx.cs; ++r) rs_st_cluster_u32(rs_mapa(a, (uint32_t)r), __float_as_uint(v));
+            } else {
+                *reinterpret_cast<float*>(cx.smem + slot_base + (uint32_t)(ob + lane) * 4u) = v;
+            }
+        }
+    }
+}
+
+__global__ void __launch_bounds__(kRsMaxThreads, 1)
+sr_resident_kernel(const unsigned char* __restrict__ blobs, int blob_stride, const SrFrameCtl* __restrict__ ctl, int T, int cs)
+{
+    extern __shared__ __align__(1024) unsigned char smem[];
+    const int tid = threadIdx.x, nthr = blockDim.x;
+    const uint32_t rank = cs > 1 ? rs_cluster_rank() : 0u;
+    const int b = blockIdx.x / cs;                                    // the sequence this cluster rolls out
+    {
+        const uint4* src = reinterpret_cast<const uint4*>(blobs + (size_t)rank * blob_stride);
+        const int n16 = reinterpret_cast<const RsHeader*>(src)->blob_bytes >> 4;
+        for (int i = tid; i < n16; i += nthr) reinterpret_cast<uint4*>(smem)[i] = src[i];
+    }
+    __syncthreads();
+    RsCtx cx;
+    cx.smem = smem;
+    cx.sbase = rs_smem_u32(smem);
+    cx.H = reinterpret_cast<const RsHeader*>(smem);
+    cx.nodes = reinterpret_cast<const RsNode*>(smem + cx.H->off_nodes);
+    cx.edges = reinterpret_cast<const RsEdge*>(smem + cx.H->off_edges);
+    cx.rank = rank;
+    cx.cs = cs;
+    cx.lane = tid & 31;
+    const RsHeader& H = *cx.H;
+    const RsUnit* units = reinterpret_cast<const RsUnit*>(smem + H.off_units);
+    const int32_t* ubegin = reinterpret_cast<const int32_t*>(smem + H.off_ubegin);
+    const int warp = tid >> 5;
+    if (tid < 32) reinterpret_cast<uint32_t*>(smem + H.zero_off)[tid] = 0u;
+    // parameters: packed convolution weights, dense weight slices, biases
+    {
+        const RsCopy* cp = reinterpret_cast<const RsCopy*>(smem + H.off_copies);
+        for (int c = 0; c < H.n_copies; ++c)
+            for (int i = tid * 16; i < cp[c].bytes; i += nthr * 16) rs_cp_async16(cx.sbase + cp[c].dst + i, cp[c].src + i);
+    }
+    // frame t of every node (relative frame 0), and the first input frame of the run (relative frame 1)
+    const long long t0 = ctl->t, run0 = ctl->run_t;
+    const int par0 = (int)(t0 & 1);
+    for (int v = 0; v < H.n_nodes; ++v) {
+        const RsNode& nd = cx.nodes[v];
+        if (nd.kind == RS_DENSE) {
+            const uint16_t* g = reinterpret_cast<const uint16_t*>(nd.gstate[par0]) + (size_t)b * nd.C;
+            for (int i = tid; i < nd.C; i += nthr) reinterpret_cast<uint16_t*>(smem + nd.buf[0])[i] = g[i];
+        } else if (nd.kind == RS_CONV) {
+            const int nq = (nd.shi - nd.slo) * nd.W * (nd.C >> 3);
+            const char* g = nd.gstate[par0] + ((size_t)b * nd.H + nd.slo) * nd.W * nd.C * 2;
+            for (int q = tid; q < nq; q += nthr) rs_cp_async16(cx.sbase + nd.buf[0] + rs_swz((uint32_t)q) * 16u, g + (size_t)q * 16);
+        } else {
+            const int nw = (nd.shi - nd.slo) * nd.W * nd.C / 2;       // 4-byte words (W * C is even)
+            const size_t row0 = ((size_t)b * nd.H + nd.slo) * nd.W * nd.C * 2;
+            const char* g0 = nd.gstate[par0] + row0;
+            const char* g1 = static_cast<const char*>(ctl->in_base[nd.input_slot]) + run0 * ctl->in_stride_bytes[nd.input_slot] + row0;
+            for (int i = tid; i < nw; i += nthr) {
+                rs_cp_async4(cx.sbase + nd.buf[0] + i * 4, g0 + (size_t)i * 4);
+                rs_cp_async4(cx.sbase + nd.buf[1] + i * 4, g1 + (size_t)i * 4);
+            }
+        }
+    }
+    rs_cp_async_wait_all();
+    rs_level_barrier(cs);             // also: every CTA of the cluster runs before any remote store is issued
+
+    for (int f = 0; f < T; ++f) {
+        // input frame of the NEXT update, fetched while this one computes
+        if (f + 1 < T) {
+            for (int v = 0; v < H.n_nodes; ++v) {
+                const RsNode& nd = cx.nodes[v];
+                if (nd.kind != RS_INPUT) continue;
+                const int nw = (nd.shi - nd.slo) * nd.W * nd.C / 2;
+                const char* g = static_cast<const char*>(ctl->in_base[nd.input_slot]) +
+                                (run0 + f + 1) * ctl->in_stride_bytes[nd.input_slot] + ((size_t)b * nd.H + nd.slo) * nd.W * nd.C * 2;
+                const uint32_t dst = cx.sbase + nd.buf[(f + 2) % 3];
+                for (int i = tid; i < nw; i += nthr) rs_cp_async4(dst + i * 4, g + (size_t)i * 4);
+            }
+        }
+        for (int l = 0; l < H.n_levels; ++l) {
+            const int ub = ubegin[l * H.n_warps + warp], ue = ubegin[l * H.n_warps + warp + 1];
+            for (int u = ub; u < ue; ++u) {
+                const RsUnit& un = units[u];
+                const RsNode& nd = cx.nodes[un.node];
+                if (un.kind == RS_U_CONV) rs_conv_unit(cx, nd, un.a, un.b, f);
+                else rs_dense_unit(cx, nd, cx.edges[un.a], un.b, un.c, un.d, f);
+            }
+            if (l == H.n_levels - 1) rs_cp_async_wait_all();
+            rs_level_barrier(cs);
+            if ((H.dense_level_mask >> l) & 1) {
+                // dense nodes of this level: fixed-order sum of the slots, bias, activation
+                for (int v = 0; v < H.n_nodes; ++v) {
+                    const RsNode& nd = cx.nodes[v];
+                    if (nd.kind != RS_DENSE || nd.level != l) continue;
+                    const float* slots = reinterpret_cast<const float*>(smem + nd.slot_off) + ((f + 1) & 1) * nd.n_slots * nd.C;
+                    const float* bias = reinterpret_cast<const float*>(smem + nd.bias_off);
+                    for (int o = tid; o < nd.C; o += nthr) {
+                        float z = 0.f;
+                        for (int s = 0; s < nd.n_slots; ++s) z += slots[s * nd.C + o];
+                        z += bias[o];
+                        if (nd.act == 1) z = fmaxf(z, 0.f);
+                        reinterpret_cast<__nv_bfloat16*>(smem + nd.buf[(f + 1) & 1])[o] = __float2bfloat16_rn(z);
+                        if (nd.is_output && rank == 0 && ctl->out_base)
+                            ctl->out_base[(run0 + f) * ctl->out_stride + (long long)b * nd.C + o] = z;
+                    }
+                }
+                if (H.sync_after_finalize) __syncthreads();
+            }
+        }
+    }
+
+    // relative frame T back to the state buffers in global memory (parity of t + T)
+    const int parT = (int)((t0 + T) & 1);
+    for (int v = 0; v < H.n_nodes; ++v) {
+        const RsNode& nd = cx.nodes[v];
+        if (nd.kind == RS_DENSE) {
+            if (rank == 0) {
+                uint16_t* g = reinterpret_cast<uint16_t*>(nd.gstate[parT]) + (size_t)b * nd.C;
+                for (int i = tid; i < nd.C; i += nthr) g[i] = reinterpret_cast<const uint16_t*>(smem + nd.buf[T & 1])[i];
+            }
+        } else if (nd.kind == RS_CONV) {
+            const int nch = nd.C >> 3, nq = (nd.hi - nd.lo) * nd.W * nch, q0 = (nd.lo - nd.slo) * nd.W * nch;
+            char* g = nd.gstate[parT] + ((size_t)b * nd.H + nd.lo) * nd.W * nd.C * 2;
+            for (int q = tid; q < nq; q += nthr)
+                *reinterpret_cast<uint4*>(g + (size_t)q * 16) =
+                    *reinterpret_cast<const uint4*>(smem + nd.buf[T & 1] + rs_swz((uint32_t)(q + q0)) * 16u);
+        } else {
+            const int nw = (nd.hi - nd.lo) * nd.W * nd.C / 2, w0 = (nd.lo - nd.slo) * nd.W * nd.C / 2;
+            char* g = nd.gstate[parT] + ((size_t)b * nd.H + nd.lo) * nd.W * nd.C * 2;
+            for (int i = tid; i < nw; i += nthr)
+                reinterpret_cast<uint32_t*>(g)[i] = reinterpret_cast<const uint32_t*>(smem + nd.buf[T % 3])[w0 + i];
+        }
+    }
+}
+
+// ------------------------------------------------------------------------------------------------ host side
+struct RsPlanNode {
+    int kind = RS_INPUT;
+    int lo[kRsMaxCluster + 1] = {0}, slo[kRsMaxCluster] = {0}, shi[kRsMaxCluster] = {0};
+    int buf[3] = {0, 0, 0}, buf_bytes = 0, bias_off = 0, w_off = 0, slot_off = 0, n_slots = 0, pix_off = 0, pix_entries = 0;
+    int first_edge = 0, ksteps = 0;
+    size_t w_global = 0;            // byte offset of the packed weights inside the convolution-weight region
+    bool has_consumers = false;
+};
+
+struct RsPlanEdge {
+    int host_edge = -1, type = RS_E_MMA, ksteps = 0, ks0 = 0, lut_off = 0, Kreal = 0;
+    size_t wd_global = 0;           // dense: byte offset inside the dense-weight region
+    int wd_off[kRsMaxCluster] = {-1, -1, -1, -1};
+};
+
+struct RsEngine {
+    int cs = 1, warps = 16, smem_bytes = 0, blob_bytes = 0, n_levels = 1;
+    std::vector<RsPlanNode> pn;
+    std::vector<RsPlanEdge> pe;                 // ordered by target node, then by the node's in-edge order
+    std::vector<int> pe_of_host_edge;
+    std::vector<std::vector<RsUnit>> units;     // per rank, sorted by (level, warp)
+    std::vector<std::vector<int>> ubegin;       // per rank
+    std::vector<std::vector<uint32_t>> luts;    // per plan edge (gather edges only)
+    int zero_off = 0;
+    bool dense_in_smem = false;
+    SrRegion r_blobs, r_wconv, r_wdense;
+    bool attr_set = false;
+};
+
+int rs_row_lo(int H, int r, int cs) { return (H * r + cs / 2) / cs; }
+int rs_up16(int x) { return (x + 15) / 16 * 16; }
+int rs_up128(int x) { return (x + 127) / 128 * 128; }
+
+// Lays the engine out for a cluster of `cs` CTAs; false if the network does not fit.
+bool rs_layout(const sr_graph* g, RsEngine& E, int cs, int warps)
+{
+    const int n_nodes = (int)g->nodes.size();
+    E.cs = cs;
+    E.warps = warps;
+    E.n_levels = (int)g->groups.size();
+    // row ownership and stored ranges
+    for (int v = 0; v < n_nodes; ++v) {
+        RsPlanNode& p = E.pn[v];
+        const sr_node_desc& d = g->nodes[v].d;
+        if (p.kind == RS_DENSE) {
+            for (int r = 0; r <= cs; ++r) p.lo[r] = r == 0 ? 0 : 1;
+            for (int r = 0; r < cs; ++r) {
+                p.slo[r] = 0;
+                p.shi[r] = 1;
+            }
+            continue;
+        }
+        if (d.h < cs) return false;
+        for (int r = 0; r <= cs; ++r) p.lo[r] = rs_row_lo(d.h, r, cs);
+        for (int r = 0; r < cs; ++r) {
+            p.slo[r] = p.lo[r];
+            p.shi[r] = p.lo[r + 1];
+        }
+    }
+    for (const RsPlanEdge& pe : E.pe) {
+        const SrHostEdge& he = g->edges[pe.host_edge];
+        if (he.d.kind != SR_EDGE_CONV) continue;
+        RsPlanNode& s = E.pn[he.d.src];
+        const RsPlanNode& t = E.pn[he.d.tgt];
+        const int Hs = g->nodes[he.d.src].d.h;
+        for (int r = 0; r < cs; ++r) {
+            const int clo = t.lo[r], chi = t.lo[r + 1];
+            if (chi <= clo) continue;
+            const int need_lo = std::max(0, he.stride_eff * clo - he.pad_eff);
+            const int need_hi = std::min(Hs, he.stride_eff * (chi - 1) - he.pad_eff + he.k_eff);
+            s.slo[r] = std::min(s.slo[r], need_lo);
+            s.shi[r] = std::max(s.shi[r], need_hi);
+        }
+    }
+    // a halo row must belong to a direct neighbour (its owner mirrors it there)
+    for (int v = 0; v < n_nodes; ++v) {
+        const RsPlanNode& p = E.pn[v];
+        if (p.kind == RS_DENSE) continue;
+        for (int r = 0; r < cs; ++r) {
+            if (r > 0 && p.slo[r] < p.lo[r - 1]) return false;
+            if (r + 1 < cs && p.shi[r] > p.lo[r + 2]) return false;
+        }
+    }
+    // units per rank
+    E.units.assign(cs, std::vector<RsUnit>());
+    E.ubegin.assign(cs, std::vector<int>());
+    std::vector<int> slot_count(n_nodes, 0);
+    struct Cand { RsUnit u; int level; long cost; };
+    std::vector<std::vector<Cand>> cand(cs);
+    for (int v = 0; v < n_nodes; ++v) {
+        const RsPlanNode& p = E.pn[v];
+        const SrHostNode& hn = g->nodes[v];
+        if (p.kind == RS_INPUT) continue;
+        const int level = hn.level - 1;
+        if (p.kind == RS_CONV) {
+            long cost = 80;                       // estimated warp instructions of a unit
+            for (int ei = 0; ei < (int)hn.in_edges.size(); ++ei) {
+                const RsPlanEdge& pe = E.pe[p.first_edge + ei];
+                const SrHostEdge& he = g->edges[pe.host_edge];
+                if (pe.type == RS_E_MMA) cost += (long)he.k_eff * he.k_eff * 12 + (long)pe.ksteps * 8;
+                else cost += (long)pe.ksteps * 90;
+            }
+            for (int r = 0; r < cs; ++r) {
+                const int npix = (p.lo[r + 1] - p.lo[r]) * hn.d.w;
+                for (int j0 = 0; j0 < npix; j0 += 16)
+                    for (int n0 = 0; n0 < hn.d.c; n0 += 32) cand[r].push_back(Cand{RsUnit{RS_U_CONV, v, j0, n0, 0, 0}, level, cost});
+            }
+        } else {
+            for (int ei = 0; ei < (int)hn.in_edges.size(); ++ei) {
+                const SrHostEdge& he = g->edges[hn.in_edges[ei]];
+                const RsPlanNode& sp = E.pn[he.d.src];
+                const sr_node_desc& sd = g->nodes[he.d.src].d;
+                for (int r = 0; r < cs; ++r) {
+                    int n = 0;
+                    if (sp.kind == RS_CONV) n = (sp.lo[r + 1] - sp.lo[r]) * sd.w * (sd.c / 8);
+                    else if (r == 0) n = sd.c / 8;
+                    if (n == 0) continue;
+                    const int parts = (n + kRsDenseUnitChunks - 1) / kRsDenseUnitChunks;
+                    const int per = (n + parts - 1) / parts;
+                    for (int c0 = 0; c0 < n; c0 += per) {
+                        const int c1 = std::min(n, c0 + per);
+                        const long ob = (hn.d.c + 7) / 8;
+                        const long cost = 30 + ob * ((long)((c1 - c0 + 31) / 32) * 150 + 50);
+                        cand[r].push_back(Cand{RsUnit{RS_U_DENSE, v, p.first_edge + ei, c0, c1, slot_count[v]++}, level, cost});
+                    }
+                }
+            }
+        }
+    }
+    for (int v = 0; v < n_nodes; ++v) E.pn[v].n_slots = slot_count[v];
+    for (int r = 0; r < cs; ++r) {
+        // longest-processing-time-first: level by level, to the least loaded scheduler partition
+        // (warp id mod 4), then to its least loaded warp
+        std::vector<std::vector<std::vector<RsUnit>>> lists(E.n_levels, std::vector<std::vector<RsUnit>>(warps));
+        for (int l = 0; l < E.n_levels; ++l) {
+            std::vector<Cand> cs_l;
+            for (const Cand& c : cand[r])
+                if (c.level == l) cs_l.push_back(c);
+            std::stable_sort(cs_l.begin(), cs_l.end(), [](const Cand& a, const Cand& b) { return a.cost > b.cost; });
+            std::vector<long> wl(warps, 0), pl(4, 0);
+            for (const Cand& c : cs_l) {
+                int bp = 0;
+                for (int p = 1; p < std::min(4, warps); ++p)
+                    if (pl[p] < pl[bp]) bp = p;
+                int bw = bp;
+                for (int w = bp; w < warps; w += 4)
+                    if (wl[w] < wl[bw]) bw = w;
+                wl[bw] += c.cost;
+                pl[bp] += c.cost;
+                lists[l][bw].push_back(c.u);
+            }
+        }
+        for (int l = 0; l < E.n_levels; ++l)
+            for (int w = 0; w < warps; ++w) {
+                E.ubegin[r].push_back((int)E.units[r].size());
+                for (const RsUnit& u : lists[l][w]) E.units[r].push_back(u);
+            }
+        E.ubegin[r].push_back((int)E.units[r].size());
+    }
+    // tables
+    size_t max_units = 0;
+    for (int r = 0; r < cs; ++r) max_units = std::max(max_units, E.units[r].size());
+    int off = (int)sizeof(RsHeader);
+    auto take = [&](int bytes, int align) {
+        off = (off + align - 1) / align * align;
+        const int o = off;
+        off += bytes;
+        return o;
+    };
+    const int off_nodes = take((int)sizeof(RsNode) * n_nodes, 16);
+    const int off_edges = take((int)sizeof(RsEdge) * (int)E.pe.size(), 16);
+    const int off_units = take((int)(sizeof(RsUnit) * std::max<size_t>(1, max_units)), 16);
+    const int off_ubegin = take((int)sizeof(int32_t) * (E.n_levels * warps + 1), 16);
+    int n_copies = 0;
+    for (int v = 0; v < n_nodes; ++v)
+        if (E.pn[v].kind != RS_INPUT) n_copies += 1 + (E.pn[v].kind == RS_CONV ? 1 : 0);
+    int dense_rows = 0;
+    for (const RsPlanEdge& pe : E.pe) {
+        const SrHostEdge& he = g->edges[pe.host_edge];
+        if (he.d.kind != SR_EDGE_CONV) dense_rows += g->nodes[he.d.tgt].d.c;
+    }
+    const int off_copies = take((int)sizeof(RsCopy) * (n_copies + dense_rows), 16);
+    for (size_t i = 0; i < E.pe.size(); ++i)
+        if (E.pe[i].type == RS_E_GATHER) E.pe[i].lut_off = take((int)E.luts[i].size() * 4, 16);
+    for (int v = 0; v < n_nodes; ++v) {
+        RsPlanNode& p = E.pn[v];
+        if (p.kind != RS_CONV) continue;
+        int npix = 0;
+        for (int r = 0; r < cs; ++r) npix = std::max(npix, (p.lo[r + 1] - p.lo[r]) * g->nodes[v].d.w);
+        p.pix_entries = (npix + 15) / 16 * 16;
+        p.pix_off = take(p.pix_entries * 4, 16);
+    }
+    E.blob_bytes = rs_up16(off);
+    off = E.blob_bytes;
+    E.zero_off = take(128, 128);
+    for (int v = 0; v < n_nodes; ++v) {
+        RsPlanNode& p = E.pn[v];
+        const sr_node_desc& d = g->nodes[v].d;
+        if (p.kind != RS_INPUT) p.bias_off = take(rs_up16(d.c * 4), 16);
+        if (p.kind == RS_DENSE) p.slot_off = take(2 * std::max(1, p.n_slots) * d.c * 4, 16);
+    }
+    for (int v = 0; v < n_nodes; ++v) {
+        RsPlanNode& p = E.pn[v];
+        const sr_node_desc& d = g->nodes[v].d;
+        int rows = 0;
+        for (int r = 0; r < cs; ++r) rows = std::max(rows, p.shi[r] - p.slo[r]);
+        if (p.kind == RS_DENSE) p.buf_bytes = rs_up16(d.c * 2);
+        else if (p.kind == RS_INPUT) p.buf_bytes = rs_up16(rows * d.w * d.c * 2);
+        else p.buf_bytes = rs_up128(rows * d.w * d.c * 2);
+        const int nb = p.kind == RS_INPUT ? 3 : 2;
+        for (int i = 0; i < nb; ++i) p.buf[i] = take(p.buf_bytes, 128);
+    }
+    for (int v = 0; v < n_nodes; ++v) {
+        RsPlanNode& p = E.pn[v];
+        if (p.kind == RS_CONV) p.w_off = take(p.ksteps * (g->nodes[v].d.c / 32) * 1024, 128);
+    }
+    if (off > kRsSmemMax) return false;
+    // dense weights in shared memory if every slice fits, else they are read from global memory (L2)
+    const int before_dense = off;
+    E.dense_in_smem = true;
+    for (RsPlanEdge& pe : E.pe) {
+        const SrHostEdge& he = g->edges[pe.host_edge];
+        if (he.d.kind == SR_EDGE_CONV) continue;
+        const RsPlanNode& sp = E.pn[he.d.src];
+        const sr_node_desc& sd = g->nodes[he.d.src].d;
+        const int Cout = g->nodes[he.d.tgt].d.c;
+        int max_slice = 0;
+        for (int r = 0; r < cs; ++r) {
+            int n = 0;
+            if (he.d.kind == SR_EDGE_MEAN_DENSE) n = sd.c;
+            else if (sp.kind == RS_CONV) n = (sp.lo[r + 1] - sp.lo[r]) * sd.w * sd.c;
+            else n = r == 0 ? sd.c : 0;
+            max_slice = std::max(max_slice, n);
+        }
+        const int o = take(Cout * max_slice * 2, 16);
+        for (int r = 0; r < cs; ++r) pe.wd_off[r] = o;
+    }
+    if (off > kRsSmemMax) {
+        off = before_dense;
+        E.dense_in_smem = false;
+        for (RsPlanEdge& pe : E.pe)
+            for (int r = 0; r < kRsMaxCluster; ++r) pe.wd_off[r] = -1;
+    }
+    E.smem_bytes = rs_up128(off);
+    (void)off_nodes; (void)off_edges; (void)off_units; (void)off_ubegin; (void)off_copies;   // see rs_table_offsets
+    return true;
+}
+
+struct RsOffsets { int nodes, edges, units, ubegin, copies; };
+
+RsOffsets rs_table_offsets(const sr_graph* g, const RsEngine& E)
+{
+    size_t max_units = 0;
+    for (int r = 0; r < E.cs; ++r) max_units = std::max(max_units, E.units[r].size());
+    int off = (int)sizeof(RsHeader);
+    auto take = [&](int bytes, int align) {
+        off = (off + align - 1) / align * align;
+        const int o = off;
+        off += bytes;
+        return o;
+    };
+    RsOffsets o;
+    o.nodes = take((int)sizeof(RsNode) * (int)g->nodes.size(), 16);
+    o.edges = take((int)sizeof(RsEdge) * (int)E.pe.size(), 16);
+    o.units = take((int)(sizeof(RsUnit) * std::max<size_t>(1, max_units)), 16);
+    o.ubegin = take((int)sizeof(int32_t) * (E.n_levels * E.warps + 1), 16);
+    o.copies = take(0, 16);
+    return o;
+}
+
+RsEngine* rs_of(const sr_graph* g) { return static_cast<RsEngine*>(g->rs); }
+
+}  // namespace
+
+void sr_rs_destroy(sr_graph* g)
+{
+    delete rs_of(g);
+    g->rs = nullptr;
+}
+
+bool sr_rs_available(const sr_graph* g) { return g->rs != nullptr; }
+
+void sr_rs_describe(const sr_graph* g, int* cluster_size, int* warps, int* smem_bytes)
+{
+    const RsEngine* E = rs_of(g);
+    *cluster_size = E ? E->cs : 0;
+    *warps = E ? E->warps : 0;
+    *smem_bytes = E ? E->smem_bytes : 0;
+}
+
+sr_status sr_rs_plan(sr_graph* g, size_t& offset)
+{
+    sr_rs_destroy(g);
+    if (!g->opt_resident || g->opt_engine != 0 || g->dtype != SR_DTYPE_BF16) return SR_OK;
+    const int n_nodes = (int)g->nodes.size(), n_edges = (int)g->edges.size();
+    if (n_nodes > 32 || n_edges > 64 || g->groups.size() > 30 || g->groups.empty()) return SR_OK;
+    if ((int)g->input_nodes.size() > SR_MAX_INPUTS) return SR_OK;
+    RsEngine* E = new RsEngine();
+    E->pn.assign(n_nodes, RsPlanNode());
+    E->pe_of_host_edge.assign(n_edges, -1);
+    bool ok = true;
+    // node kinds
+    for (int v = 0; v < n_nodes && ok; ++v) {
+        const SrHostNode& n = g->nodes[v];
+        RsPlanNode& p = E->pn[v];
+        if (n.is_input) {
+            p.kind = RS_INPUT;
+            if ((n.d.w * n.d.c) % 2 != 0) ok = false;
+        } else if (n.dense_target) {
+            p.kind = RS_DENSE;
+            if (n.d.c > kRsMaxDenseC) ok = false;
+        } else {
+            p.kind = RS_CONV;
+            if (n.d.c % 32 != 0 || n.d.c > 256) ok = false;
+        }
+    }
+    if (ok && E->pn[g->info.output_node].kind != RS_DENSE) ok = false;
+    // edges, grouped by target
+    for (int v = 0; v < n_nodes && ok; ++v) {
+        const SrHostNode& n = g->nodes[v];
+        RsPlanNode& p = E->pn[v];
+        p.first_edge = (int)E->pe.size();
+        int ks = 0;
+        for (int e : n.in_edges) {
+            const SrHostEdge& he = g->edges[e];
+            const RsPlanNode& sp = E->pn[he.d.src];
+            const sr_node_desc& sd = g->nodes[he.d.src].d;
+            RsPlanEdge pe;
+            pe.host_edge = e;
+            if (he.d.kind == SR_EDGE_CONV) {
+                if (p.kind != RS_CONV || sp.kind == RS_DENSE || he.k_eff > 15) ok = false;
+                if (sp.kind == RS_CONV) {
+                    pe.type = RS_E_MMA;
+                    pe.ksteps = he.k_eff * he.k_eff * (sd.c / 16);
+                } else {
+                    // input nodes are stored unswizzled and read by the table-driven path
+                    pe.type = RS_E_GATHER;
+                    pe.Kreal = he.k_eff * he.k_eff * sd.c;
+                    if (pe.Kreal > 64 || sd.c > 255) ok = false;
+                    pe.ksteps = (pe.Kreal + 15) / 16;
+                }
+                pe.ks0 = ks;
+                ks += pe.ksteps;
+            } else {
+                if (p.kind != RS_DENSE || sp.kind == RS_INPUT || sd.c % 8 != 0) ok = false;
+                pe.type = he.d.kind == SR_EDGE_DENSE ? RS_E_DENSE : RS_E_MEAN;
+                if (sp.kind == RS_DENSE && pe.type == RS_E_MEAN) pe.type = RS_E_DENSE;   // mean over one pixel
+            }
+            E->pe_of_host_edge[e] = (int)E->pe.size();
+            E->pe.push_back(pe);
+            E->pn[he.d.src].has_consumers = true;
+        }
+        p.ksteps = ks;
+    }
+    if (!ok) {
+        delete E;
+        return SR_OK;
+    }
+    // lookup tables of the few-channel edges: (ky, kx, channel) of every k index, valid bit 31
+    E->luts.assign(E->pe.size(), std::vector<uint32_t>());
+    for (size_t i = 0; i < E->pe.size(); ++i) {
+        const RsPlanEdge& pe = E->pe[i];
+        if (pe.type != RS_E_GATHER) continue;
+        const SrHostEdge& he = g->edges[pe.host_edge];
+        const int Cs = g->nodes[he.d.src].d.c;
+        std::vector<uint32_t>& L = E->luts[i];
+        L.assign((size_t)pe.ksteps * 16, 0u);
+        for (int kk = 0; kk < pe.Kreal; ++kk) {
+            const int tap = kk / Cs, ci = kk % Cs;
+            L[kk] = (uint32_t)(tap / he.k_eff) | ((uint32_t)(tap % he.k_eff) << 4) | ((uint32_t)ci << 8) | 0x80000000u;
+        }
+    }
+    // cluster size: the largest that still gives every sequence its own cluster in one wave, else the
+    // smallest that fits
+    int sms = 148, dev = 0;
+    if (cudaGetDevice(&dev) == cudaSuccess) cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+    std::vector<int> order;
+    if (g->opt_rs_cluster > 0) {
+        order.push_back(g->opt_rs_cluster);
+    } else {
+        for (int c = kRsMaxCluster; c >= 1; c >>= 1)
+            if (g->batch * c <= sms) order.push_back(c);
+        for (int c = 1; c <= kRsMaxCluster; c <<= 1)
+            if (g->batch * c > sms) order.push_back(c);
+    }
+    const int warps = g->opt_rs_warps > 0 ? g->opt_rs_warps : 16;
+    bool placed = false;
+    for (int c : order)
+        if (rs_layout(g, *E, c, warps)) {
+            placed = true;
+            break;
+        }
+    if (!placed) {
+        delete E;
+        return SR_OK;
+    }
+    // workspace regions: per-rank tables, packed convolution weights, dense weights
+    auto take = [&](size_t bytes) {
+        SrRegion r;
+        r.offset = offset;
+        r.bytes = bytes;
+        offset = sr_align_up(offset + bytes, 256);
+        return r;
+    };
+    size_t wconv = 0, wdense = 0;
+    for (int v = 0; v < n_nodes; ++v) {
+        RsPlanNode& p = E->pn[v];
+        if (p.kind != RS_CONV) continue;
+        p.w_global = wconv;
+        wconv += (size_t)p.ksteps * (g->nodes[v].d.c / 32) * 1024;
+    }
+    for (RsPlanEdge& pe : E->pe) {
+        const SrHostEdge& he = g->edges[pe.host_edge];
+        if (he.d.kind == SR_EDGE_CONV) continue;
+        pe.wd_global = wdense;
+        wdense += sr_align_up((size_t)g->nodes[he.d.tgt].d.c * he.K * 2, 16);
+    }
+    E->r_blobs = take((size_t)E->cs * E->blob_bytes);
+    E->r_wconv = take(std::max<size_t>(16, wconv));
+    E->r_wdense = take(std::max<size_t>(16, wdense));
+    g->rs = E;
+    return SR_OK;
+}
+
+sr_status sr_rs_bind(sr_graph* g)
+{
+    RsEngine* Ep = rs_of(g);
+    if (!Ep) return SR_OK;
+    RsEngine& E = *Ep;
+    const int n_nodes = (int)g->nodes.size();
+    const RsOffsets O = rs_table_offsets(g, E);
+    for (int r = 0; r < E.cs; ++r) {
+        std::vector<unsigned char> blob((size_t)E.blob_bytes, 0);
+        RsHeader* H = reinterpret_cast<RsHeader*>(blob.data());
+        RsNode* nodes = reinterpret_cast<RsNode*>(blob.data() + O.nodes);
+        RsEdge* edges = reinterpret_cast<RsEdge*>(blob.data() + O.edges);
+        RsUnit* units = reinterpret_cast<RsUnit*>(blob.data() + O.units);
+        int32_t* ubegin = reinterpret_cast<int32_t*>(blob.data() + O.ubegin);
+        RsCopy* copies = reinterpret_cast<RsCopy*>(blob.data() + O.copies);
+        int n_copies = 0, dense_mask = 0, sync_after = 0;
+        for (int v = 0; v < n_nodes; ++v) {
+            const SrHostNode& hn = g->nodes[v];
+            const RsPlanNode& p = E.pn[v];
+            RsNode& d = nodes[v];
+            d.kind = p.kind;
+            d.H = hn.d.h; d.W = hn.d.w; d.C = hn.d.c; d.act = hn.d.act;
+            d.level = hn.level - 1;
+            d.lo = p.lo[r]; d.hi = p.lo[r + 1];
+            d.slo = p.slo[r]; d.shi = p.shi[r];
+            d.is_output = v == g->info.output_node;
+            d.input_slot = hn.input_slot;
+            for (int i = 0; i < 3; ++i) d.buf[i] = p.buf[i];
+            d.bias_off = p.bias_off;
+            d.w_off = p.w_off;
+            d.first_edge = p.first_edge;
+            d.n_edges = (int)hn.in_edges.size();
+            d.buf_bytes = p.buf_bytes;
+            d.up_lo = d.up_hi = d.up_slo = d.dn_lo = d.dn_hi = d.dn_slo = 0;
+            if (p.kind != RS_DENSE) {
+                if (r > 0) {
+                    d.up_lo = d.lo;
+                    d.up_hi = std::min(d.hi, p.shi[r - 1]);
+                    d.up_slo = p.slo[r - 1];
+                }
+                if (r + 1 < E.cs) {
+                    d.dn_lo = std::max(d.lo, p.slo[r + 1]);
+                    d.dn_hi = d.hi;
+                    d.dn_slo = p.slo[r + 1];
+                }
+            }
+            d.slot_off = p.slot_off;
+            d.n_slots = p.n_slots;
+            d.has_consumers = p.has_consumers;
+            d.pix_off = p.pix_off;
+            if (p.kind == RS_CONV) {
+                uint32_t* pix = reinterpret_cast<uint32_t*>(blob.data() + p.pix_off);
+                const int npix = (d.hi - d.lo) * d.W;
+                for (int j = 0; j < p.pix_entries; ++j)
+                    pix[j] = j < npix ? ((uint32_t)(d.lo + j / d.W) << 16) | (uint32_t)(j % d.W) : 0xFFFFFFFFu;
+            }
+            d.gstate[0] = g->ws + hn.state[0].offset;
+            d.gstate[1] = g->ws + hn.state[1].offset;
+            if (p.kind == RS_DENSE) {
+                dense_mask |= 1 << d.level;
+                if (p.has_consumers) sync_after = 1;
+            }
+            if (p.kind != RS_INPUT) copies[n_copies++] = RsCopy{g->ws + hn.bias.offset, p.bias_off, rs_up16(hn.d.c * 4)};
+            if (p.kind == RS_CONV)
+                copies[n_copies++] = RsCopy{g->ws + E.r_wconv.offset + p.w_global, p.w_off, p.ksteps * (hn.d.c / 32) * 1024};
+        }
+        for (size_t i = 0; i < E.pe.size(); ++i) {
+            const RsPlanEdge& pe = E.pe[i];
+            const SrHostEdge& he = g->edges[pe.host_edge];
+            const RsPlanNode& sp = E.pn[he.d.src];
+            const sr_node_desc& sd = g->nodes[he.d.src].d;
+            RsEdge& d = edges[i];
+            d.src = he.d.src;
+            d.type = pe.type;
+            d.k = he.k_eff; d.stride = he.stride_eff; d.pad = he.pad_eff;
+            d.R = he.R;
+            d.ksteps = pe.ksteps;
+            d.lut_off = pe.lut_off;
+            d.Kreal = pe.Kreal;
+            d.wd_off = -1; d.wd_ld = 0; d.n_chunks = 0; d.x_chunk0 = 0; d.wchunk_mod = 0;
+            d.scale = 1.f;
+            d.wd_global = nullptr;
+            d.wd_gld = 0;
+            if (pe.type == RS_E_GATHER)
+                std::memcpy(blob.data() + pe.lut_off, E.luts[i].data(), E.luts[i].size() * 4);
+            if (he.d.kind != SR_EDGE_CONV) {
+                const int Cout = g->nodes[he.d.tgt].d.c;
+                const int nch = sd.c / 8;
+                int k_begin = 0, k_len = 0;          // this rank's slice of the flattened source, in elements
+                if (sp.kind == RS_CONV) {
+                    k_begin = sp.lo[r] * sd.w * sd.c;
+                    k_len = (sp.lo[r + 1] - sp.lo[r]) * sd.w * sd.c;
+                    d.x_chunk0 = (sp.lo[r] - sp.slo[r]) * sd.w * nch;
+                } else if (r == 0) {
+                    k_len = sd.c;
+                }
+                d.n_chunks = k_len / 8;
+                const char* wg = g->ws + E.r_wdense.offset + pe.wd_global;
+                if (pe.type == RS_E_MEAN) {
+                    d.wchunk_mod = nch;
+                    d.scale = 1.f / (float)(sd.h * sd.w);
+                    d.wd_global = wg;
+                    d.wd_gld = sd.c;
+                    if (pe.wd_off[r] >= 0) {
+                        d.wd_off = pe.wd_off[r];
+                        d.wd_ld = sd.c;
+                        for (int o = 0; o < Cout; ++o)
+                            copies[n_copies++] = RsCopy{wg + (size_t)o * sd.c * 2, d.wd_off + o * sd.c * 2, sd.c * 2};
+                    }
+                } else {
+                    d.wd_global = wg + (size_t)k_begin * 2;
+                    d.wd_gld = he.K;
+                    if (pe.wd_off[r] >= 0 && k_len > 0) {
+                        d.wd_off = pe.wd_off[r];
+                        d.wd_ld = k_len;
+                        for (int o = 0; o < Cout; ++o)
+                            copies[n_copies++] =
+                                RsCopy{wg + ((size_t)o * he.K + k_begin) * 2, d.wd_off + o * k_len * 2, k_len * 2};
+                    }
+                }
+            }
+        }
+        std::memcpy(units, E.units[r].data(), sizeof(RsUnit) * E.units[r].size());
+        std::memcpy(ubegin, E.ubegin[r].data(), sizeof(int32_t) * E.ubegin[r].size());
+        H->n_nodes = n_nodes;
+        H->n_edges = (int)E.pe.size();
+        H->n_levels = E.n_levels;
+        H->n_warps = E.warps;
+        H->off_nodes = O.nodes; H->off_edges = O.edges; H->off_units = O.units; H->off_ubegin = O.ubegin;
+        H->off_copies = O.copies;
+        H->n_copies = n_copies;
+        H->zero_off = E.zero_off;
+        H->smem_bytes = E.smem_bytes;
+        H->dense_level_mask = dense_mask;
+        H->sync_after_finalize = sync_after;
+        H->blob_bytes = E.blob_bytes;
+        if (cudaMemcpy(g->ws + E.r_blobs.offset + (size_t)r * E.blob_bytes, blob.data(), blob.size(), cudaMemcpyHostToDevice) !=
+            cudaSuccess)
+            return SR_ERR_CUDA;
+    }
+    return SR_OK;
+}
+
+sr_status sr_rs_set_weights(sr_graph* g, int edge, const float* w_eff)
+{
+    RsEngine* Ep = rs_of(g);
+    if (!Ep) return SR_OK;
+    RsEngine& E = *Ep;
+    const RsPlanEdge& pe = E.pe[E.pe_of_host_edge[edge]];
+    const SrHostEdge& he = g->edges[edge];
+    const int Cout = g->nodes[he.d.tgt].d.c, Cs = g->nodes[he.d.src].d.c;
+    auto bf16 = [](float f) {
+        uint32_t u;
+        std::memcpy(&u, &f, 4);
+        if ((u & 0x7F800000u) != 0x7F800000u) u += 0x7FFFu + ((u >> 16) & 1u);
+        return (uint16_t)(u >> 16);
+    };
+    if (he.d.kind == SR_EDGE_CONV) {
+        // ldmatrix order: per k-step and 32 output channels two 512-byte blocks; lane l of a block holds 8
+        // consecutive k, starting at k = ((l >> 3) & 1) * 8, of column (l & 7) of n-tile hb * 2 + (l >> 4).
+        // Column c of n-tile nt is output channel (c >> 1) * 8 + nt * 2 + (c & 1) of the 32, which makes the
+        // eight accumulator columns of a lane consecutive channels
+        const int nb = Cout / 32, nc16 = Cs / 16;
+        std::vector<uint16_t> pk((size_t)pe.ksteps * nb * 512, 0);
+        for (int ks = 0; ks < pe.ksteps; ++ks)
+            for (int b = 0; b < nb; ++b)
+                for (int hb = 0; hb < 2; ++hb)
+                    for (int l = 0; l < 32; ++l) {
+                        const int nt = hb * 2 + (l >> 4), col = l & 7, kh = (l >> 3) & 1;
+                        const int n = b * 32 + (col >> 1) * 8 + nt * 2 + (col & 1);
+                        for (int j = 0; j < 8; ++j) {
+                            float w = 0.f;
+                            if (pe.type == RS_E_MMA) {
+                                const int tap = ks / nc16, c = (ks % nc16) * 16 + kh * 8 + j;
+                                w = w_eff[(size_t)n * he.K + (size_t)tap * Cs + c];
+                            } else {
+                                const int kk = ks * 16 + kh * 8 + j;
+                                if (kk < pe.Kreal) w = w_eff[(size_t)n * he.K + kk];
+                            }
+                            pk[(((size_t)ks * nb + b) * 2 + hb) * 256 + l * 8 + j] = bf16(w);
+                        }
+                    }
+        const RsPlanNode& p = E.pn[he.d.tgt];
+        char* dst = g->ws + E.r_wconv.offset + p.w_global + (size_t)pe.ks0 * nb * 1024;
+        if (cudaMemcpy(dst, pk.data(), pk.size() * 2, cudaMemcpyHostToDevice) != cudaSuccess) return SR_ERR_CUDA;
+    } else {
+        std::vector<uint16_t> pk((size_t)Cout * he.K);
+        for (size_t i = 0; i < pk.size(); ++i) pk[i] = bf16(w_eff[i]);
+        if (cudaMemcpy(g->ws + E.r_wdense.offset + pe.wd_global, pk.data(), pk.size() * 2, cudaMemcpyHostToDevice) != cudaSuccess)
+            return SR_ERR_CUDA;
+    }
+    return SR_OK;
+}
+
+sr_status sr_rs_launch(sr_graph* g, int T, cudaStream_t s)
+{
+    RsEngine* E = rs_of(g);
+    if (!E) return SR_ERR_STATE;
+    if (!E->attr_set) {
+        if (cudaFuncSetAttribute(sr_resident_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, E->smem_bytes) != cudaSuccess)
+            return SR_ERR_CUDA;
+        E->attr_set = true;
+    }
+    cudaLaunchConfig_t cfg{};
+    cfg.gridDim = dim3((unsigned)(g->batch * E->cs));
+    cfg.blockDim = dim3((unsigned)(E->warps * 32));
+    cfg.dynamicSmemBytes = (size_t)E->smem_bytes;
+    cfg.stream = s;
+    cudaLaunchAttribute at[1];
+    at[0].id = cudaLaunchAttributeClusterDimension;
+    at[0].val.clusterDim.x = (unsigned)E->cs;
+    at[0].val.clusterDim.y = 1;
+    at[0].val.clusterDim.z = 1;
+    cfg.attrs = at;
+    cfg.numAttrs = E->cs > 1 ? 1 : 0;
+    const unsigned char* blobs = reinterpret_cast<const unsigned char*>(g->ws + E->r_blobs.offset);
+    const SrFrameCtl* ctl = reinterpret_cast<const SrFrameCtl*>(g->ws + g->r_ctl.offset);
+    if (cudaLaunchKernelEx(&cfg, sr_resident_kernel, blobs, E->blob_bytes, ctl, T, E->cs) != cudaSuccess) return SR_ERR_CUDA;
+    return SR_OK;
+}

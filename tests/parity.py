@@ -16,10 +16,10 @@ def to_device(spec, arr, device="cuda:0"):
     return t.to(torch.bfloat16).contiguous() if spec.dtype == "bf16" else t.contiguous()
 
 
-def make_graph(spec, pattern, engine="auto", graph_frames=0, weights=None, biases=None):
+def make_graph(spec, pattern, engine="auto", graph_frames=0, weights=None, biases=None, **options):
     from paper_1806_04965_b200 import Graph
     G = Graph(spec.nodes, spec.edges, spec.patterns[pattern], batch=spec.batch, dtype=spec.dtype, engine=engine,
-              graph_frames=graph_frames)
+              graph_frames=graph_frames, **options)
     G.set_weights(weights, biases)
     return G
 
@@ -55,13 +55,16 @@ def check_stepwise(spec, pattern, engine="auto", samples=None, zero_bias=False, 
     return worst
 
 
-def check_run(spec, pattern, engine="auto", graph_frames=0, samples=None, frames=None, tol=None):
+def check_run(spec, pattern, engine="auto", graph_frames=0, samples=None, frames=None, tol=None, expect_resident=None,
+              **options):
     """One sr_rollout_run over all frames; compare the output sequence and the final states."""
     X, W, Bi = data.make_inputs(spec), data.make_weights(spec), data.make_biases(spec)
     T = spec.frames if frames is None else frames
     samples = list(range(spec.batch)) if samples is None else samples
     want = fu.rollout_spec(spec, pattern, X, W, Bi, samples=samples, frames=T)
-    G = make_graph(spec, pattern, engine, graph_frames, W, Bi)
+    G = make_graph(spec, pattern, engine, graph_frames, W, Bi, **options)
+    if expect_resident is not None:
+        assert G.info["resident_cluster"] == expect_resident, G.info
     ins = G.input_nodes
     out = G.rollout([to_device(spec, X[v][:T + 1]) for v in ins])
     G.sync_status()

@@ -14,7 +14,8 @@ pytestmark = pytest.mark.gpu
 def test_c2_full_size_all_patterns():
     g = graphs.build("c2")
     for p in g.patterns:
-        parity.check_run(g, p, graph_frames=16, samples=[0, 31, 63])
+        parity.check_run(g, p, graph_frames=16, samples=[0, 31, 63], expect_resident=2)      # the resident kernel
+        parity.check_run(g, p, graph_frames=16, samples=[0, 31, 63], resident=False)         # per-frame launches
 
 
 def test_c3_full_size_all_patterns():

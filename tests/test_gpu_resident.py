@@ -1,0 +1,78 @@
+"""GPU parity of the resident kernel (one thread-block cluster per sequence, all frames of a run in one
+launch, states in shared memory) against the oracle: every edge kind, every cluster size, streaming,
+sequential and hybrid patterns, runs split in two and runs continued by single steps of the launch path."""
+import numpy as np
+import pytest
+
+from oracle import frame_update as fu
+from tests import parity
+from workloads import data, graphs
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.mark.parametrize("cluster", [1, 2, 4])
+def test_mini_cnn_every_pattern(cluster):
+    g = graphs.build("mini", batch=3, frames=5)
+    for p in g.patterns:
+        parity.check_run(g, p, expect_resident=cluster, resident_cluster=cluster)
+
+
+@pytest.mark.parametrize("cluster,warps", [(2, 16), (2, 8), (2, 5), (4, 12)])
+def test_c2_reduced(cluster, warps):
+    g = graphs.build("c2", batch=3, frames=6)
+    for p in g.patterns:
+        parity.check_run(g, p, expect_resident=cluster, resident_cluster=cluster, resident_warps=warps)
+
+
+def test_default_choice_and_opt_out():
+    from paper_1806_04965_b200 import Graph
+    g = graphs.build("c2", batch=4, frames=2)
+    assert Graph(g.nodes, g.edges, g.patterns["streaming"], batch=4).info["resident_cluster"] == 4
+    assert Graph(g.nodes, g.edges, g.patterns["streaming"], batch=64).info["resident_cluster"] == 2
+    # states and weights of one sequence exceed one CTA's shared memory: two CTAs per sequence, in waves
+    assert Graph(g.nodes, g.edges, g.patterns["streaming"], batch=100).info["resident_cluster"] == 2
+    assert Graph(g.nodes, g.edges, g.patterns["streaming"], batch=4, resident_cluster=1).info["resident_cluster"] == 0
+    assert Graph(g.nodes, g.edges, g.patterns["streaming"], batch=4, resident=False).info["resident_cluster"] == 0
+    assert Graph(g.nodes, g.edges, g.patterns["streaming"], batch=4, engine="direct").info["resident_cluster"] == 0
+    assert Graph(g.nodes, g.edges, g.patterns["streaming"], batch=4, dtype="fp32").info["resident_cluster"] == 0
+    big = graphs.build("c3", batch=2, frames=2)        # megabytes of weights: stays on the launch path
+    assert Graph(big.nodes, big.edges, big.patterns["streaming"], batch=2).info["resident_cluster"] == 0
+
+
+@pytest.mark.parametrize("pattern", ["streaming", "sequential"])
+def test_split_runs_and_steps_continue_each_other(pattern):
+    """run(3) -> step, step -> run(4): the resident kernel picks the states up from, and hands them back to,
+    the buffers the launch path uses; every output and the final states match the oracle."""
+    import torch
+    g = graphs.build("mini", batch=4, frames=9)
+    X, W, Bi = data.make_inputs(g), data.make_weights(g), data.make_biases(g, zero=False)
+    want = fu.rollout_spec(g, pattern, X, W, Bi)
+    G = parity.make_graph(g, pattern, "auto", 0, W, Bi, resident_cluster=2)
+    assert G.info["resident_cluster"] == 2
+    x = parity.to_device(g, X[0])
+    o = G.output_node
+    out = torch.zeros((9, g.batch, 10), dtype=torch.float32, device="cuda:0")
+    G.reset([x[0]])
+    G.run([x[1:4]], out[0:3])
+    G.step([x[4]], out[3])
+    G.step([x[5]], out[4])
+    G.run([x[6:10]], out[5:9])
+    G.sync_status()
+    assert G.frame() == 9
+    assert parity.rel_err(out.cpu().numpy().reshape(want[o][1:].shape), want[o][1:]) <= parity.TOL["bf16"]
+    for v in range(len(g.nodes)):
+        assert parity.rel_err(G.get_state(v).float().cpu().numpy(), want[v][9]) <= parity.TOL["bf16"], g.nodes[v].name
+
+
+def test_resident_and_launch_path_agree_at_full_size():
+    g = graphs.build("c2")
+    X, W, Bi = data.make_inputs(g), data.make_weights(g), data.make_biases(g)
+    outs = []
+    for resident in (True, False):
+        G = parity.make_graph(g, "streaming", "auto", 16, W, Bi, resident=resident)
+        assert (G.info["resident_cluster"] > 0) == resident
+        outs.append(G.rollout([parity.to_device(g, X[0])]).cpu().numpy())
+        G.sync_status()
+    assert np.abs(outs[1]).max() > 0
+    assert parity.rel_err(outs[0], outs[1].astype(np.float64)) <= parity.TOL["bf16"]

@@ -272,7 +272,22 @@ def c5_stress(batch: int = 32, frames: int = 128, size: int = 64, dtype: str = "
     return g
 
 
-BUILDERS = {"c1": c1_mlp, "c2": c2_small_cnn, "c3": c3_six_node, "c4": c4_ten_node, "c5": c5_stress}
+def mini_cnn(batch: int = 3, frames: int = 5, dtype: str = "bf16") -> GraphSpec:
+    """A small image network with every kind of edge the frame update knows: a few-channel first layer,
+    a pooling edge, recurrence, 1x1 skips with stride (one straight from the input), a hidden dense
+    node, and an output that sums a dense and a global-average dense edge."""
+    nodes = [Node("in", 16, 16, 3, IDENTITY), Node("n1", 16, 16, 32), Node("n2", 8, 8, 32), Node("n3", 4, 4, 64),
+             Node("d", 1, 1, 16), Node("out", 1, 1, 10, IDENTITY)]
+    edges = [Edge(0, 1, CONV, 3, 1), Edge(1, 2, CONV, 3, 1, 2), Edge(2, 2, CONV, 3, 1), Edge(2, 3, CONV, 3, 2),
+             Edge(1, 3, CONV, 1, 4), Edge(0, 3, CONV, 1, 4), Edge(3, 4, DENSE), Edge(4, 5, DENSE), Edge(3, 5, GAP_DENSE),
+             Edge(1, 1, CONV, 3, 1)]
+    g = GraphSpec("mini", nodes, edges, batch, frames, dtype, seed=1010)
+    g.patterns = {"streaming": streaming_pattern(g), "sequential": sequential_pattern(g),
+                  "hybrid": [0, 1, 1, 0, 1, 0, 0, 1, 0, 1]}
+    return g
+
+
+BUILDERS = {"mini": mini_cnn, "c1": c1_mlp, "c2": c2_small_cnn, "c3": c3_six_node, "c4": c4_ten_node, "c5": c5_stress}
 
 
 def build(name: str, **overrides) -> GraphSpec:
