@@ -56,9 +56,10 @@ struct RsNode {
     int32_t slo, shi, is_output, input_slot; // [slo, shi) rows stored (own + halo)
     int32_t buf[3], bias_off;                // byte offsets in shared memory (inputs rotate over three buffers)
     int32_t w_off, first_edge, n_edges, buf_bytes;
+    int32_t ksteps, pad3, pad4, pad5;
     int32_t up_lo, up_hi, up_slo, dn_lo;     // own rows that the previous / next CTA of the cluster also stores
     int32_t dn_hi, dn_slo, slot_off, n_slots;
-    int32_t has_consumers, pix_off, pad1, pad2;   // pix_off: table of (row << 16 | col) of the CTA's own pixels
+    int32_t has_consumers, pix_off, pad1, pad2;   // pix_off: table of the CTA's own pixels
     char* gstate[2];                         // the node's two state buffers in global memory
 };
 
@@ -80,7 +81,7 @@ struct RsHeader {
     int32_t n_nodes, n_edges, n_levels, n_warps;
     int32_t off_nodes, off_edges, off_units, off_ubegin;
     int32_t off_copies, n_copies, zero_off, smem_bytes;
-    int32_t dense_level_mask, sync_after_finalize, blob_bytes, pad_;
+    int32_t dense_level_mask, sync_after_finalize, blob_bytes, input_words_max;   // input_words_max: 4-byte words of the largest input slab
 };
 
 // ------------------------------------------------------------------------------------------------ device helpers
@@ -148,12 +149,6 @@ __device__ __forceinline__ void rs_level_barrier(int cs)
     }
 }
 
-__device__ __forceinline__ uint32_t rs_pack_bf16(float lo, float hi)
-{
-    const __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
-    return *reinterpret_cast<const uint32_t*>(&v);
-}
-
 struct RsCtx {
     unsigned char* smem;
     uint32_t sbase;
@@ -164,107 +159,187 @@ struct RsCtx {
     int cs, lane;
 };
 
-template <int NK>
-__device__ __forceinline__ void rs_mma_steps(float (&acc)[4][4], const uint32_t (&aaddr)[NK], uint32_t waddr, uint32_t wstride)
+// Operand fragments of G consecutive k-steps (16 channels each) of one filter tap.
+template <int G>
+struct RsFrag {
+    uint32_t a[G][4], b[G][2][4];
+};
+
+// Chunk q of a swizzled state buffer lives at q ^ ((q >> 3) & 7).  Two consecutive k-steps of a tap read the
+// chunks q and q + 2; a pixel starts on an even chunk and holds at least four chunks whenever a tap has
+// more than one k-step, so the second address is the first XOR 32.  `waddr` points at the first k-step's
+// weights (1 KiB per k-step and 32 output channels).
+template <int G>
+__device__ __forceinline__ void rs_load_group(RsFrag<G>& fr, bool ok, int q0, uint32_t sb, uint32_t zaddr, uint32_t waddr)
 {
-    uint32_t a[NK][4], bq[NK][2][4];
+    const uint32_t q = (uint32_t)q0;
+    const uint32_t base = sb + ((q ^ ((q >> 3) & 7u)) << 4);
 #pragma unroll
-    for (int i = 0; i < NK; ++i) {
-        rs_ldsm4(a[i], aaddr[i]);
-        rs_ldsm4(bq[i][0], waddr + i * wstride);
-        rs_ldsm4(bq[i][1], waddr + i * wstride + 512);
+    for (int i = 0; i < G; ++i) rs_ldsm4(fr.a[i], ok ? (base ^ (uint32_t)(32 * i)) : zaddr);
+#pragma unroll
+    for (int i = 0; i < G; ++i) {
+        rs_ldsm4(fr.b[i][0], waddr + i * 1024);
+        rs_ldsm4(fr.b[i][1], waddr + i * 1024 + 512);
     }
+}
+
+template <int G>
+__device__ __forceinline__ void rs_mma_group(float (&acc)[4][4], const RsFrag<G>& fr)
+{
 #pragma unroll
-    for (int i = 0; i < NK; ++i)
+    for (int i = 0; i < G; ++i)
 #pragma unroll
-        for (int nt = 0; nt < 4; ++nt) rs_mma(acc[nt], a[i], bq[i][nt >> 1][(nt & 1) * 2], bq[i][nt >> 1][(nt & 1) * 2 + 1]);
+        for (int nt = 0; nt < 4; ++nt)
+            rs_mma(acc[nt], fr.a[i], fr.b[i][nt >> 1][(nt & 1) * 2], fr.b[i][nt >> 1][(nt & 1) * 2 + 1]);
+}
+
+// All taps of a K x K edge whose source has NC16 * 16 channels, unrolled in groups of up to two k-steps, the
+// operand loads of a group issued before the multiply-adds of the previous one.  `rowm` / `colm`: this
+// lane's valid filter rows / columns; `anym`: taps valid for at least one lane of the warp (the others are
+// skipped by the whole warp); q00: the lane's chunk index at tap (0, 0); the weights of the unit's k-steps
+// are contiguous (the offsets below are compile-time constants after unrolling).
+template <int K, int NC16>
+__device__ __forceinline__ void rs_mma_edge_unrolled(float (&acc)[4][4], uint32_t rowm, uint32_t colm, uint32_t anym, int q00,
+                                                     int qrow, int nch, uint32_t sb, uint32_t zaddr, uint32_t waddr)
+{
+    constexpr int G = NC16 >= 2 ? 2 : 1, GPT = NC16 / G, S = K * K * GPT;      // groups per tap, groups in all
+    if (NC16 > 2) {
+        // more groups than the register file lets this loop pipeline: load and multiply group by group
+#pragma unroll
+        for (int s = 0; s < S; ++s) {
+            const int tap = s / GPT, part = s % GPT, ky = tap / K, kx = tap % K;
+            if ((anym >> tap) & 1u) {
+                RsFrag<G> one;
+                int qb = q00;
+                asm volatile("" : "+r"(qb));
+                rs_load_group<G>(one, ((rowm >> ky) & 1u) && ((colm >> kx) & 1u), qb + ky * qrow + kx * nch + part * 2 * G, sb,
+                                 zaddr, waddr + s * G * 1024);
+                rs_mma_group<G>(acc, one);
+            }
+        }
+        return;
+    }
+    RsFrag<G> fr[2];
+    if (anym & 1u) rs_load_group<G>(fr[0], (rowm & 1u) && (colm & 1u), q00, sb, zaddr, waddr);
+#pragma unroll
+    for (int s = 0; s < S; ++s) {
+        if (s + 1 < S) {
+            const int tap = (s + 1) / GPT, part = (s + 1) % GPT, ky = tap / K, kx = tap % K;
+            if ((anym >> tap) & 1u) {
+                const bool ok = ((rowm >> ky) & 1u) && ((colm >> kx) & 1u);
+                int qb = q00;
+                asm volatile("" : "+r"(qb));         // keeps the address arithmetic of each group next to its loads
+                rs_load_group<G>(fr[(s + 1) & 1], ok, qb + ky * qrow + kx * nch + part * 2 * G, sb, zaddr,
+                                 waddr + (s + 1) * G * 1024);
+            }
+        }
+        if ((anym >> (s / GPT)) & 1u) rs_mma_group<G>(acc, fr[s & 1]);
+    }
+}
+
+// The same for any filter size and channel count (not unrolled).
+__device__ __forceinline__ void rs_mma_edge_generic(float (&acc)[4][4], int k, int nc16, uint32_t rowm, uint32_t colm, uint32_t anym,
+                                                    int q00, int qrow, int nch, uint32_t sb, uint32_t zaddr, uint32_t waddr)
+{
+    int tap = 0;
+    for (int ky = 0; ky < k; ++ky) {
+        const bool rv = (rowm >> ky) & 1u;
+        int q0 = q00 + ky * qrow;
+        for (int kx = 0; kx < k; ++kx, ++tap, q0 += nch, waddr += nc16 * 1024) {
+            if (!((anym >> (tap & 31)) & 1u)) continue;
+            const bool ok = rv && ((colm >> kx) & 1u);
+            for (int c = 0; c < nc16; ++c) {
+                RsFrag<1> fr;
+                const uint32_t q = (uint32_t)(q0 + 2 * c);
+                rs_ldsm4(fr.a[0], ok ? sb + ((q ^ ((q >> 3) & 7u)) << 4) : zaddr);
+                rs_ldsm4(fr.b[0][0], waddr + c * 1024);
+                rs_ldsm4(fr.b[0][1], waddr + c * 1024 + 512);
+                rs_mma_group<1>(acc, fr);
+            }
+        }
+    }
 }
 
 // One (16 pixels x 32 channels) tile of a convolutional node: all k-steps of all incoming edges into one
 // accumulator, then bias, activation, bf16 cast and the stores into the next frame's buffer (own copy and,
 // for halo rows, the neighbour's).  `f` is the frame index relative to the start of the run: the update
-// computes relative frame f + 1.
+// computes relative frame f + 1.  Table fields are copied to registers before the loops that use them.
 __device__ __forceinline__ void rs_conv_unit(const RsCtx& cx, const RsNode& nd, int j0, int n0, int f)
 {
     const int lane = cx.lane;
-    const int W = nd.W, npix = (nd.hi - nd.lo) * W;
+    const int W = nd.W, C = nd.C, nslo = nd.slo, n_edges = nd.n_edges, first_edge = nd.first_edge;
     const uint32_t zaddr = cx.sbase + cx.H->zero_off;
+    // Column c of n-tile nt holds output channel n0 + (c >> 1) * 8 + nt * 2 + (c & 1) (the host packs the weights
+    // that way), so this lane's eight accumulator columns are the consecutive channels n0 + tq * 8 .. + 7: one
+    // 16-byte chunk per pixel.  The accumulators start at the bias.
     float acc[4][4];
-#pragma unroll
-    for (int i = 0; i < 4; ++i)
-#pragma unroll
-        for (int j = 0; j < 4; ++j) acc[i][j] = 0.f;
+    {
+        const float* bias = reinterpret_cast<const float*>(cx.smem + nd.bias_off) + n0 + (lane & 3) * 8;
+        const float4 bl = *reinterpret_cast<const float4*>(bias), bh = *reinterpret_cast<const float4*>(bias + 4);
+        acc[0][0] = acc[0][2] = bl.x; acc[0][1] = acc[0][3] = bl.y;
+        acc[1][0] = acc[1][2] = bl.z; acc[1][1] = acc[1][3] = bl.w;
+        acc[2][0] = acc[2][2] = bh.x; acc[2][1] = acc[2][3] = bh.y;
+        acc[3][0] = acc[3][2] = bh.z; acc[3][1] = acc[3][3] = bh.w;
+    }
     // the pixel whose row address this lane supplies to ldmatrix, and the 8-channel half it points at
-    // (the table is padded to a multiple of 16 pixels with 0xFFFFFFFF)
+    // (table entry: bit 31 / 30 = the previous / next CTA keeps the pixel's row as halo, row << 15 | column;
+    // padded to a multiple of 16 pixels with 0xFFFFFFFF)
     const uint32_t* pix = reinterpret_cast<const uint32_t*>(cx.smem + nd.pix_off);
     const uint32_t tl = pix[j0 + (lane & 15)];
     const bool vl = tl != 0xFFFFFFFFu;
-    const int oyl = (int)(tl >> 16), oxl = (int)(tl & 0xFFFFu);
+    const int oyl = (int)((tl >> 15) & 0x7FFFu), oxl = (int)(tl & 0x7FFFu);
     const int khalf = lane >> 4;
-    // the two pixels whose accumulator rows this lane holds
-    const int g = lane >> 2, tq = lane & 3;
-    int oy[2], ox[2];
-    bool pv[2];
-#pragma unroll
-    for (int r = 0; r < 2; ++r) {
-        const uint32_t t = pix[j0 + g + 8 * r];
-        pv[r] = t != 0xFFFFFFFFu;
-        oy[r] = (int)(t >> 16);
-        ox[r] = (int)(t & 0xFFFFu);
-    }
-    (void)npix;
-    const uint32_t wstride = (uint32_t)(nd.C >> 5) * 1024u;
-    uint32_t waddr = cx.sbase + nd.w_off + (uint32_t)(n0 >> 5) * 1024u + lane * 16;
-    for (int ei = 0; ei < nd.n_edges; ++ei) {
-        const RsEdge& e = cx.edges[nd.first_edge + ei];
+    const int g = lane >> 2, tq = lane & 3;       // accumulator rows g and g + 8, columns 2 * tq, 2 * tq + 1 of every n-tile
+    // the packed weights of this unit's 32 channels: 1 KiB per k-step, k-steps of all edges in order
+    uint32_t waddr = cx.sbase + nd.w_off + (uint32_t)(n0 >> 5) * (uint32_t)nd.ksteps * 1024u + lane * 16;
+    for (int ei = 0; ei < n_edges; ++ei) {
+        const RsEdge& e = cx.edges[first_edge + ei];
+        const int etype = e.type, k = e.k, stride = e.stride, pad = e.pad, ksteps = e.ksteps, lut_off = e.lut_off;
         const RsNode& sn = cx.nodes[e.src];
         const int fb = f + 1 - e.R;                                   // relative frame of the source state (Eq. 2)
         const int sbuf = sn.kind == RS_INPUT ? sn.buf[fb % 3] : sn.buf[fb & 1];
-        const int Hs = sn.H, Ws = sn.W;
-        if (e.type == RS_E_MMA) {
+        const int Ws = sn.W, Cs = sn.C, slo = sn.slo, shi = sn.shi;
+        if (etype == RS_E_MMA) {
             const uint32_t sb = cx.sbase + sbuf;
-            const int nch = sn.C >> 3, nc16 = sn.C >> 4;
-            const int iy0 = oyl * e.stride - e.pad, ix0 = oxl * e.stride - e.pad;
-            for (int ky = 0; ky < e.k; ++ky) {
-                const int iy = iy0 + ky;
-                const bool rowok = vl && iy >= sn.slo && iy < sn.shi;   // stored rows cover every in-image row a tile reads
-                const int rowq = (iy - sn.slo) * Ws * nch + khalf;
-                for (int kx = 0; kx < e.k; ++kx) {
-                    const int ix = ix0 + kx;
-                    const bool ok = rowok && (unsigned)ix < (unsigned)Ws;
-                    if (!__any_sync(0xffffffffu, ok)) {
-                        waddr += nc16 * wstride;
-                        continue;
-                    }
-                    const uint32_t q0 = (uint32_t)(rowq + ix * nch);
-                    int c = 0;
-                    for (; c + 2 <= nc16; c += 2) {
-                        uint32_t aa[2];
-                        aa[0] = ok ? sb + rs_swz(q0 + 2 * c) * 16 : zaddr;
-                        aa[1] = ok ? sb + rs_swz(q0 + 2 * c + 2) * 16 : zaddr;
-                        rs_mma_steps<2>(acc, aa, waddr, wstride);
-                        waddr += 2 * wstride;
-                    }
-                    if (c < nc16) {
-                        uint32_t aa[1];
-                        aa[0] = ok ? sb + rs_swz(q0 + 2 * c) * 16 : zaddr;
-                        rs_mma_steps<1>(acc, aa, waddr, wstride);
-                        waddr += wstride;
-                    }
-                }
+            const int nch = Cs >> 3, nc16 = Cs >> 4;
+            const int iy0 = oyl * stride - pad, ix0 = oxl * stride - pad;
+            uint32_t rowm = 0, colm = 0;
+            for (int t = 0; t < k; ++t) {
+                rowm |= (uint32_t)(vl && iy0 + t >= slo && iy0 + t < shi) << t;    // stored rows cover every in-image row read
+                colm |= (uint32_t)((unsigned)(ix0 + t) < (unsigned)Ws) << t;
             }
+            uint32_t anym = 0xFFFFFFFFu;
+            if (k * k <= 32) {
+                uint32_t m = 0;
+                for (int t = 0; t < k; ++t)
+                    if ((rowm >> t) & 1u) m |= colm << (t * k);
+                anym = __reduce_or_sync(0xffffffffu, m);
+            }
+            const int q00 = ((iy0 - slo) * Ws + ix0) * nch + khalf, qrow = Ws * nch;
+            const int sel = (k == 3 ? 0 : k == 1 ? 4 : 8) + (nc16 == 2 ? 0 : nc16 == 4 ? 1 : 3);
+            switch (sel) {
+                case 0: rs_mma_edge_unrolled<3, 2>(acc, rowm, colm, anym, q00, qrow, nch, sb, zaddr, waddr); break;
+                case 1: rs_mma_edge_unrolled<3, 4>(acc, rowm, colm, anym, q00, qrow, nch, sb, zaddr, waddr); break;
+                case 4: rs_mma_edge_unrolled<1, 2>(acc, rowm, colm, anym, q00, qrow, nch, sb, zaddr, waddr); break;
+                case 5: rs_mma_edge_unrolled<1, 4>(acc, rowm, colm, anym, q00, qrow, nch, sb, zaddr, waddr); break;
+                default: rs_mma_edge_generic(acc, k, nc16, rowm, colm, anym, q00, qrow, nch, sb, zaddr, waddr); break;
+            }
+            waddr += (uint32_t)ksteps * 1024u;
         } else {
             // few-channel edge: A fragments from scalar loads; the table gives (ky, kx, channel) of every k index
             const uint16_t* src = reinterpret_cast<const uint16_t*>(cx.smem + sbuf);
-            const uint32_t* lut = reinterpret_cast<const uint32_t*>(cx.smem + e.lut_off);
-            const int Cs = sn.C;
-            int iy0[2], ix0[2];
+            const uint32_t* lut = reinterpret_cast<const uint32_t*>(cx.smem + lut_off);
+            int base[2], iy0[2], ix0[2];
+            bool pv[2];
 #pragma unroll
             for (int r = 0; r < 2; ++r) {
-                iy0[r] = oy[r] * e.stride - e.pad;
-                ix0[r] = ox[r] * e.stride - e.pad;
+                const uint32_t t = pix[j0 + g + 8 * r];
+                pv[r] = t != 0xFFFFFFFFu;
+                iy0[r] = (int)((t >> 15) & 0x7FFFu) * stride - pad;
+                ix0[r] = (int)(t & 0x7FFFu) * stride - pad;
+                base[r] = ((iy0[r] - slo) * Ws + ix0[r]) * Cs;
             }
-            for (int ks = 0; ks < e.ksteps; ++ks) {
+            for (int ks = 0; ks < ksteps; ++ks) {
                 uint32_t a[4];
 #pragma unroll
                 for (int h = 0; h < 2; ++h) {
@@ -275,9 +350,10 @@ __device__ __forceinline__ void rs_conv_unit(const RsCtx& cx, const RsNode& nd, 
 #pragma unroll
                         for (int z = 0; z < 2; ++z) {
                             const uint32_t t = z ? L.y : L.x;
-                            const int iy = iy0[r] + (int)(t & 15u), ix = ix0[r] + (int)((t >> 4) & 15u);
-                            const bool ok = pv[r] && (t >> 31) && iy >= sn.slo && iy < sn.shi && ix >= 0 && ix < Ws;
-                            v[z] = ok ? (uint32_t)src[((iy - sn.slo) * Ws + ix) * Cs + (int)((t >> 8) & 255u)] : 0u;
+                            const int dy = (int)(t & 15u), dx = (int)((t >> 4) & 15u);
+                            const int iy = iy0[r] + dy, ix = ix0[r] + dx;
+                            const bool ok = pv[r] && (t >> 31) && iy >= slo && iy < shi && (unsigned)ix < (unsigned)Ws;
+                            v[z] = ok ? (uint32_t)src[base[r] + (dy * Ws + dx) * Cs + (int)((t >> 8) & 255u)] : 0u;
                         }
                         a[h * 2 + r] = v[0] | (v[1] << 16);
                     }
@@ -289,43 +365,38 @@ __device__ __forceinline__ void rs_conv_unit(const RsCtx& cx, const RsNode& nd, 
                 rs_mma(acc[1], a, b0[2], b0[3]);
                 rs_mma(acc[2], a, b1[0], b1[1]);
                 rs_mma(acc[3], a, b1[2], b1[3]);
-                waddr += wstride;
+                waddr += 1024;
             }
-            (void)Hs;
         }
     }
-    // epilogue.  Column c of n-tile nt holds output channel n0 + (c >> 1) * 8 + nt * 2 + (c & 1) (the host packs
-    // the weights that way), so this lane's eight accumulator columns are the consecutive channels
-    // n0 + tq * 8 .. + 7: one 16-byte chunk per pixel.
-    const float* bias = reinterpret_cast<const float*>(cx.smem + nd.bias_off) + n0 + tq * 8;
-    const float4 bl = *reinterpret_cast<const float4*>(bias), bh = *reinterpret_cast<const float4*>(bias + 4);
-    const float bb[8] = {bl.x, bl.y, bl.z, bl.w, bh.x, bh.y, bh.z, bh.w};
-    const uint32_t nchd = (uint32_t)(nd.C >> 3), ch = (uint32_t)((n0 >> 3) + tq);
-    const uint32_t dbuf = (uint32_t)nd.buf[(f + 1) & 1];
+    // epilogue: activation, bf16, one 16-byte store per pixel (and one into the neighbour's halo where the
+    // pixel table says so)
+    const uint32_t nchd = (uint32_t)(C >> 3), ch = (uint32_t)((n0 >> 3) + tq);
+    const uint32_t dbuf = (uint32_t)nd.buf[(f + 1) & 1], buf_bytes = (uint32_t)nd.buf_bytes;
     const bool relu = nd.act == 1;
+    const int d_up = (nslo - nd.up_slo) * W, d_dn = (nslo - nd.dn_slo) * W;
 #pragma unroll
     for (int r = 0; r < 2; ++r) {
-        if (!pv[r]) continue;
-        const int y = oy[r], x = ox[r];
+        const uint32_t t = pix[j0 + g + 8 * r];
+        if (t == 0xFFFFFFFFu) continue;
+        const int y = (int)((t >> 15) & 0x7FFFu), x = (int)(t & 0x7FFFu);
         uint32_t pk[4];
 #pragma unroll
         for (int nt = 0; nt < 4; ++nt) {
-            float v0 = acc[nt][2 * r] + bb[2 * nt], v1 = acc[nt][2 * r + 1] + bb[2 * nt + 1];
-            if (relu) {
-                v0 = fmaxf(v0, 0.f);
-                v1 = fmaxf(v1, 0.f);
-            }
-            pk[nt] = rs_pack_bf16(v0, v1);
+            __nv_bfloat162 v = __floats2bfloat162_rn(acc[nt][2 * r], acc[nt][2 * r + 1]);
+            if (relu) v = __hmax2(v, __floats2bfloat162_rn(0.f, 0.f));
+            pk[nt] = *reinterpret_cast<const uint32_t*>(&v);
         }
-        const uint32_t off = rs_swz((uint32_t)((y - nd.slo) * W + x) * nchd + ch) * 16u;
-        if (off < (uint32_t)nd.buf_bytes) *reinterpret_cast<uint4*>(cx.smem + dbuf + off) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
-        if (cx.rank > 0 && y >= nd.up_lo && y < nd.up_hi) {
-            const uint32_t o2 = rs_swz((uint32_t)((y - nd.up_slo) * W + x) * nchd + ch) * 16u;
-            if (o2 < (uint32_t)nd.buf_bytes) rs_st_cluster_v4(rs_mapa(cx.sbase + dbuf + o2, cx.rank - 1), pk);
+        const int lin = (y - nslo) * W + x;
+        const uint32_t off = rs_swz((uint32_t)lin * nchd + ch) * 16u;
+        if (off < buf_bytes) *reinterpret_cast<uint4*>(cx.smem + dbuf + off) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
+        if (t & 0x80000000u) {                     // the previous CTA of the cluster keeps this row as halo
+            const uint32_t o2 = rs_swz((uint32_t)(lin + d_up) * nchd + ch) * 16u;
+            if (o2 < buf_bytes) rs_st_cluster_v4(rs_mapa(cx.sbase + dbuf + o2, cx.rank - 1), pk);
         }
-        if ((int)cx.rank + 1 < cx.cs && y >= nd.dn_lo && y < nd.dn_hi) {
-            const uint32_t o2 = rs_swz((uint32_t)((y - nd.dn_slo) * W + x) * nchd + ch) * 16u;
-            if (o2 < (uint32_t)nd.buf_bytes) rs_st_cluster_v4(rs_mapa(cx.sbase + dbuf + o2, cx.rank + 1), pk);
+        if (t & 0x40000000u) {                     // the next one does
+            const uint32_t o2 = rs_swz((uint32_t)(lin + d_dn) * nchd + ch) * 16u;
+            if (o2 < buf_bytes) rs_st_cluster_v4(rs_mapa(cx.sbase + dbuf + o2, cx.rank + 1), pk);
         }
     }
 }
@@ -352,20 +423,23 @@ __device__ __forceinline__ void rs_dense_unit(const RsCtx& cx, const RsNode& nd,
     const char* wb = e.wd_off >= 0 ? reinterpret_cast<const char*>(cx.smem + e.wd_off) : e.wd_global;
     const long long ld = e.wd_off >= 0 ? (long long)e.wd_ld : (long long)e.wd_gld;
     const uint32_t slot_base = (uint32_t)nd.slot_off + (uint32_t)((((f + 1) & 1) * nd.n_slots + slot) * nd.C) * 4u;
-    for (int ob = 0; ob < nd.C; ob += 8) {
-        float acc[8];
+    const int C = nd.C, wmod = e.wchunk_mod, x0 = e.x_chunk0;
+    const float scale = e.scale;
+    for (int ob = 0; ob < C; ob += 16) {
+        float acc[16];
 #pragma unroll
-        for (int j = 0; j < 8; ++j) acc[j] = 0.f;
+        for (int j = 0; j < 16; ++j) acc[j] = 0.f;
         for (int cl = c_begin + lane; cl < c_end; cl += 32) {
-            const uint32_t q = (uint32_t)(e.x_chunk0 + cl);
+            const uint32_t q = (uint32_t)(x0 + cl);
             const uint4 xq = *reinterpret_cast<const uint4*>(xb + (swz ? rs_swz(q) : q) * 16u);
             float x[8];
             rs_unpack8(xq, x);
-            const int wc = e.wchunk_mod ? cl % e.wchunk_mod : cl;
+            const int wc = wmod ? cl % wmod : cl;
+            const char* wp = wb + ((long long)ob * ld + (long long)wc * 8) * 2;
 #pragma unroll
-            for (int j = 0; j < 8; ++j) {
-                if (ob + j < nd.C) {
-                    const uint4 wq = *reinterpret_cast<const uint4*>(wb + ((long long)(ob + j) * ld + (long long)wc * 8) * 2);
+            for (int j = 0; j < 16; ++j) {
+                if (ob + j < C) {
+                    const uint4 wq = *reinterpret_cast<const uint4*>(wp + (long long)j * ld * 2);
                     float w[8];
                     rs_unpack8(wq, w);
 #pragma unroll
@@ -374,16 +448,18 @@ __device__ __forceinline__ void rs_dense_unit(const RsCtx& cx, const RsNode& nd,
             }
         }
 #pragma unroll
-        for (int j = 0; j < 8; ++j) {
+        for (int j = 0; j < 16; ++j) {
+            if (ob + j < C) {
 #pragma unroll
-            for (int s = 16; s >= 1; s >>= 1) acc[j] += __shfl_xor_sync(0xffffffffu, acc[j], s);
+                for (int s = 16; s >= 1; s >>= 1) acc[j] += __shfl_xor_sync(0xffffffffu, acc[j], s);
+            }
         }
-        if (lane < 8 && ob + lane < nd.C) {
+        if (lane < 16 && ob + lane < C) {
             float v = 0.f;
 #pragma unroll
-            for (int j = 0; j < 8; ++j)
+            for (int j = 0; j < 16; ++j)
                 if (j == lane) v = acc[j];
-            v *= e.scale;
+            v *= scale;
             const uint32_t a = cx.sbase + slot_base + (uint32_t)(ob + lane) * 4u;
             if (cx.cs > 1) {
                 for (int r = 0; r < cx.cs; ++r) rs_st_cluster_u32(rs_mapa(a, (uint32_t)r), __float_as_uint(v));
@@ -428,7 +504,8 @@ sr_resident_kernel(const unsigned char* __restrict__ blobs, int blob_stride, con
             for (int i = tid * 16; i < cp[c].bytes; i += nthr * 16) rs_cp_async16(cx.sbase + cp[c].dst + i, cp[c].src + i);
     }
     // frame t of every node (relative frame 0), and the first input frame of the run (relative frame 1)
-    const long long t0 = ctl->t, run0 = ctl->run_t;
+    const long long t0 = ctl->t, run0 = ctl->run_t, out_stride = ctl->out_stride;
+    float* const out_base = ctl->out_base;
     const int par0 = (int)(t0 & 1);
     for (int v = 0; v < H.n_nodes; ++v) {
         const RsNode& nd = cx.nodes[v];
@@ -455,7 +532,7 @@ sr_resident_kernel(const unsigned char* __restrict__ blobs, int blob_stride, con
 
     for (int f = 0; f < T; ++f) {
         // input frame of the NEXT update, fetched while this one computes
-        if (f + 1 < T) {
+        if (f + 1 < T && tid < H.input_words_max) {
             for (int v = 0; v < H.n_nodes; ++v) {
                 const RsNode& nd = cx.nodes[v];
                 if (nd.kind != RS_INPUT) continue;
@@ -477,20 +554,22 @@ sr_resident_kernel(const unsigned char* __restrict__ blobs, int blob_stride, con
             if (l == H.n_levels - 1) rs_cp_async_wait_all();
             rs_level_barrier(cs);
             if ((H.dense_level_mask >> l) & 1) {
-                // dense nodes of this level: fixed-order sum of the slots, bias, activation
-                for (int v = 0; v < H.n_nodes; ++v) {
-                    const RsNode& nd = cx.nodes[v];
-                    if (nd.kind != RS_DENSE || nd.level != l) continue;
-                    const float* slots = reinterpret_cast<const float*>(smem + nd.slot_off) + ((f + 1) & 1) * nd.n_slots * nd.C;
-                    const float* bias = reinterpret_cast<const float*>(smem + nd.bias_off);
-                    for (int o = tid; o < nd.C; o += nthr) {
-                        float z = 0.f;
-                        for (int s = 0; s < nd.n_slots; ++s) z += slots[s * nd.C + o];
-                        z += bias[o];
-                        if (nd.act == 1) z = fmaxf(z, 0.f);
-                        reinterpret_cast<__nv_bfloat16*>(smem + nd.buf[(f + 1) & 1])[o] = __float2bfloat16_rn(z);
-                        if (nd.is_output && rank == 0 && ctl->out_base)
-                            ctl->out_base[(run0 + f) * ctl->out_stride + (long long)b * nd.C + o] = z;
+                // dense nodes of this level: fixed-order sum of the slots (the bias is slot-independent), activation
+                if (warp == 0) {
+                    for (int v = 0; v < H.n_nodes; ++v) {
+                        const RsNode& nd = cx.nodes[v];
+                        if (nd.kind != RS_DENSE || nd.level != l) continue;
+                        const int C = nd.C, n_slots = nd.n_slots;
+                        const float* slots = reinterpret_cast<const float*>(smem + nd.slot_off) + ((f + 1) & 1) * n_slots * C;
+                        const float* bias = reinterpret_cast<const float*>(smem + nd.bias_off);
+                        for (int o = tid; o < C; o += 32) {
+                            float z = 0.f;
+                            for (int s = 0; s < n_slots; ++s) z += slots[s * C + o];
+                            z += bias[o];
+                            if (nd.act == 1) z = fmaxf(z, 0.f);
+                            reinterpret_cast<__nv_bfloat16*>(smem + nd.buf[(f + 1) & 1])[o] = __float2bfloat16_rn(z);
+                            if (nd.is_output && rank == 0 && out_base) out_base[(run0 + f) * out_stride + (long long)b * C + o] = z;
+                        }
                     }
                 }
                 if (H.sync_after_finalize) __syncthreads();
@@ -644,8 +723,7 @@ bool rs_layout(const sr_graph* g, RsEngine& E, int cs, int warps)
                     const int per = (n + parts - 1) / parts;
                     for (int c0 = 0; c0 < n; c0 += per) {
                         const int c1 = std::min(n, c0 + per);
-                        const long ob = (hn.d.c + 7) / 8;
-                        const long cost = 30 + ob * ((long)((c1 - c0 + 31) / 32) * 150 + 50);
+                        const long cost = 40 + (long)((c1 - c0 + 31) / 32) * (12 + 17 * hn.d.c) + 7 * hn.d.c;
                         cand[r].push_back(Cand{RsUnit{RS_U_DENSE, v, p.first_edge + ei, c0, c1, slot_count[v]++}, level, cost});
                     }
                 }
@@ -980,6 +1058,7 @@ sr_status sr_rs_bind(sr_graph* g)
             d.first_edge = p.first_edge;
             d.n_edges = (int)hn.in_edges.size();
             d.buf_bytes = p.buf_bytes;
+            d.ksteps = p.ksteps;
             d.up_lo = d.up_hi = d.up_slo = d.dn_lo = d.dn_hi = d.dn_slo = 0;
             if (p.kind != RS_DENSE) {
                 if (r > 0) {
@@ -1000,8 +1079,12 @@ sr_status sr_rs_bind(sr_graph* g)
             if (p.kind == RS_CONV) {
                 uint32_t* pix = reinterpret_cast<uint32_t*>(blob.data() + p.pix_off);
                 const int npix = (d.hi - d.lo) * d.W;
-                for (int j = 0; j < p.pix_entries; ++j)
-                    pix[j] = j < npix ? ((uint32_t)(d.lo + j / d.W) << 16) | (uint32_t)(j % d.W) : 0xFFFFFFFFu;
+                for (int j = 0; j < p.pix_entries; ++j) {
+                    const int y = d.lo + j / d.W, x = j % d.W;
+                    const uint32_t up = (r > 0 && y >= d.up_lo && y < d.up_hi) ? 0x80000000u : 0u;
+                    const uint32_t dn = (r + 1 < E.cs && y >= d.dn_lo && y < d.dn_hi) ? 0x40000000u : 0u;
+                    pix[j] = j < npix ? (up | dn | ((uint32_t)y << 15) | (uint32_t)x) : 0xFFFFFFFFu;
+                }
             }
             d.gstate[0] = g->ws + hn.state[0].offset;
             d.gstate[1] = g->ws + hn.state[1].offset;
@@ -1083,6 +1166,10 @@ sr_status sr_rs_bind(sr_graph* g)
         H->dense_level_mask = dense_mask;
         H->sync_after_finalize = sync_after;
         H->blob_bytes = E.blob_bytes;
+        H->input_words_max = 0;
+        for (int v = 0; v < n_nodes; ++v)
+            if (E.pn[v].kind == RS_INPUT)
+                H->input_words_max = std::max(H->input_words_max, (E.pn[v].shi[r] - E.pn[v].slo[r]) * g->nodes[v].d.w * g->nodes[v].d.c / 2);
         if (cudaMemcpy(g->ws + E.r_blobs.offset + (size_t)r * E.blob_bytes, blob.data(), blob.size(), cudaMemcpyHostToDevice) !=
             cudaSuccess)
             return SR_ERR_CUDA;
@@ -1126,12 +1213,16 @@ sr_status sr_rs_set_weights(sr_graph* g, int edge, const float* w_eff)
                                 const int kk = ks * 16 + kh * 8 + j;
                                 if (kk < pe.Kreal) w = w_eff[(size_t)n * he.K + kk];
                             }
-                            pk[(((size_t)ks * nb + b) * 2 + hb) * 256 + l * 8 + j] = bf16(w);
+                            pk[(((size_t)b * pe.ksteps + ks) * 2 + hb) * 256 + l * 8 + j] = bf16(w);
                         }
                     }
+        // in the node's region the 32-channel blocks are outermost, then the k-steps of all edges in order
         const RsPlanNode& p = E.pn[he.d.tgt];
-        char* dst = g->ws + E.r_wconv.offset + p.w_global + (size_t)pe.ks0 * nb * 1024;
-        if (cudaMemcpy(dst, pk.data(), pk.size() * 2, cudaMemcpyHostToDevice) != cudaSuccess) return SR_ERR_CUDA;
+        for (int b = 0; b < nb; ++b) {
+            char* dst = g->ws + E.r_wconv.offset + p.w_global + ((size_t)b * p.ksteps + pe.ks0) * 1024;
+            if (cudaMemcpy(dst, pk.data() + (size_t)b * pe.ksteps * 512, (size_t)pe.ksteps * 1024, cudaMemcpyHostToDevice) != cudaSuccess)
+                return SR_ERR_CUDA;
+        }
     } else {
         std::vector<uint16_t> pk((size_t)Cout * he.K);
         for (size_t i = 0; i < pk.size(); ++i) pk[i] = bf16(w_eff[i]);

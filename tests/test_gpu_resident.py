@@ -18,6 +18,23 @@ def test_mini_cnn_every_pattern(cluster):
         parity.check_run(g, p, expect_resident=cluster, resident_cluster=cluster)
 
 
+@pytest.mark.parametrize("cin,cout,k,stride,pool,size,cluster", [
+    (32, 32, 3, 1, 0, 12, 2), (64, 64, 3, 1, 0, 8, 1), (64, 32, 3, 2, 0, 16, 2), (128, 32, 3, 1, 0, 8, 2), (64, 96, 1, 2, 0, 8, 1),
+    (32, 64, 5, 1, 0, 10, 2), (32, 32, 7, 4, 0, 28, 2), (64, 32, 3, 1, 2, 16, 4), (96, 32, 3, 1, 0, 9, 1), (32, 64, 1, 1, 0, 6, 2),
+])
+def test_single_conv_edge(cin, cout, k, stride, pool, size, cluster):
+    """Source channel counts (k-step loops of every shape), filter sizes, strides, a pooled edge, odd image sizes."""
+    from workloads.graphs import CONV, GAP_DENSE, IDENTITY, Edge, GraphSpec, Node, check_shapes
+    out = size // stride // (2 if pool else 1)
+    nodes = [Node("in", size, size, 2, IDENTITY), Node("a", size, size, cin), Node("n", out, out, cout), Node("o", 1, 1, 6, IDENTITY)]
+    edges = [Edge(0, 1, CONV, 3, 1), Edge(1, 2, CONV, k, stride, pool), Edge(2, 2, CONV, 3, 1), Edge(2, 3, GAP_DENSE)]
+    for R in ([1, 1, 1, 1], [0, 0, 1, 0]):
+        g = GraphSpec("edge", nodes, edges, batch=2, frames=3, dtype="bf16", seed=99)
+        g.patterns = {"p": R}
+        check_shapes(g)
+        parity.check_run(g, "p", expect_resident=cluster, resident_cluster=cluster)
+
+
 @pytest.mark.parametrize("cluster,warps", [(2, 16), (2, 8), (2, 5), (4, 12)])
 def test_c2_reduced(cluster, warps):
     g = graphs.build("c2", batch=3, frames=6)
