@@ -28,6 +28,8 @@ from workloads import data, graphs  # noqa: E402
 # dram__bytes_read.sum + dram__bytes_write.sum of one tensor-core group launch from the ncu captures summarised under
 # profiles/ (null where no capture of the current kernel exists)
 TRAFFIC = {"c2": 5.78e6, "c3": 264.1e6, "c4": 157.5e6, "c5": 612.4e6}
+# the same for one launch of the resident kernel (all T frames of the workload); null until captured for the current kernel
+TRAFFIC_RESIDENT = {}
 
 METRIC = "streaming_rollout_frames_per_sec"
 UNIT = "frames/s"
@@ -187,10 +189,10 @@ def run_reference(args):
 
 
 # ----------------------------------------------------------------------------- the CUDA library
-def time_pattern(torch, spec, pattern, W, Bi, dev_in, steps, warmup, graph_frames, engine, flush):
+def time_pattern(torch, spec, pattern, W, Bi, dev_in, steps, warmup, graph_frames, engine, flush, resident=(1, 0, 0)):
     from paper_1806_04965_b200 import Graph
     G = Graph(spec.nodes, spec.edges, spec.patterns[pattern], batch=spec.batch, dtype=spec.dtype, engine=engine,
-              graph_frames=graph_frames)
+              graph_frames=graph_frames, resident=bool(resident[0]), resident_cluster=resident[1], resident_warps=resident[2])
     G.set_weights(W, Bi)
     T = spec.frames
     out = torch.empty((T, spec.batch, spec.nodes[G.output_node].c), dtype=torch.float32, device="cuda")
@@ -217,7 +219,8 @@ def time_pattern(torch, spec, pattern, W, Bi, dev_in, steps, warmup, graph_frame
     ms = float(np.mean(times))
     return G, out, {"ms_per_step": ms, "frames_per_s": T / ms * 1e3, "us_per_frame": ms * 1e3 / T,
                     "ms_min": float(np.min(times)), "launches": launches, "groups_per_frame": G.info["n_groups"],
-                    "tensor_core_nodes": G.info["n_tensor_core_nodes"], "direct_nodes": G.info["n_direct_nodes"]}
+                    "tensor_core_nodes": G.info["n_tensor_core_nodes"], "direct_nodes": G.info["n_direct_nodes"],
+                    "resident_cluster": G.info["resident_cluster"]}
 
 
 def run_cuda(args):
@@ -255,7 +258,7 @@ def run_cuda(args):
         if p == args.pattern:
             sampler = ClockSampler(local)
         G, out, r = time_pattern(torch, spec, p, W, Bi, dev_in, args.steps, args.warmup, args.graph_frames, args.engine,
-                                 flush)
+                                 flush, (args.resident, args.resident_cluster, args.resident_warps))
         barrier()
         if p == args.pattern:
             clocks = sampler.stop()
@@ -290,7 +293,22 @@ def run_cuda(args):
     # the dominant kernel alone: every tensor-core group launch of a few plain (non-graph) runs is bracketed
     # with CUDA events on the launching stream by the library
     kernel_us, kernel_n = None, 0
-    if main["tensor_core_nodes"] > 0:
+    resident = main["resident_cluster"] > 0
+    if resident:
+        # the resident kernel: ONE launch per step walks all T frames; event-timed by the library
+        main_G.set_option(5, 1)
+        ins0, ins = [x[0] for x in dev_in], [x[1:] for x in dev_in]
+        main_G.reset(ins0)
+        main_G.run(ins, main_out)
+        main_G.kernel_time()
+        for _ in range(5):
+            flush.add_(1)
+            main_G.reset(ins0)
+            main_G.run(ins, main_out)
+        k_ms, kernel_n = main_G.kernel_time()
+        main_G.set_option(5, 0)
+        kernel_us = 1e3 * k_ms / max(1, kernel_n)
+    elif main["tensor_core_nodes"] > 0:
         main_G.set_option(1, 0)
         main_G.set_option(5, 1)
         ins0, ins = [x[0] for x in dev_in], [x[1:] for x in dev_in]
@@ -309,7 +327,19 @@ def run_cuda(args):
     conv_fl = 2.0 * spec.batch * sum(
         (16 if e.pool == 2 else e.k * e.k) * spec.nodes[e.src].c * spec.nodes[e.tgt].h * spec.nodes[e.tgt].w * spec.nodes[e.tgt].c
         for e in spec.edges if e.kind == graphs.CONV)
-    if tensor_bound:
+    if resident:
+        # algorithmic bytes of the T frames one launch covers / its duration.  The states stay on chip, so the
+        # kernel's own DRAM traffic is far below the algorithmic bytes (which assume every state is read and
+        # written once per frame): the HBM roofline is the classification the workload has on a per-frame
+        # launch path, not what limits this kernel.
+        ach = by * T / (kernel_us * 1e-6) / 1e9
+        roof = {"bound": "hbm", "achieved": ach, "peak": pk["hbm_gbs"], "unit": "GB/s", "frac": ach / pk["hbm_gbs"],
+                "traffic": TRAFFIC_RESIDENT.get(spec.name),
+                "kernel": "sr_resident_kernel, mean of %d event-timed launches (%.1f us each = %.2f us per frame, %d frames per launch, "
+                          "%d CTAs per sequence)" % (kernel_n, kernel_us, kernel_us / T, T, main["resident_cluster"]),
+                "tensor": {"achieved_tflops": fl * T / (kernel_us * 1e-6) / 1e12,
+                           "note": "mma.sync path; states and weights resident in shared memory"}}
+    elif tensor_bound:
         if kernel_us:
             ach = conv_fl / groups / (kernel_us * 1e-6) / 1e12     # average over the group launches of a frame
             what = "sr_tc_group_kernel, mean of %d event-timed launches (%.1f us each, %d per frame)" % (kernel_n, kernel_us, groups)
@@ -335,9 +365,10 @@ def run_cuda(args):
             "dtype": "bf16" if spec.dtype == "bf16" else "f32", "data": "synthetic",
             "config": {"workload": spec.name, "pattern": args.pattern, "batch": spec.batch, "frames_per_step": T,
                        "l2": "flushed between timed steps (192 MiB write)", "engine": args.engine,
-                       "graph_frames": args.graph_frames, "parallelism": "replicas x%d" % world},
+                       "graph_frames": args.graph_frames, "parallelism": "replicas x%d" % world,
+                       "resident_cluster": main["resident_cluster"]},
             "us_per_frame": us_frame, "sample_frames_per_s": world * spec.batch * T / ms * 1e3,
-            "patterns": {p: {k: r[k] for k in ("frames_per_s", "us_per_frame", "groups_per_frame", "launches")}
+            "patterns": {p: {k: r[k] for k in ("frames_per_s", "us_per_frame", "groups_per_frame", "launches", "resident_cluster")}
                          for p, r in results.items()},
             "e2e": {"value": whole_job_frames_per_s(world, T, e2e), "unit": UNIT,
                     "h2d_bytes_per_step": int(sum(h.numel() * h.element_size() for h in host_in)),
@@ -367,6 +398,9 @@ def main():
     ap.add_argument("--frames", type=int, default=0)
     ap.add_argument("--engine", default="auto", choices=["auto", "direct"])
     ap.add_argument("--graph-frames", type=int, default=16, help="frames per CUDA graph inside sr_rollout_run (0 = plain launches)")
+    ap.add_argument("--resident", type=int, default=1, help="1: sr_rollout_run may use the shared-memory-resident kernel; 0: per-frame launches")
+    ap.add_argument("--resident-cluster", type=int, default=0)
+    ap.add_argument("--resident-warps", type=int, default=0)
     ap.add_argument("--only-main", action="store_true", help="time only --pattern, not the other rollout patterns")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     args = ap.parse_args()

@@ -161,8 +161,9 @@ sr_status sr_graph_set_node_bias(sr_graph* g, int node, const float* bias_host);
  *           key 4 "overlap": 1 (default) runs independent launches of a frame on a second, library-owned
  *                  stream (the CUDA-core and the tensor-core kernel of a group; the next frame's input
  *                  copy when no input edge has R = 0), joined before the frame ends; 0 = one stream.
- *           key 5 "kernel timing": 1 brackets every tensor-core group launch with CUDA events on the launching
- *                  stream (plain launches only, not inside CUDA graphs); read with sr_graph_kernel_time.
+ *           key 5 "kernel timing": 1 brackets every tensor-core group launch and every resident launch with CUDA
+ *                  events on the launching stream (plain launches only, not inside CUDA graphs); read with
+ *                  sr_graph_kernel_time.
  *           key 6 "resident": 1 (default) lets sr_rollout_run use the resident kernel when the network qualifies
  *                  (bfloat16; per-sequence states and convolution weights fit in the shared memory of a
  *                  thread-block cluster): one cluster per sequence walks all T frames in one launch with
@@ -207,8 +208,8 @@ sr_status sr_graph_set_state(sr_graph* g, int node, const void* src_dev, void* s
 sr_status sr_graph_frame(const sr_graph* g, int64_t* t);
 /* Kernels launched by this graph so far (counts launches inside replayed CUDA graphs as well). */
 sr_status sr_graph_launch_count(const sr_graph* g, int64_t* n);
-/* Sum of the event-timed durations (milliseconds) and the number of tensor-core group launches since the
- * previous call (option key 5); waits for those launches to finish. */
+/* Sum of the event-timed durations (milliseconds) and the number of tensor-core group launches and resident
+ * launches since the previous call (option key 5); waits for those launches to finish. */
 sr_status sr_graph_kernel_time(sr_graph* g, double* ms, int64_t* launches);
 /* Synchronises `stream` and reports SR_ERR_CUDA / SR_ERR_TIMEOUT if queued work failed. */
 sr_status sr_graph_sync_status(sr_graph* g, void* stream);

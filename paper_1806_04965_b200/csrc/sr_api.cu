@@ -666,9 +666,12 @@ sr_status sr_graph_kernel_time(sr_graph* g, double* ms, int64_t* launches)
 {
     if (!g || !ms || !launches) return SR_ERR_INVALID_ARG;
     if (g->batch <= 0 || !g->ws) return SR_ERR_STATE;
-    long long n = 0;
-    const sr_status st = sr_tc_timing(g, ms, &n);
-    *launches = n;
+    long long n = 0, n_rs = 0;
+    double ms_rs = 0.0;
+    sr_status st = sr_tc_timing(g, ms, &n);
+    if (st == SR_OK) st = sr_rs_timing(g, &ms_rs, &n_rs);
+    *ms += ms_rs;
+    *launches = n + n_rs;
     return st;
 }
 

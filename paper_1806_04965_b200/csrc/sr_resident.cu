@@ -629,6 +629,8 @@ struct RsEngine {
     bool dense_in_smem = false;
     SrRegion r_blobs, r_wconv, r_wdense;
     bool attr_set = false;
+    std::vector<cudaEvent_t> ev;                // pairs bracketing timed launches (option "kernel timing")
+    size_t ev_used = 0;
 };
 
 int rs_row_lo(int H, int r, int cs) { return (H * r + cs / 2) / cs; }
@@ -877,6 +879,8 @@ RsEngine* rs_of(const sr_graph* g) { return static_cast<RsEngine*>(g->rs); }
 
 void sr_rs_destroy(sr_graph* g)
 {
+    if (RsEngine* E = rs_of(g))
+        for (cudaEvent_t e : E->ev) cudaEventDestroy(e);
     delete rs_of(g);
     g->rs = nullptr;
 }
@@ -1255,6 +1259,40 @@ sr_status sr_rs_launch(sr_graph* g, int T, cudaStream_t s)
     cfg.numAttrs = E->cs > 1 ? 1 : 0;
     const unsigned char* blobs = reinterpret_cast<const unsigned char*>(g->ws + E->r_blobs.offset);
     const SrFrameCtl* ctl = reinterpret_cast<const SrFrameCtl*>(g->ws + g->r_ctl.offset);
+    cudaStreamCaptureStatus cap = cudaStreamCaptureStatusNone;
+    bool timed = g->opt_time_tc != 0 && cudaStreamIsCapturing(s, &cap) == cudaSuccess && cap == cudaStreamCaptureStatusNone;
+    if (timed && E->ev_used + 2 > E->ev.size()) {
+        if (E->ev.size() >= 4096) timed = false;
+        for (int i = 0; timed && i < 2; ++i) {
+            cudaEvent_t e = nullptr;
+            if (cudaEventCreate(&e) != cudaSuccess) timed = false;
+            else E->ev.push_back(e);
+        }
+        if (E->ev_used + 2 > E->ev.size()) timed = false;
+    }
+    if (timed) cudaEventRecord(E->ev[E->ev_used], s);
     if (cudaLaunchKernelEx(&cfg, sr_resident_kernel, blobs, E->blob_bytes, ctl, T, E->cs) != cudaSuccess) return SR_ERR_CUDA;
+    if (timed) {
+        cudaEventRecord(E->ev[E->ev_used + 1], s);
+        E->ev_used += 2;
+    }
+    return SR_OK;
+}
+
+// Sum of the event-timed durations of the resident launches since the last call (synchronises).
+sr_status sr_rs_timing(sr_graph* g, double* ms, long long* launches)
+{
+    RsEngine* E = rs_of(g);
+    *ms = 0.0;
+    *launches = 0;
+    if (!E) return SR_OK;
+    for (size_t i = 0; i + 1 < E->ev_used; i += 2) {
+        if (cudaEventSynchronize(E->ev[i + 1]) != cudaSuccess) return SR_ERR_CUDA;
+        float t = 0.f;
+        if (cudaEventElapsedTime(&t, E->ev[i], E->ev[i + 1]) != cudaSuccess) return SR_ERR_CUDA;
+        *ms += t;
+        *launches += 1;
+    }
+    E->ev_used = 0;
     return SR_OK;
 }

@@ -11,4 +11,5 @@ bool sr_rs_available(const sr_graph* g);
 // Queues ONE kernel that performs the T frame updates described by the frame control block.
 sr_status sr_rs_launch(sr_graph* g, int T, cudaStream_t s);
 void sr_rs_describe(const sr_graph* g, int* cluster_size, int* warps, int* smem_bytes);
+sr_status sr_rs_timing(sr_graph* g, double* ms, long long* launches);   // event-timed resident launches since the last call
 void sr_rs_destroy(sr_graph* g);
