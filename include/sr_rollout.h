@@ -90,6 +90,9 @@ typedef struct {
     int32_t n_direct_nodes;            /* nodes updated by the CUDA-core kernels                          */
     int32_t resident_cluster;          /* CTAs per sequence of the shared-memory-resident kernel that
                                           sr_rollout_run uses for this graph; 0 = it does not apply       */
+    int32_t resident_smem_bytes;       /* shared memory per CTA of that kernel                            */
+    int32_t resident_heads_on_chip;    /* 1 if the dense / mean-dense weights are resident as well, 0 if they
+                                          are read from global memory every frame                         */
 } sr_info;
 
 /*

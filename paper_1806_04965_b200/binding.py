@@ -40,7 +40,7 @@ class _Info(ctypes.Structure):
     _fields_ = [(n, ctypes.c_int32) for n in
                 ("n_nodes", "n_edges", "n_inputs", "inference_factor", "n_groups", "streaming_parallel",
                  "output_node", "first_response_frame", "first_response_step", "response_interval",
-                 "n_tensor_core_nodes", "n_direct_nodes", "resident_cluster")]
+                 "n_tensor_core_nodes", "n_direct_nodes", "resident_cluster", "resident_smem_bytes", "resident_heads_on_chip")]
 
 
 def load_library(path: Optional[str] = None):

@@ -149,8 +149,8 @@ sr_status plan(sr_graph* g)
         if (!n.is_input) (n.use_tc ? n_tc : n_direct)++;
     g->info.n_tensor_core_nodes = n_tc;
     g->info.n_direct_nodes = n_direct;
-    int rs_warps = 0, rs_smem = 0;
-    sr_rs_describe(g, &g->info.resident_cluster, &rs_warps, &rs_smem);
+    int rs_warps = 0;
+    sr_rs_describe(g, &g->info.resident_cluster, &rs_warps, &g->info.resident_smem_bytes, &g->info.resident_heads_on_chip);
     return SR_OK;
 }
 
@@ -231,6 +231,16 @@ SrFrameCtl make_ctl(const sr_graph* g, const void* const* in, bool sequence, flo
     c.out_base = out;
     c.out_stride = (int64_t)g->batch * g->nodes[g->info.output_node].d.c;
     return c;
+}
+
+// What the launch path derives from the input nodes' current state (staged few-channel edges) is brought up to
+// date after a resident run.
+void refresh_staging(sr_graph* g, cudaStream_t s)
+{
+    if (g->stage_dirty) {
+        g->launches += sr_tc_after_state_change(g, s);
+        g->stage_dirty = false;
+    }
 }
 
 }  // namespace
@@ -537,6 +547,7 @@ sr_status sr_graph_reset(sr_graph* g, const void* const* in0_dev, void* stream)
         }
     }
     g->t = 0;
+    g->stage_dirty = false;
     g->launches += sr_tc_after_state_change(g, s);
     return cuda_ok(cudaGetLastError()) ? SR_OK : SR_ERR_CUDA;
 }
@@ -549,6 +560,7 @@ sr_status sr_rollout_step(sr_graph* g, const void* const* in_next_dev, float* ou
     for (size_t i = 0; i < g->input_nodes.size(); ++i)
         if (!in_next_dev[i]) return SR_ERR_INVALID_ARG;
     cudaStream_t s = static_cast<cudaStream_t>(stream);
+    refresh_staging(g, s);
     sr_launch_set_ctl(g, make_ctl(g, in_next_dev, false, out_dev), s);
     g->launches += 1 + enqueue_frames(g, 0, 1, s);
     g->t += 1;
@@ -564,8 +576,6 @@ sr_status sr_rollout_run(sr_graph* g, const void* const* in_seq_dev, int T, floa
         if (!in_seq_dev[i]) return SR_ERR_INVALID_ARG;
     if (T == 0) return SR_OK;
     cudaStream_t s = static_cast<cudaStream_t>(stream);
-    sr_launch_set_ctl(g, make_ctl(g, in_seq_dev, true, out_seq_dev), s);
-    g->launches += 1;
     if (sr_rs_available(g)) {
         bool aligned = true;                                     // the resident kernel fetches input rows in 4-byte words
         for (size_t i = 0; i < g->input_nodes.size(); ++i)
@@ -573,15 +583,17 @@ sr_status sr_rollout_run(sr_graph* g, const void* const* in_seq_dev, int T, floa
         if (aligned) {
             // one launch walks all T frames with the states in shared memory, then the frame counter
             // advances and whatever the launch path derives from the input state is refreshed
-            st = sr_rs_launch(g, T, s);
+            st = sr_rs_launch(g, T, make_ctl(g, in_seq_dev, true, out_seq_dev), s);
             if (st != SR_OK) return st;
-            sr_launch_advance(g, T, s);
-            g->launches += 2;
+            g->launches += 1;
             g->t += T;
-            g->launches += sr_tc_after_state_change(g, s);
+            g->stage_dirty = true;             // refreshed when the launch path is used next
             return cuda_ok(cudaGetLastError()) ? SR_OK : SR_ERR_CUDA;
         }
     }
+    refresh_staging(g, s);
+    sr_launch_set_ctl(g, make_ctl(g, in_seq_dev, true, out_seq_dev), s);
+    g->launches += 1;
     int done = 0;
     const int gf = g->opt_graph_frames;
     if (gf > 0 && T >= gf) {

@@ -102,6 +102,7 @@ struct sr_graph {
     void* graphs = nullptr;                        // CUDA-graph cache (opaque here)
     void* side = nullptr;                          // side stream and fork / join events (opaque here)
     bool input_feeds_same_frame = false;           // some edge that leaves an input node has R = 0
+    bool stage_dirty = false;                      // the resident kernel ran: staged copies of the input state are stale
 };
 
 // sr_compile.cpp

@@ -41,10 +41,12 @@
 namespace {
 
 constexpr int kRsMaxCluster = 4;
-constexpr int kRsSmemMax = 232448;            // 227 KiB of dynamic shared memory per CTA
+constexpr int kRsSmemMax = 232448 - 128;      // 227 KiB per CTA minus the kernel's static shared memory
 constexpr int kRsMaxThreads = 512;
 constexpr int kRsDenseUnitChunks = 64;        // 16-byte chunks of the source per dense unit
 constexpr int kRsMaxDenseC = 64;
+constexpr int kRsFinalizeWarp = 0;            // sums the dense slots after a level's barrier
+constexpr int kRsFetchWarp = 1;               // fetches the next input frame
 
 enum { RS_INPUT = 0, RS_CONV = 1, RS_DENSE = 2 };
 enum { RS_E_MMA = 0, RS_E_GATHER = 1, RS_E_DENSE = 2, RS_E_MEAN = 3 };
@@ -57,6 +59,8 @@ struct RsNode {
     int32_t buf[3], bias_off;                // byte offsets in shared memory (inputs rotate over three buffers)
     int32_t w_off, first_edge, n_edges, buf_bytes;
     int32_t ksteps, pad3, pad4, pad5;
+    // input nodes: zero-padded plain layout [top pad + rows + bottom pad][in_pitch] (+ a zero tail), see rs_input_fetch
+    int32_t in_pitch, in_pt, in_ple, in_tail, in_wpr, in_magic, in_nb, in_lead;
     int32_t up_lo, up_hi, up_slo, dn_lo;     // own rows that the previous / next CTA of the cluster also stores
     int32_t dn_hi, dn_slo, slot_off, n_slots;
     int32_t has_consumers, pix_off, pad1, pad2;   // pix_off: table of the CTA's own pixels
@@ -69,7 +73,8 @@ struct RsEdge {
     int32_t Kreal, wd_off, wd_ld, n_chunks;  // dense: weights in shared memory at wd_off (row pitch wd_ld elements) or < 0
     int32_t x_chunk0, wchunk_mod;            // dense: first source chunk of this CTA's slice; mean-dense: chunks per pixel
     float scale;
-    int32_t pad_;
+    int32_t g_const;                         // few-channel edge: element offset of the window of output pixel (0, 0)
+    int32_t g_ys, g_xs, pad_a, pad_b;        // ... and its step per output row / column
     const char* wd_global;                   // dense weights in global memory, already at this CTA's slice
     int64_t wd_gld;                          // row pitch there, in elements
 };
@@ -159,6 +164,17 @@ struct RsCtx {
     int cs, lane;
 };
 
+// Rows [slo, shi) of an input frame from global memory into the node's zero-padded buffer: 4-byte words, word i
+// belongs to row i / in_wpr (by multiplication with in_magic = ceil(2^20 / in_wpr), checked on the host).
+__device__ __forceinline__ void rs_input_fetch(const RsCtx& cx, const RsNode& nd, const char* g, int bufoff, int tid, int nthr)
+{
+    const int wpr = nd.in_wpr, nw = (nd.shi - nd.slo) * wpr, magic = nd.in_magic, pt = nd.in_pt, pitch = nd.in_pitch, ple = nd.in_ple;
+    for (int i = tid; i < nw; i += nthr) {
+        const int row = (int)(((unsigned)i * (unsigned)magic) >> 20), col = i - row * wpr;
+        rs_cp_async4(cx.sbase + bufoff + (((row + pt) * pitch + ple) << 1) + col * 4, g + (size_t)i * 4);
+    }
+}
+
 // Operand fragments of G consecutive k-steps (16 channels each) of one filter tap.
 template <int G>
 struct RsFrag {
@@ -193,47 +209,46 @@ __device__ __forceinline__ void rs_mma_group(float (&acc)[4][4], const RsFrag<G>
             rs_mma(acc[nt], fr.a[i], fr.b[i][nt >> 1][(nt & 1) * 2], fr.b[i][nt >> 1][(nt & 1) * 2 + 1]);
 }
 
-// All taps of a K x K edge whose source has NC16 * 16 channels, unrolled in groups of up to two k-steps, the
-// operand loads of a group issued before the multiply-adds of the previous one.  `rowm` / `colm`: this
-// lane's valid filter rows / columns; `anym`: taps valid for at least one lane of the warp (the others are
-// skipped by the whole warp); q00: the lane's chunk index at tap (0, 0); the weights of the unit's k-steps
-// are contiguous (the offsets below are compile-time constants after unrolling).
+// All taps of a K x K edge whose source has NC16 * 16 channels (2 or 4: at most one 128-byte line per pixel).
+// First the A address of every tap (independent arithmetic, nothing waits on anything), then a pure
+// load / multiply-add sequence in groups of two k-steps, the loads of a group issued before the
+// multiply-adds of the previous one; no branch inside (a conditional load into registers that live across
+// groups makes the compiler copy the whole fragment set at every merge).  Chunk q of the swizzled buffer
+// lives at q ^ ((q >> 3) & 7); the k-steps of a tap read chunks q, q + 2, q + 4, q + 6 of one line, i.e. the
+// first address XOR 32, 64, 96 (the zero line used by out-of-image taps is 128 bytes long, so the XOR applies
+// to it as well).  `rowm` / `colm`: this lane's valid filter rows / columns; q00: the lane's chunk index at
+// tap (0, 0); the weights of the unit's k-steps are contiguous, 1 KiB each (constant offsets after unrolling).
 template <int K, int NC16>
-__device__ __forceinline__ void rs_mma_edge_unrolled(float (&acc)[4][4], uint32_t rowm, uint32_t colm, uint32_t anym, int q00,
-                                                     int qrow, int nch, uint32_t sb, uint32_t zaddr, uint32_t waddr)
+__device__ __forceinline__ void rs_mma_edge_unrolled(float (&acc)[4][4], uint32_t rowm, uint32_t colm, int q00, int qrow, int nch,
+                                                     uint32_t sb, uint32_t zaddr, uint32_t waddr)
 {
-    constexpr int G = NC16 >= 2 ? 2 : 1, GPT = NC16 / G, S = K * K * GPT;      // groups per tap, groups in all
-    if (NC16 > 2) {
-        // more groups than the register file lets this loop pipeline: load and multiply group by group
+    constexpr int GPT = NC16 / 2, S = K * K * GPT;          // groups of two k-steps per tap, groups in all
+    uint32_t ad[K * K];
 #pragma unroll
-        for (int s = 0; s < S; ++s) {
-            const int tap = s / GPT, part = s % GPT, ky = tap / K, kx = tap % K;
-            if ((anym >> tap) & 1u) {
-                RsFrag<G> one;
-                int qb = q00;
-                asm volatile("" : "+r"(qb));
-                rs_load_group<G>(one, ((rowm >> ky) & 1u) && ((colm >> kx) & 1u), qb + ky * qrow + kx * nch + part * 2 * G, sb,
-                                 zaddr, waddr + s * G * 1024);
-                rs_mma_group<G>(acc, one);
-            }
-        }
-        return;
-    }
-    RsFrag<G> fr[2];
-    if (anym & 1u) rs_load_group<G>(fr[0], (rowm & 1u) && (colm & 1u), q00, sb, zaddr, waddr);
+    for (int ky = 0; ky < K; ++ky)
 #pragma unroll
-    for (int s = 0; s < S; ++s) {
-        if (s + 1 < S) {
-            const int tap = (s + 1) / GPT, part = (s + 1) % GPT, ky = tap / K, kx = tap % K;
-            if ((anym >> tap) & 1u) {
-                const bool ok = ((rowm >> ky) & 1u) && ((colm >> kx) & 1u);
-                int qb = q00;
-                asm volatile("" : "+r"(qb));         // keeps the address arithmetic of each group next to its loads
-                rs_load_group<G>(fr[(s + 1) & 1], ok, qb + ky * qrow + kx * nch + part * 2 * G, sb, zaddr,
-                                 waddr + (s + 1) * G * 1024);
-            }
+        for (int kx = 0; kx < K; ++kx) {
+            const uint32_t q = (uint32_t)(q00 + ky * qrow + kx * nch);
+            const bool ok = ((rowm >> ky) & 1u) && ((colm >> kx) & 1u);
+            ad[ky * K + kx] = ok ? sb + ((q ^ ((q >> 3) & 7u)) << 4) : zaddr;
         }
-        if ((anym >> (s / GPT)) & 1u) rs_mma_group<G>(acc, fr[s & 1]);
+    RsFrag<2> f0, f1;
+    auto load = [&](RsFrag<2>& fr, int s) {
+        const uint32_t a0 = ad[s / GPT] ^ (uint32_t)((s % GPT) * 64);
+        rs_ldsm4(fr.a[0], a0);
+        rs_ldsm4(fr.a[1], a0 ^ 32u);
+        rs_ldsm4(fr.b[0][0], waddr + s * 2048);
+        rs_ldsm4(fr.b[0][1], waddr + s * 2048 + 512);
+        rs_ldsm4(fr.b[1][0], waddr + s * 2048 + 1024);
+        rs_ldsm4(fr.b[1][1], waddr + s * 2048 + 1536);
+    };
+    load(f0, 0);
+#pragma unroll
+    for (int s = 0; s < S; s += 2) {
+        if (s + 1 < S) load(f1, s + 1);
+        rs_mma_group<2>(acc, f0);
+        if (s + 2 < S) load(f0, s + 2);
+        if (s + 1 < S) rs_mma_group<2>(acc, f1);
     }
 }
 
@@ -297,8 +312,9 @@ __device__ __forceinline__ void rs_conv_unit(const RsCtx& cx, const RsNode& nd, 
         const int etype = e.type, k = e.k, stride = e.stride, pad = e.pad, ksteps = e.ksteps, lut_off = e.lut_off;
         const RsNode& sn = cx.nodes[e.src];
         const int fb = f + 1 - e.R;                                   // relative frame of the source state (Eq. 2)
-        const int sbuf = sn.kind == RS_INPUT ? sn.buf[fb % 3] : sn.buf[fb & 1];
+        const int sbuf = sn.kind == RS_INPUT ? sn.buf[fb % sn.in_nb] : sn.buf[fb & 1];
         const int Ws = sn.W, Cs = sn.C, slo = sn.slo, shi = sn.shi;
+        (void)Cs;
         if (etype == RS_E_MMA) {
             const uint32_t sb = cx.sbase + sbuf;
             const int nch = Cs >> 3, nc16 = Cs >> 4;
@@ -308,36 +324,38 @@ __device__ __forceinline__ void rs_conv_unit(const RsCtx& cx, const RsNode& nd, 
                 rowm |= (uint32_t)(vl && iy0 + t >= slo && iy0 + t < shi) << t;    // stored rows cover every in-image row read
                 colm |= (uint32_t)((unsigned)(ix0 + t) < (unsigned)Ws) << t;
             }
-            uint32_t anym = 0xFFFFFFFFu;
-            if (k * k <= 32) {
-                uint32_t m = 0;
-                for (int t = 0; t < k; ++t)
-                    if ((rowm >> t) & 1u) m |= colm << (t * k);
-                anym = __reduce_or_sync(0xffffffffu, m);
-            }
             const int q00 = ((iy0 - slo) * Ws + ix0) * nch + khalf, qrow = Ws * nch;
             const int sel = (k == 3 ? 0 : k == 1 ? 4 : 8) + (nc16 == 2 ? 0 : nc16 == 4 ? 1 : 3);
             switch (sel) {
-                case 0: rs_mma_edge_unrolled<3, 2>(acc, rowm, colm, anym, q00, qrow, nch, sb, zaddr, waddr); break;
-                case 1: rs_mma_edge_unrolled<3, 4>(acc, rowm, colm, anym, q00, qrow, nch, sb, zaddr, waddr); break;
-                case 4: rs_mma_edge_unrolled<1, 2>(acc, rowm, colm, anym, q00, qrow, nch, sb, zaddr, waddr); break;
-                case 5: rs_mma_edge_unrolled<1, 4>(acc, rowm, colm, anym, q00, qrow, nch, sb, zaddr, waddr); break;
-                default: rs_mma_edge_generic(acc, k, nc16, rowm, colm, anym, q00, qrow, nch, sb, zaddr, waddr); break;
+                case 0: rs_mma_edge_unrolled<3, 2>(acc, rowm, colm, q00, qrow, nch, sb, zaddr, waddr); break;
+                case 1: rs_mma_edge_unrolled<3, 4>(acc, rowm, colm, q00, qrow, nch, sb, zaddr, waddr); break;
+                case 4: rs_mma_edge_unrolled<1, 2>(acc, rowm, colm, q00, qrow, nch, sb, zaddr, waddr); break;
+                case 5: rs_mma_edge_unrolled<1, 4>(acc, rowm, colm, q00, qrow, nch, sb, zaddr, waddr); break;
+                default: {
+                    // other filter sizes and channel counts: a plain loop; taps no lane of the warp needs are skipped
+                    uint32_t anym = 0xFFFFFFFFu;
+                    if (k * k <= 32) {
+                        uint32_t m = 0;
+                        for (int t = 0; t < k; ++t)
+                            if ((rowm >> t) & 1u) m |= colm << (t * k);
+                        anym = __reduce_or_sync(0xffffffffu, m);
+                    }
+                    rs_mma_edge_generic(acc, k, nc16, rowm, colm, anym, q00, qrow, nch, sb, zaddr, waddr);
+                    break;
+                }
             }
             waddr += (uint32_t)ksteps * 1024u;
         } else {
-            // few-channel edge: A fragments from scalar loads; the table gives (ky, kx, channel) of every k index
+            // few-channel edge (source = an input node, stored zero-padded): A fragments from scalar loads; the
+            // table gives the offset of every k index inside a pixel's window, so no bounds are checked
             const uint16_t* src = reinterpret_cast<const uint16_t*>(cx.smem + sbuf);
             const uint32_t* lut = reinterpret_cast<const uint32_t*>(cx.smem + lut_off);
-            int base[2], iy0[2], ix0[2];
-            bool pv[2];
+            const int g_const = e.g_const, g_ys = e.g_ys, g_xs = e.g_xs, tail = sn.in_tail;
+            int base[2];
 #pragma unroll
             for (int r = 0; r < 2; ++r) {
                 const uint32_t t = pix[j0 + g + 8 * r];
-                pv[r] = t != 0xFFFFFFFFu;
-                iy0[r] = (int)((t >> 15) & 0x7FFFu) * stride - pad;
-                ix0[r] = (int)(t & 0x7FFFu) * stride - pad;
-                base[r] = ((iy0[r] - slo) * Ws + ix0[r]) * Cs;
+                base[r] = t != 0xFFFFFFFFu ? g_const + (int)((t >> 15) & 0x7FFFu) * g_ys + (int)(t & 0x7FFFu) * g_xs : tail;
             }
             for (int ks = 0; ks < ksteps; ++ks) {
                 uint32_t a[4];
@@ -345,18 +363,8 @@ __device__ __forceinline__ void rs_conv_unit(const RsCtx& cx, const RsNode& nd, 
                 for (int h = 0; h < 2; ++h) {
                     const uint2 L = *reinterpret_cast<const uint2*>(lut + ks * 16 + h * 8 + 2 * tq);
 #pragma unroll
-                    for (int r = 0; r < 2; ++r) {
-                        uint32_t v[2];
-#pragma unroll
-                        for (int z = 0; z < 2; ++z) {
-                            const uint32_t t = z ? L.y : L.x;
-                            const int dy = (int)(t & 15u), dx = (int)((t >> 4) & 15u);
-                            const int iy = iy0[r] + dy, ix = ix0[r] + dx;
-                            const bool ok = pv[r] && (t >> 31) && iy >= slo && iy < shi && (unsigned)ix < (unsigned)Ws;
-                            v[z] = ok ? (uint32_t)src[base[r] + (dy * Ws + dx) * Cs + (int)((t >> 8) & 255u)] : 0u;
-                        }
-                        a[h * 2 + r] = v[0] | (v[1] << 16);
-                    }
+                    for (int r = 0; r < 2; ++r)
+                        a[h * 2 + r] = (uint32_t)src[base[r] + (int)L.x] | ((uint32_t)src[base[r] + (int)L.y] << 16);
                 }
                 uint32_t b0[4], b1[4];
                 rs_ldsm4(b0, waddr);
@@ -447,18 +455,19 @@ __device__ __forceinline__ void rs_dense_unit(const RsCtx& cx, const RsNode& nd,
                 }
             }
         }
+        // reduce-scatter over the warp: every step halves the values a lane keeps and adds the partner's copy of
+        // them (16 shuffles for 16 outputs instead of 80); lane l ends with the total of output ob + (l & 15)
+        float v8[8], v4[4], v2[2];
+        const bool h3 = lane & 8, h2 = lane & 4, h1 = lane & 2, h0 = lane & 1;
 #pragma unroll
-        for (int j = 0; j < 16; ++j) {
-            if (ob + j < C) {
+        for (int i = 0; i < 8; ++i) v8[i] = (h3 ? acc[i + 8] : acc[i]) + __shfl_xor_sync(0xffffffffu, h3 ? acc[i] : acc[i + 8], 8);
 #pragma unroll
-                for (int s = 16; s >= 1; s >>= 1) acc[j] += __shfl_xor_sync(0xffffffffu, acc[j], s);
-            }
-        }
+        for (int i = 0; i < 4; ++i) v4[i] = (h2 ? v8[i + 4] : v8[i]) + __shfl_xor_sync(0xffffffffu, h2 ? v8[i] : v8[i + 4], 4);
+#pragma unroll
+        for (int i = 0; i < 2; ++i) v2[i] = (h1 ? v4[i + 2] : v4[i]) + __shfl_xor_sync(0xffffffffu, h1 ? v4[i] : v4[i + 2], 2);
+        float v = (h0 ? v2[1] : v2[0]) + __shfl_xor_sync(0xffffffffu, h0 ? v2[0] : v2[1], 1);
+        v += __shfl_xor_sync(0xffffffffu, v, 16);
         if (lane < 16 && ob + lane < C) {
-            float v = 0.f;
-#pragma unroll
-            for (int j = 0; j < 16; ++j)
-                if (j == lane) v = acc[j];
             v *= scale;
             const uint32_t a = cx.sbase + slot_base + (uint32_t)(ob + lane) * 4u;
             if (cx.cs > 1) {
@@ -471,9 +480,10 @@ __device__ __forceinline__ void rs_dense_unit(const RsCtx& cx, const RsNode& nd,
 }
 
 __global__ void __launch_bounds__(kRsMaxThreads, 1)
-sr_resident_kernel(const unsigned char* __restrict__ blobs, int blob_stride, const SrFrameCtl* __restrict__ ctl, int T, int cs)
+sr_resident_kernel(const unsigned char* __restrict__ blobs, int blob_stride, SrFrameCtl* __restrict__ ctl_out,
+                   const __grid_constant__ SrFrameCtl init, int T, int cs)
 {
-    extern __shared__ __align__(1024) unsigned char smem[];
+    extern __shared__ __align__(128) unsigned char smem[];
     const int tid = threadIdx.x, nthr = blockDim.x;
     const uint32_t rank = cs > 1 ? rs_cluster_rank() : 0u;
     const int b = blockIdx.x / cs;                                    // the sequence this cluster rolls out
@@ -497,13 +507,33 @@ sr_resident_kernel(const unsigned char* __restrict__ blobs, int blob_stride, con
     const int32_t* ubegin = reinterpret_cast<const int32_t*>(smem + H.off_ubegin);
     const int warp = tid >> 5;
     if (tid < 32) reinterpret_cast<uint32_t*>(smem + H.zero_off)[tid] = 0u;
+    // the input buffers' padding stays zero for the whole run
+    for (int v = 0; v < H.n_nodes; ++v) {
+        const RsNode& nd = cx.nodes[v];
+        if (nd.kind != RS_INPUT) continue;
+        for (int k = 0; k < nd.in_nb; ++k)
+            for (int i = tid; i < (nd.buf_bytes >> 2); i += nthr) reinterpret_cast<uint32_t*>(smem + nd.buf[k])[i] = 0u;
+    }
+    __syncthreads();
     // parameters: packed convolution weights, dense weight slices, biases
     {
         const RsCopy* cp = reinterpret_cast<const RsCopy*>(smem + H.off_copies);
-        for (int c = 0; c < H.n_copies; ++c)
-            for (int i = tid * 16; i < cp[c].bytes; i += nthr * 16) rs_cp_async16(cx.sbase + cp[c].dst + i, cp[c].src + i);
+        // every cluster reads the same parameter blocks: each starts at a different 2 KiB-aligned place inside a
+        // block, so that at any moment the clusters pull different lines out of L2
+        for (int c = 0; c < H.n_copies; ++c) {
+            const int bytes = cp[c].bytes;
+            const int rot = (int)(((unsigned)b * 2048u) % (unsigned)bytes) & ~15;
+            for (int i = tid * 16; i < bytes; i += nthr * 16) {
+                int j = i + rot;
+                if (j >= bytes) j -= bytes;
+                rs_cp_async16(cx.sbase + cp[c].dst + j, cp[c].src + j);
+            }
+        }
     }
     // frame t of every node (relative frame 0), and the first input frame of the run (relative frame 1)
+    // `init` is the frame control block of this run (frame counter, the caller's input sequences and output);
+    // the block in global memory is brought up to date at the end, for the launches that follow
+    const SrFrameCtl* const ctl = &init;
     const long long t0 = ctl->t, run0 = ctl->run_t, out_stride = ctl->out_stride;
     float* const out_base = ctl->out_base;
     const int par0 = (int)(t0 & 1);
@@ -517,30 +547,33 @@ sr_resident_kernel(const unsigned char* __restrict__ blobs, int blob_stride, con
             const char* g = nd.gstate[par0] + ((size_t)b * nd.H + nd.slo) * nd.W * nd.C * 2;
             for (int q = tid; q < nq; q += nthr) rs_cp_async16(cx.sbase + nd.buf[0] + rs_swz((uint32_t)q) * 16u, g + (size_t)q * 16);
         } else {
-            const int nw = (nd.shi - nd.slo) * nd.W * nd.C / 2;       // 4-byte words (W * C is even)
+            // relative frame 0 from the state buffer; frames 1 .. in_lead - 1 from the caller's sequence
             const size_t row0 = ((size_t)b * nd.H + nd.slo) * nd.W * nd.C * 2;
-            const char* g0 = nd.gstate[par0] + row0;
-            const char* g1 = static_cast<const char*>(ctl->in_base[nd.input_slot]) + run0 * ctl->in_stride_bytes[nd.input_slot] + row0;
-            for (int i = tid; i < nw; i += nthr) {
-                rs_cp_async4(cx.sbase + nd.buf[0] + i * 4, g0 + (size_t)i * 4);
-                rs_cp_async4(cx.sbase + nd.buf[1] + i * 4, g1 + (size_t)i * 4);
-            }
+            rs_input_fetch(cx, nd, nd.gstate[par0] + row0, nd.buf[0], tid, nthr);
+            for (int k = 1; k < nd.in_lead && k <= T; ++k)
+                rs_input_fetch(cx, nd, static_cast<const char*>(ctl->in_base[nd.input_slot]) +
+                                           (run0 + k - 1) * ctl->in_stride_bytes[nd.input_slot] + row0, nd.buf[k % nd.in_nb], tid, nthr);
         }
+    }
+    __shared__ const char* in_ptr[SR_MAX_INPUTS];      // the caller's frame sequences, read once
+    __shared__ long long in_stride[SR_MAX_INPUTS];
+    if (tid < SR_MAX_INPUTS) {
+        in_stride[tid] = ctl->in_stride_bytes[tid];
+        in_ptr[tid] = static_cast<const char*>(ctl->in_base[tid]) + run0 * ctl->in_stride_bytes[tid];
     }
     rs_cp_async_wait_all();
     rs_level_barrier(cs);             // also: every CTA of the cluster runs before any remote store is issued
 
     for (int f = 0; f < T; ++f) {
-        // input frame of the NEXT update, fetched while this one computes
-        if (f + 1 < T && tid < H.input_words_max) {
+        // the input frame a later update reads (relative frame f + in_lead), fetched by one warp while this update
+        // computes (the host gave that warp fewer units)
+        if (warp == kRsFetchWarp) {
             for (int v = 0; v < H.n_nodes; ++v) {
                 const RsNode& nd = cx.nodes[v];
-                if (nd.kind != RS_INPUT) continue;
-                const int nw = (nd.shi - nd.slo) * nd.W * nd.C / 2;
-                const char* g = static_cast<const char*>(ctl->in_base[nd.input_slot]) +
-                                (run0 + f + 1) * ctl->in_stride_bytes[nd.input_slot] + ((size_t)b * nd.H + nd.slo) * nd.W * nd.C * 2;
-                const uint32_t dst = cx.sbase + nd.buf[(f + 2) % 3];
-                for (int i = tid; i < nw; i += nthr) rs_cp_async4(dst + i * 4, g + (size_t)i * 4);
+                if (nd.kind != RS_INPUT || f + nd.in_lead > T) continue;
+                const int fr = f + nd.in_lead;
+                rs_input_fetch(cx, nd, in_ptr[nd.input_slot] + (size_t)(fr - 1) * in_stride[nd.input_slot] +
+                                           ((size_t)b * nd.H + nd.slo) * nd.W * nd.C * 2, nd.buf[fr % nd.in_nb], cx.lane, 32);
             }
         }
         for (int l = 0; l < H.n_levels; ++l) {
@@ -555,14 +588,14 @@ sr_resident_kernel(const unsigned char* __restrict__ blobs, int blob_stride, con
             rs_level_barrier(cs);
             if ((H.dense_level_mask >> l) & 1) {
                 // dense nodes of this level: fixed-order sum of the slots (the bias is slot-independent), activation
-                if (warp == 0) {
+                if (warp == kRsFinalizeWarp) {
                     for (int v = 0; v < H.n_nodes; ++v) {
                         const RsNode& nd = cx.nodes[v];
                         if (nd.kind != RS_DENSE || nd.level != l) continue;
                         const int C = nd.C, n_slots = nd.n_slots;
                         const float* slots = reinterpret_cast<const float*>(smem + nd.slot_off) + ((f + 1) & 1) * n_slots * C;
                         const float* bias = reinterpret_cast<const float*>(smem + nd.bias_off);
-                        for (int o = tid; o < C; o += 32) {
+                        for (int o = cx.lane; o < C; o += 32) {
                             float z = 0.f;
                             for (int s = 0; s < n_slots; ++s) z += slots[s * C + o];
                             z += bias[o];
@@ -577,6 +610,13 @@ sr_resident_kernel(const unsigned char* __restrict__ blobs, int blob_stride, con
         }
     }
 
+    if (blockIdx.x == 0 && tid == 0) {
+        SrFrameCtl c = init;
+        c.t += T;
+        c.run_t += T;
+        c.error = ctl_out->error;
+        *ctl_out = c;
+    }
     // relative frame T back to the state buffers in global memory (parity of t + T)
     const int parT = (int)((t0 + T) & 1);
     for (int v = 0; v < H.n_nodes; ++v) {
@@ -593,10 +633,14 @@ sr_resident_kernel(const unsigned char* __restrict__ blobs, int blob_stride, con
                 *reinterpret_cast<uint4*>(g + (size_t)q * 16) =
                     *reinterpret_cast<const uint4*>(smem + nd.buf[T & 1] + rs_swz((uint32_t)(q + q0)) * 16u);
         } else {
-            const int nw = (nd.hi - nd.lo) * nd.W * nd.C / 2, w0 = (nd.lo - nd.slo) * nd.W * nd.C / 2;
+            const int wpr = nd.in_wpr, nw = (nd.hi - nd.lo) * wpr, r0 = nd.lo - nd.slo + nd.in_pt;
             char* g = nd.gstate[parT] + ((size_t)b * nd.H + nd.lo) * nd.W * nd.C * 2;
-            for (int i = tid; i < nw; i += nthr)
-                reinterpret_cast<uint32_t*>(g)[i] = reinterpret_cast<const uint32_t*>(smem + nd.buf[T % 3])[w0 + i];
+            const unsigned char* sbuf = smem + nd.buf[T % nd.in_nb];
+            for (int i = tid; i < nw; i += nthr) {
+                const int row = (int)(((unsigned)i * (unsigned)nd.in_magic) >> 20), col = i - row * wpr;
+                reinterpret_cast<uint32_t*>(g)[i] =
+                    *reinterpret_cast<const uint32_t*>(sbuf + (((row + r0) * nd.in_pitch + nd.in_ple) << 1) + col * 4);
+            }
         }
     }
 }
@@ -609,6 +653,8 @@ struct RsPlanNode {
     int first_edge = 0, ksteps = 0;
     size_t w_global = 0;            // byte offset of the packed weights inside the convolution-weight region
     bool has_consumers = false;
+    // input nodes: zero-padded buffer geometry (elements), buffers in rotation and how far ahead frames are fetched
+    int in_pitch = 0, in_pt = 0, in_pb = 0, in_ple = 0, in_tail_len = 0, in_wpr = 0, in_magic = 0, in_nb = 3, in_lead = 2;
 };
 
 struct RsPlanEdge {
@@ -699,12 +745,12 @@ bool rs_layout(const sr_graph* g, RsEngine& E, int cs, int warps)
         if (p.kind == RS_INPUT) continue;
         const int level = hn.level - 1;
         if (p.kind == RS_CONV) {
-            long cost = 80;                       // estimated warp instructions of a unit
+            // estimated cycles of a unit while all warps of the CTA are busy (measured on B200 with 16 warps: the
+            // warps of a scheduler share its tensor pipe and the CTA's shared-memory pipe)
+            long cost = 1700;
             for (int ei = 0; ei < (int)hn.in_edges.size(); ++ei) {
                 const RsPlanEdge& pe = E.pe[p.first_edge + ei];
-                const SrHostEdge& he = g->edges[pe.host_edge];
-                if (pe.type == RS_E_MMA) cost += (long)he.k_eff * he.k_eff * 12 + (long)pe.ksteps * 8;
-                else cost += (long)pe.ksteps * 90;
+                cost += (long)pe.ksteps * (pe.type == RS_E_MMA ? 160 : 400);
             }
             for (int r = 0; r < cs; ++r) {
                 const int npix = (p.lo[r + 1] - p.lo[r]) * hn.d.w;
@@ -725,7 +771,7 @@ bool rs_layout(const sr_graph* g, RsEngine& E, int cs, int warps)
                     const int per = (n + parts - 1) / parts;
                     for (int c0 = 0; c0 < n; c0 += per) {
                         const int c1 = std::min(n, c0 + per);
-                        const long cost = 40 + (long)((c1 - c0 + 31) / 32) * (12 + 17 * hn.d.c) + 7 * hn.d.c;
+                        const long cost = 2200 + (long)((c1 - c0 + 31) / 32) * 250 * hn.d.c;
                         cand[r].push_back(Cand{RsUnit{RS_U_DENSE, v, p.first_edge + ei, c0, c1, slot_count[v]++}, level, cost});
                     }
                 }
@@ -743,6 +789,18 @@ bool rs_layout(const sr_graph* g, RsEngine& E, int cs, int warps)
                 if (c.level == l) cs_l.push_back(c);
             std::stable_sort(cs_l.begin(), cs_l.end(), [](const Cand& a, const Cand& b) { return a.cost > b.cost; });
             std::vector<long> wl(warps, 0), pl(4, 0);
+            // fixed duties: the slot sums of the dense nodes of this level, the input fetch (last level's barrier waits for it)
+            bool dense_here = false;
+            for (int v = 0; v < n_nodes; ++v)
+                if (E.pn[v].kind == RS_DENSE && g->nodes[v].level - 1 == l) dense_here = true;
+            if (dense_here && kRsFinalizeWarp < warps) {
+                wl[kRsFinalizeWarp] += 3500;
+                pl[kRsFinalizeWarp % 4] += 3500;
+            }
+            if (l == 0 && kRsFetchWarp < warps) {
+                wl[kRsFetchWarp] += 2500;
+                pl[kRsFetchWarp % 4] += 2500;
+            }
             for (const Cand& c : cs_l) {
                 int bp = 0;
                 for (int p = 1; p < std::min(4, warps); ++p)
@@ -810,9 +868,9 @@ bool rs_layout(const sr_graph* g, RsEngine& E, int cs, int warps)
         int rows = 0;
         for (int r = 0; r < cs; ++r) rows = std::max(rows, p.shi[r] - p.slo[r]);
         if (p.kind == RS_DENSE) p.buf_bytes = rs_up16(d.c * 2);
-        else if (p.kind == RS_INPUT) p.buf_bytes = rs_up16(rows * d.w * d.c * 2);
+        else if (p.kind == RS_INPUT) p.buf_bytes = rs_up16(((p.in_pt + rows + p.in_pb) * p.in_pitch + p.in_tail_len) * 2);
         else p.buf_bytes = rs_up128(rows * d.w * d.c * 2);
-        const int nb = p.kind == RS_INPUT ? 3 : 2;
+        const int nb = p.kind == RS_INPUT ? p.in_nb : 2;
         for (int i = 0; i < nb; ++i) p.buf[i] = take(p.buf_bytes, 128);
     }
     for (int v = 0; v < n_nodes; ++v) {
@@ -887,12 +945,13 @@ void sr_rs_destroy(sr_graph* g)
 
 bool sr_rs_available(const sr_graph* g) { return g->rs != nullptr; }
 
-void sr_rs_describe(const sr_graph* g, int* cluster_size, int* warps, int* smem_bytes)
+void sr_rs_describe(const sr_graph* g, int* cluster_size, int* warps, int* smem_bytes, int* heads_on_chip)
 {
     const RsEngine* E = rs_of(g);
     *cluster_size = E ? E->cs : 0;
     *warps = E ? E->warps : 0;
     *smem_bytes = E ? E->smem_bytes : 0;
+    *heads_on_chip = E && E->dense_in_smem ? 1 : 0;
 }
 
 sr_status sr_rs_plan(sr_graph* g, size_t& offset)
@@ -963,18 +1022,53 @@ sr_status sr_rs_plan(sr_graph* g, size_t& offset)
         delete E;
         return SR_OK;
     }
-    // lookup tables of the few-channel edges: (ky, kx, channel) of every k index, valid bit 31
+    // input nodes are kept zero-padded (top / bottom rows, left / right columns as wide as any consumer's filter
+    // reaches) so that the few-channel path never checks bounds
+    for (int v = 0; v < n_nodes && ok; ++v) {
+        RsPlanNode& p = E->pn[v];
+        if (p.kind != RS_INPUT) continue;
+        const sr_node_desc& d = g->nodes[v].d;
+        int pt = 0, pb = 0, kmax = 1;
+        bool has0 = false, has1 = false;
+        for (const RsPlanEdge& pe : E->pe) {
+            const SrHostEdge& he = g->edges[pe.host_edge];
+            if (he.d.src != v) continue;
+            pt = std::max(pt, he.pad_eff);
+            pb = std::max(pb, he.k_eff - 1 - he.pad_eff);
+            kmax = std::max(kmax, he.k_eff);
+            (he.R ? has1 : has0) = true;
+        }
+        p.in_pt = pt;
+        p.in_pb = pb;
+        p.in_ple = (pt * d.c + 1) / 2 * 2;
+        p.in_pitch = (p.in_ple + d.w * d.c + pb * d.c + 1) / 2 * 2;
+        p.in_tail_len = ((kmax - 1) * p.in_pitch + kmax * d.c + 1) / 2 * 2;
+        p.in_wpr = d.w * d.c / 2;
+        p.in_magic = ((1 << 20) + p.in_wpr - 1) / p.in_wpr;
+        p.in_nb = (has0 && has1) ? 3 : 2;
+        p.in_lead = has0 ? 2 : 1;
+        const int nw = d.h * p.in_wpr;
+        if (nw > 8192) ok = false;
+        for (int i = 0; i < nw && ok; ++i)
+            if ((int)(((unsigned)i * (unsigned)p.in_magic) >> 20) != i / p.in_wpr) ok = false;
+    }
+    if (!ok) {
+        delete E;
+        return SR_OK;
+    }
+    // lookup tables of the few-channel edges: the offset of every k index (filter row, column, channel) inside a
+    // pixel's window of the padded source; padded k indices point at the window's first element (their weights are 0)
     E->luts.assign(E->pe.size(), std::vector<uint32_t>());
     for (size_t i = 0; i < E->pe.size(); ++i) {
         const RsPlanEdge& pe = E->pe[i];
         if (pe.type != RS_E_GATHER) continue;
         const SrHostEdge& he = g->edges[pe.host_edge];
-        const int Cs = g->nodes[he.d.src].d.c;
+        const int Cs = g->nodes[he.d.src].d.c, P = E->pn[he.d.src].in_pitch;
         std::vector<uint32_t>& L = E->luts[i];
         L.assign((size_t)pe.ksteps * 16, 0u);
         for (int kk = 0; kk < pe.Kreal; ++kk) {
             const int tap = kk / Cs, ci = kk % Cs;
-            L[kk] = (uint32_t)(tap / he.k_eff) | ((uint32_t)(tap % he.k_eff) << 4) | ((uint32_t)ci << 8) | 0x80000000u;
+            L[kk] = (uint32_t)((tap / he.k_eff) * P + (tap % he.k_eff) * Cs + ci);
         }
     }
     // cluster size: the largest that still gives every sequence its own cluster in one wave, else the
@@ -1079,6 +1173,14 @@ sr_status sr_rs_bind(sr_graph* g)
             d.slot_off = p.slot_off;
             d.n_slots = p.n_slots;
             d.has_consumers = p.has_consumers;
+            d.in_pitch = p.in_pitch; d.in_pt = p.in_pt; d.in_ple = p.in_ple; d.in_wpr = p.in_wpr; d.in_magic = p.in_magic;
+            d.in_nb = p.in_nb; d.in_lead = p.in_lead;
+            d.in_tail = 0;
+            if (p.kind == RS_INPUT) {
+                int rows = 0;
+                for (int rr = 0; rr < E.cs; ++rr) rows = std::max(rows, p.shi[rr] - p.slo[rr]);
+                d.in_tail = (p.in_pt + rows + p.in_pb) * p.in_pitch;
+            }
             d.pix_off = p.pix_off;
             if (p.kind == RS_CONV) {
                 uint32_t* pix = reinterpret_cast<uint32_t*>(blob.data() + p.pix_off);
@@ -1117,6 +1219,12 @@ sr_status sr_rs_bind(sr_graph* g)
             d.scale = 1.f;
             d.wd_global = nullptr;
             d.wd_gld = 0;
+            d.g_const = d.g_ys = d.g_xs = 0;
+            if (pe.type == RS_E_GATHER) {
+                d.g_const = (-he.pad_eff - sp.slo[r] + sp.in_pt) * sp.in_pitch + sp.in_ple - he.pad_eff * sd.c;
+                d.g_ys = he.stride_eff * sp.in_pitch;
+                d.g_xs = he.stride_eff * sd.c;
+            }
             if (pe.type == RS_E_GATHER)
                 std::memcpy(blob.data() + pe.lut_off, E.luts[i].data(), E.luts[i].size() * 4);
             if (he.d.kind != SR_EDGE_CONV) {
@@ -1236,7 +1344,7 @@ sr_status sr_rs_set_weights(sr_graph* g, int edge, const float* w_eff)
     return SR_OK;
 }
 
-sr_status sr_rs_launch(sr_graph* g, int T, cudaStream_t s)
+sr_status sr_rs_launch(sr_graph* g, int T, const SrFrameCtl& init, cudaStream_t s)
 {
     RsEngine* E = rs_of(g);
     if (!E) return SR_ERR_STATE;
@@ -1258,7 +1366,7 @@ sr_status sr_rs_launch(sr_graph* g, int T, cudaStream_t s)
     cfg.attrs = at;
     cfg.numAttrs = E->cs > 1 ? 1 : 0;
     const unsigned char* blobs = reinterpret_cast<const unsigned char*>(g->ws + E->r_blobs.offset);
-    const SrFrameCtl* ctl = reinterpret_cast<const SrFrameCtl*>(g->ws + g->r_ctl.offset);
+    SrFrameCtl* ctl = reinterpret_cast<SrFrameCtl*>(g->ws + g->r_ctl.offset);
     cudaStreamCaptureStatus cap = cudaStreamCaptureStatusNone;
     bool timed = g->opt_time_tc != 0 && cudaStreamIsCapturing(s, &cap) == cudaSuccess && cap == cudaStreamCaptureStatusNone;
     if (timed && E->ev_used + 2 > E->ev.size()) {
@@ -1271,7 +1379,7 @@ sr_status sr_rs_launch(sr_graph* g, int T, cudaStream_t s)
         if (E->ev_used + 2 > E->ev.size()) timed = false;
     }
     if (timed) cudaEventRecord(E->ev[E->ev_used], s);
-    if (cudaLaunchKernelEx(&cfg, sr_resident_kernel, blobs, E->blob_bytes, ctl, T, E->cs) != cudaSuccess) return SR_ERR_CUDA;
+    if (cudaLaunchKernelEx(&cfg, sr_resident_kernel, blobs, E->blob_bytes, ctl, init, T, E->cs) != cudaSuccess) return SR_ERR_CUDA;
     if (timed) {
         cudaEventRecord(E->ev[E->ev_used + 1], s);
         E->ev_used += 2;
