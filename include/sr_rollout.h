@@ -173,7 +173,7 @@ sr_status sr_graph_set_node_bias(sr_graph* g, int node, const float* bias_host);
  *                  the states on chip; 0 = always the per-frame launch path.  sr_rollout_step always uses
  *                  the launch path.
  *           key 7 "resident cluster size": CTAs per sequence, 1, 2 or 4; 0 (default) = chosen by the library.
- *           key 8 "resident warps": warps per CTA of the resident kernel, 4..16; 0 = default.
+ *           key 8 "resident warps": warps per CTA of the resident kernel, 4..32; 0 = default.
  * Must be set before sr_graph_workspace_bytes / sr_graph_bind_workspace (engine, weight ring, tile width,
  * resident keys) / before the first run (graphs). */
 sr_status sr_graph_set_option(sr_graph* g, int key, int value);

@@ -353,7 +353,7 @@ sr_status sr_graph_set_option(sr_graph* g, int key, int value)
     }
     if (key == 8) {
         if (g->ws) return SR_ERR_STATE;
-        if (value != 0 && (value < 4 || value > 16)) return SR_ERR_INVALID_ARG;
+        if (value != 0 && (value < 4 || value > 32)) return SR_ERR_INVALID_ARG;
         g->opt_rs_warps = value;
         return SR_OK;
     }
@@ -572,9 +572,9 @@ sr_status sr_rollout_run(sr_graph* g, const void* const* in_seq_dev, int T, floa
     sr_status st = ready(g);
     if (st != SR_OK) return st;
     if (!in_seq_dev || T < 0) return SR_ERR_INVALID_ARG;
+    if (T == 0) return SR_OK;                                    // an empty sequence: nothing to read, nothing changes
     for (size_t i = 0; i < g->input_nodes.size(); ++i)
         if (!in_seq_dev[i]) return SR_ERR_INVALID_ARG;
-    if (T == 0) return SR_OK;
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     if (sr_rs_available(g)) {
         bool aligned = true;                                     // the resident kernel fetches input rows in 4-byte words

@@ -42,7 +42,7 @@ namespace {
 
 constexpr int kRsMaxCluster = 4;
 constexpr int kRsSmemMax = 232448 - 128;      // 227 KiB per CTA minus the kernel's static shared memory
-constexpr int kRsMaxThreads = 512;
+constexpr int kRsMaxWarps = 32;
 constexpr int kRsDenseUnitChunks = 64;        // 16-byte chunks of the source per dense unit
 constexpr int kRsMaxDenseC = 64;
 constexpr int kRsFinalizeWarp = 0;            // sums the dense slots after a level's barrier
@@ -479,9 +479,10 @@ __device__ __forceinline__ void rs_dense_unit(const RsCtx& cx, const RsNode& nd,
     }
 }
 
-__global__ void __launch_bounds__(kRsMaxThreads, 1)
-sr_resident_kernel(const unsigned char* __restrict__ blobs, int blob_stride, SrFrameCtl* __restrict__ ctl_out,
-                   const __grid_constant__ SrFrameCtl init, int T, int cs)
+// The kernel body.  It is instantiated for 16, 24 and 32 warps per CTA (128, 80 and 64 registers per thread: the
+// code needs about 80, the compiler uses whatever the bound leaves), see the wrappers below.
+__device__ __forceinline__ void rs_kernel_body(const unsigned char* __restrict__ blobs, int blob_stride, SrFrameCtl* __restrict__ ctl_out,
+                                               const SrFrameCtl& init, int T, int cs)
 {
     extern __shared__ __align__(128) unsigned char smem[];
     const int tid = threadIdx.x, nthr = blockDim.x;
@@ -643,6 +644,14 @@ sr_resident_kernel(const unsigned char* __restrict__ blobs, int blob_stride, SrF
             }
         }
     }
+}
+
+template <int MAXT>
+__global__ void __launch_bounds__(MAXT, 1)
+sr_resident_kernel(const unsigned char* __restrict__ blobs, int blob_stride, SrFrameCtl* __restrict__ ctl_out,
+                   const __grid_constant__ SrFrameCtl init, int T, int cs)
+{
+    rs_kernel_body(blobs, blob_stride, ctl_out, init, T, cs);
 }
 
 // ------------------------------------------------------------------------------------------------ host side
@@ -1084,7 +1093,8 @@ sr_status sr_rs_plan(sr_graph* g, size_t& offset)
         for (int c = 1; c <= kRsMaxCluster; c <<= 1)
             if (g->batch * c > sms) order.push_back(c);
     }
-    const int warps = g->opt_rs_warps > 0 ? g->opt_rs_warps : 16;
+    // 24 warps (80 registers each) hide the shared-memory latencies best on B200; with 32 the 64-register build spills
+    const int warps = g->opt_rs_warps > 0 ? g->opt_rs_warps : 24;
     bool placed = false;
     for (int c : order)
         if (rs_layout(g, *E, c, warps)) {
@@ -1349,7 +1359,9 @@ sr_status sr_rs_launch(sr_graph* g, int T, const SrFrameCtl& init, cudaStream_t 
     RsEngine* E = rs_of(g);
     if (!E) return SR_ERR_STATE;
     if (!E->attr_set) {
-        if (cudaFuncSetAttribute(sr_resident_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, E->smem_bytes) != cudaSuccess)
+        if (cudaFuncSetAttribute(sr_resident_kernel<512>, cudaFuncAttributeMaxDynamicSharedMemorySize, E->smem_bytes) != cudaSuccess ||
+            cudaFuncSetAttribute(sr_resident_kernel<768>, cudaFuncAttributeMaxDynamicSharedMemorySize, E->smem_bytes) != cudaSuccess ||
+            cudaFuncSetAttribute(sr_resident_kernel<1024>, cudaFuncAttributeMaxDynamicSharedMemorySize, E->smem_bytes) != cudaSuccess)
             return SR_ERR_CUDA;
         E->attr_set = true;
     }
@@ -1379,7 +1391,11 @@ sr_status sr_rs_launch(sr_graph* g, int T, const SrFrameCtl& init, cudaStream_t 
         if (E->ev_used + 2 > E->ev.size()) timed = false;
     }
     if (timed) cudaEventRecord(E->ev[E->ev_used], s);
-    if (cudaLaunchKernelEx(&cfg, sr_resident_kernel, blobs, E->blob_bytes, ctl, init, T, E->cs) != cudaSuccess) return SR_ERR_CUDA;
+    cudaError_t le;
+    if (E->warps <= 16) le = cudaLaunchKernelEx(&cfg, sr_resident_kernel<512>, blobs, E->blob_bytes, ctl, init, T, E->cs);
+    else if (E->warps <= 24) le = cudaLaunchKernelEx(&cfg, sr_resident_kernel<768>, blobs, E->blob_bytes, ctl, init, T, E->cs);
+    else le = cudaLaunchKernelEx(&cfg, sr_resident_kernel<1024>, blobs, E->blob_bytes, ctl, init, T, E->cs);
+    if (le != cudaSuccess) return SR_ERR_CUDA;
     if (timed) {
         cudaEventRecord(E->ev[E->ev_used + 1], s);
         E->ev_used += 2;

@@ -35,11 +35,36 @@ def test_single_conv_edge(cin, cout, k, stride, pool, size, cluster):
         parity.check_run(g, "p", expect_resident=cluster, resident_cluster=cluster)
 
 
-@pytest.mark.parametrize("cluster,warps", [(2, 16), (2, 8), (2, 5), (4, 12)])
+@pytest.mark.parametrize("cluster,warps", [(2, 16), (2, 8), (2, 5), (4, 12), (2, 24), (2, 32), (4, 29)])
 def test_c2_reduced(cluster, warps):
     g = graphs.build("c2", batch=3, frames=6)
     for p in g.patterns:
         parity.check_run(g, p, expect_resident=cluster, resident_cluster=cluster, resident_warps=warps)
+
+
+@pytest.mark.parametrize("batch,frames", [(1, 1), (1, 2), (2, 3), (5, 7)])
+def test_short_runs_and_small_batches(batch, frames):
+    """One- and two-frame runs (the input look-ahead is longer than the run), a single sequence, an odd batch."""
+    g = graphs.build("mini", batch=batch, frames=frames)
+    for p in g.patterns:
+        parity.check_run(g, p, expect_resident=2, resident_cluster=2)
+    g = graphs.build("c2", batch=batch, frames=frames)
+    parity.check_run(g, "streaming", expect_resident=2, resident_cluster=2)
+
+
+def test_empty_run_is_a_no_op():
+    import torch
+    g = graphs.build("mini", batch=2, frames=2)
+    X, W, Bi = data.make_inputs(g), data.make_weights(g), data.make_biases(g, zero=False)
+    G = parity.make_graph(g, "streaming", "auto", 0, W, Bi)
+    x = parity.to_device(g, X[0])
+    G.reset([x[0]])
+    before = [G.get_state(v).clone() for v in range(len(g.nodes))]
+    G.run([x[1:1]])
+    G.sync_status()
+    assert G.frame() == 0
+    for v in range(len(g.nodes)):
+        assert torch.equal(G.get_state(v), before[v])
 
 
 def test_default_choice_and_opt_out():

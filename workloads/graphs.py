@@ -283,7 +283,9 @@ def mini_cnn(batch: int = 3, frames: int = 5, dtype: str = "bf16") -> GraphSpec:
              Edge(1, 1, CONV, 3, 1)]
     g = GraphSpec("mini", nodes, edges, batch, frames, dtype, seed=1010)
     g.patterns = {"streaming": streaming_pattern(g), "sequential": sequential_pattern(g),
-                  "hybrid": [0, 1, 1, 0, 1, 0, 0, 1, 0, 1]}
+                  "hybrid": [0, 1, 1, 0, 1, 0, 0, 1, 0, 1],
+                  # the input feeds one node inside the frame and another across frames
+                  "mixed_input": [1, 1, 1, 0, 1, 0, 0, 1, 0, 1]}
     return g
 
 
