@@ -174,6 +174,9 @@ sr_status sr_graph_set_node_bias(sr_graph* g, int node, const float* bias_host);
  *                  the launch path.
  *           key 7 "resident cluster size": CTAs per sequence, 1, 2 or 4; 0 (default) = chosen by the library.
  *           key 8 "resident warps": warps per CTA of the resident kernel, 4..32; 0 = default.
+ *           key 9 "resident tile width": 0 (default) = 16-pixel x 32-channel work units only, 1 = 16-channel units for
+ *                  every convolutional node, 2 = 16-channel units for the nodes whose 32-channel unit would be the
+ *                  longest dependent chain of a frame (more, shorter units; they load the activations twice).
  * Must be set before sr_graph_workspace_bytes / sr_graph_bind_workspace (engine, weight ring, tile width,
  * resident keys) / before the first run (graphs). */
 sr_status sr_graph_set_option(sr_graph* g, int key, int value);

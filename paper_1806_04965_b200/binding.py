@@ -106,7 +106,7 @@ class Graph:
 
     def __init__(self, nodes: Sequence, edges: Sequence, R: Sequence[int], batch: int = 0, dtype: str = "bf16",
                  engine: str = "auto", graph_frames: int = 0, device: str = "cuda:0", static_workspace: bool = False, weight_ring_units: int = 0, tile_width: int = 0,
-                 resident: bool = True, resident_cluster: int = 0, resident_warps: int = 0):
+                 resident: bool = True, resident_cluster: int = 0, resident_warps: int = 0, resident_split: int = 0):
         self._lib = load_library()
         self._h = ctypes.c_void_p()
         self.nodes, self.edges, self.R = list(nodes), list(edges), [int(r) for r in R]
@@ -133,6 +133,7 @@ class Graph:
             _check(self._lib.sr_graph_set_option(self._h, 6, 1 if resident else 0), "sr_graph_set_option")
             _check(self._lib.sr_graph_set_option(self._h, 7, int(resident_cluster)), "sr_graph_set_option")
             _check(self._lib.sr_graph_set_option(self._h, 8, int(resident_warps)), "sr_graph_set_option")
+            _check(self._lib.sr_graph_set_option(self._h, 9, int(resident_split)), "sr_graph_set_option")
             nbytes = ctypes.c_size_t()
             _check(self._lib.sr_graph_workspace_bytes(self._h, ctypes.byref(nbytes)), "sr_graph_workspace_bytes")
             self.workspace_bytes = nbytes.value

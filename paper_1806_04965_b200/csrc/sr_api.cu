@@ -351,6 +351,12 @@ sr_status sr_graph_set_option(sr_graph* g, int key, int value)
         g->opt_rs_cluster = value;
         return SR_OK;
     }
+    if (key == 9) {
+        if (g->ws) return SR_ERR_STATE;
+        if (value < 0 || value > 2) return SR_ERR_INVALID_ARG;
+        g->opt_rs_split = value;
+        return SR_OK;
+    }
     if (key == 8) {
         if (g->ws) return SR_ERR_STATE;
         if (value != 0 && (value < 4 || value > 32)) return SR_ERR_INVALID_ARG;

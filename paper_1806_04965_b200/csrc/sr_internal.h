@@ -85,7 +85,7 @@ struct sr_graph {
     std::vector<std::vector<int>> groups;          // groups[l-1] = nodes of level l
     // options
     int opt_engine = 0, opt_graph_frames = 0, opt_b_units = 0, opt_tile_w = 0, opt_overlap = 1, opt_time_tc = 0;
-    int opt_resident = 1, opt_rs_cluster = 0, opt_rs_warps = 0;
+    int opt_resident = 1, opt_rs_cluster = 0, opt_rs_warps = 0, opt_rs_split = 0;   // 16-channel work units: 0 never, 1 always, 2 by cost
     // workspace
     size_t ws_bytes = 0;
     char* ws = nullptr;

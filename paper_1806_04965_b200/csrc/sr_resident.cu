@@ -130,6 +130,11 @@ __device__ __forceinline__ void rs_st_cluster_v4(uint32_t addr, const uint32_t (
     asm volatile("st.shared::cluster.v4.u32 [%0], {%1,%2,%3,%4};" ::"r"(addr), "r"(v[0]), "r"(v[1]), "r"(v[2]), "r"(v[3]) : "memory");
 }
 
+__device__ __forceinline__ void rs_st_cluster_v2(uint32_t addr, uint32_t v0, uint32_t v1)
+{
+    asm volatile("st.shared::cluster.v2.u32 [%0], {%1,%2};" ::"r"(addr), "r"(v0), "r"(v1) : "memory");
+}
+
 __device__ __forceinline__ void rs_cp_async4(uint32_t dst, const void* src)
 {
     asm volatile("cp.async.ca.shared.global [%0], [%1], 4;" ::"r"(dst), "l"(src) : "memory");
@@ -175,37 +180,20 @@ __device__ __forceinline__ void rs_input_fetch(const RsCtx& cx, const RsNode& nd
     }
 }
 
-// Operand fragments of G consecutive k-steps (16 channels each) of one filter tap.
-template <int G>
+// Operand fragments of G consecutive k-steps (16 source channels each) of one filter tap for a tile of NB * 16
+// output channels.
+template <int G, int NB>
 struct RsFrag {
-    uint32_t a[G][4], b[G][2][4];
+    uint32_t a[G][4], b[G][NB][4];
 };
 
-// Chunk q of a swizzled state buffer lives at q ^ ((q >> 3) & 7).  Two consecutive k-steps of a tap read the
-// chunks q and q + 2; a pixel starts on an even chunk and holds at least four chunks whenever a tap has
-// more than one k-step, so the second address is the first XOR 32.  `waddr` points at the first k-step's
-// weights (1 KiB per k-step and 32 output channels).
-template <int G>
-__device__ __forceinline__ void rs_load_group(RsFrag<G>& fr, bool ok, int q0, uint32_t sb, uint32_t zaddr, uint32_t waddr)
-{
-    const uint32_t q = (uint32_t)q0;
-    const uint32_t base = sb + ((q ^ ((q >> 3) & 7u)) << 4);
-#pragma unroll
-    for (int i = 0; i < G; ++i) rs_ldsm4(fr.a[i], ok ? (base ^ (uint32_t)(32 * i)) : zaddr);
-#pragma unroll
-    for (int i = 0; i < G; ++i) {
-        rs_ldsm4(fr.b[i][0], waddr + i * 1024);
-        rs_ldsm4(fr.b[i][1], waddr + i * 1024 + 512);
-    }
-}
-
-template <int G>
-__device__ __forceinline__ void rs_mma_group(float (&acc)[4][4], const RsFrag<G>& fr)
+template <int G, int NB>
+__device__ __forceinline__ void rs_mma_group(float (&acc)[2 * NB][4], const RsFrag<G, NB>& fr)
 {
 #pragma unroll
     for (int i = 0; i < G; ++i)
 #pragma unroll
-        for (int nt = 0; nt < 4; ++nt)
+        for (int nt = 0; nt < 2 * NB; ++nt)
             rs_mma(acc[nt], fr.a[i], fr.b[i][nt >> 1][(nt & 1) * 2], fr.b[i][nt >> 1][(nt & 1) * 2 + 1]);
 }
 
@@ -218,8 +206,8 @@ __device__ __forceinline__ void rs_mma_group(float (&acc)[4][4], const RsFrag<G>
 // first address XOR 32, 64, 96 (the zero line used by out-of-image taps is 128 bytes long, so the XOR applies
 // to it as well).  `rowm` / `colm`: this lane's valid filter rows / columns; q00: the lane's chunk index at
 // tap (0, 0); the weights of the unit's k-steps are contiguous, 1 KiB each (constant offsets after unrolling).
-template <int K, int NC16>
-__device__ __forceinline__ void rs_mma_edge_unrolled(float (&acc)[4][4], uint32_t rowm, uint32_t colm, int q00, int qrow, int nch,
+template <int K, int NC16, int NB>
+__device__ __forceinline__ void rs_mma_edge_unrolled(float (&acc)[2 * NB][4], uint32_t rowm, uint32_t colm, int q00, int qrow, int nch,
                                                      uint32_t sb, uint32_t zaddr, uint32_t waddr)
 {
     constexpr int GPT = NC16 / 2, S = K * K * GPT;          // groups of two k-steps per tap, groups in all
@@ -232,28 +220,29 @@ __device__ __forceinline__ void rs_mma_edge_unrolled(float (&acc)[4][4], uint32_
             const bool ok = ((rowm >> ky) & 1u) && ((colm >> kx) & 1u);
             ad[ky * K + kx] = ok ? sb + ((q ^ ((q >> 3) & 7u)) << 4) : zaddr;
         }
-    RsFrag<2> f0, f1;
-    auto load = [&](RsFrag<2>& fr, int s) {
+    RsFrag<2, NB> f0, f1;
+    auto load = [&](RsFrag<2, NB>& fr, int s) {
         const uint32_t a0 = ad[s / GPT] ^ (uint32_t)((s % GPT) * 64);
         rs_ldsm4(fr.a[0], a0);
         rs_ldsm4(fr.a[1], a0 ^ 32u);
-        rs_ldsm4(fr.b[0][0], waddr + s * 2048);
-        rs_ldsm4(fr.b[0][1], waddr + s * 2048 + 512);
-        rs_ldsm4(fr.b[1][0], waddr + s * 2048 + 1024);
-        rs_ldsm4(fr.b[1][1], waddr + s * 2048 + 1536);
+#pragma unroll
+        for (int i = 0; i < 2; ++i)
+#pragma unroll
+            for (int j = 0; j < NB; ++j) rs_ldsm4(fr.b[i][j], waddr + s * 2048 + i * 1024 + j * 512);
     };
     load(f0, 0);
 #pragma unroll
     for (int s = 0; s < S; s += 2) {
         if (s + 1 < S) load(f1, s + 1);
-        rs_mma_group<2>(acc, f0);
+        rs_mma_group<2, NB>(acc, f0);
         if (s + 2 < S) load(f0, s + 2);
-        if (s + 1 < S) rs_mma_group<2>(acc, f1);
+        if (s + 1 < S) rs_mma_group<2, NB>(acc, f1);
     }
 }
 
 // The same for any filter size and channel count (not unrolled).
-__device__ __forceinline__ void rs_mma_edge_generic(float (&acc)[4][4], int k, int nc16, uint32_t rowm, uint32_t colm, uint32_t anym,
+template <int NB>
+__device__ __forceinline__ void rs_mma_edge_generic(float (&acc)[2 * NB][4], int k, int nc16, uint32_t rowm, uint32_t colm, uint32_t anym,
                                                     int q00, int qrow, int nch, uint32_t sb, uint32_t zaddr, uint32_t waddr)
 {
     int tap = 0;
@@ -264,37 +253,44 @@ __device__ __forceinline__ void rs_mma_edge_generic(float (&acc)[4][4], int k, i
             if (!((anym >> (tap & 31)) & 1u)) continue;
             const bool ok = rv && ((colm >> kx) & 1u);
             for (int c = 0; c < nc16; ++c) {
-                RsFrag<1> fr;
+                RsFrag<1, NB> fr;
                 const uint32_t q = (uint32_t)(q0 + 2 * c);
                 rs_ldsm4(fr.a[0], ok ? sb + ((q ^ ((q >> 3) & 7u)) << 4) : zaddr);
-                rs_ldsm4(fr.b[0][0], waddr + c * 1024);
-                rs_ldsm4(fr.b[0][1], waddr + c * 1024 + 512);
-                rs_mma_group<1>(acc, fr);
+#pragma unroll
+                for (int j = 0; j < NB; ++j) rs_ldsm4(fr.b[0][j], waddr + c * 1024 + j * 512);
+                rs_mma_group<1, NB>(acc, fr);
             }
         }
     }
 }
 
-// One (16 pixels x 32 channels) tile of a convolutional node: all k-steps of all incoming edges into one
+// One (16 pixels x NB * 16 channels) tile of a convolutional node: all k-steps of all incoming edges into one
 // accumulator, then bias, activation, bf16 cast and the stores into the next frame's buffer (own copy and,
 // for halo rows, the neighbour's).  `f` is the frame index relative to the start of the run: the update
-// computes relative frame f + 1.  Table fields are copied to registers before the loops that use them.
-__device__ __forceinline__ void rs_conv_unit(const RsCtx& cx, const RsNode& nd, int j0, int n0, int f)
+// computes relative frame f + 1.  n0 is the first channel of the 32-channel block; a 16-channel tile (NB = 1)
+// takes n-tiles 2 * half, 2 * half + 1 of the block.  Table fields are copied to registers before the loops
+// that use them.
+template <int NB>
+__device__ __forceinline__ void rs_conv_unit(const RsCtx& cx, const RsNode& nd, int j0, int n0, int half, int f)
 {
     const int lane = cx.lane;
     const int W = nd.W, C = nd.C, nslo = nd.slo, n_edges = nd.n_edges, first_edge = nd.first_edge;
     const uint32_t zaddr = cx.sbase + cx.H->zero_off;
-    // Column c of n-tile nt holds output channel n0 + (c >> 1) * 8 + nt * 2 + (c & 1) (the host packs the weights
-    // that way), so this lane's eight accumulator columns are the consecutive channels n0 + tq * 8 .. + 7: one
-    // 16-byte chunk per pixel.  The accumulators start at the bias.
-    float acc[4][4];
+    // Column c of n-tile nt of a block holds output channel n0 + (c >> 1) * 8 + nt * 2 + (c & 1) (the host packs the
+    // weights that way), so a lane's accumulator columns are consecutive channels: n0 + tq * 8 .. + 7 for a
+    // 32-channel tile (one 16-byte chunk per pixel), the lower or upper four of them for a 16-channel tile.
+    // The accumulators start at the bias.
+    float acc[2 * NB][4];
     {
-        const float* bias = reinterpret_cast<const float*>(cx.smem + nd.bias_off) + n0 + (lane & 3) * 8;
-        const float4 bl = *reinterpret_cast<const float4*>(bias), bh = *reinterpret_cast<const float4*>(bias + 4);
+        const float* bias = reinterpret_cast<const float*>(cx.smem + nd.bias_off) + n0 + (lane & 3) * 8 + (NB == 1 ? half * 4 : 0);
+        const float4 bl = *reinterpret_cast<const float4*>(bias);
         acc[0][0] = acc[0][2] = bl.x; acc[0][1] = acc[0][3] = bl.y;
         acc[1][0] = acc[1][2] = bl.z; acc[1][1] = acc[1][3] = bl.w;
-        acc[2][0] = acc[2][2] = bh.x; acc[2][1] = acc[2][3] = bh.y;
-        acc[3][0] = acc[3][2] = bh.z; acc[3][1] = acc[3][3] = bh.w;
+        if (NB == 2) {
+            const float4 bh = *reinterpret_cast<const float4*>(bias + 4);
+            acc[2 * NB - 2][0] = acc[2 * NB - 2][2] = bh.x; acc[2 * NB - 2][1] = acc[2 * NB - 2][3] = bh.y;
+            acc[2 * NB - 1][0] = acc[2 * NB - 1][2] = bh.z; acc[2 * NB - 1][1] = acc[2 * NB - 1][3] = bh.w;
+        }
     }
     // the pixel whose row address this lane supplies to ldmatrix, and the 8-channel half it points at
     // (table entry: bit 31 / 30 = the previous / next CTA keeps the pixel's row as halo, row << 15 | column;
@@ -306,7 +302,7 @@ __device__ __forceinline__ void rs_conv_unit(const RsCtx& cx, const RsNode& nd, 
     const int khalf = lane >> 4;
     const int g = lane >> 2, tq = lane & 3;       // accumulator rows g and g + 8, columns 2 * tq, 2 * tq + 1 of every n-tile
     // the packed weights of this unit's 32 channels: 1 KiB per k-step, k-steps of all edges in order
-    uint32_t waddr = cx.sbase + nd.w_off + (uint32_t)(n0 >> 5) * (uint32_t)nd.ksteps * 1024u + lane * 16;
+    uint32_t waddr = cx.sbase + nd.w_off + (uint32_t)(n0 >> 5) * (uint32_t)nd.ksteps * 1024u + lane * 16 + (NB == 1 ? half * 512 : 0);
     for (int ei = 0; ei < n_edges; ++ei) {
         const RsEdge& e = cx.edges[first_edge + ei];
         const int etype = e.type, k = e.k, stride = e.stride, pad = e.pad, ksteps = e.ksteps, lut_off = e.lut_off;
@@ -327,10 +323,10 @@ __device__ __forceinline__ void rs_conv_unit(const RsCtx& cx, const RsNode& nd, 
             const int q00 = ((iy0 - slo) * Ws + ix0) * nch + khalf, qrow = Ws * nch;
             const int sel = (k == 3 ? 0 : k == 1 ? 4 : 8) + (nc16 == 2 ? 0 : nc16 == 4 ? 1 : 3);
             switch (sel) {
-                case 0: rs_mma_edge_unrolled<3, 2>(acc, rowm, colm, q00, qrow, nch, sb, zaddr, waddr); break;
-                case 1: rs_mma_edge_unrolled<3, 4>(acc, rowm, colm, q00, qrow, nch, sb, zaddr, waddr); break;
-                case 4: rs_mma_edge_unrolled<1, 2>(acc, rowm, colm, q00, qrow, nch, sb, zaddr, waddr); break;
-                case 5: rs_mma_edge_unrolled<1, 4>(acc, rowm, colm, q00, qrow, nch, sb, zaddr, waddr); break;
+                case 0: rs_mma_edge_unrolled<3, 2, NB>(acc, rowm, colm, q00, qrow, nch, sb, zaddr, waddr); break;
+                case 1: rs_mma_edge_unrolled<3, 4, NB>(acc, rowm, colm, q00, qrow, nch, sb, zaddr, waddr); break;
+                case 4: rs_mma_edge_unrolled<1, 2, NB>(acc, rowm, colm, q00, qrow, nch, sb, zaddr, waddr); break;
+                case 5: rs_mma_edge_unrolled<1, 4, NB>(acc, rowm, colm, q00, qrow, nch, sb, zaddr, waddr); break;
                 default: {
                     // other filter sizes and channel counts: a plain loop; taps no lane of the warp needs are skipped
                     uint32_t anym = 0xFFFFFFFFu;
@@ -340,7 +336,7 @@ __device__ __forceinline__ void rs_conv_unit(const RsCtx& cx, const RsNode& nd, 
                             if ((rowm >> t) & 1u) m |= colm << (t * k);
                         anym = __reduce_or_sync(0xffffffffu, m);
                     }
-                    rs_mma_edge_generic(acc, k, nc16, rowm, colm, anym, q00, qrow, nch, sb, zaddr, waddr);
+                    rs_mma_edge_generic<NB>(acc, k, nc16, rowm, colm, anym, q00, qrow, nch, sb, zaddr, waddr);
                     break;
                 }
             }
@@ -366,46 +362,50 @@ __device__ __forceinline__ void rs_conv_unit(const RsCtx& cx, const RsNode& nd, 
                     for (int r = 0; r < 2; ++r)
                         a[h * 2 + r] = (uint32_t)src[base[r] + (int)L.x] | ((uint32_t)src[base[r] + (int)L.y] << 16);
                 }
-                uint32_t b0[4], b1[4];
-                rs_ldsm4(b0, waddr);
-                rs_ldsm4(b1, waddr + 512);
-                rs_mma(acc[0], a, b0[0], b0[1]);
-                rs_mma(acc[1], a, b0[2], b0[3]);
-                rs_mma(acc[2], a, b1[0], b1[1]);
-                rs_mma(acc[3], a, b1[2], b1[3]);
+#pragma unroll
+                for (int j = 0; j < NB; ++j) {
+                    uint32_t bj[4];
+                    rs_ldsm4(bj, waddr + j * 512);
+                    rs_mma(acc[2 * j], a, bj[0], bj[1]);
+                    rs_mma(acc[2 * j + 1], a, bj[2], bj[3]);
+                }
                 waddr += 1024;
             }
         }
     }
-    // epilogue: activation, bf16, one 16-byte store per pixel (and one into the neighbour's halo where the
-    // pixel table says so)
-    const uint32_t nchd = (uint32_t)(C >> 3), ch = (uint32_t)((n0 >> 3) + tq);
+    // epilogue: activation, bf16, one 16-byte (8-byte for a 16-channel tile) store per pixel, and one into the
+    // neighbour's halo where the pixel table says so
+    const uint32_t nchd = (uint32_t)(C >> 3), ch = (uint32_t)((n0 >> 3) + tq), sub = NB == 1 ? (uint32_t)half * 8u : 0u;
     const uint32_t dbuf = (uint32_t)nd.buf[(f + 1) & 1], buf_bytes = (uint32_t)nd.buf_bytes;
     const bool relu = nd.act == 1;
     const int d_up = (nslo - nd.up_slo) * W, d_dn = (nslo - nd.dn_slo) * W;
+    auto put = [&](uint32_t off, const uint32_t (&pk)[4], int peer) {
+        if (off >= buf_bytes) return;
+        if (peer < 0) {
+            if (NB == 2) *reinterpret_cast<uint4*>(cx.smem + dbuf + off) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
+            else *reinterpret_cast<uint2*>(cx.smem + dbuf + off + sub) = make_uint2(pk[0], pk[1]);
+        } else {
+            const uint32_t ra = rs_mapa(cx.sbase + dbuf + off + sub, (uint32_t)peer);
+            if (NB == 2) rs_st_cluster_v4(ra, pk);
+            else rs_st_cluster_v2(ra, pk[0], pk[1]);
+        }
+    };
 #pragma unroll
     for (int r = 0; r < 2; ++r) {
         const uint32_t t = pix[j0 + g + 8 * r];
         if (t == 0xFFFFFFFFu) continue;
         const int y = (int)((t >> 15) & 0x7FFFu), x = (int)(t & 0x7FFFu);
-        uint32_t pk[4];
+        uint32_t pk[4] = {0u, 0u, 0u, 0u};
 #pragma unroll
-        for (int nt = 0; nt < 4; ++nt) {
+        for (int nt = 0; nt < 2 * NB; ++nt) {
             __nv_bfloat162 v = __floats2bfloat162_rn(acc[nt][2 * r], acc[nt][2 * r + 1]);
             if (relu) v = __hmax2(v, __floats2bfloat162_rn(0.f, 0.f));
             pk[nt] = *reinterpret_cast<const uint32_t*>(&v);
         }
         const int lin = (y - nslo) * W + x;
-        const uint32_t off = rs_swz((uint32_t)lin * nchd + ch) * 16u;
-        if (off < buf_bytes) *reinterpret_cast<uint4*>(cx.smem + dbuf + off) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
-        if (t & 0x80000000u) {                     // the previous CTA of the cluster keeps this row as halo
-            const uint32_t o2 = rs_swz((uint32_t)(lin + d_up) * nchd + ch) * 16u;
-            if (o2 < buf_bytes) rs_st_cluster_v4(rs_mapa(cx.sbase + dbuf + o2, cx.rank - 1), pk);
-        }
-        if (t & 0x40000000u) {                     // the next one does
-            const uint32_t o2 = rs_swz((uint32_t)(lin + d_dn) * nchd + ch) * 16u;
-            if (o2 < buf_bytes) rs_st_cluster_v4(rs_mapa(cx.sbase + dbuf + o2, cx.rank + 1), pk);
-        }
+        put(rs_swz((uint32_t)lin * nchd + ch) * 16u, pk, -1);
+        if (t & 0x80000000u) put(rs_swz((uint32_t)(lin + d_up) * nchd + ch) * 16u, pk, (int)cx.rank - 1);   // halo of the previous CTA
+        if (t & 0x40000000u) put(rs_swz((uint32_t)(lin + d_dn) * nchd + ch) * 16u, pk, (int)cx.rank + 1);   // of the next one
     }
 }
 
@@ -582,7 +582,10 @@ __device__ __forceinline__ void rs_kernel_body(const unsigned char* __restrict__
             for (int u = ub; u < ue; ++u) {
                 const RsUnit& un = units[u];
                 const RsNode& nd = cx.nodes[un.node];
-                if (un.kind == RS_U_CONV) rs_conv_unit(cx, nd, un.a, un.b, f);
+                if (un.kind == RS_U_CONV) {
+                    if (un.c == 2) rs_conv_unit<2>(cx, nd, un.a, un.b, 0, f);
+                    else rs_conv_unit<1>(cx, nd, un.a, un.b, un.c, f);
+                }
                 else rs_dense_unit(cx, nd, cx.edges[un.a], un.b, un.c, un.d, f);
             }
             if (l == H.n_levels - 1) rs_cp_async_wait_all();
@@ -748,6 +751,33 @@ bool rs_layout(const sr_graph* g, RsEngine& E, int cs, int warps)
     std::vector<int> slot_count(n_nodes, 0);
     struct Cand { RsUnit u; int level; long cost; };
     std::vector<std::vector<Cand>> cand(cs);
+    // which nodes are cut into 16-channel tiles: those whose 32-channel tile alone would take more than half of a
+    // warp's fair share of its level
+    std::vector<char> split(n_nodes, 0);
+    if (g->opt_rs_split != 0) {
+        std::vector<long> level_cost(E.n_levels, 0), unit_cost(n_nodes, 0);
+        for (int v = 0; v < n_nodes; ++v) {
+            const RsPlanNode& p = E.pn[v];
+            const SrHostNode& hn = g->nodes[v];
+            if (p.kind == RS_INPUT) continue;
+            long c = 1700, units = 0;
+            if (p.kind == RS_CONV) {
+                for (int ei = 0; ei < (int)hn.in_edges.size(); ++ei) {
+                    const RsPlanEdge& pe = E.pe[p.first_edge + ei];
+                    c += (long)pe.ksteps * (pe.type == RS_E_MMA ? 160 : 400);
+                }
+                units = (long)(((p.lo[1] - p.lo[0]) * hn.d.w + 15) / 16) * (hn.d.c / 32);
+            } else {
+                c = 5000;
+                units = 4;
+            }
+            unit_cost[v] = c;
+            level_cost[hn.level - 1] += c * units;
+        }
+        for (int v = 0; v < n_nodes; ++v)
+            if (E.pn[v].kind == RS_CONV && (g->opt_rs_split == 1 || unit_cost[v] * 2 * warps > level_cost[g->nodes[v].level - 1]))
+                split[v] = 1;
+    }
     for (int v = 0; v < n_nodes; ++v) {
         const RsPlanNode& p = E.pn[v];
         const SrHostNode& hn = g->nodes[v];
@@ -761,10 +791,20 @@ bool rs_layout(const sr_graph* g, RsEngine& E, int cs, int warps)
                 const RsPlanEdge& pe = E.pe[p.first_edge + ei];
                 cost += (long)pe.ksteps * (pe.type == RS_E_MMA ? 160 : 400);
             }
+            // a unit is a 16-pixel x 32-channel tile (c = 2), or, for nodes with many k-steps when the CTA has more
+            // warps than such tiles, its two 16-channel halves (c = 0, 1): they load the A operand twice but halve the
+            // longest dependent chain of a frame
             for (int r = 0; r < cs; ++r) {
                 const int npix = (p.lo[r + 1] - p.lo[r]) * hn.d.w;
                 for (int j0 = 0; j0 < npix; j0 += 16)
-                    for (int n0 = 0; n0 < hn.d.c; n0 += 32) cand[r].push_back(Cand{RsUnit{RS_U_CONV, v, j0, n0, 0, 0}, level, cost});
+                    for (int n0 = 0; n0 < hn.d.c; n0 += 32) {
+                        if (split[v]) {
+                            cand[r].push_back(Cand{RsUnit{RS_U_CONV, v, j0, n0, 0, 0}, level, 1400 + (cost - 1700) * 6 / 10});
+                            cand[r].push_back(Cand{RsUnit{RS_U_CONV, v, j0, n0, 1, 0}, level, 1400 + (cost - 1700) * 6 / 10});
+                        } else {
+                            cand[r].push_back(Cand{RsUnit{RS_U_CONV, v, j0, n0, 2, 0}, level, cost});
+                        }
+                    }
             }
         } else {
             for (int ei = 0; ei < (int)hn.in_edges.size(); ++ei) {

@@ -18,6 +18,14 @@ def test_mini_cnn_every_pattern(cluster):
         parity.check_run(g, p, expect_resident=cluster, resident_cluster=cluster)
 
 
+@pytest.mark.parametrize("split", [1, 2])
+def test_both_tile_widths(split):
+    """16-channel work units for every convolutional node / for the nodes the cost rule picks (default: 32-channel units)."""
+    for g in (graphs.build("mini", batch=3, frames=4), graphs.build("c2", batch=2, frames=4)):
+        for p in g.patterns:
+            parity.check_run(g, p, expect_resident=2, resident_cluster=2, resident_split=split)
+
+
 @pytest.mark.parametrize("cin,cout,k,stride,pool,size,cluster", [
     (32, 32, 3, 1, 0, 12, 2), (64, 64, 3, 1, 0, 8, 1), (64, 32, 3, 2, 0, 16, 2), (128, 32, 3, 1, 0, 8, 2), (64, 96, 1, 2, 0, 8, 1),
     (32, 64, 5, 1, 0, 10, 2), (32, 32, 7, 4, 0, 28, 2), (64, 32, 3, 1, 2, 16, 4), (96, 32, 3, 1, 0, 9, 1), (32, 64, 1, 1, 0, 6, 2),
