@@ -75,6 +75,46 @@ def test_empty_run_is_a_no_op():
         assert torch.equal(G.get_state(v), before[v])
 
 
+def random_small_network(seed):
+    """A seeded random image network of the kind the resident kernel takes: 2-4 convolutional nodes of 32 or 64
+    channels on shrinking images, a chain plus random skips (1x1 or 3x3, stride = size ratio) and self-loops, a
+    dense or mean-dense head, and a random valid rollout pattern (forward edges drawn, recurrent edges bridge)."""
+    from workloads.graphs import CONV, DENSE, GAP_DENSE, IDENTITY, Edge, GraphSpec, Node, check_shapes
+    r = np.random.default_rng(seed)
+    size = int(r.choice([8, 12, 16, 20]))
+    nodes = [Node("in", size, size, int(r.choice([1, 2, 3])), IDENTITY)]
+    sizes = [size]
+    for i in range(int(r.integers(2, 5))):
+        s = sizes[-1] // 2 if (sizes[-1] % 2 == 0 and sizes[-1] >= 8 and r.random() < 0.5) else sizes[-1]
+        sizes.append(s)
+        nodes.append(Node("n%d" % (i + 1), s, s, int(r.choice([32, 64]))))
+    n_conv = len(nodes) - 1
+    nodes.append(Node("out", 1, 1, int(r.integers(3, 13)), IDENTITY))
+    edges = [Edge(i, i + 1, CONV, 3, sizes[i] // sizes[i + 1]) for i in range(n_conv)]
+    for i in range(n_conv + 1):
+        for j in range(i + 2, n_conv + 1):
+            if r.random() < 0.4 and sizes[i] % sizes[j] == 0:
+                edges.append(Edge(i, j, CONV, int(r.choice([1, 3])), sizes[i] // sizes[j]))
+    for i in range(1, n_conv + 1):
+        if r.random() < 0.4:
+            edges.append(Edge(i, i, CONV, 3, 1))
+    edges.append(Edge(n_conv, n_conv + 1, DENSE if r.random() < 0.5 else GAP_DENSE))
+    g = GraphSpec("rand%d" % seed, nodes, edges, batch=int(r.integers(1, 4)), frames=int(r.integers(2, 6)), dtype="bf16", seed=2000 + seed)
+    g.patterns = {"streaming": [1] * len(edges),
+                  "random": [1 if e.src >= e.tgt else int(r.random() < 0.5) for e in edges]}
+    check_shapes(g)
+    return g, int(r.choice([1, 2, 4]))
+
+
+@pytest.mark.parametrize("seed", range(12))
+def test_random_small_networks(seed):
+    g, cluster = random_small_network(seed)
+    if min(v.h for v in g.nodes[:-1]) < cluster:
+        cluster = 1
+    for p in g.patterns:
+        parity.check_run(g, p, resident_cluster=cluster)
+
+
 def test_default_choice_and_opt_out():
     from paper_1806_04965_b200 import Graph
     g = graphs.build("c2", batch=4, frames=2)
