@@ -32,6 +32,7 @@
 #include <cuda_runtime.h>
 
 #include <algorithm>
+#include <cstddef>
 #include <cstring>
 #include <vector>
 
@@ -52,32 +53,40 @@ enum { RS_INPUT = 0, RS_CONV = 1, RS_DENSE = 2 };
 enum { RS_E_MMA = 0, RS_E_GATHER = 1, RS_E_DENSE = 2, RS_E_MEAN = 3 };
 enum { RS_U_CONV = 0, RS_U_DENSE = 1 };
 
+// The first five 16-byte groups of RsNode and the first three of RsEdge are what a work unit needs; the unit
+// fetches them with 128-bit loads (a quarter of the shared-memory instructions of field-by-field reads, which
+// matter: the kernel is bound by the shared-memory pipe).  The static_asserts below pin the layout.
 struct RsNode {
-    int32_t kind, H, W, C;
-    int32_t act, level, lo, hi;              // level: 0-based tableau level; [lo, hi) rows owned by this CTA
-    int32_t slo, shi, is_output, input_slot; // [slo, shi) rows stored (own + halo)
-    int32_t buf[3], bias_off;                // byte offsets in shared memory (inputs rotate over three buffers)
-    int32_t w_off, first_edge, n_edges, buf_bytes;
-    int32_t ksteps, pad3, pad4, pad5;
-    // input nodes: zero-padded plain layout [top pad + rows + bottom pad][in_pitch] (+ a zero tail), see rs_input_fetch
-    int32_t in_pitch, in_pt, in_ple, in_tail, in_wpr, in_magic, in_nb, in_lead;
-    int32_t up_lo, up_hi, up_slo, dn_lo;     // own rows that the previous / next CTA of the cluster also stores
-    int32_t dn_hi, dn_slo, slot_off, n_slots;
-    int32_t has_consumers, pix_off, pad1, pad2;   // pix_off: table of the CTA's own pixels
+    int32_t kind, W, C, slo;                 // [slo, shi) rows stored by this CTA (own + halo)
+    int32_t shi, buf[3];                     // byte offsets of the state buffers in shared memory (inputs rotate over in_nb)
+    int32_t in_nb, in_tail, act, buf_bytes;
+    int32_t n_edges, first_edge, pix_off, bias_off;   // pix_off: table of the CTA's own pixels
+    int32_t w_off, ksteps, up_slo, dn_slo;   // up_slo / dn_slo: first stored row of the previous / next CTA of the cluster
+    int32_t H, level, lo, hi;                // level: 0-based tableau level; [lo, hi) rows owned by this CTA
+    int32_t is_output, input_slot, in_pitch, in_pt;   // input nodes: zero-padded plain layout [top pad + rows + bottom
+    int32_t in_ple, in_wpr, in_magic, in_lead;        // pad][in_pitch] (+ a zero tail), see rs_input_fetch
+    int32_t up_lo, up_hi, dn_lo, dn_hi;      // own rows that the previous / next CTA of the cluster also stores
+    int32_t slot_off, n_slots, has_consumers, pad0;
     char* gstate[2];                         // the node's two state buffers in global memory
 };
+static_assert(offsetof(RsNode, kind) == 0 && offsetof(RsNode, shi) == 16 && offsetof(RsNode, in_nb) == 32 &&
+              offsetof(RsNode, n_edges) == 48 && offsetof(RsNode, w_off) == 64 && sizeof(RsNode) % 16 == 0, "RsNode layout");
 
 struct RsEdge {
     int32_t src, type, k, stride;
     int32_t pad, R, ksteps, lut_off;
-    int32_t Kreal, wd_off, wd_ld, n_chunks;  // dense: weights in shared memory at wd_off (row pitch wd_ld elements) or < 0
-    int32_t x_chunk0, wchunk_mod;            // dense: first source chunk of this CTA's slice; mean-dense: chunks per pixel
+    int32_t g_const, g_ys, g_xs, Kreal;      // few-channel edge: element offset of the window of output pixel (0, 0) and
+                                             // its step per output row / column; Kreal = k * k * C_in
+    int32_t wd_off, wd_ld, n_chunks, x_chunk0;   // dense: weights in shared memory at wd_off (row pitch wd_ld elements) or < 0;
+                                                 // first source chunk of this CTA's slice
+    int32_t wchunk_mod;                      // mean-dense: chunks per pixel
     float scale;
-    int32_t g_const;                         // few-channel edge: element offset of the window of output pixel (0, 0)
-    int32_t g_ys, g_xs, pad_a, pad_b;        // ... and its step per output row / column
+    int32_t pad_a, pad_b;
     const char* wd_global;                   // dense weights in global memory, already at this CTA's slice
     int64_t wd_gld;                          // row pitch there, in elements
 };
+static_assert(offsetof(RsEdge, src) == 0 && offsetof(RsEdge, pad) == 16 && offsetof(RsEdge, g_const) == 32 &&
+              sizeof(RsEdge) % 16 == 0, "RsEdge layout");
 
 struct RsUnit { int32_t kind, node, a, b, c, d; };
 struct RsCopy { const char* src; int32_t dst, bytes; };
@@ -274,7 +283,9 @@ template <int NB>
 __device__ __forceinline__ void rs_conv_unit(const RsCtx& cx, const RsNode& nd, int j0, int n0, int half, int f)
 {
     const int lane = cx.lane;
-    const int W = nd.W, C = nd.C, nslo = nd.slo, n_edges = nd.n_edges, first_edge = nd.first_edge;
+    const uint4* np = reinterpret_cast<const uint4*>(&nd);
+    const uint4 nq0 = np[0], nq3 = np[3], nq4 = np[4];
+    const int W = (int)nq0.y, C = (int)nq0.z, nslo = (int)nq0.w, n_edges = (int)nq3.x, first_edge = (int)nq3.y;
     const uint32_t zaddr = cx.sbase + cx.H->zero_off;
     // Column c of n-tile nt of a block holds output channel n0 + (c >> 1) * 8 + nt * 2 + (c & 1) (the host packs the
     // weights that way), so a lane's accumulator columns are consecutive channels: n0 + tq * 8 .. + 7 for a
@@ -282,7 +293,7 @@ __device__ __forceinline__ void rs_conv_unit(const RsCtx& cx, const RsNode& nd, 
     // The accumulators start at the bias.
     float acc[2 * NB][4];
     {
-        const float* bias = reinterpret_cast<const float*>(cx.smem + nd.bias_off) + n0 + (lane & 3) * 8 + (NB == 1 ? half * 4 : 0);
+        const float* bias = reinterpret_cast<const float*>(cx.smem + nq3.w) + n0 + (lane & 3) * 8 + (NB == 1 ? half * 4 : 0);
         const float4 bl = *reinterpret_cast<const float4*>(bias);
         acc[0][0] = acc[0][2] = bl.x; acc[0][1] = acc[0][3] = bl.y;
         acc[1][0] = acc[1][2] = bl.z; acc[1][1] = acc[1][3] = bl.w;
@@ -295,21 +306,29 @@ __device__ __forceinline__ void rs_conv_unit(const RsCtx& cx, const RsNode& nd, 
     // the pixel whose row address this lane supplies to ldmatrix, and the 8-channel half it points at
     // (table entry: bit 31 / 30 = the previous / next CTA keeps the pixel's row as halo, row << 15 | column;
     // padded to a multiple of 16 pixels with 0xFFFFFFFF)
-    const uint32_t* pix = reinterpret_cast<const uint32_t*>(cx.smem + nd.pix_off);
+    const uint32_t* pix = reinterpret_cast<const uint32_t*>(cx.smem + nq3.z);
     const uint32_t tl = pix[j0 + (lane & 15)];
     const bool vl = tl != 0xFFFFFFFFu;
     const int oyl = (int)((tl >> 15) & 0x7FFFu), oxl = (int)(tl & 0x7FFFu);
     const int khalf = lane >> 4;
     const int g = lane >> 2, tq = lane & 3;       // accumulator rows g and g + 8, columns 2 * tq, 2 * tq + 1 of every n-tile
     // the packed weights of this unit's 32 channels: 1 KiB per k-step, k-steps of all edges in order
-    uint32_t waddr = cx.sbase + nd.w_off + (uint32_t)(n0 >> 5) * (uint32_t)nd.ksteps * 1024u + lane * 16 + (NB == 1 ? half * 512 : 0);
+    uint32_t waddr = cx.sbase + nq4.x + (uint32_t)(n0 >> 5) * nq4.y * 1024u + lane * 16 + (NB == 1 ? half * 512 : 0);
     for (int ei = 0; ei < n_edges; ++ei) {
         const RsEdge& e = cx.edges[first_edge + ei];
-        const int etype = e.type, k = e.k, stride = e.stride, pad = e.pad, ksteps = e.ksteps, lut_off = e.lut_off;
-        const RsNode& sn = cx.nodes[e.src];
-        const int fb = f + 1 - e.R;                                   // relative frame of the source state (Eq. 2)
-        const int sbuf = sn.kind == RS_INPUT ? sn.buf[fb % sn.in_nb] : sn.buf[fb & 1];
-        const int Ws = sn.W, Cs = sn.C, slo = sn.slo, shi = sn.shi;
+        const uint4* ep = reinterpret_cast<const uint4*>(&e);
+        const uint4 eq0 = ep[0], eq1 = ep[1];
+        const int etype = (int)eq0.y, k = (int)eq0.z, stride = (int)eq0.w, pad = (int)eq1.x, ksteps = (int)eq1.z, lut_off = (int)eq1.w;
+        const RsNode& sn = cx.nodes[eq0.x];
+        const uint4* sp = reinterpret_cast<const uint4*>(&sn);
+        const uint4 sq0 = sp[0], sq1 = sp[1];
+        const int fb = f + 1 - (int)eq1.y;                            // relative frame of the source state (Eq. 2)
+        int sbuf = (fb & 1) ? (int)sq1.z : (int)sq1.y;
+        if (sq0.x == RS_INPUT) {
+            const int bi = fb % sn.in_nb;
+            sbuf = bi == 0 ? (int)sq1.y : bi == 1 ? (int)sq1.z : (int)sq1.w;
+        }
+        const int Ws = (int)sq0.y, Cs = (int)sq0.z, slo = (int)sq0.w, shi = (int)sq1.x;
         (void)Cs;
         if (etype == RS_E_MMA) {
             const uint32_t sb = cx.sbase + sbuf;
@@ -346,7 +365,8 @@ __device__ __forceinline__ void rs_conv_unit(const RsCtx& cx, const RsNode& nd, 
             // table gives the offset of every k index inside a pixel's window, so no bounds are checked
             const uint16_t* src = reinterpret_cast<const uint16_t*>(cx.smem + sbuf);
             const uint32_t* lut = reinterpret_cast<const uint32_t*>(cx.smem + lut_off);
-            const int g_const = e.g_const, g_ys = e.g_ys, g_xs = e.g_xs, tail = sn.in_tail;
+            const uint4 eq2 = ep[2];
+            const int g_const = (int)eq2.x, g_ys = (int)eq2.y, g_xs = (int)eq2.z, tail = sn.in_tail;
             int base[2];
 #pragma unroll
             for (int r = 0; r < 2; ++r) {
@@ -376,9 +396,10 @@ __device__ __forceinline__ void rs_conv_unit(const RsCtx& cx, const RsNode& nd, 
     // epilogue: activation, bf16, one 16-byte (8-byte for a 16-channel tile) store per pixel, and one into the
     // neighbour's halo where the pixel table says so
     const uint32_t nchd = (uint32_t)(C >> 3), ch = (uint32_t)((n0 >> 3) + tq), sub = NB == 1 ? (uint32_t)half * 8u : 0u;
-    const uint32_t dbuf = (uint32_t)nd.buf[(f + 1) & 1], buf_bytes = (uint32_t)nd.buf_bytes;
-    const bool relu = nd.act == 1;
-    const int d_up = (nslo - nd.up_slo) * W, d_dn = (nslo - nd.dn_slo) * W;
+    const uint4 nq1 = np[1], nq2 = np[2], nq4e = np[4];      // fetched here, not kept in registers across the main loop
+    const uint32_t dbuf = ((f + 1) & 1) ? nq1.z : nq1.y, buf_bytes = nq2.w;
+    const bool relu = nq2.z == 1;
+    const int d_up = (nslo - (int)nq4e.z) * W, d_dn = (nslo - (int)nq4e.w) * W;
     auto put = [&](uint32_t off, const uint32_t (&pk)[4], int peer) {
         if (off >= buf_bytes) return;
         if (peer < 0) {
