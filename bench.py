@@ -29,7 +29,7 @@ from workloads import data, graphs  # noqa: E402
 # profiles/ (null where no capture of the current kernel exists)
 TRAFFIC = {"c2": 5.78e6, "c3": 264.1e6, "c4": 157.5e6, "c5": 612.4e6}
 # the same for one launch of the resident kernel (all T frames of the workload); null until captured for the current kernel
-TRAFFIC_RESIDENT = {"c2": 7.98e6}
+TRAFFIC_RESIDENT = {"c2": 8.00e6}
 
 METRIC = "streaming_rollout_frames_per_sec"
 UNIT = "frames/s"
