@@ -95,7 +95,7 @@ struct RsHeader {
     int32_t n_nodes, n_edges, n_levels, n_warps;
     int32_t off_nodes, off_edges, off_units, off_ubegin;
     int32_t off_copies, n_copies, zero_off, smem_bytes;
-    int32_t dense_level_mask, sync_after_finalize, blob_bytes, input_words_max;   // input_words_max: 4-byte words of the largest input slab
+    int32_t dense_level_mask, sync_after_finalize, blob_bytes, pad_;
 };
 
 // ------------------------------------------------------------------------------------------------ device helpers
@@ -1155,7 +1155,7 @@ sr_status sr_rs_plan(sr_graph* g, size_t& offset)
             if (g->batch * c > sms) order.push_back(c);
     }
     // 24 warps (80 registers each) hide the shared-memory latencies best on B200; with 32 the 64-register build spills
-    const int warps = g->opt_rs_warps > 0 ? g->opt_rs_warps : 24;
+    const int warps = std::min(kRsMaxWarps, g->opt_rs_warps > 0 ? g->opt_rs_warps : 24);
     bool placed = false;
     for (int c : order)
         if (rs_layout(g, *E, c, warps)) {
@@ -1349,10 +1349,6 @@ sr_status sr_rs_bind(sr_graph* g)
         H->dense_level_mask = dense_mask;
         H->sync_after_finalize = sync_after;
         H->blob_bytes = E.blob_bytes;
-        H->input_words_max = 0;
-        for (int v = 0; v < n_nodes; ++v)
-            if (E.pn[v].kind == RS_INPUT)
-                H->input_words_max = std::max(H->input_words_max, (E.pn[v].shi[r] - E.pn[v].slo[r]) * g->nodes[v].d.w * g->nodes[v].d.c / 2);
         if (cudaMemcpy(g->ws + E.r_blobs.offset + (size_t)r * E.blob_bytes, blob.data(), blob.size(), cudaMemcpyHostToDevice) !=
             cudaSuccess)
             return SR_ERR_CUDA;
