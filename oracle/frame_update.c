@@ -102,16 +102,19 @@ static void edge_transform(const sro_node* s, const sro_node* t, const sro_edge*
  * states[v] : [T+1][B][h][w][c] doubles, caller-allocated.  For input nodes the
  * caller has filled all frames; for the others this routine fills frames 0..T.
  * order[]   : the non-input nodes sorted by increasing tableau level.
+ * keep_frame0: 0 = frame 0 of every non-input node is set to zero (a rollout from the start);
+ *              1 = frame 0 is taken as the caller filled it: the window continues an earlier one, whose last
+ *                  frame becomes this window's frame 0 (Sec. 4, chaining of shallow rollout windows).
  * OpenMP spreads the independent (sample, output row) pairs of one node over the cores.
  * Returns 0, or -1 on a bad argument.
  */
 int sro_rollout(int n_nodes, const sro_node* nodes, int n_edges, const sro_edge* edges, const uint8_t* R,
                 const int32_t* order, int n_order, int B, int T,
                 const double* const* weights, const double* const* bias, double* const* states,
-                int round_states_bf16)
+                int round_states_bf16, int keep_frame0)
 {
     if (n_nodes <= 0 || n_edges <= 0 || B <= 0 || T < 0) return -1;
-    for (int i = 0; i < n_order; ++i) {                         /* frame 0: zero */
+    for (int i = 0; i < n_order && !keep_frame0; ++i) {         /* frame 0: zero */
         const sro_node* v = &nodes[order[i]];
         memset(states[order[i]], 0, sizeof(double) * (size_t)B * v->h * v->w * v->c);
     }

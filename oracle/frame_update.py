@@ -49,9 +49,11 @@ def _load():
 
 def rollout(nodes: Sequence, edges: Sequence, R: Sequence[int], batch: int, frames: int,
             inputs: Dict[int, np.ndarray], weights: List[np.ndarray], biases: List[np.ndarray],
-            round_states_bf16: bool = False) -> List[np.ndarray]:
+            round_states_bf16: bool = False, initial_states: Dict[int, np.ndarray] | None = None) -> List[np.ndarray]:
     """nodes: objects with h, w, c, act; edges: objects with src, tgt, kind, k, stride, pool.
-    inputs: {input node: [T+1][B][H][W][C]}.  Returns one float64 array [T+1][B][H][W][C] per node."""
+    inputs: {input node: [T+1][B][H][W][C]}.  Returns one float64 array [T+1][B][H][W][C] per node.
+    initial_states: {non-input node: [B][H][W][C]} makes the window continue an earlier one (its last frame is this
+    window's frame 0, paper Sec. 4); nodes left out start at zero."""
     lib = _load()
     n_nodes, n_edges = len(nodes), len(edges)
     pairs = [(e.src, e.tgt) for e in edges]
@@ -72,6 +74,8 @@ def rollout(nodes: Sequence, edges: Sequence, R: Sequence[int], batch: int, fram
             assert a.shape == (frames + 1, batch, n.h, n.w, n.c), (a.shape, vi)
         else:
             a = np.zeros((frames + 1, batch, n.h, n.w, n.c), dtype=np.float64)
+            if initial_states is not None and vi in initial_states:
+                a[0] = np.asarray(initial_states[vi], dtype=np.float64).reshape(a[0].shape)
         states.append(a)
     w64 = [np.ascontiguousarray(w, dtype=np.float64) for w in weights]
     b64 = [np.ascontiguousarray(b, dtype=np.float64) for b in biases]
@@ -80,7 +84,7 @@ def rollout(nodes: Sequence, edges: Sequence, R: Sequence[int], batch: int, fram
     c_b = (dp * n_nodes)(*[b.ctypes.data_as(dp) for b in b64])
     c_s = (dp * n_nodes)(*[s.ctypes.data_as(dp) for s in states])
     rc = lib.sro_rollout(n_nodes, c_nodes, n_edges, c_edges, c_R, c_order, len(order), batch, frames,
-                         c_w, c_b, c_s, int(round_states_bf16))
+                         c_w, c_b, c_s, int(round_states_bf16), int(initial_states is not None))
     if rc != 0:
         raise RuntimeError("sro_rollout failed: %d" % rc)
     return states

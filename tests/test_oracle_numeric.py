@@ -197,16 +197,22 @@ def test_numeric_dependence_on_input_frames_matches_theory():
 
 
 def test_resume_from_saved_states():
-    # chaining windows: running 2T frames equals running T, then restarting from the frame-T states
+    # chaining windows (Sec. 4): the last frame of a window is frame 0 of the next, so 6 frames in one go equal 3 frames,
+    # then 3 more frames started from the saved frame-3 states and fed input frames 3..6 - bit for bit, for a net with
+    # recurrence and a skip, under both rollouts; and the restart really uses the saved states (zeros give other values)
     g = graphs.mnist_net("SR", batch=2, frames=6)
     W, B = data.make_weights(g), data.make_biases(g, zero=False)
     X = {0: np.abs(randn(120, (7, 2, 28, 28, 1)))}
-    full = fu.rollout_spec(g, "streaming", X, W, B)
-    # the definition is first-order in frames: frame 4..6 from frame 3 states.  Re-run from scratch up to 3,
-    # then evaluate one more window by hand for the output node using frame-3 states.
-    part = fu.rollout_spec(g, "streaming", {0: X[0][:4]}, W, B, frames=3)
-    for v in range(len(g.nodes)):
-        assert np.array_equal(part[v][3], full[v][3])
+    for pattern in ("streaming", "sequential"):
+        full = fu.rollout_spec(g, pattern, X, W, B)
+        first = fu.rollout_spec(g, pattern, {0: X[0][:4]}, W, B, frames=3)
+        saved = {v: first[v][3] for v in range(1, len(g.nodes))}
+        second = fu.rollout_spec(g, pattern, {0: X[0][3:]}, W, B, frames=3, initial_states=saved)
+        cold = fu.rollout_spec(g, pattern, {0: X[0][3:]}, W, B, frames=3)
+        for v in range(len(g.nodes)):
+            assert np.array_equal(first[v][:4], full[v][:4])
+            assert np.array_equal(second[v], full[v][3:])
+        assert not np.array_equal(cold[3][1], full[3][4])
 
 
 def test_bf16_rounding_switch():
