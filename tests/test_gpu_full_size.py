@@ -1,8 +1,8 @@
 """GPU parity at the benchmark's full sizes, in the launch configuration bench.py times (sr_rollout_run
 with CUDA graphs of 16 frames, tensor cores where they apply).  The oracle evaluates a few whole
 sequences of the batch (sequences are independent, so those samples are exact); output sequence and
-final states of every node are compared.  c5 runs fewer frames at full size (the oracle needs about
-5 G multiply-adds per sample and frame) and all 128 frames at reduced image size."""
+final states of every node are compared.  The benchmarked runs themselves are compared in full length on one
+sequence each: c5 (64 x 64 images, all 128 frames; streaming and one hybrid) and c4 sequential (all 64 frames)."""
 import pytest
 
 from tests import parity
@@ -29,9 +29,9 @@ def test_c4_full_size_streaming():
     parity.check_run(g, "streaming", graph_frames=16, samples=[0, 127])
 
 
-def test_c4_full_batch_sequential_fewer_frames():
-    g = graphs.build("c4", frames=8)
-    parity.check_run(g, "sequential", graph_frames=0, samples=[64])
+def test_c4_full_size_sequential_all_frames():
+    g = graphs.build("c4")
+    parity.check_run(g, "sequential", graph_frames=16, samples=[64])
 
 
 def test_c5_full_size_fewer_frames():
@@ -40,6 +40,14 @@ def test_c5_full_size_fewer_frames():
     g2 = graphs.build("c5", frames=3)
     for p in ("sequential", "hybrid0", "hybrid1", "hybrid2"):
         parity.check_run(g2, p, graph_frames=0, samples=[17])
+
+
+@pytest.mark.parametrize("pattern", ["streaming", "hybrid1"])
+def test_c5_full_size_all_128_frames(pattern):
+    # the run bench.py times: batch 32, 64 x 64 images, 128 frames, CUDA graphs of 16 frames; the oracle follows one
+    # whole sequence (about 0.7 T multiply-adds), which is exact because sequences are independent
+    g = graphs.build("c5")
+    parity.check_run(g, pattern, graph_frames=16, samples=[13])
 
 
 def test_c5_all_128_frames_reduced_images():

@@ -72,3 +72,34 @@ def test_reference_arm_runs_on_rank_zero_only():
     line = json.loads(r.stdout.strip().splitlines()[-1])
     assert line["impl"] == "reference" and line["cpu_baseline"]["kind"] == "oracle" and line["value"] > 0
     assert line["e2e"]["h2d_bytes_per_step"] == 0
+
+
+def test_gpus_flag_spawns_one_process_per_rank():
+    # no WORLD_SIZE in the environment: bench.py starts the ranks itself, with the rendezvous variables set,
+    # and only rank 0's line reaches stdout
+    env = {k: v for k, v in os.environ.items() if k not in ("RANK", "WORLD_SIZE", "LOCAL_RANK", "MASTER_ADDR", "MASTER_PORT")}
+    r = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), "--impl", "reference", "--gpus", "2", "--steps", "1",
+                        "--warmup", "0", "--workload", "c1"], env=env, capture_output=True, text=True, timeout=300)
+    assert r.returncode == 0, r.stderr
+    import json
+    lines = [l for l in r.stdout.strip().splitlines() if l.startswith("{")]
+    assert len(lines) == 1
+    line = json.loads(lines[0])
+    assert line["impl"] == "reference" and line["n_gpus"] == 2 and line["config"]["parallelism"] == "replicas x2"
+
+
+def test_spawned_ranks_get_distinct_rendezvous_variables(tmp_path):
+    import bench
+    probe = tmp_path / "probe.py"
+    probe.write_text("import os, sys\n"
+                     "open(sys.argv[1] + os.environ['RANK'], 'w').write(' '.join(os.environ[k] for k in "
+                     "('RANK', 'LOCAL_RANK', 'WORLD_SIZE', 'MASTER_ADDR', 'MASTER_PORT')))\n")
+    saved = bench.__file__
+    try:
+        bench.__file__ = str(probe)
+        assert bench.spawn_ranks(3, [str(tmp_path / "rank")]) == 0
+    finally:
+        bench.__file__ = saved
+    got = [open(tmp_path / ("rank%d" % r)).read().split() for r in range(3)]
+    assert [g[0] for g in got] == ["0", "1", "2"] and [g[1] for g in got] == ["0", "1", "2"]
+    assert all(g[2] == "3" and g[3] == "127.0.0.1" for g in got) and len({g[4] for g in got}) == 1
