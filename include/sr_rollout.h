@@ -32,7 +32,8 @@
  *   - element type of states and input frames: float (dtype 0) or bfloat16 bit
  *     patterns (dtype 1).  Weights and biases are always passed as float; in
  *     bfloat16 mode weights are rounded to bfloat16 (nearest even) when stored.
- *     Outputs (`out_dev`, `out_seq_dev`) are always float.
+ *     Outputs (`out_dev`, `out_seq_dev`) are always float and have the output node's full shape,
+ *     [B][H][W][C] per frame ([B][C] for a dense output node, whose H = W = 1).
  */
 #ifndef SR_ROLLOUT_H
 #define SR_ROLLOUT_H
@@ -131,8 +132,10 @@ sr_status sr_graph_bind_workspace(sr_graph* g, void* workspace_dev, size_t bytes
  * library holds that much memory until the process exits, whether or not this call is ever made.
  *
  * Behaviour
- *   - allocates nothing on the device (no cudaMalloc / cudaFree, no allocating library call); inputs and
- *     outputs are still the caller's buffers, passed to reset / step / run as before;
+ *   - allocates no device memory (no cudaMalloc / cudaFree, no allocating library call); inputs and
+ *     outputs are still the caller's buffers, passed to reset / step / run as before.  Host-side objects are
+ *     still created later, as for any graph: the first step / run creates a stream and two events, and
+ *     sr_rollout_run with CUDA graphs enabled instantiates a graph;
  *   - the first call on a device looks the array's address up for that device (the device must be
  *     current) and remembers it; make that first call before any stream capture begins;
  *   - a graph whose sr_graph_workspace_bytes exceeds SR_STATIC_WORKSPACE_BYTES is refused with
@@ -141,7 +144,11 @@ sr_status sr_graph_bind_workspace(sr_graph* g, void* workspace_dev, size_t bytes
  *     binding clears the part the new graph uses (states start at zero) and parameters must be set
  *     again.  Only one such graph may be in use at a time: work of two graphs bound to the built-in
  *     workspace that overlaps on the GPU (different streams, or a new bind while an older graph's work
- *     is still queued) races on the same memory.  Synchronise before handing the array to the next graph.
+ *     is still queued) races on the same memory.  Synchronise before handing the array to the next graph;
+ *   - the array has one owner per device, the graph that bound it last.  A new bind takes it away from the
+ *     previous owner, which becomes unbound: its reset / step / run / get_state / set_state / parameter calls
+ *     return SR_ERR_STATE until it is bound again (to either kind of workspace) and given its parameters
+ *     again.  Concurrent binds from several host threads are serialised by the library.
  * Otherwise identical to sr_graph_bind_workspace: same kernels, same results.
  * Errors: INVALID_ARG, STATE (already bound, or theory-only graph), TOO_LARGE, CUDA.
  */
@@ -177,6 +184,11 @@ sr_status sr_graph_set_node_bias(sr_graph* g, int node, const float* bias_host);
  *           key 9 "resident tile width": 0 (default) = 16-pixel x 32-channel work units only, 1 = 16-channel units for
  *                  every convolutional node, 2 = 16-channel units for the nodes whose 32-channel unit would be the
  *                  longest dependent chain of a frame (more, shorter units; they load the activations twice).
+ *           key 10 "device wait limit": milliseconds (1..60000, default 1000) after which a wait inside a kernel (on a
+ *                  shared-memory barrier, on a descriptor queue) gives up; the kernel then records an error, waits
+ *                  for its own copies in flight, frees its tensor memory and returns, and sr_graph_sync_status
+ *                  reports SR_ERR_TIMEOUT.  0 is a test hook: every tensor-core launch reports the error at once and
+ *                  returns before it touches a barrier, a copy or an MMA.  May be set at any time.
  * Must be set before sr_graph_workspace_bytes / sr_graph_bind_workspace (engine, weight ring, tile width,
  * resident keys) / before the first run (graphs). */
 sr_status sr_graph_set_option(sr_graph* g, int key, int value);
@@ -184,7 +196,7 @@ sr_status sr_graph_set_option(sr_graph* g, int key, int value);
 /*
  * Frame 0 (Sec. A "Training details", Eq. 3): every non-input state := 0; input node i := in0_dev[i]
  * (one device pointer per input node, in increasing node order, each [B][H][W][C] of the graph dtype).
- * The frame counter returns to 0.
+ * The frame counter returns to 0 and a device-side error recorded earlier (SR_ERR_TIMEOUT) is cleared.
  */
 sr_status sr_graph_reset(sr_graph* g, const void* const* in0_dev, void* stream);
 
@@ -193,13 +205,14 @@ sr_status sr_graph_reset(sr_graph* g, const void* const* in0_dev, void* stream);
  * frame t+1; then, group by group, every node v of the group gets
  *     x_v^{t+1} = sigma_v( b_v + sum_e f_e(theta_e, x_src(e)^{t+1-R(e)}) )
  * and the buffers flip.  A streaming pattern runs ONE group.  If out_dev is not NULL it receives the
- * output node's new state as float [B][C_out].
+ * output node's new state as float [B][H][W][C_out] ([B][C_out] for a dense output node).
  */
 sr_status sr_rollout_step(sr_graph* g, const void* const* in_next_dev, float* out_dev, void* stream);
 
 /*
  * T frame updates without host round trips in between: in_seq_dev[i] points to the T frames
- * t+1..t+T of input node i, [T][B][H][W][C]; out_seq_dev (may be NULL) receives [T][B][C_out] floats.
+ * t+1..t+T of input node i, [T][B][H][W][C]; out_seq_dev (may be NULL) receives T frames of the output node's
+ * shape, [T][B][H][W][C_out] floats.
  * Equivalent to T calls of sr_rollout_step.
  */
 sr_status sr_rollout_run(sr_graph* g, const void* const* in_seq_dev, int T, float* out_seq_dev, void* stream);
@@ -217,7 +230,8 @@ sr_status sr_graph_launch_count(const sr_graph* g, int64_t* n);
 /* Sum of the event-timed durations (milliseconds) and the number of tensor-core group launches and resident
  * launches since the previous call (option key 5); waits for those launches to finish. */
 sr_status sr_graph_kernel_time(sr_graph* g, double* ms, int64_t* launches);
-/* Synchronises `stream` and reports SR_ERR_CUDA / SR_ERR_TIMEOUT if queued work failed. */
+/* Synchronises `stream` and reports SR_ERR_CUDA / SR_ERR_TIMEOUT if queued work failed.  A recorded time-out stays
+ * recorded, and is reported by every later call, until sr_graph_reset starts the rollout over. */
 sr_status sr_graph_sync_status(sr_graph* g, void* stream);
 
 const char* sr_status_str(sr_status s);

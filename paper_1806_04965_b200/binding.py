@@ -106,7 +106,8 @@ class Graph:
 
     def __init__(self, nodes: Sequence, edges: Sequence, R: Sequence[int], batch: int = 0, dtype: str = "bf16",
                  engine: str = "auto", graph_frames: int = 0, device: str = "cuda:0", static_workspace: bool = False, weight_ring_units: int = 0, tile_width: int = 0,
-                 resident: bool = True, resident_cluster: int = 0, resident_warps: int = 0, resident_split: int = 0):
+                 resident: bool = True, resident_cluster: int = 0, resident_warps: int = 0, resident_split: int = 0,
+                 wait_limit_ms: Optional[int] = None):
         self._lib = load_library()
         self._h = ctypes.c_void_p()
         self.nodes, self.edges, self.R = list(nodes), list(edges), [int(r) for r in R]
@@ -134,6 +135,8 @@ class Graph:
             _check(self._lib.sr_graph_set_option(self._h, 7, int(resident_cluster)), "sr_graph_set_option")
             _check(self._lib.sr_graph_set_option(self._h, 8, int(resident_warps)), "sr_graph_set_option")
             _check(self._lib.sr_graph_set_option(self._h, 9, int(resident_split)), "sr_graph_set_option")
+            if wait_limit_ms is not None:
+                _check(self._lib.sr_graph_set_option(self._h, 10, int(wait_limit_ms)), "sr_graph_set_option")
             nbytes = ctypes.c_size_t()
             _check(self._lib.sr_graph_workspace_bytes(self._h, ctypes.byref(nbytes)), "sr_graph_workspace_bytes")
             self.workspace_bytes = nbytes.value
@@ -191,10 +194,15 @@ class Graph:
     def reset(self, in0):
         _check(self._lib.sr_graph_reset(self._h, self._ptrs(in0), self._stream()), "sr_graph_reset")
 
+    def out_shape(self):
+        """Shape of one frame of output: the output node's state, [B][C] for a dense node, else [B][H][W][C]."""
+        nd = self.nodes[self.output_node]
+        return (self.batch, nd.c) if nd.h == 1 and nd.w == 1 else (self.batch, nd.h, nd.w, nd.c)
+
     def step(self, in_next, out=None):
         if out is not None:
             assert out.is_cuda and out.is_contiguous() and out.dtype == self._torch.float32
-            assert tuple(out.shape) == (self.batch, self.nodes[self.output_node].c)
+            assert tuple(out.shape) == self.out_shape()
         _check(self._lib.sr_rollout_step(self._h, self._ptrs(in_next), out.data_ptr() if out is not None else None,
                                          self._stream()), "sr_rollout_step")
 
@@ -202,7 +210,7 @@ class Graph:
         T = int(in_seq[0].shape[0])
         if out_seq is not None:
             assert out_seq.is_cuda and out_seq.is_contiguous() and out_seq.dtype == self._torch.float32
-            assert tuple(out_seq.shape) == (T, self.batch, self.nodes[self.output_node].c)
+            assert tuple(out_seq.shape) == (T,) + self.out_shape()
         _check(self._lib.sr_rollout_run(self._h, self._ptrs(in_seq, T), T,
                                         out_seq.data_ptr() if out_seq is not None else None, self._stream()),
                "sr_rollout_run")
@@ -245,8 +253,7 @@ class Graph:
         """frames: one tensor [T+1][B][H][W][C] per input node (frames 0..T).  Resets to frame 0,
         runs T updates, returns the outputs [T][B][C_out] (float32)."""
         T = int(frames[0].shape[0]) - 1
-        out = self._torch.empty((T, self.batch, self.nodes[self.output_node].c), dtype=self._torch.float32,
-                                device=self.device)
+        out = self._torch.empty((T,) + self.out_shape(), dtype=self._torch.float32, device=self.device)
         self.reset([f[0] for f in frames])
         self.run([f[1:] for f in frames], out)
         return out

@@ -3,7 +3,9 @@
 #include <cuda_runtime.h>
 
 #include <algorithm>
+#include <cstddef>
 #include <cstring>
+#include <mutex>
 #include <new>
 #include <vector>
 
@@ -12,7 +14,38 @@
 #include "sr_resident.h"
 #include "sr_tc.h"
 
+// Built-in workspace for callers that may not allocate device memory.  In host code the array's name
+// is only a handle: its device address is looked up once per device and that pointer is what the
+// kernels get (through the ordinary bind path).
+static __device__ __align__(256) unsigned char sr_static_workspace[SR_STATIC_WORKSPACE_BYTES];
+
 namespace {
+
+// One owner per device: the graph that bound the array last.  Binding takes the array away from the previous owner,
+// which becomes unbound (its calls then fail with SR_ERR_STATE on the host instead of running kernels on tables the
+// new owner has overwritten).
+struct StaticSlot {
+    void* address = nullptr;
+    sr_graph* owner = nullptr;
+};
+std::mutex static_mutex;
+StaticSlot static_slot[64];
+
+void unbind(sr_graph* g)
+{
+    g->ws = nullptr;
+    g->static_device = -1;
+    for (SrHostEdge& e : g->edges) e.w_set = false;
+    for (SrHostNode& n : g->nodes) n.bias_set = false;
+}
+
+void sr_release_static_workspace(sr_graph* g)
+{
+    std::lock_guard<std::mutex> lock(static_mutex);
+    if (g->static_device >= 0 && g->static_device < 64 && static_slot[g->static_device].owner == g)
+        static_slot[g->static_device].owner = nullptr;
+    g->static_device = -1;
+}
 
 struct GraphCache {
     cudaStream_t capture_stream = nullptr;
@@ -156,6 +189,7 @@ sr_status plan(sr_graph* g)
 
 bool cuda_ok(cudaError_t e) { return e == cudaSuccess; }
 
+
 sr_status ready(const sr_graph* g)
 {
     if (!g) return SR_ERR_INVALID_ARG;
@@ -229,7 +263,7 @@ SrFrameCtl make_ctl(const sr_graph* g, const void* const* in, bool sequence, flo
         c.in_stride_bytes[i] = sequence ? (int64_t)(node_elems(g, g->input_nodes[i]) * g->elem) : 0;
     }
     c.out_base = out;
-    c.out_stride = (int64_t)g->batch * g->nodes[g->info.output_node].d.c;
+    c.out_stride = (int64_t)node_elems(g, g->info.output_node);          // [B][H][W][C] floats per frame
     return c;
 }
 
@@ -271,6 +305,7 @@ sr_status sr_graph_create(const sr_node_desc* nodes, int n_nodes, const sr_edge_
 void sr_graph_destroy(sr_graph* g)
 {
     if (!g) return;
+    sr_release_static_workspace(g);
     if (g->graphs) {
         GraphCache* c = static_cast<GraphCache*>(g->graphs);
         if (c->exec) cudaGraphExecDestroy(c->exec);
@@ -363,6 +398,16 @@ sr_status sr_graph_set_option(sr_graph* g, int key, int value)
         g->opt_rs_warps = value;
         return SR_OK;
     }
+    if (key == 10) {
+        if (value < 0 || value > 60000) return SR_ERR_INVALID_ARG;
+        g->opt_wait_ms = value;
+        if (g->graphs) {                                 // recorded launches carry the old limit
+            GraphCache* c = static_cast<GraphCache*>(g->graphs);
+            if (c->exec) cudaGraphExecDestroy(c->exec);
+            c->exec = nullptr;
+        }
+        return SR_OK;
+    }
     return SR_ERR_INVALID_ARG;
 }
 
@@ -384,6 +429,11 @@ sr_status sr_graph_bind_workspace(sr_graph* g, void* workspace_dev, size_t bytes
     if (!g || !workspace_dev) return SR_ERR_INVALID_ARG;
     if (g->ws) return SR_ERR_STATE;
     if (reinterpret_cast<uintptr_t>(workspace_dev) & 255) return SR_ERR_INVALID_ARG;
+    if (g->graphs) {                                     // launches recorded for an earlier binding point at its tables
+        GraphCache* c = static_cast<GraphCache*>(g->graphs);
+        if (c->exec) cudaGraphExecDestroy(c->exec);
+        c->exec = nullptr;
+    }
     sr_status st = plan(g);
     if (st != SR_OK) return st;
     if (bytes < g->ws_bytes) return SR_ERR_INVALID_ARG;
@@ -440,28 +490,30 @@ sr_status sr_graph_bind_workspace(sr_graph* g, void* workspace_dev, size_t bytes
     return SR_OK;
 }
 
-// Built-in workspace for callers that may not allocate device memory.  In host code the array's name
-// is only a handle: its device address is looked up once per device and that pointer is what the
-// kernels get (through the ordinary bind path).
-static __device__ __align__(256) unsigned char sr_static_workspace[SR_STATIC_WORKSPACE_BYTES];
-
 sr_status sr_graph_bind_static_workspace(sr_graph* g)
 {
-    static void* address_on_device[64] = {nullptr};
     if (!g) return SR_ERR_INVALID_ARG;
     if (g->ws || g->batch <= 0) return SR_ERR_STATE;
     size_t need = 0;
-    const sr_status st = sr_graph_workspace_bytes(g, &need);
+    sr_status st = sr_graph_workspace_bytes(g, &need);
     if (st != SR_OK) return st;
     if (need > (size_t)SR_STATIC_WORKSPACE_BYTES) return SR_ERR_TOO_LARGE;
     int dev = -1;
     if (!cuda_ok(cudaGetDevice(&dev)) || dev < 0 || dev >= 64) return SR_ERR_CUDA;
-    if (!address_on_device[dev]) {
+    std::lock_guard<std::mutex> lock(static_mutex);
+    StaticSlot& slot = static_slot[dev];
+    if (!slot.address) {
         void* p = nullptr;
         if (!cuda_ok(cudaGetSymbolAddress(&p, sr_static_workspace)) || !p) return SR_ERR_CUDA;
-        address_on_device[dev] = p;
+        slot.address = p;
     }
-    return sr_graph_bind_workspace(g, address_on_device[dev], (size_t)SR_STATIC_WORKSPACE_BYTES);
+    if (slot.owner && slot.owner != g) unbind(slot.owner);
+    slot.owner = nullptr;
+    st = sr_graph_bind_workspace(g, slot.address, (size_t)SR_STATIC_WORKSPACE_BYTES);
+    if (st != SR_OK) return st;
+    slot.owner = g;
+    g->static_device = dev;
+    return SR_OK;
 }
 
 sr_status sr_graph_set_edge_weights(sr_graph* g, int edge, const float* w, int is_device)
@@ -552,6 +604,8 @@ sr_status sr_graph_reset(sr_graph* g, const void* const* in0_dev, void* stream)
             if (!cuda_ok(cudaMemsetAsync(g->ws + n.state[1].offset, 0, bytes, s))) return SR_ERR_CUDA;
         }
     }
+    // a reported device-side error (an expired wait) is cleared here: the rollout starts over
+    if (!cuda_ok(cudaMemsetAsync(g->ws + g->r_ctl.offset + offsetof(SrFrameCtl, error), 0, sizeof(int32_t), s))) return SR_ERR_CUDA;
     g->t = 0;
     g->stage_dirty = false;
     g->launches += sr_tc_after_state_change(g, s);
@@ -620,10 +674,21 @@ sr_status sr_rollout_run(sr_graph* g, const void* const* in_seq_dev, int T, floa
             int k = enqueue_frames(g, 0, gf, c->capture_stream);
             sr_launch_advance(g, gf, c->capture_stream);
             ++k;
-            if (!cuda_ok(cudaStreamEndCapture(c->capture_stream, &graph)) || !graph) return SR_ERR_CUDA;
+            // a capture that has begun is always ended, also when a launch inside it failed: a stream left in
+            // capture mode would refuse every later use
+            const bool queued = cuda_ok(cudaGetLastError());
+            const bool ended = cuda_ok(cudaStreamEndCapture(c->capture_stream, &graph));
+            if (!queued || !ended || !graph) {
+                if (graph) cudaGraphDestroy(graph);
+                cudaGetLastError();
+                return SR_ERR_CUDA;
+            }
             const cudaError_t ie = cudaGraphInstantiate(&c->exec, graph, 0);
             cudaGraphDestroy(graph);
-            if (!cuda_ok(ie)) return SR_ERR_CUDA;
+            if (!cuda_ok(ie)) {
+                c->exec = nullptr;
+                return SR_ERR_CUDA;
+            }
             c->frames = gf;
             c->kernels = k;
         }

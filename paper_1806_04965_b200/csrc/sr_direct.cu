@@ -180,6 +180,7 @@ __device__ void head_item(const SrDevNode& nd, const SrDevEdge* edges, const SrD
                           float* out_f32)
 {
     __shared__ float mean[kHeadMaxC];
+    __shared__ float part[4 * kWarps * 32];
     __shared__ float red[kWarps][kHeadCo];
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, tid = threadIdx.x;
     const int b = it.b0, co0 = it.p0;
@@ -193,10 +194,11 @@ __device__ void head_item(const SrDevNode& nd, const SrDevEdge* edges, const SrD
         const T* src = static_cast<const T*>(e.src[e.R ? prev : cur]) + (size_t)b * Kx;
         const float* w0 = e.w + (size_t)co0 * e.K;
         if (e.kind == SR_EDGE_MEAN_DENSE) {
-            __syncthreads();
-            for (int c = tid; c < e.Cs; c += blockDim.x) mean[c] = 0.f;
+            // the sums run in a fixed order (no atomics), so a frame update is bit-reproducible
             __syncthreads();
             if ((e.Cs & 3) == 0 && e.Cs / 4 <= (int)blockDim.x) {
+                // groups of Cs/4 threads share the pixels; a group's partial sums take one row of part[][Cs]
+                // (groups * Cs <= 4 * blockDim.x floats), the rows are then added in group order
                 const int vc = e.Cs / 4, groups = blockDim.x / vc;
                 const int col = tid % vc, grp = tid / vc;
                 if (grp < groups) {
@@ -208,10 +210,20 @@ __device__ void head_item(const SrDevNode& nd, const SrDevEdge* edges, const SrD
                         for (int q = 0; q < 4; ++q) s4[q] += x[q];
                     }
 #pragma unroll
-                    for (int q = 0; q < 4; ++q) atomicAdd(&mean[4 * col + q], s4[q]);
+                    for (int q = 0; q < 4; ++q) part[grp * e.Cs + 4 * col + q] = s4[q];
+                }
+                __syncthreads();
+                for (int c = tid; c < e.Cs; c += blockDim.x) {
+                    float m = 0.f;
+                    for (int gq = 0; gq < groups; ++gq) m += part[gq * e.Cs + c];
+                    mean[c] = m;
                 }
             } else {
-                for (int i = tid; i < Kx; i += blockDim.x) atomicAdd(&mean[i % e.Cs], to_f(src[i]));
+                for (int c = tid; c < e.Cs; c += blockDim.x) {
+                    float m = 0.f;
+                    for (int p = 0; p < HW; ++p) m += to_f(src[(size_t)p * e.Cs + c]);
+                    mean[c] = m;
+                }
             }
             __syncthreads();
             const float inv = 1.f / (float)HW;

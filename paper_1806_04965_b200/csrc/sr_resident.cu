@@ -696,8 +696,11 @@ struct RsPlanEdge {
     int wd_off[kRsMaxCluster] = {-1, -1, -1, -1};
 };
 
+struct RsOffsets { int nodes = 0, edges = 0, units = 0, ubegin = 0, copies = 0; };   // table offsets inside a rank's blob
+
 struct RsEngine {
     int cs = 1, warps = 16, smem_bytes = 0, blob_bytes = 0, n_levels = 1;
+    RsOffsets offs;                             // written by rs_layout, read when the blobs are filled
     std::vector<RsPlanNode> pn;
     std::vector<RsPlanEdge> pe;                 // ordered by target node, then by the node's in-edge order
     std::vector<int> pe_of_host_edge;
@@ -975,30 +978,12 @@ bool rs_layout(const sr_graph* g, RsEngine& E, int cs, int warps)
             for (int r = 0; r < kRsMaxCluster; ++r) pe.wd_off[r] = -1;
     }
     E.smem_bytes = rs_up128(off);
-    (void)off_nodes; (void)off_edges; (void)off_units; (void)off_ubegin; (void)off_copies;   // see rs_table_offsets
+    E.offs.nodes = off_nodes;
+    E.offs.edges = off_edges;
+    E.offs.units = off_units;
+    E.offs.ubegin = off_ubegin;
+    E.offs.copies = off_copies;
     return true;
-}
-
-struct RsOffsets { int nodes, edges, units, ubegin, copies; };
-
-RsOffsets rs_table_offsets(const sr_graph* g, const RsEngine& E)
-{
-    size_t max_units = 0;
-    for (int r = 0; r < E.cs; ++r) max_units = std::max(max_units, E.units[r].size());
-    int off = (int)sizeof(RsHeader);
-    auto take = [&](int bytes, int align) {
-        off = (off + align - 1) / align * align;
-        const int o = off;
-        off += bytes;
-        return o;
-    };
-    RsOffsets o;
-    o.nodes = take((int)sizeof(RsNode) * (int)g->nodes.size(), 16);
-    o.edges = take((int)sizeof(RsEdge) * (int)E.pe.size(), 16);
-    o.units = take((int)(sizeof(RsUnit) * std::max<size_t>(1, max_units)), 16);
-    o.ubegin = take((int)sizeof(int32_t) * (E.n_levels * E.warps + 1), 16);
-    o.copies = take(0, 16);
-    return o;
 }
 
 RsEngine* rs_of(const sr_graph* g) { return static_cast<RsEngine*>(g->rs); }
@@ -1200,7 +1185,7 @@ sr_status sr_rs_bind(sr_graph* g)
     if (!Ep) return SR_OK;
     RsEngine& E = *Ep;
     const int n_nodes = (int)g->nodes.size();
-    const RsOffsets O = rs_table_offsets(g, E);
+    const RsOffsets O = E.offs;
     for (int r = 0; r < E.cs; ++r) {
         std::vector<unsigned char> blob((size_t)E.blob_bytes, 0);
         RsHeader* H = reinterpret_cast<RsHeader*>(blob.data());

@@ -51,7 +51,6 @@ constexpr int kFifo = 16;                             // burst descriptors in fl
 constexpr int kMaxA = 4;                              // activation ring depth
 constexpr int kWUnit = 4096, kMaxWUnits = 32;         // weight ring: units of 4 KiB
 constexpr int kSmemBudget = 200 * 1024;
-constexpr long long kWaitCycles = 2000000000LL;       // about a second
 constexpr int kMaxNodeKb = 128;                       // K-blocks per node the shared-memory table holds
 
 // One K-block of a node's reduction: 32 bytes, staged into shared memory per node so that the two
@@ -122,7 +121,7 @@ __device__ __forceinline__ uint32_t mbar_try_wait(uint32_t bar, uint32_t parity)
     return ok;
 }
 // Bounded wait.  Returns false if the limit expired or another role already gave up.
-__device__ __noinline__ bool mbar_wait_slow(uint32_t bar, uint32_t parity, volatile int* abort_flag)
+__device__ __noinline__ bool mbar_wait_slow(uint32_t bar, uint32_t parity, volatile int* abort_flag, long long limit)
 {
     const long long t0 = clock64();
     for (;;) {
@@ -130,16 +129,24 @@ __device__ __noinline__ bool mbar_wait_slow(uint32_t bar, uint32_t parity, volat
         for (int i = 0; i < 32; ++i)
             if (mbar_try_wait(bar, parity)) return true;
         if (*abort_flag) return false;
-        if (clock64() - t0 > kWaitCycles) {
+        if (clock64() - t0 > limit) {
             *abort_flag = 1;
             return false;
         }
     }
 }
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag)
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, long long limit)
 {
     if (mbar_try_wait(bar, parity)) return true;
-    return mbar_wait_slow(bar, parity, abort_flag);
+    return mbar_wait_slow(bar, parity, abort_flag, limit);
+}
+// Wait for a copy this thread started itself, before the CTA gives up its shared memory.  It has its own limit and
+// does not look at the abort flag: after another role gave up, the copies in flight still have to land.
+__device__ __noinline__ void mbar_wait_drain(uint32_t bar, uint32_t parity, long long limit)
+{
+    const long long t0 = clock64();
+    while (!mbar_try_wait(bar, parity))
+        if (clock64() - t0 > limit) return;
 }
 
 __device__ __forceinline__ void tma_load_4d(uint32_t dst, const void* map, uint32_t bar, int c0, int c1, int c2, int c3)
@@ -203,7 +210,8 @@ __device__ __forceinline__ void tc_wait_ld() { asm volatile("tcgen05.wait::ld.sy
 __global__ void __launch_bounds__(kThreads, 1)
 sr_tc_group_kernel(const CUtensorMap* __restrict__ maps, const TcNode* __restrict__ nodes,
                    const TcKBlock* __restrict__ kbs, const TcTile* __restrict__ tiles, int n_tiles,
-                   SrFrameCtl* __restrict__ ctl, int t_off, int B, int n_a, int a_slot, int n_wu, int w_slot_units, int tmem_cols)
+                   SrFrameCtl* __restrict__ ctl, int t_off, int B, int n_a, int a_slot, int n_wu, int w_slot_units, int tmem_cols,
+                   long long wait_limit)
 {
     extern __shared__ uint8_t smem_raw[];
     __shared__ uint64_t bars[2 * kMaxA + 2 * kMaxWUnits + 4];
@@ -217,6 +225,12 @@ sr_tc_group_kernel(const CUtensorMap* __restrict__ maps, const TcNode* __restric
 
     // weight ring first: an M = 128 instruction on a node with fewer than 128 output channels reads
     // rows past its weight box, which then still lie inside this allocation
+    // A wait limit of zero (a host-side test hook) means "every wait has already expired": report it and return
+    // before any barrier, tensor memory, copy or MMA is touched.
+    if (wait_limit <= 0) {
+        if (threadIdx.x == 0) atomicExch(&ctl->error, 1);
+        return;
+    }
     const uint32_t w_ring = (smem_u32(smem_raw) + 1023u) & ~1023u;
     const uint32_t a_ring = w_ring + (uint32_t)(n_wu * kWUnit);
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -301,7 +315,7 @@ sr_tc_group_kernel(const CUtensorMap* __restrict__ maps, const TcNode* __restric
                         const TcKBlock k = tab[kb];
                         if (k.x_bytes16) {
                             const uint32_t s = a_nxt;
-                            if (!mbar_wait(bar_aempty + 8 * s, a_ph ^ 1, abortp)) { ok = false; break; }
+                            if (!mbar_wait(bar_aempty + 8 * s, a_ph ^ 1, abortp, wait_limit)) { ok = false; break; }
                             if (++a_nxt == (uint32_t)n_a) { a_nxt = 0; a_ph ^= 1; }
                             mbar_expect_tx(bar_afull + 8 * s, (uint32_t)k.x_bytes16 << 4);
                             const int par = (k.flags & 1) ? prev : cur;
@@ -311,7 +325,7 @@ sr_tc_group_kernel(const CUtensorMap* __restrict__ maps, const TcNode* __restric
                         }
                         if (k.flags & 4) {
                             ws_cur = w_nxt;
-                            if (!mbar_wait(bar_wempty + 8 * ws_cur, w_ph ^ 1, abortp)) { ok = false; break; }
+                            if (!mbar_wait(bar_wempty + 8 * ws_cur, w_ph ^ 1, abortp, wait_limit)) { ok = false; break; }
                             if (++w_nxt == n_ws) { w_nxt = 0; w_ph ^= 1; }
                         }
                         const uint32_t unit = ws_cur * (uint32_t)w_slot_units + k.w_box * box_u;
@@ -328,7 +342,7 @@ sr_tc_group_kernel(const CUtensorMap* __restrict__ maps, const TcNode* __restric
                     // waiting and address arithmetic and hands the issuer one 32-byte descriptor per weight
                     // group (up to 3 K-blocks = 12 MMAs): descriptor address words, flags, barriers to commit.
                     const uint32_t acc = (tmem_cols >= 512 && uses0 > uses1) ? 1u : 0u;   // 256 columns: one accumulator
-                    if (!mbar_wait(bar_tempty + 8 * acc, ((acc ? uses1 : uses0) & 1) ^ 1, abortp)) ok = false;
+                    if (!mbar_wait(bar_tempty + 8 * acc, ((acc ? uses1 : uses0) & 1) ^ 1, abortp, wait_limit)) ok = false;
                     int kb = 0;
                     while (kb < n_kb && ok) {
                         uint32_t lo[3] = {0u, 0u, 0u}, nt = 0, act_mask = 0, n_k16 = 0, desc_hi = 0, x_hi = 0, commit_w = 0, loads = 0;
@@ -341,7 +355,7 @@ sr_tc_group_kernel(const CUtensorMap* __restrict__ maps, const TcNode* __restric
                             if (nt > 0 && k.x_bytes16 && loads >= max_loads) break;
                             if (k.x_bytes16) {
                                 a_cur = a_nxt;
-                                if (!mbar_wait(bar_afull + 8 * a_cur, a_ph, abortp)) { ok = false; break; }
+                                if (!mbar_wait(bar_afull + 8 * a_cur, a_ph, abortp, wait_limit)) { ok = false; break; }
                                 if (++a_nxt == (uint32_t)n_a) { a_nxt = 0; a_ph ^= 1; }
                                 ++loads;
                             }
@@ -350,7 +364,7 @@ sr_tc_group_kernel(const CUtensorMap* __restrict__ maps, const TcNode* __restric
                                 if (++w_nxt == n_ws) w_nxt = 0;
                             }
                             const uint32_t unit = ws_cur * (uint32_t)w_slot_units + k.w_box * box_u;
-                            if (!mbar_wait(bar_wfull + 8 * unit, (wf_phase >> unit) & 1, abortp)) { ok = false; break; }
+                            if (!mbar_wait(bar_wfull + 8 * unit, (wf_phase >> unit) & 1, abortp, wait_limit)) { ok = false; break; }
                             wf_phase ^= 1u << unit;
                             const uint32_t x_lo = (((a_ring + a_cur * a_slot) >> 4) + k.x_off16) & 0x3FFFu;
                             const uint32_t w_lo = ((w_ring + unit * kWUnit) >> 4) & 0x3FFFu;
@@ -368,7 +382,7 @@ sr_tc_group_kernel(const CUtensorMap* __restrict__ maps, const TcNode* __restric
                         if (n_pub - fifo_read >= (uint32_t)kFifo) {          // never overwrite a descriptor not yet taken
                             const long long t0 = clock64();
                             while (n_pub - fifo_read >= (uint32_t)kFifo)
-                                if (abort_flag || clock64() - t0 > kWaitCycles) { abort_flag = 1; ok = false; break; }
+                                if (abort_flag || clock64() - t0 > wait_limit) { abort_flag = 1; ok = false; break; }
                             if (!ok) break;
                         }
                         const uint32_t fl = nt | (n_k16 << 2) | (first << 5) | (acc << 6) | (commit_w << 7) | (ws_cur << 8) | (act_mask << 11) |
@@ -395,10 +409,10 @@ sr_tc_group_kernel(const CUtensorMap* __restrict__ maps, const TcNode* __restric
             // drain: every copy this thread started must have landed before the CTA may exit
             for (uint32_t j = 0; j < (uint32_t)n_a && j < ia; ++j) {
                 const uint32_t i2 = ia - 1 - j;
-                mbar_wait(bar_afull + 8 * (i2 % n_a), (i2 / n_a) & 1, abortp);
+                mbar_wait_drain(bar_afull + 8 * (i2 % n_a), (i2 / n_a) & 1, wait_limit);
             }
             for (uint32_t v = 0; v < (uint32_t)n_wu; ++v)
-                if ((wf_used >> v) & 1) mbar_wait(bar_wfull + 8 * v, ((wf_phase >> v) & 1) ^ 1, abortp);
+                if ((wf_used >> v) & 1) mbar_wait_drain(bar_wfull + 8 * v, ((wf_phase >> v) & 1) ^ 1, wait_limit);
         }
     } else if (warp == 1) {
         // ---------------------------------------------------------------- MMA issuer
@@ -413,7 +427,7 @@ sr_tc_group_kernel(const CUtensorMap* __restrict__ maps, const TcNode* __restric
                     const long long t0 = clock64();
                     bool give_up = false;
                     while ((q0 = ld_shared_v4(e)).x != n) {
-                        if (abort_flag || clock64() - t0 > kWaitCycles) { give_up = true; break; }
+                        if (abort_flag || clock64() - t0 > wait_limit) { give_up = true; break; }
                     }
                     if (give_up) { abort_flag = 1; break; }
                 }
@@ -473,10 +487,10 @@ sr_tc_group_kernel(const CUtensorMap* __restrict__ maps, const TcNode* __restric
             const bool wide = nd.n_mh * nd.n_cols > 256;
             const uint32_t acc = (!wide && tmem_cols >= 512 && uses0 > uses1) ? 1u : 0u;
             if (wide || acc == 0) {
-                if (!mbar_wait(bar_tfull, uses0 & 1, abortp)) ok = false;
+                if (!mbar_wait(bar_tfull, uses0 & 1, abortp, wait_limit)) ok = false;
             }
             if (ok && (wide || acc == 1)) {
-                if (!mbar_wait(bar_tfull + 8, uses1 & 1, abortp)) ok = false;
+                if (!mbar_wait(bar_tfull + 8, uses1 & 1, abortp, wait_limit)) ok = false;
             }
             ok = __all_sync(0xffffffffu, ok);
             asm volatile("bar.sync 1, 128;" ::: "memory");           // the offset table is complete
@@ -1110,7 +1124,7 @@ int sr_tc_launch_group(sr_graph* g, int group, int t_off, cudaStream_t s)
         reinterpret_cast<const TcKBlock*>(g->ws + E->r_kbs.offset),
         reinterpret_cast<const TcTile*>(g->ws + E->r_tiles.offset) + E->group_tile_offset[group],
         (int)E->group_tiles[group].size(), reinterpret_cast<SrFrameCtl*>(g->ws + g->r_ctl.offset), t_off, g->batch, n_a, a_slot,
-        n_wu, E->group_w_slot[group], E->group_ctas_per_sm[group] > 1 ? 256 : 512);
+        n_wu, E->group_w_slot[group], E->group_ctas_per_sm[group] > 1 ? 256 : 512, (long long)g->opt_wait_ms * 2000000LL);
     if (timed) {
         cudaEventRecord(E->ev[E->ev_used + 1], s);
         E->ev_used += 2;

@@ -39,7 +39,7 @@ def check_stepwise(spec, pattern, engine="auto", samples=None, zero_bias=False, 
     ins = G.input_nodes
     dev = {v: to_device(spec, X[v]) for v in ins}
     G.reset([dev[v][0] for v in ins])
-    out = torch.empty((spec.batch, spec.nodes[G.output_node].c), dtype=torch.float32, device="cuda:0")
+    out = torch.empty(G.out_shape(), dtype=torch.float32, device="cuda:0")
     tol = TOL[spec.dtype] if tol is None else tol
     worst = 0.0
     for t in range(1, spec.frames + 1):

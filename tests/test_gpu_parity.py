@@ -82,3 +82,55 @@ def test_run_equals_steps_and_resume():
     D.run([x[5:9]], od)
     assert torch.equal(od, oa[4:])
     assert A.launch_count() > 0
+
+
+@pytest.mark.parametrize("dtype", ["fp32", "bf16"])
+def test_spatial_output_node_fills_a_full_frame(dtype):
+    # the output node is an image: `out` holds [B][H][W][C] floats per frame, and consecutive frames of a run do not overlap
+    import torch
+    g = graphs.build("sink", dtype=dtype)
+    for p in g.patterns:
+        parity.check_stepwise(g, p, zero_bias=False)
+        parity.check_run(g, p)
+    from paper_1806_04965_b200 import Graph
+    G = Graph(g.nodes, g.edges, g.patterns["streaming"], batch=g.batch, dtype=dtype)
+    assert G.out_shape() == (g.batch, 4, 4, 8)
+    G.set_weights(data.make_weights(g), data.make_biases(g, zero=False))
+    X = data.make_inputs(g)
+    # guard words behind the output buffer stay untouched
+    buf = torch.full((g.frames * g.batch * 4 * 4 * 8 + 64,), 7.0, dtype=torch.float32, device="cuda:0")
+    out = buf[:g.frames * g.batch * 4 * 4 * 8].view(g.frames, g.batch, 4, 4, 8)
+    x = parity.to_device(g, X[0])
+    G.reset([x[0]])
+    G.run([x[1:]], out)
+    G.sync_status()
+    assert bool((buf[-64:] == 7.0).all())
+    assert float(out.abs().max()) > 0
+
+
+def test_expired_device_wait_is_reported_and_cleared_by_reset():
+    # host-side hook only: with a wait limit of zero every tensor-core launch reports the expiry at its entry and
+    # returns before it touches a barrier, a copy or an MMA; nothing on the GPU actually waits
+    from paper_1806_04965_b200 import SrError
+    g = graphs.build("c3", batch=2, frames=3, size=16)
+    X, W, Bi = data.make_inputs(g), data.make_weights(g), data.make_biases(g)
+    G = parity.make_graph(g, "streaming", "auto", 0, W, Bi, wait_limit_ms=0)
+    assert G.info["n_tensor_core_nodes"] > 0 and G.info["resident_cluster"] == 0
+    x = parity.to_device(g, X[0])
+    G.rollout([x])
+    for _ in range(2):                                  # the error stays recorded until the rollout starts over
+        with pytest.raises(SrError) as e:
+            G.sync_status()
+        assert e.value.status == "SR_ERR_TIMEOUT"
+    G.set_option(10, 1000)
+    want = fu_rollout(g, X, W, Bi)
+    out = G.rollout([x])                                # reset clears the error word
+    G.sync_status()
+    o = G.output_node
+    assert parity.rel_err(out.cpu().numpy().reshape(want[o][1:].shape), want[o][1:]) <= parity.TOL["bf16"]
+    parity.check_run(g, "streaming")                    # and a fresh graph is unaffected
+
+
+def fu_rollout(g, X, W, Bi):
+    from oracle import frame_update as fu
+    return fu.rollout_spec(g, "streaming", X, W, Bi)

@@ -46,6 +46,32 @@ def test_built_in_workspace_matches_caller_workspace_twice():
     assert np.array_equal(got_out, want_out)
 
 
+def test_a_new_bind_takes_the_array_from_the_previous_graph_and_allocates_nothing():
+    import torch
+    from paper_1806_04965_b200 import Graph, SrError
+    spec = graphs.build("c2", batch=4, frames=3)
+    X, W, Bi = data.make_inputs(spec), data.make_weights(spec), data.make_biases(spec)
+    x = parity.to_device(spec, X[0])
+    first = Graph(spec.nodes, spec.edges, spec.patterns["streaming"], batch=spec.batch, dtype=spec.dtype, static_workspace=True)
+    first.set_weights(W, Bi)
+    want = first.rollout([x]).cpu().numpy()
+    torch.cuda.synchronize()
+    free_before, _ = torch.cuda.mem_get_info()
+    second = Graph(spec.nodes, spec.edges, spec.patterns["streaming"], batch=spec.batch, dtype=spec.dtype, static_workspace=True)
+    free_after, _ = torch.cuda.mem_get_info()
+    assert free_after == free_before                # binding the built-in array takes no device memory
+    # the first graph no longer owns the array: its calls fail on the host instead of running on the new owner's tables
+    for call in (lambda: first.reset([x[0]]), lambda: first.step([x[1]]), lambda: first.run([x[1:]]),
+                 lambda: first.get_state(1), lambda: first.set_weights(W, Bi)):
+        with pytest.raises(SrError) as e:
+            call()
+        assert e.value.status == "SR_ERR_STATE"
+    second.set_weights(W, Bi)
+    got = second.rollout([x]).cpu().numpy()
+    second.sync_status()
+    assert np.array_equal(got, want)
+
+
 def test_graph_larger_than_the_built_in_workspace_is_refused():
     from paper_1806_04965_b200 import Graph, SrError
     spec = graphs.build("c3")                      # hundreds of MiB of states

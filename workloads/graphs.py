@@ -289,7 +289,16 @@ def mini_cnn(batch: int = 3, frames: int = 5, dtype: str = "bf16") -> GraphSpec:
     return g
 
 
-BUILDERS = {"mini": mini_cnn, "c1": c1_mlp, "c2": c2_small_cnn, "c3": c3_six_node, "c4": c4_ten_node, "c5": c5_stress}
+def conv_sink(batch: int = 3, frames: int = 4, dtype: str = "bf16") -> GraphSpec:
+    """A network whose output node is an image: in -> n1 (3x3) -> n2 (3x3, stride 2), recurrence on n1."""
+    nodes = [Node("in", 8, 8, 3, IDENTITY), Node("n1", 8, 8, 16), Node("n2", 4, 4, 8, IDENTITY)]
+    edges = [Edge(0, 1, CONV, 3, 1), Edge(1, 2, CONV, 3, 2), Edge(1, 1, CONV, 3, 1)]
+    g = GraphSpec("sink", nodes, edges, batch, frames, dtype, seed=1011)
+    g.patterns = {"streaming": streaming_pattern(g), "sequential": sequential_pattern(g)}
+    return g
+
+
+BUILDERS = {"mini": mini_cnn, "sink": conv_sink, "c1": c1_mlp, "c2": c2_small_cnn, "c3": c3_six_node, "c4": c4_ten_node, "c5": c5_stress}
 
 
 def build(name: str, **overrides) -> GraphSpec:
