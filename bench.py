@@ -230,10 +230,11 @@ def run_reference(args):
 
 
 # ----------------------------------------------------------------------------- the CUDA library
-def time_pattern(torch, spec, pattern, W, Bi, dev_in, steps, warmup, graph_frames, engine, flush, resident=(1, 0, 0)):
+def time_pattern(torch, spec, pattern, W, Bi, dev_in, steps, warmup, graph_frames, engine, flush, resident=(1, 0, 0), tc_pair=0):
     from paper_1806_04965_b200 import Graph
     G = Graph(spec.nodes, spec.edges, spec.patterns[pattern], batch=spec.batch, dtype=spec.dtype, engine=engine,
-              graph_frames=graph_frames, resident=bool(resident[0]), resident_cluster=resident[1], resident_warps=resident[2])
+              graph_frames=graph_frames, resident=bool(resident[0]), resident_cluster=resident[1], resident_warps=resident[2],
+              tc_pair=tc_pair)
     G.set_weights(W, Bi)
     T = spec.frames
     out = torch.empty((T, spec.batch, spec.nodes[G.output_node].c), dtype=torch.float32, device="cuda")
@@ -332,7 +333,7 @@ def measure_workload(torch, args, name, rank, local, dist, pk, flush, steps, war
         barrier()
         sampler = ClockSampler(local) if p == first else None
         G, out, r = time_pattern(torch, spec, p, W, Bi, dev_in, steps, warmup, args.graph_frames, args.engine, flush,
-                                 (args.resident, args.resident_cluster, args.resident_warps))
+                                 (args.resident, args.resident_cluster, args.resident_warps), args.tc_pair)
         barrier()
         if p == first:
             clocks = sampler.stop()
@@ -512,6 +513,7 @@ def main():
     ap.add_argument("--resident", type=int, default=1, help="1: sr_rollout_run may use the shared-memory-resident kernel; 0: per-frame launches")
     ap.add_argument("--resident-cluster", type=int, default=0)
     ap.add_argument("--resident-warps", type=int, default=0)
+    ap.add_argument("--tc-pair", type=int, default=0, help="tensor-core work items: 0 = library decides, 1 = single tiles, 2 = pairs of tiles")
     ap.add_argument("--only-main", action="store_true", help="time only --workload and --pattern")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     args = ap.parse_args()

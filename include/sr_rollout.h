@@ -163,8 +163,8 @@ sr_status sr_graph_set_node_bias(sr_graph* g, int node, const float* bias_host);
 /* Options.  key 0 "engine": 0 = tensor cores where a node qualifies (default), 1 = CUDA-core kernels only.
  *           key 1 "frames per CUDA graph" used by sr_rollout_run: 0 = plain launches, n >= 1 = graphs
  *                  of n frames (default 0).
- *           key 2 "weight ring": 4 KiB units of shared memory the tensor-core kernel gives to weight tiles
- *                  (8, 16, 24 or 32; 0 = default); the rest of the shared memory holds activation tiles.
+ *           key 2 "weight ring": weight boxes the tensor-core kernel keeps in flight in shared memory
+ *                  (2..8; 0 = default); the rest of the shared memory holds activation boxes.
  *           key 3 "tile width": width in pixels (8, 16 or 32; 0 = default) of the 128-pixel output tiles of
  *                  nodes that have a stride-1 k x k incoming edge (narrow tiles reload less halo, wide
  *                  tiles read longer contiguous runs).
@@ -189,7 +189,10 @@ sr_status sr_graph_set_node_bias(sr_graph* g, int node, const float* bias_host);
  *                  for its own copies in flight, frees its tensor memory and returns, and sr_graph_sync_status
  *                  reports SR_ERR_TIMEOUT.  0 is a test hook: every tensor-core launch reports the error at once and
  *                  returns before it touches a barrier, a copy or an MMA.  May be set at any time.
- * Must be set before sr_graph_workspace_bytes / sr_graph_bind_workspace (engine, weight ring, tile width,
+ *           key 11 "tile pairs": the tensor-core kernel's work item is a pair of neighbouring pixel tiles that share every
+ *                  weight box (half the weight traffic, twice the work per item).  0 (default) = pairs in launch
+ *                  groups with many tiles per SM, 1 = single tiles only, 2 = pairs wherever the geometry allows.
+ * Must be set before sr_graph_workspace_bytes / sr_graph_bind_workspace (engine, weight ring, tile width, tile pairs,
  * resident keys) / before the first run (graphs). */
 sr_status sr_graph_set_option(sr_graph* g, int key, int value);
 

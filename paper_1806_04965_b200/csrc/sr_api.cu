@@ -370,7 +370,7 @@ sr_status sr_graph_set_option(sr_graph* g, int key, int value)
     }
     if (key == 2) {
         if (g->ws) return SR_ERR_STATE;
-        if (value < 0 || value > 32) return SR_ERR_INVALID_ARG;
+        if (value < 0 || value > 8 || value == 1) return SR_ERR_INVALID_ARG;
         g->opt_b_units = value;
         return SR_OK;
     }
@@ -396,6 +396,12 @@ sr_status sr_graph_set_option(sr_graph* g, int key, int value)
         if (g->ws) return SR_ERR_STATE;
         if (value != 0 && (value < 4 || value > 32)) return SR_ERR_INVALID_ARG;
         g->opt_rs_warps = value;
+        return SR_OK;
+    }
+    if (key == 11) {
+        if (g->ws) return SR_ERR_STATE;
+        if (value < 0 || value > 2) return SR_ERR_INVALID_ARG;
+        g->opt_tc_pair = value;
         return SR_OK;
     }
     if (key == 10) {

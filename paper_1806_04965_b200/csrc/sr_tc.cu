@@ -6,10 +6,10 @@
 // tile simply walks the K-blocks of every incoming edge, tap by tap, into one TMEM accumulator.
 //
 // GEMM shape.  D[c_out][pixel] = sum_k W[c_out][k] * X[pixel][k]: the weights are the M operand
-// (128 rows per instruction, two halves for C_out > 128), up to 256 output pixels are the N operand.
+// (128 rows per instruction, one tile per 128 output channels), up to 256 output pixels are the N operand.
 // Measured on B200, one tcgen05.mma of M = 128 costs about 110 cycles however small N is and 128
 // cycles at N = 256, and a tcgen05.commit is only free if about eight MMAs lie between commits; so
-// every instruction is given N = 256 pixels and weight tiles are released in groups.
+// every instruction is given N = 256 pixels and commits come once per eight MMAs.
 //
 // Operands.  K-block = one filter tap x up to 64 input channels.  Activation tiles come straight from
 // the NHWC state of the source node through 4-D TMA boxes (zero fill outside the image = zero
@@ -25,12 +25,21 @@
 // This makes the k taps of one filter column row-shifted windows of ONE box: the box is loaded once
 // per filter column and the shared-memory descriptor of tap ky just starts ky * tw rows further down.
 //
-// Warp roles in a CTA of 192 threads: warp 0 = TMA producer, warp 1 = MMA issuer (owns TMEM),
-// warps 2..5 = epilogue (TMEM lane = output channel; bias, ReLU, bf16, NHWC stores in which a warp
-// writes 32 consecutive channels of one pixel).  Two accumulators in TMEM let the epilogue of a tile
-// overlap the main loop of the next when they fit.  CTAs are persistent and walk a tile list sorted
-// by decreasing work.  Every wait is bounded; on expiry the kernel records an error in the frame
-// control block, drains its own copies, frees TMEM and returns.
+// Two pixel tiles per weight box.  What limits the kernel is the traffic from L2 into shared memory, and
+// most of it is weights: every tile re-fetches its node's weight boxes.  So a work item is a PAIR of
+// neighbouring pixel tiles ("lanes") that share every weight box: lane 0 accumulates in TMEM columns
+// 0..255, lane 1 in columns 256..511, and each weight box that arrives feeds the MMAs of both.  The
+// two tiles are neighbours in x (8-wide tiles) or consecutive samples (tiles that span the image), so
+// ONE activation box covers both and lane 1's operand window is lane 0's, a fixed number of bytes
+// further on.  Launch groups with few tiles keep single tiles (two accumulators alternate instead).
+//
+// Warp roles in a CTA of 384 threads: warp 0 = TMA producer; warp 2 = scout (all barrier waits and
+// address arithmetic; publishes one 16-byte burst descriptor per eight or so MMAs); warp 1 = MMA
+// issuer (owns TMEM; reads descriptors and issues, nothing else); warps 4..11 = epilogue (TMEM lane
+// = output channel; bias, ReLU, bf16, NHWC stores in which a warp writes 32 consecutive channels of one
+// pixel).  CTAs are persistent and walk a work list sorted by decreasing work.  Every wait is bounded;
+// on expiry the kernel records an error in the frame control block, waits for its own copies, frees
+// TMEM and returns.
 #include <cuda.h>
 #include <cuda_bf16.h>
 #include <cuda_runtime.h>
@@ -45,49 +54,74 @@
 
 namespace {
 
-constexpr int kMaxCols = 256;                         // pixels (N of the MMA) per tile
-constexpr int kThreads = 224;
+constexpr int kMaxCols = 256;                         // pixels (N of the MMA) per lane
+constexpr int kThreads = 384;
+constexpr int kEpiWarps = 8;                          // warps 4..11
 constexpr int kFifo = 16;                             // burst descriptors in flight between scout and issuer
 constexpr int kMaxA = 4;                              // activation ring depth
-constexpr int kWUnit = 4096, kMaxWUnits = 32;         // weight ring: units of 4 KiB
-constexpr int kSmemBudget = 200 * 1024;
-constexpr int kMaxNodeKb = 128;                       // K-blocks per node the shared-memory table holds
+constexpr int kMaxW = 8;                              // weight ring depth (one weight box per slot)
+constexpr int kSmemBudget = 203 * 1024;               // dynamic shared memory; the static part takes the rest of 227 KiB
+constexpr int kMaxNodeKb = 128;                       // K-blocks per node the shared-memory tables hold
 
-// One K-block of a node's reduction: 32 bytes, staged into shared memory per node so that the two
-// single-thread roles never wait on global memory between barrier waits.
-struct TcKBlock {
-    uint32_t k_off;         // first K column in the node's weight matrix
-    uint32_t desc_hi;       // upper word of the shared-memory matrix descriptors (swizzle, SBO, version)
-    uint16_t x_map0, x_map1;// tensor map of the activation box for source frame parity 0 / 1
-    uint16_t w_map;         // tensor map of the weight box
-    int8_t qx, qy;          // box origin relative to the tile origin (columns, rows)
-    uint16_t c0;            // first channel of the box
-    uint16_t x_off16;       // (byte offset of this tap's window inside the activation slot) / 16
-    uint16_t x_bytes16;     // (bytes of the activation box this block loads into a fresh slot) / 16; 0 = reuse the slot
-    uint16_t w_bytes16;     // (bytes of the weight box) / 16
-    uint8_t n_k16;          // MMA steps (K = 16 each) in this block
-    uint8_t flags;          // 1: the edge reads frame t (R = 1), else frame t+1; 2: last reader of the activation
-                            // slot; 4: first box of a weight group; 8: last box of a weight group
-    uint8_t w_box;          // index of this block's weight box inside its group
-    uint8_t x_sbo16;        // (bytes between 8-pixel groups of the activation operand) / 16: one image row of the box
-    uint8_t pad_[4];
+// One weight group (consecutive K-blocks of equal channel-block width, fetched by ONE copy) as the weight producer
+// sees it (8 bytes).  A thread that waits for a slot, arms the barrier and starts a copy gets through about one
+// copy per 420 cycles (measured on B200), so copies must be large: a group, not a K-block.
+struct TcKbWeight {
+    uint16_t blk;           // index of the group's first K-block in its tensor map (a run of equally wide blocks)
+    uint16_t w_map;         // tensor map of that run: dims (channels of a block, output channels, blocks)
+    uint16_t w_bytes16;     // (bytes of the whole group) / 16
+    uint16_t pad_;
 };
-static_assert(sizeof(TcKBlock) == 32, "K-block table entries are copied as two 16-byte words");
+static_assert(sizeof(TcKbWeight) == 8, "copied as one 8-byte word");
+
+// One activation box of a node's reduction as the activation producer sees it (16 bytes); only the K-blocks that
+// open a fresh box have one.
+struct TcKbAct {
+    uint16_t x_map0, x_map1;// tensor map of the activation box for source frame parity 0 / 1
+    uint16_t x_bytes16;     // (bytes of the activation box) / 16
+    int8_t qx, qy;          // box origin relative to the tile origin (columns, rows)
+    uint8_t c0_16;          // (first channel of the box) / 16
+    uint8_t flags;          // 1: the edge reads frame t (R = 1), else frame t+1
+    uint8_t pad_[6];
+};
+static_assert(sizeof(TcKbAct) == 16, "copied as one 16-byte word");
+
+// One burst (= one weight group: one or two K-blocks of equal descriptor state) as the scout sees it (8 bytes).  The
+// scout is a single thread whose every shared-memory access or barrier probe costs tens to hundreds of cycles, so
+// everything that can be worked out on the host is.
+struct TcBurst {
+    uint16_t xa_off16;      // (byte offset of the first block's operand window inside its activation slot) / 16
+    uint16_t xb_off16;      // two blocks: the same for the second block; one block: for lane 1's window of that block
+    uint8_t flags;          // 1 / 2: the first / second block opens a fresh activation slot; 4 / 8: the first / second
+                            // block is the last reader of its slot; 16: the burst has two blocks
+    uint8_t state;          // descriptor state of the burst: index into the node's state table
+    uint16_t pad_;
+};
+static_assert(sizeof(TcBurst) == 8, "copied as one 8-byte word");
+
+// Descriptor state shared by consecutive bursts of a node (16 bytes).
+struct TcState {
+    uint32_t desc_hi;       // upper word of the weight descriptors (swizzle, SBO, version)
+    uint32_t x_hi;          // upper word of the activation descriptors (SBO = one image row of the box)
+    uint16_t n_k16;         // MMA steps (K = 16 each) per K-block
+    uint16_t w_step16;      // (bytes of one block's weights) / 16
+    uint32_t pad_;
+};
+static_assert(sizeof(TcState) == 16, "read as one 16-byte word");
 
 struct TcNode {
     void* state[2];
     const float* bias;
     int32_t H, W, C, act;
-    int32_t tw, th, tb, sep;        // tile geometry (see the file comment)
-    int32_t n_cols;                 // N of the MMA: stacked rows of a tile, rounded up to 32
-    int32_t n_mh;                   // halves of 128 output channels
-    int32_t first_kb, n_kb;
-    uint32_t idesc;
-    int32_t w_box_units, w_group_units;
-    int32_t pad_;
+    int32_t tw, th, tb, sep;        // geometry of one lane's tile (see the file comment)
+    int32_t n_cols;                 // N of the MMA: stacked rows of a lane's tile, rounded up to 32
+    int32_t l1_dw, l1_db;           // where lane 1's tile lies relative to lane 0's: columns, samples
+    int32_t first_state, pad_;      // first entry of the node in the state table
+    int32_t first_act, n_act;       // range in the activation-box table
+    int32_t first_wg, n_wg;         // range in the weight-group table and in the burst table (one burst per group)
 };
 
-struct TcTile { int32_t node, b0, h0, w0, m0, pad_[3]; };   // m0: first output channel of the tile (0 or 128)
+struct TcTile { int32_t node, b0, h0, w0, m0, lanes, pad_[2]; };   // m0: first output channel; lanes: 1 or 2 pixel tiles
 
 struct TcStem {             // a few-channel input edge staged as im2col rows
     const void* src[2];
@@ -155,11 +189,11 @@ __device__ __forceinline__ void tma_load_4d(uint32_t dst, const void* map, uint3
         "cp.async.bulk.tensor.4d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5, %6}], [%2];"
         ::"r"(dst), "l"(map), "r"(bar), "r"(c0), "r"(c1), "r"(c2), "r"(c3) : "memory");
 }
-__device__ __forceinline__ void tma_load_2d(uint32_t dst, const void* map, uint32_t bar, int c0, int c1)
+__device__ __forceinline__ void tma_load_3d(uint32_t dst, const void* map, uint32_t bar, int c0, int c1, int c2)
 {
     asm volatile(
-        "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
-        ::"r"(dst), "l"(map), "r"(bar), "r"(c0), "r"(c1) : "memory");
+        "cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5}], [%2];"
+        ::"r"(dst), "l"(map), "r"(bar), "r"(c0), "r"(c1), "r"(c2) : "memory");
 }
 
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
@@ -207,55 +241,70 @@ __device__ __forceinline__ void tc_wait_ld() { asm volatile("tcgen05.wait::ld.sy
 
 
 // ------------------------------------------------------------------------------------------ the kernel
-__global__ void __launch_bounds__(kThreads, 1)
+// Burst descriptors (scout -> issuer): 16 bytes, written and read as one 128-bit access.
+//   x : bits 0-15 sequence number; 16 kind (1 = state); 29 stop
+//       burst: 17-18 K-blocks in the burst (1 or 2); 19 first MMA of each lane overwrites its accumulator;
+//              20-21 lanes to issue; 22-23 lanes whose accumulator is complete after this burst; 24-27 activation
+//              slots to hand back; 28 hand the weight slot of the burst back
+//       state: 17-19 K = 16 steps per K-block; 20 / 21 accumulator of lane 0 / 1; 22-27 MMA columns / 8
+//   y, z, w (burst): lower descriptor words, ready to use: y the weights of the (first) K-block.  A burst of ONE
+//       K-block applies it to every lane named: z = lane 0's activation window, w = lane 1's.  A burst of TWO
+//       K-blocks belongs to a single tile (lane 0's accumulator): z = first block's window, w = second block's, whose
+//       weights lie one block further on in the slot (the step is part of the state).
+//       w bits 24-31 repeat the low sequence bits (a torn read would show).
+//   y, z (state): upper descriptor words of the weight and of the activation operand; w bits 0-15: the weight step / 16
+constexpr uint32_t kDescState = 1u << 16, kDescStop = 1u << 29;
+
+__global__ void __launch_bounds__(kThreads, 2)
 sr_tc_group_kernel(const CUtensorMap* __restrict__ maps, const TcNode* __restrict__ nodes,
-                   const TcKBlock* __restrict__ kbs, const TcTile* __restrict__ tiles, int n_tiles,
-                   SrFrameCtl* __restrict__ ctl, int t_off, int B, int n_a, int a_slot, int n_wu, int w_slot_units, int tmem_cols,
-                   long long wait_limit)
+                   const TcKbWeight* __restrict__ kb_weight, const TcKbAct* __restrict__ kb_act, const TcBurst* __restrict__ bursts, const TcState* __restrict__ states,
+                   const TcTile* __restrict__ tiles, int n_tiles, SrFrameCtl* __restrict__ ctl, int t_off, int B,
+                   int n_a, int a_slot, int n_w, int w_slot, int tmem_cols, long long wait_limit)
 {
     extern __shared__ uint8_t smem_raw[];
-    __shared__ uint64_t bars[2 * kMaxA + 2 * kMaxWUnits + 4];
+    __shared__ uint64_t bars[2 * kMaxA + 2 * kMaxW + 4];
     __shared__ uint32_t tmem_slot;
     __shared__ int abort_flag;
-    __shared__ uint4 kb_tab[2][2 * kMaxNodeKb];            // K-block tables of the producer's and the issuer's current node
-    __shared__ __align__(16) uint16_t epi_buf[4][32 * 32]; // per epilogue warp: 32 pixels x 32 channels, bf16
-    __shared__ int pix_off[kMaxCols];                      // element offset of every pixel of the current tile, -1 = not stored
-    __shared__ __align__(16) uint4 fifo[kFifo][2];         // burst descriptors, scout -> issuer
+    __shared__ int epi_stop;
+    __shared__ uint2 w_tab[kMaxNodeKb];                    // K-block records of the weight producer's current node,
+    __shared__ uint4 a_tab[kMaxNodeKb];                    // of the activation producer's
+    __shared__ uint2 m_tab[kMaxNodeKb];                    // and the burst records of the scout's
+    __shared__ __align__(16) uint16_t epi_buf[kEpiWarps][32 * 32];   // per epilogue warp: 32 pixels x 32 channels, bf16
+    __shared__ int pix_off[2 * kMaxCols];                  // element offset of every pixel of both lanes, -1 = not stored
+    __shared__ __align__(16) uint4 fifo[kFifo];            // burst descriptors, scout -> issuer
     __shared__ volatile uint32_t fifo_read;                // descriptors the issuer has taken
 
-    // weight ring first: an M = 128 instruction on a node with fewer than 128 output channels reads
-    // rows past its weight box, which then still lie inside this allocation
     // A wait limit of zero (a host-side test hook) means "every wait has already expired": report it and return
     // before any barrier, tensor memory, copy or MMA is touched.
     if (wait_limit <= 0) {
         if (threadIdx.x == 0) atomicExch(&ctl->error, 1);
         return;
     }
+    // weight ring first: an M = 128 instruction on a node with fewer than 128 output channels reads
+    // rows past its weight box, which then still lie inside this allocation
     const uint32_t w_ring = (smem_u32(smem_raw) + 1023u) & ~1023u;
-    const uint32_t a_ring = w_ring + (uint32_t)(n_wu * kWUnit);
+    const uint32_t a_ring = w_ring + (uint32_t)(n_w * w_slot);
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const uint32_t bar_afull = smem_u32(&bars[0]), bar_aempty = smem_u32(&bars[kMaxA]);
-    const uint32_t bar_wfull = smem_u32(&bars[2 * kMaxA]), bar_wempty = smem_u32(&bars[2 * kMaxA + kMaxWUnits]);
-    const uint32_t bar_tfull = smem_u32(&bars[2 * kMaxA + 2 * kMaxWUnits]), bar_tempty = bar_tfull + 16;
+    const uint32_t bar_wfull = smem_u32(&bars[2 * kMaxA]), bar_wempty = smem_u32(&bars[2 * kMaxA + kMaxW]);
+    const uint32_t bar_tfull = smem_u32(&bars[2 * kMaxA + 2 * kMaxW]), bar_tempty = bar_tfull + 16;
 
-    if (threadIdx.x < kFifo) {
-        fifo[threadIdx.x][0] = make_uint4(0, 0, 0, 0);
-        fifo[threadIdx.x][1] = make_uint4(0, 0, 0, 0);
-    }
+    if (threadIdx.x < kFifo) fifo[threadIdx.x] = make_uint4(0, 0, 0, 0);
     if (threadIdx.x == 0) {
         abort_flag = 0;
+        epi_stop = 0;
         fifo_read = 0;
         for (int s = 0; s < n_a; ++s) {
             mbar_init(bar_afull + 8 * s, 1);
             mbar_init(bar_aempty + 8 * s, 1);
         }
-        for (int s = 0; s < n_wu; ++s) {
+        for (int s = 0; s < n_w; ++s) {
             mbar_init(bar_wfull + 8 * s, 1);
             mbar_init(bar_wempty + 8 * s, 1);
         }
         for (int a = 0; a < 2; ++a) {
             mbar_init(bar_tfull + 8 * a, 1);
-            mbar_init(bar_tempty + 8 * a, 4);
+            mbar_init(bar_tempty + 8 * a, kEpiWarps);
         }
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
@@ -273,238 +322,337 @@ sr_tc_group_kernel(const CUtensorMap* __restrict__ maps, const TcNode* __restric
     const long long t = ctl->t + t_off;                     // this launch computes frame t+1 from frame t
     const int prev = (int)(t & 1), cur = prev ^ 1;
 
-    // Accumulator buffers: a tile whose n_mh * n_cols columns fit into 256 takes the less used of the
-    // two 256-column buffers, a wider tile takes both.  uses[] counts the tiles a buffer has served;
-    // the issuer and the epilogue warps walk the same tile list and make the same choice.
-    uint32_t uses0 = 0, uses1 = 0;
-
-    if (warp == 0 || warp == 6) {
-        // The producer (warp 0) and the scout (warp 6) walk the same tile list.  At every change of node the whole warp
-        // copies the node's K-block table into its own shared-memory buffer; lane 0 then runs the
-        // block loop out of shared memory.
-        uint4* my_tab = kb_tab[warp == 0 ? 0 : 1];
-        uint32_t n_pub = 0;                                   // bursts published so far (scout)
+    if (warp == 0) {
+        // ---------------------------------------------------------------- weight producer
+        // The three feeding roles (weights, activations, scout) walk the same work list independently.  At every
+        // change of node the whole warp copies its view of the node's K-block table into shared memory; lane 0 then
+        // runs out of shared memory.  Both rings are plain rings: slot after slot, one phase bit per lap.  Weights and
+        // activations have a producer each, so that an activation box (needed once per filter) is requested as soon
+        // as its slot is free and not only when the weight ring has advanced to it.
         int cached_node = -1;
-        // The weight ring is a ring of slots of w_slot_units 4 KiB units (the largest weight group of
-        // the launch), handed back through one "empty" barrier per slot.  Box i of a group starts at
-        // unit i * w_box_units of its slot and signals arrival on that unit's "full" barrier (a full
-        // barrier per group would let the issuer wait for boxes whose activation slots it still
-        // holds).  Which units lead a box depends on the node, and a unit's barrier flips phase only
-        // when used, so both roles keep one phase bit per unit.
-        const uint32_t n_ws = (uint32_t)(n_wu / w_slot_units);
-        uint32_t ia = 0, wf_phase = 0, wf_used = 0, ws_cur = 0, a_cur = 0;
-        uint32_t a_nxt = 0, a_ph = 0, w_nxt = 0, w_ph = 0;    // next slot of each ring and the phase of its barriers
+        uint32_t w_nxt = 0, w_ph = 0, w_used = 0, w_par = 0;  // next slot, phase; slots filled, parity of the latest fill
         bool ok = true;
         for (int ti = blockIdx.x; ti < n_tiles; ti += gridDim.x) {
             const TcTile tl = tiles[ti];
-            const int first_kb = nodes[tl.node].first_kb, n_kb = nodes[tl.node].n_kb;
-            const uint32_t box_u = (uint32_t)nodes[tl.node].w_box_units;
-            const uint32_t idesc = nodes[tl.node].idesc;
+            if (tl.node < 0) break;                                   // the rest of this CTA's column of the work list is padding
+            const int first_wg = nodes[tl.node].first_wg, n_wg = nodes[tl.node].n_wg;
             if (tl.node != cached_node) {
                 __syncwarp();
-                const uint4* src = reinterpret_cast<const uint4*>(kbs + first_kb);
-                for (int i = lane; i < 2 * n_kb; i += 32) my_tab[i] = src[i];
+                for (int i = lane; i < n_wg; i += 32) w_tab[i] = reinterpret_cast<const uint2*>(kb_weight)[first_wg + i];
                 cached_node = tl.node;
                 __syncwarp();
             }
-            if (lane == 0 && ok) {
-                const TcKBlock* tab = reinterpret_cast<const TcKBlock*>(my_tab);
-                if (warp == 0) {
-                    // ------------------------------------------------------ TMA producer
-                    for (int kb = 0; kb < n_kb; ++kb) {
-                        const TcKBlock k = tab[kb];
-                        if (k.x_bytes16) {
-                            const uint32_t s = a_nxt;
-                            if (!mbar_wait(bar_aempty + 8 * s, a_ph ^ 1, abortp, wait_limit)) { ok = false; break; }
-                            if (++a_nxt == (uint32_t)n_a) { a_nxt = 0; a_ph ^= 1; }
-                            mbar_expect_tx(bar_afull + 8 * s, (uint32_t)k.x_bytes16 << 4);
-                            const int par = (k.flags & 1) ? prev : cur;
-                            tma_load_4d(a_ring + s * a_slot, &maps[par ? k.x_map1 : k.x_map0], bar_afull + 8 * s, k.c0,
-                                        tl.w0 + k.qx, tl.h0 + k.qy, tl.b0);
-                            ++ia;
-                        }
-                        if (k.flags & 4) {
-                            ws_cur = w_nxt;
-                            if (!mbar_wait(bar_wempty + 8 * ws_cur, w_ph ^ 1, abortp, wait_limit)) { ok = false; break; }
-                            if (++w_nxt == n_ws) { w_nxt = 0; w_ph ^= 1; }
-                        }
-                        const uint32_t unit = ws_cur * (uint32_t)w_slot_units + k.w_box * box_u;
-                        mbar_expect_tx(bar_wfull + 8 * unit, (uint32_t)k.w_bytes16 << 4);
-                        tma_load_2d(w_ring + unit * kWUnit, &maps[k.w_map], bar_wfull + 8 * unit, (int)k.k_off, tl.m0);
-                        wf_phase ^= 1u << unit;
-                        wf_used |= 1u << unit;
-                    }
-                } else {
-                    // ------------------------------------------------------ scout
-                    // Measured: whatever the issuing thread executes between two tcgen05.mma costs tensor-pipe
-                    // time one for one (a probe of a ready barrier ~165 cycles, a shared-memory load ~110, a
-                    // commit ~50), except for ~200 cycles per burst of >= 8 MMAs.  So this thread does all the
-                    // waiting and address arithmetic and hands the issuer one 32-byte descriptor per weight
-                    // group (up to 3 K-blocks = 12 MMAs): descriptor address words, flags, barriers to commit.
-                    const uint32_t acc = (tmem_cols >= 512 && uses0 > uses1) ? 1u : 0u;   // 256 columns: one accumulator
-                    if (!mbar_wait(bar_tempty + 8 * acc, ((acc ? uses1 : uses0) & 1) ^ 1, abortp, wait_limit)) ok = false;
-                    int kb = 0;
-                    while (kb < n_kb && ok) {
-                        uint32_t lo[3] = {0u, 0u, 0u}, nt = 0, act_mask = 0, n_k16 = 0, desc_hi = 0, x_hi = 0, commit_w = 0, loads = 0;
-                        const uint32_t first = kb == 0;
-                        // a burst stays inside one weight group and never holds so many fresh activation slots
-                        // that the producer could not load the next one (it would wait for this very burst)
-                        const uint32_t max_loads = n_a > 2 ? (uint32_t)n_a - 1 : 1u;
-                        while (nt < 3 && kb < n_kb) {
-                            const TcKBlock k = tab[kb];
-                            if (nt > 0 && k.x_bytes16 && loads >= max_loads) break;
-                            if (k.x_bytes16) {
-                                a_cur = a_nxt;
-                                if (!mbar_wait(bar_afull + 8 * a_cur, a_ph, abortp, wait_limit)) { ok = false; break; }
-                                if (++a_nxt == (uint32_t)n_a) { a_nxt = 0; a_ph ^= 1; }
-                                ++loads;
-                            }
-                            if (k.flags & 4) {
-                                ws_cur = w_nxt;
-                                if (++w_nxt == n_ws) w_nxt = 0;
-                            }
-                            const uint32_t unit = ws_cur * (uint32_t)w_slot_units + k.w_box * box_u;
-                            if (!mbar_wait(bar_wfull + 8 * unit, (wf_phase >> unit) & 1, abortp, wait_limit)) { ok = false; break; }
-                            wf_phase ^= 1u << unit;
-                            const uint32_t x_lo = (((a_ring + a_cur * a_slot) >> 4) + k.x_off16) & 0x3FFFu;
-                            const uint32_t w_lo = ((w_ring + unit * kWUnit) >> 4) & 0x3FFFu;
-                            lo[nt] = w_lo | (x_lo << 16);
-                            if (k.flags & 2) act_mask |= 1u << a_cur;
-                            n_k16 = k.n_k16;
-                            desc_hi = k.desc_hi;
-                            x_hi = (k.desc_hi & ~0x3FFFu) | k.x_sbo16;
-                            ++nt;
-                            ++kb;
-                            if (k.flags & 8) { commit_w = 1; break; }
-                        }
-                        if (!ok) break;
-                        ++n_pub;
-                        if (n_pub - fifo_read >= (uint32_t)kFifo) {          // never overwrite a descriptor not yet taken
-                            const long long t0 = clock64();
-                            while (n_pub - fifo_read >= (uint32_t)kFifo)
-                                if (abort_flag || clock64() - t0 > wait_limit) { abort_flag = 1; ok = false; break; }
-                            if (!ok) break;
-                        }
-                        const uint32_t fl = nt | (n_k16 << 2) | (first << 5) | (acc << 6) | (commit_w << 7) | (ws_cur << 8) | (act_mask << 11) |
-                                            ((kb == n_kb ? 1u : 0u) << 15);
-                        const uint32_t e = smem_u32(&fifo[n_pub & (kFifo - 1)][0]);
-                        st_shared_v4(e + 16, lo[0], lo[1], lo[2], x_hi);
-                        __threadfence_block();
-                        st_shared_v4(e, n_pub, desc_hi, idesc, fl);
-                    }
-                    if (acc == 0) ++uses0; else ++uses1;
+            if (lane == 0) {
+                const TcKbWeight* tab = reinterpret_cast<const TcKbWeight*>(w_tab);
+                for (int kb = 0; kb < n_wg; ++kb) {
+                    const TcKbWeight k = tab[kb];
+                    const uint32_t s = w_nxt;
+                    if (!mbar_wait(bar_wempty + 8 * s, w_ph ^ 1, abortp, wait_limit)) { ok = false; break; }
+                    w_used |= 1u << s;
+                    w_par = (w_par & ~(1u << s)) | (w_ph << s);
+                    if (++w_nxt == (uint32_t)n_w) { w_nxt = 0; w_ph ^= 1; }
+                    mbar_expect_tx(bar_wfull + 8 * s, (uint32_t)k.w_bytes16 << 4);
+                    tma_load_3d(w_ring + s * w_slot, &maps[k.w_map], bar_wfull + 8 * s, 0, tl.m0, (int)k.blk);
                 }
             }
             ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
             if (!ok) break;
         }
-        if (warp == 6 && lane == 0) {
-            ++n_pub;                                                                // tell the issuer to stop
-            const uint32_t e = smem_u32(&fifo[n_pub & (kFifo - 1)][0]);
-            st_shared_v4(e + 16, 0, 0, 0, n_pub);
-            __threadfence_block();
-            st_shared_v4(e, n_pub, 0, 0, 1u << 16);
-        }
-        if (warp == 0 && lane == 0) {
-            // drain: every copy this thread started must have landed before the CTA may exit
-            for (uint32_t j = 0; j < (uint32_t)n_a && j < ia; ++j) {
-                const uint32_t i2 = ia - 1 - j;
-                mbar_wait_drain(bar_afull + 8 * (i2 % n_a), (i2 / n_a) & 1, wait_limit);
+        if (lane == 0)                       // every copy this thread started must have landed before the CTA may exit
+            for (uint32_t v = 0; v < (uint32_t)n_w; ++v)
+                if ((w_used >> v) & 1) mbar_wait_drain(bar_wfull + 8 * v, (w_par >> v) & 1, wait_limit);
+    } else if (warp == 3) {
+        // ---------------------------------------------------------------- activation producer
+        int cached_node = -1;
+        uint32_t a_nxt = 0, a_ph = 0, a_used = 0, a_par = 0;
+        bool ok = true;
+        for (int ti = blockIdx.x; ti < n_tiles; ti += gridDim.x) {
+            const TcTile tl = tiles[ti];
+            if (tl.node < 0) break;
+            const int first_act = nodes[tl.node].first_act, n_act = nodes[tl.node].n_act;
+            if (tl.node != cached_node) {
+                __syncwarp();
+                for (int i = lane; i < n_act; i += 32) a_tab[i] = reinterpret_cast<const uint4*>(kb_act)[first_act + i];
+                cached_node = tl.node;
+                __syncwarp();
             }
-            for (uint32_t v = 0; v < (uint32_t)n_wu; ++v)
-                if ((wf_used >> v) & 1) mbar_wait_drain(bar_wfull + 8 * v, ((wf_phase >> v) & 1) ^ 1, wait_limit);
+            if (lane == 0) {
+                const TcKbAct* tab = reinterpret_cast<const TcKbAct*>(a_tab);
+                for (int i = 0; i < n_act; ++i) {
+                    const TcKbAct k = tab[i];
+                    const uint32_t s = a_nxt;
+                    if (!mbar_wait(bar_aempty + 8 * s, a_ph ^ 1, abortp, wait_limit)) { ok = false; break; }
+                    a_used |= 1u << s;
+                    a_par = (a_par & ~(1u << s)) | (a_ph << s);
+                    if (++a_nxt == (uint32_t)n_a) { a_nxt = 0; a_ph ^= 1; }
+                    mbar_expect_tx(bar_afull + 8 * s, (uint32_t)k.x_bytes16 << 4);
+                    const int par = (k.flags & 1) ? prev : cur;
+                    tma_load_4d(a_ring + s * a_slot, &maps[par ? k.x_map1 : k.x_map0], bar_afull + 8 * s, (int)k.c0_16 << 4,
+                                tl.w0 + k.qx, tl.h0 + k.qy, tl.b0);
+                }
+            }
+            ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
+            if (!ok) break;
+        }
+        if (lane == 0)
+            for (uint32_t v = 0; v < (uint32_t)n_a; ++v)
+                if ((a_used >> v) & 1) mbar_wait_drain(bar_afull + 8 * v, (a_par >> v) & 1, wait_limit);
+    } else if (warp == 2) {
+        // ---------------------------------------------------------------- scout
+        int cached_node = -1;
+        uint32_t a_nxt = 0, a_ph = 0, w_nxt = 0, w_ph = 0;    // next slot of each ring and the phase of its barriers
+        uint32_t n_pub = 0, a_cur = 0, a_base16 = 0;          // descriptors published, activation slot in use and its address / 16
+        uint32_t cur_state = 0xFFFFFFFFu, w_hi = 0, x_hi = 0, nk = 0, w_step = 0;   // descriptor state of the current burst
+        uint32_t st_w_hi = 0xFFFFFFFFu, st_x_hi = 0xFFFFFFFFu, st_misc = 0xFFFFFFFFu;   // state the issuer holds
+        uint32_t uses0 = 0, uses1 = 0;                        // tiles each accumulator has served
+        bool ok = true;
+        // hand one descriptor to the issuer; never overwrites a descriptor not yet taken
+        uint32_t seen_read = 0;                               // the issuer's progress as last looked up
+        auto publish = [&](uint32_t x, uint32_t y, uint32_t z, uint32_t w) -> bool {
+            ++n_pub;
+            if (n_pub - seen_read >= (uint32_t)kFifo) {
+                const long long t0 = clock64();
+                while (n_pub - (seen_read = fifo_read) >= (uint32_t)kFifo)
+                    if (abort_flag || clock64() - t0 > wait_limit) { abort_flag = 1; return false; }
+            }
+            st_shared_v4(smem_u32(&fifo[n_pub & (kFifo - 1)]), (n_pub & 0xFFFFu) | x, y, z, (w & 0x00FFFFFFu) | (n_pub << 24));
+            return true;
+        };
+        for (int ti = blockIdx.x; ti < n_tiles; ti += gridDim.x) {
+            const TcTile tl = tiles[ti];
+            if (tl.node < 0) break;
+            const int first_wg = nodes[tl.node].first_wg, n_bursts = nodes[tl.node].n_wg, first_state = nodes[tl.node].first_state;
+            const uint32_t ncols8 = (uint32_t)nodes[tl.node].n_cols >> 3;
+            if (tl.node != cached_node) {
+                __syncwarp();
+                for (int i = lane; i < n_bursts; i += 32) m_tab[i] = reinterpret_cast<const uint2*>(bursts)[first_wg + i];
+                cached_node = tl.node;
+                cur_state = 0xFFFFFFFFu;
+                __syncwarp();
+            }
+            if (lane == 0 && ok) {
+                {
+                    // ------------------------------------------------------ scout
+                    // Measured: whatever the issuing thread executes between two tcgen05.mma costs tensor-pipe
+                    // time one for one (a probe of a ready barrier ~165 cycles, a shared-memory load ~110, a
+                    // commit ~50), except for ~200 cycles per burst of >= 8 MMAs.  So this thread does all the
+                    // waiting and address arithmetic and hands the issuer one 16-byte descriptor per burst: one
+                    // weight box applied to both lanes of a pair, or two boxes applied to a single tile (8 MMAs
+                    // at 64 channels per K-block either way).
+                    const uint32_t lanes = (uint32_t)tl.lanes;
+                    const uint32_t acc0 = lanes == 2 ? 0u : ((tmem_cols >= 512 && uses0 > uses1) ? 1u : 0u);
+                    const uint32_t lane_all = lanes == 2 ? 3u : 1u;
+                    int kb = 0;
+                    const int n_kb = n_bursts;
+                    bool first = true;
+                    while (kb < n_kb && ok) {
+                        const uint2 rec = m_tab[kb];
+                        ++kb;
+                        const uint32_t fl = rec.y & 0xFFu, st = (rec.y >> 8) & 0xFFu;
+                        if (st != cur_state) {
+                            const uint4 sv = __ldg(reinterpret_cast<const uint4*>(states) + first_state + st);
+                            w_hi = sv.x;
+                            x_hi = sv.y;
+                            nk = sv.z & 0xFFFFu;
+                            w_step = sv.z >> 16;
+                            cur_state = st;
+                        }
+                        uint32_t act_mask = 0;
+                        if (fl & 1u) {
+                            a_cur = a_nxt;
+                            if (!mbar_wait(bar_afull + 8 * a_cur, a_ph, abortp, wait_limit)) { ok = false; break; }
+                            if (++a_nxt == (uint32_t)n_a) { a_nxt = 0; a_ph ^= 1; }
+                            a_base16 = (a_ring + a_cur * a_slot) >> 4;
+                        }
+                        const uint32_t z = ((a_base16 + (rec.x & 0xFFFFu)) & 0x3FFFu) | 0x10000u;
+                        if (fl & 4u) act_mask |= 1u << a_cur;
+                        if (fl & 2u) {
+                            a_cur = a_nxt;
+                            if (!mbar_wait(bar_afull + 8 * a_cur, a_ph, abortp, wait_limit)) { ok = false; break; }
+                            if (++a_nxt == (uint32_t)n_a) { a_nxt = 0; a_ph ^= 1; }
+                            a_base16 = (a_ring + a_cur * a_slot) >> 4;
+                        }
+                        const uint32_t w = ((a_base16 + (rec.x >> 16)) & 0x3FFFu) | 0x10000u;
+                        if (fl & 8u) act_mask |= 1u << a_cur;
+                        if (!mbar_wait(bar_wfull + 8 * w_nxt, w_ph, abortp, wait_limit)) { ok = false; break; }
+                        const uint32_t y = (((w_ring + w_nxt * w_slot) >> 4) & 0x3FFFu) | 0x10000u;
+                        if (++w_nxt == (uint32_t)n_w) { w_nxt = 0; w_ph ^= 1; }
+                        const uint32_t nt = (fl & 16u) ? 2u : 1u;
+                        const uint32_t misc = nk | (acc0 << 3) | (1u << 4) | (ncols8 << 5) | (w_step << 11);
+                        if (w_hi != st_w_hi || x_hi != st_x_hi || misc != st_misc) {
+                            if (!publish(kDescState | ((misc & 0x7FFu) << 17), w_hi, x_hi, w_step)) { ok = false; break; }
+                            st_w_hi = w_hi; st_x_hi = x_hi; st_misc = misc;
+                        }
+                        const uint32_t last = kb == n_kb ? 1u : 0u;
+                        const uint32_t base = nt << 17;
+                        if (first) {
+                            // the accumulators come back from the epilogue one after the other (lane 0's first): lane 0
+                            // starts as soon as its own is free
+                            if (!mbar_wait(bar_tempty + 8 * acc0, ((acc0 ? uses1 : uses0) & 1) ^ 1, abortp, wait_limit)) { ok = false; break; }
+                            if (lanes == 2) {
+                                if (!publish(base | (1u << 19) | (1u << 20) | (last << 22), y, z, w)) { ok = false; break; }
+                                if (!mbar_wait(bar_tempty + 8, (uses1 & 1) ^ 1, abortp, wait_limit)) { ok = false; break; }
+                                if (!publish(base | (1u << 19) | (2u << 20) | ((last * 2u) << 22) | (act_mask << 24) | (1u << 28), y, z, w)) { ok = false; break; }
+                            } else {
+                                if (!publish(base | (1u << 19) | (1u << 20) | (last << 22) | (act_mask << 24) | (1u << 28), y, z, w)) { ok = false; break; }
+                            }
+                            first = false;
+                        } else {
+                            if (!publish(base | (lane_all << 20) | ((last * lane_all) << 22) | (act_mask << 24) | (1u << 28), y, z, w)) { ok = false; break; }
+                        }
+                    }
+                    if (lanes == 2) { ++uses0; ++uses1; }
+                    else if (acc0 == 0) ++uses0;
+                    else ++uses1;
+                }
+            }
+            ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
+            if (!ok) break;
+        }
+        if (lane == 0) {
+            ++n_pub;                                                                // tell the issuer to stop (this slot may be
+            st_shared_v4(smem_u32(&fifo[n_pub & (kFifo - 1)]), (n_pub & 0xFFFFu) | kDescStop, 0, 0, n_pub << 24);   // taken only after an abort)
         }
     } else if (warp == 1) {
         // ---------------------------------------------------------------- MMA issuer
         // One thread; it reads burst descriptors and issues, nothing else (see the scout).
         if (lane == 0) {
-            uint32_t n = 0;
+            uint32_t n = 0, w_hi = 0, x_hi = 0, idesc = 0, nk = 0, acc_of[2] = {0u, 1u}, w_rel = 0, w_step = 0;
             for (;;) {
                 ++n;
-                const uint32_t e = smem_u32(&fifo[n & (kFifo - 1)][0]);
-                uint4 q0 = ld_shared_v4(e);
-                if (q0.x != n) {
+                const uint32_t e = smem_u32(&fifo[n & (kFifo - 1)]);
+                uint4 q = ld_shared_v4(e);
+                if ((q.x & 0xFFFFu) != (n & 0xFFFFu) || (q.w >> 24) != (n & 0xFFu)) {
                     const long long t0 = clock64();
                     bool give_up = false;
-                    while ((q0 = ld_shared_v4(e)).x != n) {
+                    for (;;) {
+                        q = ld_shared_v4(e);
+                        if ((q.x & 0xFFFFu) == (n & 0xFFFFu) && (q.w >> 24) == (n & 0xFFu)) break;
                         if (abort_flag || clock64() - t0 > wait_limit) { give_up = true; break; }
                     }
                     if (give_up) { abort_flag = 1; break; }
                 }
-                __threadfence_block();
-                const uint4 q1 = ld_shared_v4(e + 16);
+                const uint32_t fl = q.x;
                 fifo_read = n;
-                const uint32_t fl = q0.w;
-                if (fl & (1u << 16)) break;
-                const uint32_t w_hi = q0.y, x_hi = q1.w, idesc = q0.z, nt = fl & 3u, nk = (fl >> 2) & 7u, acc = (fl >> 6) & 1u;
-                const uint32_t d_tmem = tmem_base + acc * 256;
-                if (fl & 32u) tc_fence_after();                          // first burst of a tile: the accumulator was just handed back
-                uint32_t accum = (fl & 32u) ? 0u : 1u;
-                const uint32_t los[3] = {q1.x, q1.y, q1.z};
-#pragma unroll
-                for (uint32_t t = 0; t < 3; ++t) {
-                    if (t < nt) {
-                        const uint32_t wl = (los[t] & 0x3FFFu) | 0x10000u, xl = (los[t] >> 16) | 0x10000u;
-                        // a K = 16 step moves both operands 32 bytes along K: +2 in the descriptors' address field
+                if (fl & kDescStop) break;
+                if (fl & kDescState) {
+                    const uint32_t misc = fl >> 17;
+                    nk = misc & 7u;
+                    acc_of[0] = (misc >> 3) & 1u;
+                    acc_of[1] = (misc >> 4) & 1u;
+                    // instruction descriptor: D = f32, A = B = bf16, both K-major, M = 128 output channels, N = pixels
+                    idesc = (1u << 4) | (1u << 7) | (1u << 10) | (((misc >> 5) & 63u) << 17) | ((uint32_t)(128 >> 4) << 24);
+                    w_hi = q.y;
+                    x_hi = q.z;
+                    w_step = q.w & 0xFFFFu;
+                    continue;
+                }
+                const uint32_t first = fl & (1u << 19);
+                const uint32_t xw = q.w & 0x1FFFFu;
+                if (first) tc_fence_after();                             // the accumulator was just handed back
+                // a K = 16 step moves both operands 32 bytes along K: +2 in the descriptors' address field
+                if (((fl >> 17) & 3u) == 2u) {
+                    // two K-blocks of a single tile
+                    const uint32_t d_tmem = tmem_base + acc_of[0] * 256, wb = q.y + w_step;
+                    if (nk == 4) {
+                        tc_mma_bf16_lohi(d_tmem, q.y, w_hi, q.z, x_hi, idesc, first ? 0u : 1u);
+                        tc_mma_bf16_lohi(d_tmem, q.y + 2, w_hi, q.z + 2, x_hi, idesc, 1u);
+                        tc_mma_bf16_lohi(d_tmem, q.y + 4, w_hi, q.z + 4, x_hi, idesc, 1u);
+                        tc_mma_bf16_lohi(d_tmem, q.y + 6, w_hi, q.z + 6, x_hi, idesc, 1u);
+                        tc_mma_bf16_lohi(d_tmem, wb, w_hi, xw, x_hi, idesc, 1u);
+                        tc_mma_bf16_lohi(d_tmem, wb + 2, w_hi, xw + 2, x_hi, idesc, 1u);
+                        tc_mma_bf16_lohi(d_tmem, wb + 4, w_hi, xw + 4, x_hi, idesc, 1u);
+                        tc_mma_bf16_lohi(d_tmem, wb + 6, w_hi, xw + 6, x_hi, idesc, 1u);
+                    } else {
+                        uint32_t accum = first ? 0u : 1u;
                         for (uint32_t j = 0; j < nk; ++j) {
-                            tc_mma_bf16_lohi(d_tmem, wl + 2 * j, w_hi, xl + 2 * j, x_hi, idesc, accum);
+                            tc_mma_bf16_lohi(d_tmem, q.y + 2 * j, w_hi, q.z + 2 * j, x_hi, idesc, accum);
                             accum = 1u;
                         }
+                        for (uint32_t j = 0; j < nk; ++j) tc_mma_bf16_lohi(d_tmem, wb + 2 * j, w_hi, xw + 2 * j, x_hi, idesc, 1u);
+                    }
+                    if ((fl >> 22) & 1u) tc_commit(bar_tfull + 8 * acc_of[0]);
+                } else {
+#pragma unroll
+                    for (uint32_t l = 0; l < 2; ++l) {
+                        if (!((fl >> (20 + l)) & 1u)) continue;
+                        const uint32_t d_tmem = tmem_base + acc_of[l] * 256;
+                        const uint32_t xa = l == 0 ? q.z : xw;
+                        if (nk == 4) {
+                            tc_mma_bf16_lohi(d_tmem, q.y, w_hi, xa, x_hi, idesc, first ? 0u : 1u);
+                            tc_mma_bf16_lohi(d_tmem, q.y + 2, w_hi, xa + 2, x_hi, idesc, 1u);
+                            tc_mma_bf16_lohi(d_tmem, q.y + 4, w_hi, xa + 4, x_hi, idesc, 1u);
+                            tc_mma_bf16_lohi(d_tmem, q.y + 6, w_hi, xa + 6, x_hi, idesc, 1u);
+                        } else {
+                            uint32_t accum = first ? 0u : 1u;
+                            for (uint32_t j = 0; j < nk; ++j) {
+                                tc_mma_bf16_lohi(d_tmem, q.y + 2 * j, w_hi, xa + 2 * j, x_hi, idesc, accum);
+                                accum = 1u;
+                            }
+                        }
+                        if ((fl >> (22 + l)) & 1u) tc_commit(bar_tfull + 8 * acc_of[l]);   // this lane's accumulator is complete
                     }
                 }
-                if (fl & 128u) tc_commit(bar_wempty + 8 * ((fl >> 8) & 7u));   // hands the weight slot back
-                uint32_t m = (fl >> 11) & 15u;
+                if (fl & (1u << 28)) {                                   // hand the weight slot of this burst back (ring order)
+                    tc_commit(bar_wempty + 8 * w_rel);
+                    if (++w_rel == (uint32_t)n_w) w_rel = 0;
+                }
+                uint32_t m = (fl >> 24) & 15u;
                 while (m) {                                              // activation slots this burst read last
                     const uint32_t sl = __ffs(m) - 1;
                     tc_commit(bar_aempty + 8 * sl);
                     m &= m - 1;
                 }
-                if (fl & (1u << 15)) tc_commit(bar_tfull + 8 * acc);     // accumulator complete
             }
         }
-    } else {
-        // ---------------------------------------------------------------- epilogue (warps 2..5)
-        // TMEM lane = output channel, TMEM column = pixel.  A warp turns 32 channels x 32 pixels into
-        // NHWC order through a 2 KiB shared-memory buffer: every thread writes its channel of 32 pixels
-        // (bias, ReLU, bf16), then reads back 8 consecutive channels of one pixel and stores them as one
-        // 16-byte word, so a pixel's 32 channels leave the warp as one 64-byte run.  The element offset
-        // of every pixel of the tile (or -1 for the separator rows and for pixels outside the image) is
-        // tabulated once per tile.
-        const int quarter = warp & 3;                       // TMEM lanes 32*quarter .. +31 belong to this warp
-        const int et = threadIdx.x - 64;                    // 0..127 among the epilogue threads
-        uint16_t* tbuf = &epi_buf[warp - 2][0];
+    } else if (warp >= 4) {
+        // ---------------------------------------------------------------- epilogue (warps 4..11)
+        // TMEM lane = output channel, TMEM column = pixel.  Two warps share each quarter of the 128 lanes and take
+        // alternate 32-column chunks.  A warp turns 32 channels x 32 pixels into NHWC order through a 2 KiB
+        // shared-memory buffer: every thread writes its channel of 32 pixels (bias, ReLU, bf16), then reads back
+        // 8 consecutive channels of one pixel and stores them as one 16-byte word, so a pixel's 32 channels leave
+        // the warp as one 64-byte run.  The element offset of every pixel of the work item (or -1 for separator
+        // rows and pixels outside the image) is tabulated once per item.  Lane 0's accumulator is drained first and
+        // handed back first.
+        const int ew = warp - 4, quarter = ew & 3, half = ew >> 2;      // TMEM lanes 32*quarter .. +31 belong to this warp
+        const int et = threadIdx.x - 128;                               // 0..255 among the epilogue threads
+        uint16_t* tbuf = &epi_buf[ew][0];
+        uint32_t uses0 = 0, uses1 = 0;
         bool ok = true;
-        for (int ti = blockIdx.x; ti < n_tiles && ok; ti += gridDim.x) {
+        for (int ti = blockIdx.x; ti < n_tiles; ti += gridDim.x) {
             const TcTile tl = tiles[ti];
+            if (tl.node < 0) break;
             const TcNode nd = nodes[tl.node];
             const int rows = nd.th + nd.sep;
-            for (int n = et; n < nd.n_cols; n += 128) {
-                const int x = n % nd.tw, q = n / nd.tw, r = q % rows, bi = q / rows;
-                const int b = tl.b0 + bi, y = tl.h0 + r, xx = tl.w0 + x;
-                const bool v = r < nd.th && bi < nd.tb && b < B && y < nd.H && xx < nd.W;
-                pix_off[n] = v ? (int)((((size_t)b * nd.H + y) * nd.W + xx) * nd.C) : -1;
+            for (int idx = et; idx < tl.lanes * kMaxCols; idx += kEpiWarps * 32) {
+                const int l = idx >> 8, n = idx & (kMaxCols - 1);
+                int off = -1;
+                if (n < nd.n_cols) {
+                    const int x = n % nd.tw, q = n / nd.tw, r = q % rows, bi = q / rows;
+                    const int b = tl.b0 + bi + l * nd.l1_db, y = tl.h0 + r, xx = tl.w0 + x + l * nd.l1_dw;
+                    if (r < nd.th && bi < nd.tb && b < B && y < nd.H && xx < nd.W) off = (int)((((size_t)b * nd.H + y) * nd.W + xx) * nd.C);
+                }
+                pix_off[idx] = off;
             }
-            const bool wide = nd.n_mh * nd.n_cols > 256;
-            const uint32_t acc = (!wide && tmem_cols >= 512 && uses0 > uses1) ? 1u : 0u;
-            if (wide || acc == 0) {
-                if (!mbar_wait(bar_tfull, uses0 & 1, abortp, wait_limit)) ok = false;
-            }
-            if (ok && (wide || acc == 1)) {
-                if (!mbar_wait(bar_tfull + 8, uses1 & 1, abortp, wait_limit)) ok = false;
-            }
-            ok = __all_sync(0xffffffffu, ok);
-            asm volatile("bar.sync 1, 128;" ::: "memory");           // the offset table is complete
-            if (abort_flag) ok = false;
-            if (!ok) break;
-            tc_fence_after();
+            if (!ok) abort_flag = 1;
+            if (et == 0) epi_stop = abort_flag;                      // one decision for all eight warps
+            asm volatile("bar.sync 1, 256;" ::: "memory");           // the offset table is complete
+            if (epi_stop) break;
+            const uint32_t acc0 = tl.lanes == 2 ? 0u : ((tmem_cols >= 512 && uses0 > uses1) ? 1u : 0u);
             __nv_bfloat16* out = static_cast<__nv_bfloat16*>(nd.state[cur]);
-            for (int h = 0; h < nd.n_mh; ++h) {
-                const int co_w = tl.m0 + h * 128 + quarter * 32;        // first channel of this warp
-                const int co = co_w + lane;                             // TMEM lane = output channel
-                const float bias = co < nd.C ? __ldg(nd.bias + co) : 0.f;
-                const bool gvalid = co_w + (lane & 3) * 8 < nd.C;       // this thread's group of 8 channels exists
-                const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + acc * 256 + h * nd.n_cols;
-                for (int c0 = 0; c0 < nd.n_cols; c0 += 32) {
+            const int co_w = tl.m0 + quarter * 32;                  // first channel of this warp
+            const int co = co_w + lane;                             // TMEM lane = output channel
+            const float bias = co < nd.C ? __ldg(nd.bias + co) : 0.f;
+            const bool gvalid = co_w + (lane & 3) * 8 < nd.C;       // this thread's group of 8 channels exists
+            for (int l = 0; l < tl.lanes && ok; ++l) {
+                const uint32_t acc = l == 0 ? acc0 : 1u;
+                if (!mbar_wait(bar_tfull + 8 * acc, (acc ? uses1 : uses0) & 1, abortp, wait_limit)) ok = false;
+                ok = __all_sync(0xffffffffu, ok);
+                if (!ok) break;
+                tc_fence_after();
+                const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + acc * 256;
+                const int* poff = pix_off + l * kMaxCols;
+                for (int c0 = half * 32; c0 < nd.n_cols; c0 += 64) {
                     uint32_t v[32];
                     tc_ld32(taddr + c0, v);
                     tc_wait_ld();
@@ -519,7 +667,7 @@ sr_tc_group_kernel(const CUtensorMap* __restrict__ maps, const TcNode* __restric
 #pragma unroll
                     for (int pass = 0; pass < 4; ++pass) {
                         const int p = pass * 8 + (lane >> 2);
-                        const int o = pix_off[c0 + p];
+                        const int o = poff[c0 + p];
                         if (o >= 0 && gvalid) {
                             const uint4 w = *reinterpret_cast<const uint4*>(tbuf + p * 32 + (lane & 3) * 8);
                             *reinterpret_cast<uint4*>(out + (size_t)o + co_w + (lane & 3) * 8) = w;
@@ -527,15 +675,14 @@ sr_tc_group_kernel(const CUtensorMap* __restrict__ maps, const TcNode* __restric
                     }
                     __syncwarp();
                 }
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(bar_tempty + 8 * acc);
             }
-            tc_fence_before();
-            asm volatile("bar.sync 1, 128;" ::: "memory");           // everybody is done with the offset table
-            if (lane == 0) {
-                if (wide || acc == 0) mbar_arrive(bar_tempty);
-                if (wide || acc == 1) mbar_arrive(bar_tempty + 8);
-            }
-            if (wide || acc == 0) ++uses0;
-            if (wide || acc == 1) ++uses1;
+            asm volatile("bar.sync 1, 256;" ::: "memory");           // everybody is done with the offset table
+            if (tl.lanes == 2) { ++uses0; ++uses1; }
+            else if (acc0 == 0) ++uses0;
+            else ++uses1;
         }
     }
     __syncwarp();
@@ -607,20 +754,38 @@ struct KbHost {
     int k_off;
     bool x_load;       // loads a fresh activation box (else: reuses the box loaded earlier for this channel block)
     int x_shift;       // pixels by which this tap's window is shifted inside the box
-    int x_width;       // pixels per image row of the box (tile width, plus the pixel range of the taps it serves)
+    int x_width;       // pixels per image row of the box (lane width, plus the pixel range of the taps it serves)
     bool x_release;
     int box_qy = 0, box_qx = 0, box_ry = 0, box_rx = 0;   // origin and residue class of the box (loading block)
+    int src_col = 0;   // first column of this block in the edge's own weight matrix [C_out][k * k * C_in]
+    int run = 0;       // run of equally wide K-blocks this block belongs to, and its index inside the run
+    int blk = 0;
+    bool w_first = false, w_last = false;   // first / last block of a weight group
+    int w_off = 0;     // byte offset of this block's weights inside the group's slot
 };
+
+// Consecutive K-blocks of equal channel-block width: one 3-D view (channels of a block, output channels, blocks) of
+// the node's weight matrix, whose columns are stored in the order the K loop walks them.
+struct WRun { int bk, first_col, n_blocks; };
+// what the MMAs of one K-block need (host-side; folded into burst records and descriptor states at bind time)
+struct KmHost {
+    uint32_t desc_hi = 0, x_off16 = 0, x_l1off16 = 0, x_sbo16 = 0, n_k16 = 0, w_step16 = 0;
+    bool x_load = false, x_release = false;
+};
+struct WGroup { int run, blk, n, bytes; };
 
 struct NodePlan {
     int node;
-    int tw, th, tb, sep, n_cols, n_mh;
+    int tw, th, tb, sep, n_cols;
     bool one_box;                   // tw == 8: one activation box per channel block serves all k x k taps
-    int group;                      // weight boxes per group
+    int pair;                       // 0: single tiles; 1: lane 1 is the tile tw columns to the right; 2: the next tb samples
     int k_total;                    // columns of the concatenated weight matrix
     std::vector<KbHost> kbs;
+    std::vector<WRun> runs;
+    std::vector<WGroup> wgroups;
     SrRegion wcat;
-    std::vector<int> edge_k_off;    // first column of each incoming edge (index parallel to in_edges)
+    int lane_w() const { return pair == 1 ? 2 * tw : tw; }           // columns of the activation box that hold pixels
+    int box_tb() const { return pair == 2 ? 2 * tb : tb; }           // samples of the activation box
 };
 
 struct StemPlan {
@@ -635,8 +800,8 @@ struct TcEngine {
     std::vector<StemPlan> stems;
     std::vector<int> stem_of_edge;
     std::vector<std::vector<TcTile>> group_tiles;
-    std::vector<int> group_tile_offset, group_a_slot, group_n_a, group_n_wu, group_w_slot, group_grid, group_ctas_per_sm;
-    SrRegion r_maps, r_nodes, r_kbs, r_tiles, r_stems;
+    std::vector<int> group_tile_offset, group_a_slot, group_n_a, group_n_w, group_w_slot, group_grid, group_ctas_per_sm;
+    SrRegion r_maps, r_nodes, r_kb_weight, r_kb_act, r_bursts, r_states, r_tiles, r_stems;
     int n_maps = 0, n_kbs = 0, n_tiles = 0;
     int sm_count = 148;
     // optional timing of the group launches with CUDA events on the launching stream
@@ -709,9 +874,165 @@ void choose_tile(int H, int W, int B, int sep, int forced_tw, NodePlan& P)
     }
 }
 
+void tap_q(int tap, int pad, int st, int& q, int& r)
+{
+    const int a = tap - pad;
+    q = (a >= 0) ? a / st : -((-a + st - 1) / st);
+    r = a - q * st;
+}
+
+// The K-blocks of a node for its tile geometry and pairing mode (the stems' staging buffers exist already).
+void build_kblocks(const sr_graph* g, const TcEngine* E, NodePlan& P)
+{
+    const SrHostNode& n = g->nodes[P.node];
+    P.kbs.clear();
+    // one_box: every class of an edge gets a box as wide as the widest class of the node needs, so that all
+    // K-blocks of equal channel-block width share one activation descriptor state
+    int span = 0;
+    if (P.one_box)
+        for (int e : n.in_edges) {
+            const SrHostEdge& he = g->edges[e];
+            if (is_stem(g, he)) continue;
+            for (int r0 = 0; r0 < he.stride_eff; ++r0) {
+                int lo = 1 << 20, hi = -(1 << 20);
+                for (int t = 0; t < he.k_eff; ++t) {
+                    int q, r;
+                    tap_q(t, he.pad_eff, he.stride_eff, q, r);
+                    if (r == r0) { lo = std::min(lo, q); hi = std::max(hi, q); }
+                }
+                if (hi >= lo) span = std::max(span, hi - lo);
+            }
+        }
+    // The order of the reduction is free (a sum): edges with wider channel blocks come first, so that K-blocks of
+    // equal width form one run each and a run's weights are one 3-D tensor.
+    std::vector<int> order(n.in_edges.begin(), n.in_edges.end());
+    auto width_of = [&](int e) {
+        const SrHostEdge& he = g->edges[e];
+        return is_stem(g, he) ? E->stems[E->stem_of_edge[e]].Kp : block_k(g->nodes[he.d.src].d.c);
+    };
+    std::stable_sort(order.begin(), order.end(), [&](int a, int b) { return width_of(a) > width_of(b); });
+    for (int e : order) {
+        const SrHostEdge& he = g->edges[e];
+        const SrHostNode& s = g->nodes[he.d.src];
+        if (is_stem(g, he)) {
+            const int si = E->stem_of_edge[e], Kp = E->stems[si].Kp;
+            P.kbs.push_back(KbHost{e, true, si, 0, 0, 0, Kp, 0, true, 0, P.lane_w(), true});
+        } else {
+            // Taps whose input pixels fall into the same residue class of the stride read the same view of the
+            // source, shifted by whole pixels: they share ONE activation box and differ only in where their window
+            // starts inside it (rows always; pixels too when the tile is 8 wide, because then the 8-pixel groups of
+            // the operand are simply one box row apart, whatever the row length).
+            const int bk = block_k(s.d.c), k = he.k_eff, st = he.stride_eff;
+            struct Tap { int ky, kx, qy, qx; };
+            std::map<std::tuple<int, int, int>, std::vector<Tap>> classes;      // (ry, rx, qx or 0) -> taps
+            for (int ky = 0; ky < k; ++ky)
+                for (int kx = 0; kx < k; ++kx) {
+                    int qy, ry, qx, rx;
+                    tap_q(ky, he.pad_eff, st, qy, ry);
+                    tap_q(kx, he.pad_eff, st, qx, rx);
+                    classes[std::make_tuple(ry, rx, P.one_box ? 0 : qx)].push_back(Tap{ky, kx, qy, qx});
+                }
+            for (int c0 = 0; c0 < s.d.c; c0 += bk)
+                for (auto& cl : classes) {
+                    const std::vector<Tap>& taps = cl.second;
+                    int qy0 = 1 << 20, qx0 = 1 << 20;
+                    for (const Tap& t : taps) { qy0 = std::min(qy0, t.qy); qx0 = std::min(qx0, t.qx); }
+                    const int bw = P.lane_w() + span;
+                    for (size_t i = 0; i < taps.size(); ++i) {
+                        const Tap& t = taps[i];
+                        // the first tap of the class carries the box origin (qy0, qx0)
+                        KbHost kb{e, false, -1, t.ky, t.kx, c0, bk, 0,
+                                  i == 0, (t.qy - qy0) * bw + (t.qx - qx0), bw, i + 1 == taps.size()};
+                        kb.src_col = (t.ky * k + t.kx) * s.d.c + c0;
+                        kb.box_qy = qy0;
+                        kb.box_qx = qx0;
+                        kb.box_ry = std::get<0>(cl.first);
+                        kb.box_rx = std::get<1>(cl.first);
+                        P.kbs.push_back(kb);
+                    }
+                }
+        }
+    }
+    // columns in loop order; runs of equal block width; weight groups: up to two blocks of a run when tiles are single,
+    // one when they come in pairs (a pair already gives eight MMAs per block), never two blocks that each open a
+    // fresh activation box (the ring may have only two slots)
+    P.runs.clear();
+    P.wgroups.clear();
+    const int rows = std::min(n.d.c, 128), per_group = P.pair ? 1 : 2;
+    int k_off = 0;
+    for (size_t i = 0; i < P.kbs.size(); ++i) {
+        KbHost& kb = P.kbs[i];
+        kb.k_off = k_off;
+        k_off += kb.bk;
+        if (P.runs.empty() || P.runs.back().bk != kb.bk) P.runs.push_back(WRun{kb.bk, kb.k_off, 0});
+        kb.run = (int)P.runs.size() - 1;
+        kb.blk = P.runs.back().n_blocks++;
+        bool open = P.wgroups.empty() || P.wgroups.back().run != kb.run || P.wgroups.back().n >= per_group;
+        if (!open && kb.x_load) {
+            bool had_load = false;
+            for (int j = 0; j < P.wgroups.back().n; ++j) had_load |= P.kbs[i - 1 - j].x_load;
+            open = had_load;
+        }
+        if (open) {
+            if (i > 0) P.kbs[i - 1].w_last = true;
+            P.wgroups.push_back(WGroup{kb.run, kb.blk, 0, 0});
+            kb.w_first = true;
+        }
+        kb.w_off = P.wgroups.back().bytes;
+        P.wgroups.back().n += 1;
+        P.wgroups.back().bytes += rows * kb.bk * 2;
+    }
+    if (!P.kbs.empty()) P.kbs.back().w_last = true;
+    P.k_total = k_off;
+}
+
+// Pixels by which lane 1's operand window lies behind lane 0's inside a box of row length x_width.
+int lane1_shift_px(const NodePlan& P, int x_width)
+{
+    if (P.pair == 1) return P.tw;
+    if (P.pair == 2) return P.tb * (P.th + P.sep) * x_width;
+    return 0;
+}
+
+int act_slot_bytes(const NodePlan& P)
+{
+    int a_slot = 1024;
+    for (const KbHost& kb : P.kbs) {
+        const size_t box_px = (size_t)kb.x_width * (P.th + P.sep) * P.box_tb();
+        // the last 8-pixel group a window reads: shift + (n_cols / 8 - 1) rows of the box + 8 pixels
+        const size_t reach_px = (size_t)kb.x_shift + lane1_shift_px(P, kb.x_width) + (size_t)(P.n_cols / 8 - 1) * (kb.x_width * 8 / P.tw) + 8;
+        a_slot = std::max(a_slot, (int)sr_align_up(std::max(box_px, reach_px) * kb.bk * 2, 1024));
+    }
+    return a_slot;
+}
+
+int weight_slot_bytes(const sr_graph*, const NodePlan& P)
+{
+    int w = 1024;
+    for (const WGroup& wg : P.wgroups) w = std::max(w, (int)sr_align_up((size_t)wg.bytes, 1024));
+    return w;
+}
+
+std::vector<TcTile> node_tiles(const sr_graph* g, const NodePlan& P, int node_index)
+{
+    const SrHostNode& n = g->nodes[P.node];
+    std::vector<TcTile> out;
+    const int db = P.tb * (P.pair == 2 ? 2 : 1), dw = P.tw * (P.pair == 1 ? 2 : 1);
+    for (int b0 = 0; b0 < g->batch; b0 += db)
+        for (int h0 = 0; h0 < n.d.h; h0 += P.th)
+            for (int w0 = 0; w0 < n.d.w; w0 += dw)
+                for (int m0 = 0; m0 < n.d.c; m0 += 128) {
+                    int lanes = 1;
+                    if (P.pair == 1 && w0 + P.tw < n.d.w) lanes = 2;
+                    if (P.pair == 2 && b0 + P.tb < g->batch) lanes = 2;
+                    out.push_back(TcTile{node_index, b0, h0, w0, m0, lanes, {0, 0}});
+                }
+    return out;
+}
+
 }  // namespace
 
-// A node goes to the tensor cores if it sums convolutions only, has 16..256 output channels in
+// A node goes to the tensor cores if it sums convolutions only, has at least 16 output channels in
 // multiples of 8, and every incoming edge either has C_in % 16 == 0 or is a few-channel input edge.
 void sr_tc_select_nodes(sr_graph* g)
 {
@@ -719,7 +1040,7 @@ void sr_tc_select_nodes(sr_graph* g)
         SrHostNode& n = g->nodes[v];
         n.use_tc = false;
         if (n.is_input || n.dense_target || (int)v == g->info.output_node) continue;
-        if (n.d.c % 8 != 0 || n.d.c < 16 || n.d.c > 256) continue;
+        if (n.d.c % 8 != 0 || n.d.c < 16 || n.d.c > 1024) continue;
         bool ok = true;
         int n_blocks = 0;
         for (int e : n.in_edges) {
@@ -742,6 +1063,9 @@ sr_status sr_tc_plan(sr_graph* g, size_t& off)
     if (!any) return SR_OK;
     TcEngine* E = new TcEngine();
     g->tc = E;
+    int dev = 0;
+    if (cudaGetDevice(&dev) == cudaSuccess) cudaDeviceGetAttribute(&E->sm_count, cudaDevAttrMultiProcessorCount, dev);
+    if (E->sm_count <= 0) E->sm_count = 148;
     E->node_of.assign(g->nodes.size(), -1);
     E->stem_of_edge.assign(g->edges.size(), -1);
     auto take = [&](size_t bytes) {
@@ -751,21 +1075,27 @@ sr_status sr_tc_plan(sr_graph* g, size_t& off)
         off = sr_align_up(off + bytes, 1024);
         return r;
     };
+    // tile geometry and staging buffers
     for (size_t v = 0; v < g->nodes.size(); ++v) {
         const SrHostNode& n = g->nodes[v];
         if (!n.use_tc) continue;
         NodePlan P{};
         P.node = (int)v;
         // sep: how many image rows the taps that share one activation box are apart at most
-        auto tap_q = [](int tap, int pad, int st, int& q, int& r) {
-            const int a = tap - pad;
-            q = (a >= 0) ? a / st : -((-a + st - 1) / st);
-            r = a - q * st;
-        };
         P.sep = 0;
         for (int e : n.in_edges) {
             const SrHostEdge& he = g->edges[e];
-            if (is_stem(g, he)) continue;
+            if (is_stem(g, he)) {
+                StemPlan S;
+                S.edge = e;
+                S.Kp = stem_kp(he.K);
+                const size_t bytes = (size_t)g->batch * n.d.h * n.d.w * S.Kp * 2;
+                S.buf[0] = take(bytes);
+                S.buf[1] = take(bytes);
+                E->stem_of_edge[e] = (int)E->stems.size();
+                E->stems.push_back(S);
+                continue;
+            }
             for (int r0 = 0; r0 < he.stride_eff; ++r0) {
                 int lo = 1 << 20, hi = -(1 << 20);
                 for (int t = 0; t < he.k_eff; ++t) {
@@ -778,118 +1108,116 @@ sr_status sr_tc_plan(sr_graph* g, size_t& off)
         }
         choose_tile(n.d.h, n.d.w, g->batch, P.sep, g->opt_tile_w, P);
         P.one_box = P.tw == 8;
-        P.n_mh = 1;                                   // a node with more than 128 output channels is tiled in halves
-        P.group = 3;
-        int k_off = 0;
-        for (int e : n.in_edges) {
-            const SrHostEdge& he = g->edges[e];
-            const SrHostNode& s = g->nodes[he.d.src];
-            P.edge_k_off.push_back(k_off);
-            if (is_stem(g, he)) {
-                StemPlan S;
-                S.edge = e;
-                S.Kp = stem_kp(he.K);
-                const size_t bytes = (size_t)g->batch * n.d.h * n.d.w * S.Kp * 2;
-                S.buf[0] = take(bytes);
-                S.buf[1] = take(bytes);
-                E->stem_of_edge[e] = (int)E->stems.size();
-                E->stems.push_back(S);
-                P.kbs.push_back(KbHost{e, true, (int)E->stems.size() - 1, 0, 0, 0, S.Kp, k_off, true, 0, P.tw, true});
-                k_off += S.Kp;
-            } else {
-                // Taps whose input pixels fall into the same residue class of the stride read the same view of the
-                // source, shifted by whole pixels: they share ONE activation box and differ only in where their window
-                // starts inside it (rows always; pixels too when the tile is 8 wide, because then the 8-pixel groups of
-                // the operand are simply one box row apart, whatever the row length).
-                const int bk = block_k(s.d.c), k = he.k_eff, st = he.stride_eff;
-                const int edge_off = k_off;
-                struct Tap { int ky, kx, qy, qx; };
-                std::map<std::tuple<int, int, int>, std::vector<Tap>> classes;      // (ry, rx, qx or 0) -> taps
-                for (int ky = 0; ky < k; ++ky)
-                    for (int kx = 0; kx < k; ++kx) {
-                        int qy, ry, qx, rx;
-                        tap_q(ky, he.pad_eff, st, qy, ry);
-                        tap_q(kx, he.pad_eff, st, qx, rx);
-                        classes[std::make_tuple(ry, rx, P.one_box ? 0 : qx)].push_back(Tap{ky, kx, qy, qx});
-                    }
-                for (int c0 = 0; c0 < s.d.c; c0 += bk)
-                    for (auto& cl : classes) {
-                        const std::vector<Tap>& taps = cl.second;
-                        int qy0 = 1 << 20, qx0 = 1 << 20, qx1 = -(1 << 20);
-                        for (const Tap& t : taps) { qy0 = std::min(qy0, t.qy); qx0 = std::min(qx0, t.qx); qx1 = std::max(qx1, t.qx); }
-                        const int bw = P.tw + (qx1 - qx0);
-                        for (size_t i = 0; i < taps.size(); ++i) {
-                            const Tap& t = taps[i];
-                            // the first tap of the class carries the box origin (qy0, qx0) through its ky / kx fields
-                            KbHost kb{e, false, -1, t.ky, t.kx, c0, bk, edge_off + (t.ky * k + t.kx) * s.d.c + c0,
-                                      i == 0, (t.qy - qy0) * bw + (t.qx - qx0), bw, i + 1 == taps.size()};
-                            kb.box_qy = qy0;
-                            kb.box_qx = qx0;
-                            kb.box_ry = std::get<0>(cl.first);
-                            kb.box_rx = std::get<1>(cl.first);
-                            P.kbs.push_back(kb);
-                        }
-                    }
-                k_off += k * k * s.d.c;
-            }
-        }
-        P.k_total = k_off;
-        P.wcat = take((size_t)n.d.c * P.k_total * 2);
+        P.pair = 0;
         E->node_of[v] = (int)E->nodes.size();
         E->nodes.push_back(P);
     }
-    // tiles per group, largest reduction first
+    // per launch group: pairing, K-blocks, work list (largest reduction first), ring geometry
     E->group_tiles.assign(g->groups.size(), {});
-    int n_tiles = 0, n_kbs = 0;
+    int n_tiles = 0;
     for (size_t gi = 0; gi < g->groups.size(); ++gi) {
-        std::vector<std::pair<long long, TcTile>> tl;
-        int a_slot = 1024, w_slot = 1;
-        for (int v : g->groups[gi]) {
-            if (E->node_of[v] < 0) continue;
-            const NodePlan& P = E->nodes[E->node_of[v]];
-            const SrHostNode& n = g->nodes[v];
-            for (int b0 = 0; b0 < g->batch; b0 += P.tb)
-                for (int h0 = 0; h0 < n.d.h; h0 += P.th)
-                    for (int w0 = 0; w0 < n.d.w; w0 += P.tw)
-                        for (int m0 = 0; m0 < n.d.c; m0 += 128)
-                            tl.push_back({(long long)P.kbs.size() * P.n_cols, TcTile{E->node_of[v], b0, h0, w0, m0, {0, 0, 0}}});
-            w_slot = std::max(w_slot, std::max(1, (std::min(n.d.c, 128) * 128 + kWUnit - 1) / kWUnit) * P.group);
-            // a window starts up to sep * tw rows into the box and the MMA reads n_cols rows from there
-            for (const KbHost& kb : P.kbs) {
-                const size_t box_px = (size_t)kb.x_width * (P.th + P.sep) * P.tb;
-                // the last 8-pixel group a window reads: shift + (n_cols / 8 - 1) rows of the box + 8 pixels
-                const size_t reach_px = (size_t)kb.x_shift + (size_t)(P.n_cols / 8 - 1) * (kb.x_width * 8 / P.tw) + 8;
-                a_slot = std::max(a_slot, (int)sr_align_up(std::max(box_px, reach_px) * kb.bk * 2, 1024));
-            }
+        std::vector<int> members;
+        for (int v : g->groups[gi])
+            if (E->node_of[v] >= 0) members.push_back(E->node_of[v]);
+        size_t single_tiles = 0;
+        for (int ni : members) {
+            build_kblocks(g, E, E->nodes[ni]);
+            single_tiles += node_tiles(g, E->nodes[ni], ni).size();
         }
-        std::stable_sort(tl.begin(), tl.end(), [](const auto& a, const auto& b) { return a.first > b.first; });
-        for (auto& p : tl) E->group_tiles[gi].push_back(p.second);
-        E->group_tile_offset.push_back(n_tiles);
-        n_tiles += (int)tl.size();
-        int n_wu = g->opt_b_units > 0 ? g->opt_b_units : 24;
-        n_wu = std::max(2 * w_slot, std::min(kMaxWUnits, n_wu)) / w_slot * w_slot;
-        int n_a = std::max(2, std::min(kMaxA, (kSmemBudget - n_wu * kWUnit) / a_slot));
+        // Pairs halve the weight traffic but double the size of a work item, expose the epilogue (both accumulators
+        // are busy) and leave room for fewer weight slots; with copies issued group-wise the L2 keeps single tiles
+        // fed, so pairs are used on request only.  Option "pair": 0 / 1 = single tiles, 2 = pairs wherever the
+        // geometry allows.
+        (void)single_tiles;
+        bool pair = g->opt_tc_pair == 2;
+        int a_slot = 1024, w_slot = 1024, n_a = 2, n_w = 2, per_sm = 1;
+        for (int attempt = 0; attempt < 2; ++attempt) {
+            a_slot = 1024;
+            w_slot = 1024;
+            for (int ni : members) {
+                NodePlan& P = E->nodes[ni];
+                const SrHostNode& n = g->nodes[P.node];
+                P.pair = 0;
+                if (pair) {
+                    if (P.tw == 8 && n.d.w > P.tw) P.pair = 1;
+                    else if (P.th == n.d.h && g->batch > P.tb) P.pair = 2;
+                }
+                build_kblocks(g, E, P);
+                a_slot = std::max(a_slot, act_slot_bytes(P));
+                w_slot = std::max(w_slot, weight_slot_bytes(g, P));
+            }
+            // two activation slots (a box usually serves a whole filter, and its producer runs ahead on its own), the
+            // weight ring as deep as it gets; more activation slots only once the weight ring is full
+            const int avail = kSmemBudget - 1024;
+            const int w_max = g->opt_b_units > 0 ? std::min(kMaxW, std::max(2, g->opt_b_units)) : kMaxW;
+            n_a = 2;
+            while (n_a < kMaxA && (n_a + 1) * a_slot + w_max * w_slot <= avail) ++n_a;
+            n_w = std::min(w_max, (avail - n_a * a_slot) / w_slot);
+            if (n_w >= 3 || !pair) break;
+            pair = false;                                  // the paired boxes do not leave room for a weight ring: single tiles
+        }
+        if (!members.empty() && n_w < 2) return SR_ERR_UNSUPPORTED;
         // Small launches (a few tiles per SM) are bound by the latency of one tile, not by throughput: give every
         // CTA the smallest rings and one accumulator, so that two CTAs share an SM and twice as many tiles are in flight.
-        int per_sm = 1;
-        if ((int)tl.size() <= 4 * 148 && 2 * w_slot * kWUnit + 2 * a_slot <= 88 * 1024) {
-            per_sm = 2;
-            n_wu = 2 * w_slot;
-            n_a = 2;
+        std::vector<std::pair<long long, TcTile>> tl;
+        for (int ni : members) {
+            const NodePlan& P = E->nodes[ni];
+            long long mma_cycles = 0;                        // one lane's MMAs: about max(110, N / 2) cycles each
+            for (const KbHost& kb : P.kbs) mma_cycles += (long long)(kb.bk / 16) * std::max(110, P.n_cols / 2);
+            for (const TcTile& t : node_tiles(g, P, ni))
+                tl.push_back({mma_cycles * t.lanes + (t.lanes == 2 ? 6000 : 1500), t});    // plus start-up and exposed epilogue
         }
+        if (!pair && (int)tl.size() <= 4 * E->sm_count && 2 * a_slot + 3 * w_slot + 1024 <= 88 * 1024) {
+            per_sm = 2;
+            n_a = 2;
+            n_w = std::min(kMaxW, (88 * 1024 - 1024 - 2 * a_slot) / w_slot);
+        }
+        // Work lists: the items go, longest first, to the CTA with the least work so far; CTA c then walks column c
+        // of a matrix with one row per round (entries of node -1 pad the shorter columns).
+        std::stable_sort(tl.begin(), tl.end(), [](const auto& a, const auto& b) { return a.first > b.first; });
+        const int grid = (int)std::min<size_t>(tl.size(), (size_t)E->sm_count * per_sm);
+        std::vector<std::vector<TcTile>> lists(std::max(grid, 1));
+        {
+            std::vector<std::pair<long long, int>> heap;     // (-load, cta): the standard heap keeps the largest on top
+            for (int c = 0; c < grid; ++c) heap.push_back({0, -c});
+            std::make_heap(heap.begin(), heap.end());
+            for (auto& it : tl) {
+                std::pop_heap(heap.begin(), heap.end());
+                std::pair<long long, int> top = heap.back();
+                lists[-top.second].push_back(it.second);
+                top.first -= it.first;
+                heap.back() = top;
+                std::push_heap(heap.begin(), heap.end());
+            }
+        }
+        size_t n_rows = 0;
+        for (auto& l : lists) n_rows = std::max(n_rows, l.size());
+        for (size_t r = 0; r < n_rows; ++r)
+            for (int c = 0; c < grid; ++c)
+                E->group_tiles[gi].push_back(r < lists[c].size() ? lists[c][r] : TcTile{-1, 0, 0, 0, 0, 0, {0, 0}});
+        E->group_grid.push_back(grid);
+        E->group_tile_offset.push_back(n_tiles);
+        n_tiles += (int)E->group_tiles[gi].size();
         E->group_ctas_per_sm.push_back(per_sm);
         E->group_a_slot.push_back(a_slot);
         E->group_n_a.push_back(n_a);
-        E->group_n_wu.push_back(n_wu);
+        E->group_n_w.push_back(n_w);
         E->group_w_slot.push_back(w_slot);
     }
-    for (const NodePlan& P : E->nodes) n_kbs += (int)P.kbs.size();
+    int n_kbs = 0;
+    for (NodePlan& P : E->nodes) {
+        n_kbs += (int)P.kbs.size();
+        P.wcat = take((size_t)g->nodes[P.node].d.c * P.k_total * 2);
+    }
     E->n_tiles = n_tiles;
     E->n_kbs = n_kbs;
     // upper bound on distinct tensor maps: two parities per K-block plus one weight map per (node, bk)
-    E->r_maps = take(sizeof(CUtensorMap) * (size_t)(2 * n_kbs + 3 * E->nodes.size() + 1));
+    E->r_maps = take(sizeof(CUtensorMap) * (size_t)(4 * n_kbs + 1));
     E->r_nodes = take(sizeof(TcNode) * E->nodes.size());
-    E->r_kbs = take(sizeof(TcKBlock) * (size_t)std::max(1, n_kbs));
+    E->r_kb_weight = take(sizeof(TcKbWeight) * (size_t)std::max(1, n_kbs));
+    E->r_kb_act = take(sizeof(TcKbAct) * (size_t)std::max(1, n_kbs));
+    E->r_bursts = take(sizeof(TcBurst) * (size_t)std::max(1, n_kbs));
+    E->r_states = take(sizeof(TcState) * (size_t)std::max(1, n_kbs));
     E->r_tiles = take(sizeof(TcTile) * (size_t)std::max(1, n_tiles));
     E->r_stems = take(sizeof(TcStem) * std::max<size_t>(1, E->stems.size()));
     return SR_OK;
@@ -901,10 +1229,7 @@ sr_status sr_tc_bind(sr_graph* g)
     if (!E) return SR_OK;
     EncodeTiledFn encode = encode_fn();
     if (!encode) return SR_ERR_CUDA;
-    int dev = 0;
-    cudaGetDevice(&dev);
-    cudaDeviceGetAttribute(&E->sm_count, cudaDevAttrMultiProcessorCount, dev);
-    if (cudaFuncSetAttribute(sr_tc_group_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBudget + 1024) != cudaSuccess)
+    if (cudaFuncSetAttribute(sr_tc_group_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBudget) != cudaSuccess)
         return SR_ERR_CUDA;
     char* ws = g->ws;
     std::vector<CUtensorMap> maps;
@@ -915,6 +1240,7 @@ sr_status sr_tc_bind(sr_graph* g)
         auto key = std::make_tuple((uintptr_t)base, C, Wv, Hv, (int)stride_w, bk, tw, rows, tb);
         auto it = cache.find(key);
         if (it != cache.end()) return it->second;
+        if (tw > 256 || rows > 256 || tb > 256) return -1;
         CUtensorMap m;
         cuuint64_t dims[4] = {(cuuint64_t)C, (cuuint64_t)Wv, (cuuint64_t)Hv, (cuuint64_t)g->batch};
         cuuint64_t strides[3] = {(cuuint64_t)stride_w, (cuuint64_t)stride_h, (cuuint64_t)stride_b};
@@ -928,7 +1254,10 @@ sr_status sr_tc_bind(sr_graph* g)
         return (int)maps.size() - 1;
     };
     std::vector<TcNode> dn;
-    std::vector<TcKBlock> dk;
+    std::vector<TcKbWeight> dw;
+    std::vector<TcKbAct> da;
+    std::vector<TcBurst> db;
+    std::vector<TcState> ds;
     for (const NodePlan& P : E->nodes) {
         const SrHostNode& n = g->nodes[P.node];
         TcNode d{};
@@ -937,67 +1266,74 @@ sr_status sr_tc_bind(sr_graph* g)
         d.bias = reinterpret_cast<const float*>(ws + n.bias.offset);
         d.H = n.d.h; d.W = n.d.w; d.C = n.d.c; d.act = n.d.act;
         d.tw = P.tw; d.th = P.th; d.tb = P.tb; d.sep = P.sep;
-        d.n_cols = P.n_cols; d.n_mh = P.n_mh;
-        d.first_kb = (int)dk.size();
-        d.n_kb = (int)P.kbs.size();
-        // instruction descriptor: D = f32, A = B = bf16, both K-major, M = 128 output channels, N = pixels
-        d.idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(P.n_cols >> 3) << 17) | ((uint32_t)(128 >> 4) << 24);
-        d.w_box_units = std::max(1, (std::min(n.d.c, 128) * 128 + kWUnit - 1) / kWUnit);
-        d.w_group_units = d.w_box_units * P.group;
-        const int rows = P.th + P.sep;
-        std::map<int, int> wmap;                      // bk -> weight tensor map
-        for (const KbHost& kb : P.kbs) {
-            if (wmap.count(kb.bk)) continue;
+        d.n_cols = P.n_cols;
+        d.l1_dw = P.pair == 1 ? P.tw : 0;
+        d.l1_db = P.pair == 2 ? P.tb : 0;
+        d.first_state = (int)ds.size();
+        d.first_act = (int)da.size();
+        std::vector<KmHost> dm;                       // per K-block of this node
+        d.first_wg = (int)dw.size();
+        d.n_wg = (int)P.wgroups.size();
+        const int rows = P.th + P.sep, box_tb = P.box_tb();
+        if (P.k_total > 65535) return SR_ERR_UNSUPPORTED;
+        // one 3-D view per run: (channels of a block, output channels, blocks of the run); a box of g blocks lands in
+        // shared memory block after block, each an ordinary K-major swizzled tile
+        std::map<std::pair<int, int>, int> run_map;   // (run, blocks in the box) -> tensor map
+        for (const WGroup& wg : P.wgroups) {
+            if (run_map.count({wg.run, wg.n})) continue;
+            const WRun& R = P.runs[wg.run];
             CUtensorMap m;
-            cuuint64_t dims[2] = {(cuuint64_t)P.k_total, (cuuint64_t)n.d.c};
-            cuuint64_t strides[1] = {(cuuint64_t)P.k_total * 2};
-            cuuint32_t box[2] = {(cuuint32_t)kb.bk, (cuuint32_t)std::min(n.d.c, 128)};
-            cuuint32_t es[2] = {1, 1};
-            if (encode(&m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, ws + P.wcat.offset, dims, strides, box, es,
-                       CU_TENSOR_MAP_INTERLEAVE_NONE, swizzle_of(kb.bk), CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+            cuuint64_t dims[3] = {(cuuint64_t)R.bk, (cuuint64_t)n.d.c, (cuuint64_t)R.n_blocks};
+            cuuint64_t strides[2] = {(cuuint64_t)P.k_total * 2, (cuuint64_t)R.bk * 2};
+            cuuint32_t box[3] = {(cuuint32_t)R.bk, (cuuint32_t)std::min(n.d.c, 128), (cuuint32_t)wg.n};
+            cuuint32_t es[3] = {1, 1, 1};
+            if (encode(&m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, ws + P.wcat.offset + (size_t)R.first_col * 2, dims, strides, box, es,
+                       CU_TENSOR_MAP_INTERLEAVE_NONE, swizzle_of(R.bk), CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
                        CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
                 return SR_ERR_CUDA;
             maps.push_back(m);
-            wmap[kb.bk] = (int)maps.size() - 1;
+            run_map[{wg.run, wg.n}] = (int)maps.size() - 1;
         }
-        // weight groups: up to P.group consecutive K-blocks of equal channel-block width
-        std::vector<int> box_of(P.kbs.size(), 0);
-        std::vector<char> starts(P.kbs.size(), 0), ends(P.kbs.size(), 0);
-        for (size_t i = 0, in_group = 0; i < P.kbs.size(); ++i) {
-            if (in_group == 0 || (int)in_group == P.group || P.kbs[i].bk != P.kbs[i - 1].bk || P.kbs[i].x_width != P.kbs[i - 1].x_width) {
-                starts[i] = 1;
-                if (i > 0) ends[i - 1] = 1;
-                in_group = 0;
-            }
-            box_of[i] = (int)in_group++;
+        for (const WGroup& wg : P.wgroups) {
+            TcKbWeight kw{};
+            const size_t bytes = (size_t)wg.bytes;
+            const int mi = run_map[{wg.run, wg.n}];
+            if (wg.blk > 65535 || mi > 65535 || (bytes >> 4) > 65535) return SR_ERR_UNSUPPORTED;
+            kw.blk = (uint16_t)wg.blk;
+            kw.w_map = (uint16_t)mi;
+            kw.w_bytes16 = (uint16_t)(bytes >> 4);
+            dw.push_back(kw);
         }
-        if (!P.kbs.empty()) ends[P.kbs.size() - 1] = 1;
         for (size_t i = 0; i < P.kbs.size(); ++i) {
             const KbHost& kb = P.kbs[i];
             const SrHostEdge& he = g->edges[kb.edge];
             const SrHostNode& s = g->nodes[he.d.src];
-            TcKBlock k{};
+            TcKbAct kl{};
+            KmHost km;
             int map0 = -1, map1 = -1, qxv = 0, qyv = 0;
-            const bool g_start = starts[i] != 0, g_end = ends[i] != 0;
-            k.flags = (uint8_t)((he.R ? 1 : 0) | (kb.x_release ? 2 : 0) | (g_start ? 4 : 0) | (g_end ? 8 : 0));
-            k.w_box = (uint8_t)box_of[i];
-            k.w_map = (uint16_t)wmap[kb.bk];
-            k.k_off = (uint32_t)kb.k_off;
-            k.n_k16 = (uint8_t)(kb.bk / 16);
-            k.desc_hi = desc_hi_of(kb.bk);
-            k.x_bytes16 = kb.x_load ? (uint16_t)((kb.bk * 2 * kb.x_width * rows * P.tb) >> 4) : 0;
-            k.x_sbo16 = (uint8_t)((kb.x_width * 8 / P.tw * kb.bk * 2) >> 4);
-            k.w_bytes16 = (uint16_t)((kb.bk * 2 * std::min(n.d.c, 128)) >> 4);
-            k.x_off16 = (uint16_t)((kb.x_shift * kb.bk * 2) >> 4);
+            kl.flags = (uint8_t)(he.R ? 1 : 0);
+            km.x_load = kb.x_load;
+            km.x_release = kb.x_release;
+            km.w_step16 = (uint32_t)((std::min(n.d.c, 128) * kb.bk * 2) >> 4);
+            km.n_k16 = (uint32_t)(kb.bk / 16);
+            km.desc_hi = desc_hi_of(kb.bk);
+            const size_t x_bytes = (size_t)kb.bk * 2 * kb.x_width * rows * box_tb;
+            const size_t l1_bytes = (size_t)lane1_shift_px(P, kb.x_width) * kb.bk * 2;
+            const size_t sbo_bytes = (size_t)kb.x_width * 8 / P.tw * kb.bk * 2;
+            if ((x_bytes >> 4) > 65535 || (l1_bytes >> 4) > 65535 || (sbo_bytes >> 4) > 0x3FFF) return SR_ERR_UNSUPPORTED;
+            kl.x_bytes16 = (uint16_t)(x_bytes >> 4);
+            km.x_sbo16 = (uint32_t)(sbo_bytes >> 4);
+            km.x_l1off16 = (uint32_t)(l1_bytes >> 4);
+            km.x_off16 = (uint32_t)((kb.x_shift * kb.bk * 2) >> 4);
             if (kb.stem) {
                 const StemPlan& S = E->stems[kb.stem_index];
                 for (int par = 0; par < 2; ++par)
                     (par ? map1 : map0) = act_map(ws + S.buf[par].offset, S.Kp, n.d.w, n.d.h, (size_t)S.Kp * 2,
-                                                  (size_t)n.d.w * S.Kp * 2, (size_t)n.d.h * n.d.w * S.Kp * 2, S.Kp, P.tw, rows, P.tb);
-                k.c0 = 0;
+                                                  (size_t)n.d.w * S.Kp * 2, (size_t)n.d.h * n.d.w * S.Kp * 2, S.Kp, kb.x_width, rows, box_tb);
+                kl.c0_16 = 0;
             } else if (!kb.x_load) {
-                map0 = map1 = 0;                         // reuses the box the first tap of this filter column loaded
-                k.c0 = (uint16_t)kb.c0;
+                map0 = map1 = 0;                         // reuses the box the first tap of its class loaded
+                kl.c0_16 = (uint8_t)(kb.c0 / 16);
             } else {
                 // input pixel = stride * (output pixel + q) + r, q = floor((tap - pad) / stride), r the residue:
                 // the residue-class view of the source makes the tap a dense box starting at (w0 + qx, h0 + qy)
@@ -1008,15 +1344,47 @@ sr_status sr_tc_bind(sr_graph* g)
                 for (int par = 0; par < 2; ++par) {
                     char* base = ws + s.state[par].offset + ((size_t)ry * s.d.w + rx) * s.d.c * 2;
                     (par ? map1 : map0) = act_map(base, s.d.c, Wv, Hv, (size_t)st * s.d.c * 2, (size_t)st * s.d.w * s.d.c * 2,
-                                                  (size_t)s.d.h * s.d.w * s.d.c * 2, kb.bk, kb.x_width, rows, P.tb);
+                                                  (size_t)s.d.h * s.d.w * s.d.c * 2, kb.bk, kb.x_width, rows, box_tb);
                 }
-                qxv = qx; qyv = qy; k.c0 = (uint16_t)kb.c0;
+                qxv = qx; qyv = qy; kl.c0_16 = (uint8_t)(kb.c0 / 16);
             }
             if (map0 < 0 || map1 < 0) return SR_ERR_CUDA;
-            if (map0 > 65535 || map1 > 65535 || qxv < -128 || qxv > 127 || qyv < -128 || qyv > 127) return SR_ERR_UNSUPPORTED;
-            k.x_map0 = (uint16_t)map0; k.x_map1 = (uint16_t)map1;
-            k.qx = (int8_t)qxv; k.qy = (int8_t)qyv;
-            dk.push_back(k);
+            if (map0 > 65535 || map1 > 65535 || qxv < -128 || qxv > 127 || qyv < -128 || qyv > 127 || kb.c0 / 16 > 255) return SR_ERR_UNSUPPORTED;
+            kl.x_map0 = (uint16_t)map0; kl.x_map1 = (uint16_t)map1;
+            kl.qx = (int8_t)qxv; kl.qy = (int8_t)qyv;
+            if (kb.x_load) da.push_back(kl);
+            dm.push_back(km);
+        }
+        d.n_act = (int)da.size() - d.first_act;
+        // bursts: one per weight group; descriptor states: the distinct (weight, activation) upper words of the node
+        size_t i0 = 0;
+        for (const WGroup& wg : P.wgroups) {
+            const KmHost& a = dm[i0];
+            TcState st{};
+            st.desc_hi = a.desc_hi;
+            st.x_hi = (a.desc_hi & ~0x3FFFu) | a.x_sbo16;
+            st.n_k16 = (uint16_t)a.n_k16;
+            st.w_step16 = (uint16_t)a.w_step16;
+            size_t si = (size_t)d.first_state;
+            for (; si < ds.size(); ++si)
+                if (std::memcmp(&ds[si], &st, sizeof(st)) == 0) break;
+            if (si == ds.size()) ds.push_back(st);
+            if (si - d.first_state > 255 || wg.n > 2 || (wg.n == 2 && P.pair != 0)) return SR_ERR_UNSUPPORTED;
+            TcBurst b{};
+            b.state = (uint8_t)(si - d.first_state);
+            b.xa_off16 = (uint16_t)a.x_off16;
+            b.flags = (uint8_t)((a.x_load ? 1 : 0) | (a.x_release ? 4 : 0));
+            if (wg.n == 2) {
+                const KmHost& c = dm[i0 + 1];
+                if (c.desc_hi != a.desc_hi || c.x_sbo16 != a.x_sbo16) return SR_ERR_UNSUPPORTED;
+                b.xb_off16 = (uint16_t)c.x_off16;
+                b.flags |= (uint8_t)(16 | (c.x_load ? 2 : 0) | (c.x_release ? 8 : 0));
+            } else {
+                if (a.x_off16 + a.x_l1off16 > 65535) return SR_ERR_UNSUPPORTED;
+                b.xb_off16 = (uint16_t)(a.x_off16 + a.x_l1off16);
+            }
+            db.push_back(b);
+            i0 += (size_t)wg.n;
         }
         dn.push_back(d);
     }
@@ -1042,12 +1410,10 @@ sr_status sr_tc_bind(sr_graph* g)
         return bytes == 0 || cudaMemcpy(ws + r.offset, p, bytes, cudaMemcpyHostToDevice) == cudaSuccess;
     };
     if (!up(E->r_maps, maps.data(), maps.size() * sizeof(CUtensorMap)) || !up(E->r_nodes, dn.data(), dn.size() * sizeof(TcNode)) ||
-        !up(E->r_kbs, dk.data(), dk.size() * sizeof(TcKBlock)) || !up(E->r_tiles, tiles.data(), tiles.size() * sizeof(TcTile)) ||
-        !up(E->r_stems, stems.data(), stems.size() * sizeof(TcStem)))
+        !up(E->r_kb_weight, dw.data(), dw.size() * sizeof(TcKbWeight)) || !up(E->r_kb_act, da.data(), da.size() * sizeof(TcKbAct)) ||
+        !up(E->r_bursts, db.data(), db.size() * sizeof(TcBurst)) || !up(E->r_states, ds.data(), ds.size() * sizeof(TcState)) ||
+        !up(E->r_tiles, tiles.data(), tiles.size() * sizeof(TcTile)) || !up(E->r_stems, stems.data(), stems.size() * sizeof(TcStem)))
         return SR_ERR_CUDA;
-    E->group_grid.clear();
-    for (size_t gi = 0; gi < E->group_tiles.size(); ++gi)
-        E->group_grid.push_back((int)std::min<size_t>(E->group_tiles[gi].size(), (size_t)E->sm_count * E->group_ctas_per_sm[gi]));
     return SR_OK;
 }
 
@@ -1060,21 +1426,25 @@ sr_status sr_tc_set_weights(sr_graph* g, int edge, const float* w_eff)
     if (ni < 0) return SR_ERR_STATE;
     const NodePlan& P = E->nodes[ni];
     const SrHostNode& t = g->nodes[he.d.tgt];
-    int k_off = -1, width = he.K;
-    for (size_t i = 0; i < t.in_edges.size(); ++i)
-        if (t.in_edges[i] == edge) k_off = P.edge_k_off[i];
-    if (k_off < 0) return SR_ERR_STATE;
-    if (E->stem_of_edge[edge] >= 0) width = E->stems[E->stem_of_edge[edge]].Kp;
-    std::vector<uint16_t> h((size_t)t.d.c * width, 0);
-    for (int co = 0; co < t.d.c; ++co)
-        for (int k = 0; k < he.K; ++k) {
-            const __nv_bfloat16 b = __float2bfloat16_rn(w_eff[(size_t)co * he.K + k]);
-            std::memcpy(&h[(size_t)co * width + k], &b, 2);
-        }
-    char* dst = g->ws + P.wcat.offset + (size_t)k_off * 2;
-    if (cudaMemcpy2D(dst, (size_t)P.k_total * 2, h.data(), (size_t)width * 2, (size_t)width * 2, t.d.c,
-                     cudaMemcpyHostToDevice) != cudaSuccess)
-        return SR_ERR_CUDA;
+    // the node's weight matrix keeps its columns in the order the K loop walks them: every K-block of this edge
+    // takes its slice [C_out][block width] of the edge's own matrix (a staged edge: all of it, zero-padded)
+    bool any = false;
+    for (const KbHost& kb : P.kbs) {
+        if (kb.edge != edge) continue;
+        any = true;
+        const int n_src = kb.stem ? he.K : kb.bk;
+        std::vector<uint16_t> h((size_t)t.d.c * kb.bk, 0);
+        for (int co = 0; co < t.d.c; ++co)
+            for (int k = 0; k < n_src; ++k) {
+                const __nv_bfloat16 b = __float2bfloat16_rn(w_eff[(size_t)co * he.K + kb.src_col + k]);
+                std::memcpy(&h[(size_t)co * kb.bk + k], &b, 2);
+            }
+        char* dst = g->ws + P.wcat.offset + (size_t)kb.k_off * 2;
+        if (cudaMemcpy2D(dst, (size_t)P.k_total * 2, h.data(), (size_t)kb.bk * 2, (size_t)kb.bk * 2, t.d.c,
+                         cudaMemcpyHostToDevice) != cudaSuccess)
+            return SR_ERR_CUDA;
+    }
+    if (!any) return SR_ERR_STATE;
     return SR_OK;
 }
 
@@ -1102,8 +1472,8 @@ int sr_tc_launch_group(sr_graph* g, int group, int t_off, cudaStream_t s)
 {
     TcEngine* E = eng(g);
     if (!E || E->group_tiles[group].empty()) return 0;
-    const int n_a = E->group_n_a[group], a_slot = E->group_a_slot[group], n_wu = E->group_n_wu[group];
-    const size_t smem = (size_t)n_a * a_slot + (size_t)n_wu * kWUnit + 1024;
+    const int n_a = E->group_n_a[group], a_slot = E->group_a_slot[group], n_w = E->group_n_w[group], w_slot = E->group_w_slot[group];
+    const size_t smem = (size_t)n_a * a_slot + (size_t)n_w * w_slot + 1024;
     cudaStreamCaptureStatus cap = cudaStreamCaptureStatusNone;
     bool timed = g->opt_time_tc != 0 && cudaStreamIsCapturing(s, &cap) == cudaSuccess && cap == cudaStreamCaptureStatusNone;
     if (timed) {
@@ -1121,10 +1491,11 @@ int sr_tc_launch_group(sr_graph* g, int group, int t_off, cudaStream_t s)
     }
     sr_tc_group_kernel<<<E->group_grid[group], kThreads, smem, s>>>(
         reinterpret_cast<const CUtensorMap*>(g->ws + E->r_maps.offset), reinterpret_cast<const TcNode*>(g->ws + E->r_nodes.offset),
-        reinterpret_cast<const TcKBlock*>(g->ws + E->r_kbs.offset),
+        reinterpret_cast<const TcKbWeight*>(g->ws + E->r_kb_weight.offset), reinterpret_cast<const TcKbAct*>(g->ws + E->r_kb_act.offset),
+        reinterpret_cast<const TcBurst*>(g->ws + E->r_bursts.offset), reinterpret_cast<const TcState*>(g->ws + E->r_states.offset),
         reinterpret_cast<const TcTile*>(g->ws + E->r_tiles.offset) + E->group_tile_offset[group],
         (int)E->group_tiles[group].size(), reinterpret_cast<SrFrameCtl*>(g->ws + g->r_ctl.offset), t_off, g->batch, n_a, a_slot,
-        n_wu, E->group_w_slot[group], E->group_ctas_per_sm[group] > 1 ? 256 : 512, (long long)g->opt_wait_ms * 2000000LL);
+        n_w, w_slot, E->group_ctas_per_sm[group] > 1 ? 256 : 512, (long long)g->opt_wait_ms * 2000000LL);
     if (timed) {
         cudaEventRecord(E->ev[E->ev_used + 1], s);
         E->ev_used += 2;

@@ -29,13 +29,13 @@ def rel_err(got: np.ndarray, want: np.ndarray) -> float:
     return float(np.abs(got.astype(np.float64) - want).max()) / scale
 
 
-def check_stepwise(spec, pattern, engine="auto", samples=None, zero_bias=False, tol=None):
+def check_stepwise(spec, pattern, engine="auto", samples=None, zero_bias=False, tol=None, **options):
     """Step frame by frame; compare EVERY node state at EVERY frame with the oracle on `samples`."""
     import torch
     X, W, Bi = data.make_inputs(spec), data.make_weights(spec), data.make_biases(spec, zero=zero_bias)
     samples = list(range(spec.batch)) if samples is None else samples
     want = fu.rollout_spec(spec, pattern, X, W, Bi, samples=samples)
-    G = make_graph(spec, pattern, engine, 0, W, Bi)
+    G = make_graph(spec, pattern, engine, 0, W, Bi, **options)
     ins = G.input_nodes
     dev = {v: to_device(spec, X[v]) for v in ins}
     G.reset([dev[v][0] for v in ins])

@@ -17,10 +17,13 @@ def tiny(name, nodes, edges, batch=3, frames=3, R=None):
 
 
 def run(g):
+    # single tiles, then pairs of tiles that share every weight box (forced: these graphs are too small for the
+    # library to choose pairs by itself)
     from paper_1806_04965_b200 import Graph
     G = Graph(g.nodes, g.edges, g.patterns["p"], batch=g.batch, dtype="bf16")
     assert G.info["n_tensor_core_nodes"] >= 1, G.info
-    return parity.check_stepwise(g, "p", zero_bias=False)
+    parity.check_stepwise(g, "p", zero_bias=False, tc_pair=1)
+    return parity.check_stepwise(g, "p", zero_bias=False, tc_pair=2)
 
 
 @pytest.mark.parametrize("cin,cout,k,stride,size", [
@@ -71,4 +74,16 @@ def test_configs_reduced_tensor_cores(name, kw):
     g = build(name, **kw)
     for p in g.patterns:
         parity.check_stepwise(g, p, engine="auto", zero_bias=False)
+        parity.check_stepwise(g, p, engine="auto", zero_bias=False, tc_pair=2)
         parity.check_run(g, p, engine="auto", graph_frames=2)
+        parity.check_run(g, p, engine="auto", graph_frames=2, tc_pair=2, resident=False)
+
+
+@pytest.mark.parametrize("batch", [1, 2, 7])
+def test_pairs_with_ragged_batches_and_widths(batch):
+    # lane 1 of the last pair falls outside the batch (sample pairs) or outside the image (column pairs)
+    g = tiny("ragged", [Node("in", 20, 20, 64, IDENTITY), Node("a", 20, 20, 128), Node("b", 10, 10, 128), Node("c", 5, 5, 256),
+                        Node("o", 1, 1, 4, IDENTITY)],
+             [Edge(0, 1, CONV, 3, 1), Edge(1, 1, CONV, 3, 1), Edge(1, 2, CONV, 3, 2), Edge(2, 2, CONV, 3, 1), Edge(2, 3, CONV, 3, 2),
+              Edge(0, 3, CONV, 1, 4), Edge(3, 4, GAP_DENSE)], batch=batch, frames=3)
+    run(g)
