@@ -220,6 +220,29 @@ sr_status sr_rollout_step(sr_graph* g, const void* const* in_next_dev, float* ou
  */
 sr_status sr_rollout_run(sr_graph* g, const void* const* in_seq_dev, int T, float* out_seq_dev, void* stream);
 
+/*
+ * Deep rollout windows, W > 1 (Sec. 3, Definition "rollout pattern and window", Eq. 2; inference tableau, Eq. 4).
+ *
+ * sr_graph_window_tableau: T((i, v)) of the window of size W for i = 0..W, row-major [W + 1][n_nodes] on the host: the
+ * update step at which node v of frame i becomes computable when the whole window is evaluated at once (0 for frame
+ * 0 and for input nodes).  All nodes with the same value form one update step.  Pure host work; any valid pattern.
+ *
+ * sr_rollout_window: evaluates the W frame updates t+1 .. t+W as ONE window instead of W chained windows of size 1.
+ * Implemented for patterns whose frames do not depend on each other - every edge that bridges a frame leaves an
+ * input node (e.g. the sequential rollout of a network without recurrence) -, where T((i, v)) = level(v) for every
+ * frame i: level by level, the nodes of ALL W frames are updated in one launch group over a batch of W * B samples
+ * (the equal-compute comparison of Sec. 4, "classifications of the first 8 images in parallel").  Other patterns
+ * return SR_ERR_UNSUPPORTED.  in_seq_dev / out_seq_dev as for sr_rollout_run; afterwards the graph stands at frame
+ * t + W and can be stepped on.  Results equal those of W calls of sr_rollout_step.
+ * The window needs a workspace of its own (states of all W frames): ask for its size, allocate, bind; binding copies
+ * the parameters set so far, so set weights and biases first (later changes do not reach the window).
+ * Errors: INVALID_ARG, STATE (not bound, parameters missing, other W than bound), UNSUPPORTED, CUDA.
+ */
+sr_status sr_graph_window_tableau(const sr_graph* g, int W, int32_t* T_host);
+sr_status sr_graph_window_workspace_bytes(sr_graph* g, int W, size_t* bytes);
+sr_status sr_graph_bind_window(sr_graph* g, int W, void* workspace_dev, size_t bytes);
+sr_status sr_rollout_window(sr_graph* g, const void* const* in_seq_dev, int W, float* out_seq_dev, void* stream);
+
 /* Copy the current (frame t) state of a node out of / into the graph, [B][H][W][C] of the graph dtype.
  * Restoring all states and continuing to step resumes a rollout (Sec. 5: the next window starts
  * from the last frame of the previous one). */

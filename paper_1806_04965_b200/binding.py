@@ -77,6 +77,12 @@ def load_library(path: Optional[str] = None):
     lib.sr_graph_sync_status.argtypes = [vp, vp]
     lib.sr_graph_kernel_time.argtypes = [vp, ctypes.POINTER(ctypes.c_double), ctypes.POINTER(ctypes.c_int64)]
     lib.sr_graph_kernel_time.restype = ctypes.c_int
+    lib.sr_graph_window_tableau.argtypes = [vp, ip, ctypes.POINTER(ctypes.c_int32)]
+    lib.sr_graph_window_workspace_bytes.argtypes = [vp, ip, ctypes.POINTER(ctypes.c_size_t)]
+    lib.sr_graph_bind_window.argtypes = [vp, ip, vp, ctypes.c_size_t]
+    lib.sr_rollout_window.argtypes = [vp, ctypes.POINTER(vp), ip, vp, vp]
+    for name in ("sr_graph_window_tableau", "sr_graph_window_workspace_bytes", "sr_graph_bind_window", "sr_rollout_window"):
+        getattr(lib, name).restype = ctypes.c_int
     lib.sr_status_str.argtypes = [ip]
     lib.sr_status_str.restype = ctypes.c_char_p
     for name in ("sr_graph_create", "sr_graph_info", "sr_graph_levels", "sr_graph_workspace_bytes",
@@ -215,6 +221,31 @@ class Graph:
         _check(self._lib.sr_rollout_run(self._h, self._ptrs(in_seq, T), T,
                                         out_seq.data_ptr() if out_seq is not None else None, self._stream()),
                "sr_rollout_run")
+
+    def window_tableau(self, W: int) -> List[List[int]]:
+        """T((i, v)) of the rollout window of size W, one row per frame i = 0..W (Eq. 4)."""
+        n = len(self.nodes)
+        buf = (ctypes.c_int32 * ((W + 1) * n))()
+        _check(self._lib.sr_graph_window_tableau(self._h, W, buf), "sr_graph_window_tableau")
+        return [list(buf[i * n:(i + 1) * n]) for i in range(W + 1)]
+
+    def bind_window(self, W: int):
+        """Allocates and binds the workspace of a window of W frames (after the parameters have been set)."""
+        nbytes = ctypes.c_size_t()
+        _check(self._lib.sr_graph_window_workspace_bytes(self._h, W, ctypes.byref(nbytes)), "sr_graph_window_workspace_bytes")
+        self._window_ws = self._torch.empty(nbytes.value + 256, dtype=self._torch.uint8, device=self.device)
+        base = (self._window_ws.data_ptr() + 255) // 256 * 256
+        _check(self._lib.sr_graph_bind_window(self._h, W, base, nbytes.value), "sr_graph_bind_window")
+
+    def rollout_window(self, in_seq, out_seq=None):
+        """The W = in_seq[0].shape[0] frame updates t+1 .. t+W evaluated as one window."""
+        W = int(in_seq[0].shape[0])
+        if out_seq is not None:
+            assert out_seq.is_cuda and out_seq.is_contiguous() and out_seq.dtype == self._torch.float32
+            assert tuple(out_seq.shape) == (W,) + self.out_shape()
+        _check(self._lib.sr_rollout_window(self._h, self._ptrs(in_seq, W), W,
+                                           out_seq.data_ptr() if out_seq is not None else None, self._stream()),
+               "sr_rollout_window")
 
     def get_state(self, node: int):
         nd = self.nodes[node]

@@ -305,6 +305,8 @@ sr_status sr_graph_create(const sr_node_desc* nodes, int n_nodes, const sr_edge_
 void sr_graph_destroy(sr_graph* g)
 {
     if (!g) return;
+    if (g->window) sr_graph_destroy(g->window);
+    g->window = nullptr;
     sr_release_static_workspace(g);
     if (g->graphs) {
         GraphCache* c = static_cast<GraphCache*>(g->graphs);
@@ -537,6 +539,8 @@ sr_status sr_graph_set_edge_weights(sr_graph* g, int edge, const float* w, int i
     } else {
         std::memcpy(u.data(), w, n_user * sizeof(float));
     }
+    if (g->kept_weights.size() != g->edges.size()) g->kept_weights.assign(g->edges.size(), std::vector<float>());
+    g->kept_weights[edge] = u;                                   // as set by the caller: a window graph gets the same
     if (g->dtype == SR_DTYPE_BF16)
         for (float& x : u) x = round_bf16_host(x);
     // the convolution actually executed: [C_out][k'][k'][Cs]; a pooled edge gets the box-filtered kernel
@@ -588,6 +592,8 @@ sr_status sr_graph_set_node_bias(sr_graph* g, int node, const float* bias_host)
     if (!cuda_ok(cudaMemcpy(g->ws + n.bias.offset, bias_host, (size_t)n.d.c * sizeof(float), cudaMemcpyHostToDevice)))
         return SR_ERR_CUDA;
     n.bias_set = true;
+    if (g->kept_bias.size() != g->nodes.size()) g->kept_bias.assign(g->nodes.size(), std::vector<float>());
+    g->kept_bias[node].assign(bias_host, bias_host + n.d.c);
     return SR_OK;
 }
 
@@ -711,6 +717,122 @@ sr_status sr_rollout_run(sr_graph* g, const void* const* in_seq_dev, int T, floa
         g->launches += 1;
     }
     g->t += T;
+    return cuda_ok(cudaGetLastError()) ? SR_OK : SR_ERR_CUDA;
+}
+
+// ------------------------------------------------------------------ deep windows (W > 1)
+sr_status sr_graph_window_tableau(const sr_graph* g, int W, int32_t* T_host)
+{
+    if (!g || !T_host || W < 1 || W > 4096) return SR_ERR_INVALID_ARG;
+    sr_window_tableau(g, W, T_host);
+    return SR_OK;
+}
+
+static bool frames_independent(const sr_graph* g)
+{
+    for (const SrHostEdge& e : g->edges)
+        if (e.R == 1 && !g->nodes[e.d.src].is_input) return false;
+    return true;
+}
+
+sr_status sr_graph_window_workspace_bytes(sr_graph* g, int W, size_t* bytes)
+{
+    if (!g || !bytes || W < 1 || W > 4096) return SR_ERR_INVALID_ARG;
+    if (g->batch <= 0) return SR_ERR_STATE;
+    if (!frames_independent(g)) return SR_ERR_UNSUPPORTED;
+    if (g->window && g->window_frames != W) {
+        if (g->window->ws) return SR_ERR_STATE;                  // a bound window keeps its size
+        sr_graph_destroy(g->window);
+        g->window = nullptr;
+    }
+    if (!g->window) {
+        std::vector<sr_node_desc> nd;
+        std::vector<sr_edge_desc> ed;
+        std::vector<uint8_t> R;
+        for (const SrHostNode& n : g->nodes) nd.push_back(n.d);
+        for (const SrHostEdge& e : g->edges) {
+            ed.push_back(e.d);
+            R.push_back((uint8_t)e.R);
+        }
+        sr_graph* w = nullptr;
+        const sr_status st = sr_graph_create(nd.data(), (int)nd.size(), ed.data(), (int)ed.size(), R.data(), g->batch * W, g->dtype, &w);
+        if (st != SR_OK) return st;
+        w->opt_engine = g->opt_engine;
+        w->opt_b_units = g->opt_b_units;
+        w->opt_tile_w = g->opt_tile_w;
+        w->opt_overlap = g->opt_overlap;
+        w->opt_tc_pair = g->opt_tc_pair;
+        w->opt_wait_ms = g->opt_wait_ms;
+        w->opt_resident = 0;                                     // a window is one update of a large batch: the launch path
+        g->window = w;
+        g->window_frames = W;
+    }
+    return sr_graph_workspace_bytes(g->window, bytes);
+}
+
+sr_status sr_graph_bind_window(sr_graph* g, int W, void* workspace_dev, size_t bytes)
+{
+    if (!g || !workspace_dev) return SR_ERR_INVALID_ARG;
+    sr_status st = ready(g);
+    if (st != SR_OK) return st;
+    size_t need = 0;
+    st = sr_graph_window_workspace_bytes(g, W, &need);
+    if (st != SR_OK) return st;
+    if (g->window->ws) return SR_ERR_STATE;
+    if (g->kept_weights.size() != g->edges.size()) return SR_ERR_STATE;
+    st = sr_graph_bind_workspace(g->window, workspace_dev, bytes);
+    if (st != SR_OK) return st;
+    for (size_t e = 0; e < g->edges.size(); ++e) {
+        st = sr_graph_set_edge_weights(g->window, (int)e, g->kept_weights[e].data(), 0);
+        if (st != SR_OK) return st;
+    }
+    for (size_t v = 0; v < g->nodes.size() && v < g->kept_bias.size(); ++v)
+        if (!g->kept_bias[v].empty()) {
+            st = sr_graph_set_node_bias(g->window, (int)v, g->kept_bias[v].data());
+            if (st != SR_OK) return st;
+        }
+    return SR_OK;
+}
+
+sr_status sr_rollout_window(sr_graph* g, const void* const* in_seq_dev, int W, float* out_seq_dev, void* stream)
+{
+    sr_status st = ready(g);
+    if (st != SR_OK) return st;
+    sr_graph* w = g->window;
+    if (!w || !w->ws || g->window_frames != W) return SR_ERR_STATE;
+    if (!in_seq_dev) return SR_ERR_INVALID_ARG;
+    for (size_t i = 0; i < g->input_nodes.size(); ++i)
+        if (!in_seq_dev[i]) return SR_ERR_INVALID_ARG;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    // frames t .. t+W-1 of the input nodes side by side: what edges that bridge a frame read (Eq. 2: frame i - R(e))
+    for (size_t i = 0; i < g->input_nodes.size(); ++i) {
+        const int v = g->input_nodes[i];
+        const size_t frame = node_elems(g, v) * g->elem;
+        char* dst = w->ws + w->nodes[v].state[0].offset;
+        if (!cuda_ok(cudaMemcpyAsync(dst, g->ws + g->nodes[v].state[g->t & 1].offset, frame, cudaMemcpyDeviceToDevice, s))) return SR_ERR_CUDA;
+        if (W > 1 && !cuda_ok(cudaMemcpyAsync(dst + frame, in_seq_dev[i], frame * (size_t)(W - 1), cudaMemcpyDeviceToDevice, s)))
+            return SR_ERR_CUDA;
+    }
+    w->t = 0;
+    w->stage_dirty = false;
+    w->launches += sr_tc_after_state_change(w, s);
+    // ONE update of the window graph computes all W frames: its batch is [W][B], which is how in_seq and out_seq lie in memory
+    st = sr_rollout_step(w, in_seq_dev, out_seq_dev, stream);
+    if (st != SR_OK) return st;
+    // the last frame of the window becomes the current frame of this graph (Sec. 4: windows chain)
+    const int64_t t_new = g->t + W;
+    for (size_t v = 0; v < g->nodes.size(); ++v) {
+        const size_t frame = node_elems(g, (int)v) * g->elem;
+        char* dst = g->ws + g->nodes[v].state[t_new & 1].offset;
+        const char* src = g->nodes[v].is_input
+                              ? static_cast<const char*>(in_seq_dev[g->nodes[v].input_slot]) + frame * (size_t)(W - 1)
+                              : w->ws + w->nodes[v].state[1].offset + frame * (size_t)(W - 1);
+        if (!cuda_ok(cudaMemcpyAsync(dst, src, frame, cudaMemcpyDeviceToDevice, s))) return SR_ERR_CUDA;
+    }
+    g->t = t_new;
+    g->stage_dirty = true;
+    g->launches += w->launches;
+    w->launches = 0;
     return cuda_ok(cudaGetLastError()) ? SR_OK : SR_ERR_CUDA;
 }
 

@@ -176,3 +176,28 @@ sr_status sr_compile(sr_graph* g, const sr_node_desc* nodes, int n_nodes, const 
     I.response_interval = F;
     return SR_OK;
 }
+
+// Inference tableau of the rollout window of size W (Eq. 4): T((i, v)) for i = 0..W, row-major [W + 1][n_nodes].
+// Frame 0 and the input nodes are given (T = 0); every other node of the window becomes computable one update step
+// after the last of its predecessors ((i - R(e), u) for every edge e = (u, v)), which is also the length of the longest
+// admissible path that ends in it.  Frames are visited in increasing order and, inside a frame, nodes in increasing
+// level, so every predecessor is final when it is read.
+void sr_window_tableau(const sr_graph* g, int W, int32_t* T)
+{
+    const int n = (int)g->nodes.size();
+    std::vector<int> order;
+    for (const std::vector<int>& grp : g->groups)
+        for (int v : grp) order.push_back(v);
+    for (int v = 0; v < n; ++v) T[v] = 0;
+    for (int i = 1; i <= W; ++i) {
+        for (int v = 0; v < n; ++v) T[(size_t)i * n + v] = 0;
+        for (int v : order) {
+            int t = 0;
+            for (int e : g->nodes[v].in_edges) {
+                const SrHostEdge& he = g->edges[e];
+                t = std::max(t, T[(size_t)(i - he.R) * n + he.d.src]);
+            }
+            T[(size_t)i * n + v] = t + 1;
+        }
+    }
+}

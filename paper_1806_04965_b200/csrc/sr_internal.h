@@ -104,6 +104,11 @@ struct sr_graph {
     void* graphs = nullptr;                        // CUDA-graph cache (opaque here)
     void* side = nullptr;                          // side stream and fork / join events (opaque here)
     bool input_feeds_same_frame = false;           // some edge that leaves an input node has R = 0
+    // deep-window mode: a second graph of the same network whose batch holds the W frames of a window side by side
+    sr_graph* window = nullptr;
+    int window_frames = 0;
+    std::vector<std::vector<float>> kept_weights;  // the parameters as the caller set them (host copies), for that graph
+    std::vector<std::vector<float>> kept_bias;
     int static_device = -1;                        // >= 0: bound to the built-in workspace of that device
     bool stage_dirty = false;                      // the resident kernel ran: staged copies of the input state are stale
 };
@@ -111,5 +116,7 @@ struct sr_graph {
 // sr_compile.cpp
 sr_status sr_compile(sr_graph* g, const sr_node_desc* nodes, int n_nodes, const sr_edge_desc* edges, int n_edges,
                      const uint8_t* R);
+
+void sr_window_tableau(const sr_graph* g, int W, int32_t* T /* [W + 1][n_nodes] */);
 
 inline size_t sr_align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }

@@ -189,6 +189,12 @@ __device__ __forceinline__ void tma_load_4d(uint32_t dst, const void* map, uint3
         "cp.async.bulk.tensor.4d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5, %6}], [%2];"
         ::"r"(dst), "l"(map), "r"(bar), "r"(c0), "r"(c1), "r"(c2), "r"(c3) : "memory");
 }
+// Ask for a box to be brought into L2 (no shared memory, no barrier: fire and forget).
+__device__ __forceinline__ void tma_prefetch_4d(const void* map, int c0, int c1, int c2, int c3)
+{
+    asm volatile("cp.async.bulk.prefetch.tensor.4d.L2.global.tile [%0, {%1, %2, %3, %4}];"
+                 ::"l"(map), "r"(c0), "r"(c1), "r"(c2), "r"(c3) : "memory");
+}
 __device__ __forceinline__ void tma_load_3d(uint32_t dst, const void* map, uint32_t bar, int c0, int c1, int c2)
 {
     asm volatile(
@@ -378,8 +384,24 @@ sr_tc_group_kernel(const CUtensorMap* __restrict__ maps, const TcNode* __restric
             }
             if (lane == 0) {
                 const TcKbAct* tab = reinterpret_cast<const TcKbAct*>(a_tab);
+                // With two or three slots a box is requested only about one filter ahead of its use, and a box that
+                // comes from DRAM takes longer than that.  So every request is accompanied by an L2 prefetch of the
+                // box two further on (of the next work item when this one ends, if it belongs to the same node).
+                TcTile nx = tl;
+                nx.node = -1;
+                if (ti + (int)gridDim.x < n_tiles) nx = tiles[ti + gridDim.x];
                 for (int i = 0; i < n_act; ++i) {
                     const TcKbAct k = tab[i];
+                    {
+                        const int j = i + 2 < n_act ? i + 2 : i + 2 - n_act;
+                        const bool here = i + 2 < n_act;
+                        if ((here || nx.node == tl.node) && j < n_act) {
+                            const TcKbAct p = tab[j];
+                            const TcTile& pt = here ? tl : nx;
+                            const int par = (p.flags & 1) ? prev : cur;
+                            tma_prefetch_4d(&maps[par ? p.x_map1 : p.x_map0], (int)p.c0_16 << 4, pt.w0 + p.qx, pt.h0 + p.qy, pt.b0);
+                        }
+                    }
                     const uint32_t s = a_nxt;
                     if (!mbar_wait(bar_aempty + 8 * s, a_ph ^ 1, abortp, wait_limit)) { ok = false; break; }
                     a_used |= 1u << s;
@@ -700,13 +722,13 @@ sr_tc_group_kernel(const CUtensorMap* __restrict__ maps, const TcNode* __restric
 __global__ void sr_tc_stage_kernel(const TcStem* __restrict__ stems, int n_stems, const SrFrameCtl* __restrict__ ctl,
                                    int t_off, int fixed_parity, int B)
 {
-    __shared__ int tap_off[64];     // offset of element kk relative to the (unpadded) window origin, -1 = padding
-    __shared__ short tap_dy[64], tap_dx[64];
+    __shared__ int tap_off[128];    // offset of element kk relative to the (unpadded) window origin, -1 = padding
+    __shared__ short tap_dy[128], tap_dx[128];
     const int cur = fixed_parity >= 0 ? fixed_parity : (int)((ctl->t + t_off + 1) & 1);
     for (int si = 0; si < n_stems; ++si) {
         const TcStem st = stems[si];
         __syncthreads();
-        if (threadIdx.x < 64) {
+        if (threadIdx.x < 128) {
             const int kk = threadIdx.x;
             if (kk < st.K) {
                 const int ci = kk % st.Cs, tap = kk / st.Cs, kx = tap % st.k, ky = tap / st.k;
@@ -814,11 +836,11 @@ struct TcEngine {
 TcEngine* eng(const sr_graph* g) { return static_cast<TcEngine*>(g->tc); }
 
 int block_k(int cs) { return cs % 64 == 0 ? 64 : (cs % 32 == 0 ? 32 : 16); }
-int stem_kp(int K) { return K <= 16 ? 16 : (K <= 32 ? 32 : 64); }
+int stem_kp(int K) { return K <= 16 ? 16 : (K <= 32 ? 32 : (K <= 64 ? 64 : 128)); }
 bool is_stem(const sr_graph* g, const SrHostEdge& e)
 {
     const SrHostNode& s = g->nodes[e.d.src];
-    return s.is_input && (s.d.c % 16) != 0 && e.K <= 64;
+    return s.is_input && (s.d.c % 16) != 0 && e.K <= 128;
 }
 
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
@@ -908,15 +930,20 @@ void build_kblocks(const sr_graph* g, const TcEngine* E, NodePlan& P)
     std::vector<int> order(n.in_edges.begin(), n.in_edges.end());
     auto width_of = [&](int e) {
         const SrHostEdge& he = g->edges[e];
-        return is_stem(g, he) ? E->stems[E->stem_of_edge[e]].Kp : block_k(g->nodes[he.d.src].d.c);
+        return is_stem(g, he) ? std::min(64, E->stems[E->stem_of_edge[e]].Kp) : block_k(g->nodes[he.d.src].d.c);
     };
     std::stable_sort(order.begin(), order.end(), [&](int a, int b) { return width_of(a) > width_of(b); });
     for (int e : order) {
         const SrHostEdge& he = g->edges[e];
         const SrHostNode& s = g->nodes[he.d.src];
         if (is_stem(g, he)) {
-            const int si = E->stem_of_edge[e], Kp = E->stems[si].Kp;
-            P.kbs.push_back(KbHost{e, true, si, 0, 0, 0, Kp, 0, true, 0, P.lane_w(), true});
+            // a staged edge: its im2col rows are one K-block of 16 / 32 / 64 columns, or two of 64
+            const int si = E->stem_of_edge[e], Kp = E->stems[si].Kp, bk = std::min(64, Kp);
+            for (int c0 = 0; c0 < Kp; c0 += bk) {
+                KbHost kb{e, true, si, 0, 0, c0, bk, 0, true, 0, P.lane_w(), true};
+                kb.src_col = c0;
+                P.kbs.push_back(kb);
+            }
         } else {
             // Taps whose input pixels fall into the same residue class of the stride read the same view of the
             // source, shifted by whole pixels: they share ONE activation box and differ only in where their window
@@ -1049,7 +1076,7 @@ void sr_tc_select_nodes(sr_graph* g)
             if (he.d.kind != SR_EDGE_CONV) ok = false;
             else if (s.d.c % 16 != 0 && !is_stem(g, he)) ok = false;
             else if (he.k_eff > 8) ok = false;
-            else n_blocks += is_stem(g, he) ? 1 : he.k_eff * he.k_eff * (s.d.c / block_k(s.d.c));
+            else n_blocks += is_stem(g, he) ? 2 : he.k_eff * he.k_eff * (s.d.c / block_k(s.d.c));
         }
         if (ok && n_blocks >= 1 && n_blocks <= kMaxNodeKb) n.use_tc = true;
     }
@@ -1329,8 +1356,8 @@ sr_status sr_tc_bind(sr_graph* g)
                 const StemPlan& S = E->stems[kb.stem_index];
                 for (int par = 0; par < 2; ++par)
                     (par ? map1 : map0) = act_map(ws + S.buf[par].offset, S.Kp, n.d.w, n.d.h, (size_t)S.Kp * 2,
-                                                  (size_t)n.d.w * S.Kp * 2, (size_t)n.d.h * n.d.w * S.Kp * 2, S.Kp, kb.x_width, rows, box_tb);
-                kl.c0_16 = 0;
+                                                  (size_t)n.d.w * S.Kp * 2, (size_t)n.d.h * n.d.w * S.Kp * 2, kb.bk, kb.x_width, rows, box_tb);
+                kl.c0_16 = (uint8_t)(kb.c0 / 16);
             } else if (!kb.x_load) {
                 map0 = map1 = 0;                         // reuses the box the first tap of its class loaded
                 kl.c0_16 = (uint8_t)(kb.c0 / 16);
@@ -1432,7 +1459,7 @@ sr_status sr_tc_set_weights(sr_graph* g, int edge, const float* w_eff)
     for (const KbHost& kb : P.kbs) {
         if (kb.edge != edge) continue;
         any = true;
-        const int n_src = kb.stem ? he.K : kb.bk;
+        const int n_src = kb.stem ? std::max(0, std::min(kb.bk, he.K - kb.src_col)) : kb.bk;
         std::vector<uint16_t> h((size_t)t.d.c * kb.bk, 0);
         for (int co = 0; co < t.d.c; ++co)
             for (int k = 0; k < n_src; ++k) {

@@ -134,3 +134,55 @@ def test_expired_device_wait_is_reported_and_cleared_by_reset():
 def fu_rollout(g, X, W, Bi):
     from oracle import frame_update as fu
     return fu.rollout_spec(g, "streaming", X, W, Bi)
+
+
+@pytest.mark.parametrize("name,kw,W", [("c4ff", dict(batch=3, frames=9, size=16), 4), ("dsr2", dict(batch=2, frames=7, h1_recurrence=False), 3),
+                                        ("mini_ff", dict(), 5)])
+def test_deep_window_equals_chained_windows(name, kw, W):
+    # a network without recurrence under the sequential rollout: the W frames of a window do not depend on each other and
+    # are evaluated at once (one launch group per level over W * B samples); results equal W single steps, the graph
+    # stands at frame t + W afterwards and can be stepped on (two windows, then single steps to the end)
+    import torch
+    from workloads.graphs import CONV, GAP_DENSE, IDENTITY, Edge, GraphSpec, Node, sequential_pattern, streaming_pattern
+    if name == "mini_ff":
+        # a streaming input edge (reads the previous input frame) beside within-frame edges
+        nodes = [Node("in", 16, 16, 3, IDENTITY), Node("a", 16, 16, 32), Node("b", 8, 8, 64), Node("o", 1, 1, 5, IDENTITY)]
+        edges = [Edge(0, 1, CONV, 3, 1), Edge(1, 2, CONV, 3, 2), Edge(0, 2, CONV, 1, 2), Edge(2, 3, GAP_DENSE)]
+        g = GraphSpec("mini_ff", nodes, edges, batch=3, frames=12, dtype="bf16", seed=77)
+        g.patterns = {"sequential": [0, 0, 1, 0]}
+    elif name == "dsr2":
+        g = graphs.dsr(2, **kw)
+    else:
+        g = graphs.build(name, **kw)
+    from oracle import frame_update as fu
+    X, Wt, Bi = data.make_inputs(g), data.make_weights(g), data.make_biases(g, zero=False)
+    want = fu.rollout_spec(g, "sequential", X, Wt, Bi)
+    G = parity.make_graph(g, "sequential", "auto", 0, Wt, Bi)
+    G.bind_window(W)
+    x = {v: parity.to_device(g, X[v]) for v in G.input_nodes}
+    G.reset([x[v][0] for v in G.input_nodes])
+    o, tol = G.output_node, parity.TOL[g.dtype]
+    t = 0
+    for _ in range(2):
+        out = torch.empty((W,) + G.out_shape(), dtype=torch.float32, device="cuda:0")
+        G.rollout_window([x[v][t + 1:t + 1 + W] for v in G.input_nodes], out)
+        assert G.frame() == t + W
+        assert parity.rel_err(out.cpu().numpy().reshape(want[o][t + 1:t + 1 + W].shape), want[o][t + 1:t + 1 + W]) <= tol
+        t += W
+        for v in range(len(g.nodes)):
+            assert parity.rel_err(G.get_state(v).float().cpu().numpy(), want[v][t]) <= tol, (g.nodes[v].name, t)
+    while t < g.frames:
+        G.step([x[v][t + 1] for v in G.input_nodes])
+        t += 1
+        for v in range(len(g.nodes)):
+            assert parity.rel_err(G.get_state(v).float().cpu().numpy(), want[v][t]) <= tol, (g.nodes[v].name, t)
+    G.sync_status()
+
+
+def test_deep_window_refuses_patterns_with_recurrence():
+    from paper_1806_04965_b200 import SrError
+    g = graphs.build("c2", batch=2, frames=3)
+    G = parity.make_graph(g, "streaming", "auto", 0, data.make_weights(g), data.make_biases(g))
+    with pytest.raises(SrError) as e:
+        G.bind_window(4)
+    assert e.value.status == "SR_ERR_UNSUPPORTED"

@@ -87,3 +87,29 @@ def test_pairs_with_ragged_batches_and_widths(batch):
              [Edge(0, 1, CONV, 3, 1), Edge(1, 1, CONV, 3, 1), Edge(1, 2, CONV, 3, 2), Edge(2, 2, CONV, 3, 1), Edge(2, 3, CONV, 3, 2),
               Edge(0, 3, CONV, 1, 4), Edge(3, 4, GAP_DENSE)], batch=batch, frames=3)
     run(g)
+
+
+@pytest.mark.parametrize("k", [0, 2, 6])
+def test_paper_cifar10_networks_on_tensor_cores(k):
+    # DSR0 / DSR2 / DSR6 (Sec. A, paragraph CIFAR10): receptive field 5 on the 3-channel input (75 columns, staged as two
+    # K-blocks), 32- and 64-channel blocks with dense skips, stride-4 edges into the 4 x 4 x 512 node (four channel
+    # tiles); every convolutional node runs on the tensor cores, only the dense output node does not
+    from paper_1806_04965_b200 import Graph
+    from workloads import graphs
+    g = graphs.dsr(k, batch=3, frames=4)
+    G = Graph(g.nodes, g.edges, g.patterns["streaming"], batch=g.batch, dtype="bf16")
+    assert G.info["n_direct_nodes"] == 1 and G.info["n_tensor_core_nodes"] == len(g.nodes) - 2, G.info
+    assert G.info["first_response_step"] == 4
+    S = Graph(g.nodes, g.edges, g.patterns["sequential"], batch=0)
+    assert S.info["first_response_step"] == 4 + k and S.info["inference_factor"] == 4 + k
+    for p in g.patterns:
+        parity.check_stepwise(g, p, zero_bias=False, tc_pair=1)
+        parity.check_stepwise(g, p, zero_bias=False, tc_pair=2)
+        parity.check_run(g, p, graph_frames=2)
+
+
+def test_gtsrb_network_variant():
+    # DSR4 without the H1 recurrence and with 43 classes (Sec. A, paragraph GTSRB)
+    from workloads import graphs
+    g = graphs.dsr(4, batch=2, frames=3, classes=43, h1_recurrence=False)
+    parity.check_stepwise(g, "streaming", zero_bias=False)

@@ -68,6 +68,7 @@ def test_compiler_matches_oracle_on_all_small_networks():
 def test_compiler_on_benchmark_graphs_and_paper_networks():
     specs = [graphs.build(c) for c in ("c1", "c2", "c3", "c4", "c5")] + [graphs.mnist_net(k) for k in ("FF", "S", "SR")]
     specs += [graphs.chain_with_shortcut(4 + k) for k in range(7)] + [graphs.worked_example()]
+    specs += [graphs.dsr(k) for k in range(7)] + [graphs.dsr(4, classes=43, h1_recurrence=False)]
     for g in specs:
         es = [(e.src, e.tgt) for e in g.edges]
         for name, R in g.patterns.items():
@@ -78,6 +79,12 @@ def test_compiler_on_benchmark_graphs_and_paper_networks():
                 rt.first_response(len(g.nodes), es, R, G.info["output_node"]), (g.name, name)
             if name == "streaming":
                 assert G.info["n_groups"] == 1
+    # the paper's CIFAR10 nets themselves (Sec. 4): streaming answers after 4 update steps whatever the depth, the
+    # sequential rollout after 4 + k; DSR2 has shortest path 4 and longest path 6
+    for k in range(7):
+        g = graphs.dsr(k)
+        assert Graph(g.nodes, g.edges, g.patterns["streaming"]).info["first_response_step"] == 4
+        assert Graph(g.nodes, g.edges, g.patterns["sequential"]).info["first_response_step"] == 4 + k
     sr = graphs.mnist_net("SR")
     assert Graph(sr.nodes, sr.edges, sr.patterns["sequential"]).info["inference_factor"] == 3   # paper Sec. 4
     assert Graph(sr.nodes, sr.edges, sr.patterns["streaming"]).info["inference_factor"] == 1
@@ -116,3 +123,34 @@ def test_theory_only_graph_refuses_device_calls():
     assert lib.sr_graph_workspace_bytes(G._h, ctypes.byref(n)) == 8            # SR_ERR_STATE
     assert lib.sr_rollout_step(G._h, None, None, None) == 8
     assert lib.sr_graph_info(None, None) == 1
+
+
+def test_window_tableau_matches_the_oracle_for_every_window_size():
+    # Eq. 4 for W = 1..4: the compiler's closed recursion against the oracle's iteration of the update step U on the
+    # explicit window, on every valid pattern of the small networks and on the named graphs
+    from tests.test_oracle_theory import NETS
+    checked = 0
+    cases = [(n, es, None) for (n, es) in NETS[:60]]
+    for g in [graphs.worked_example(), graphs.mnist_net("SR"), graphs.dsr(2), graphs.build("c3", batch=1, frames=1)]:
+        cases.append((len(g.nodes), [(e.src, e.tgt) for e in g.edges], g))
+    for n, es, g in cases:
+        patterns = list(g.patterns.values()) if g is not None else [R for R in rt.all_patterns(len(es)) if rt.is_valid(n, es, R)]
+        for R in patterns:
+            nodes, edges = (g.nodes, g.edges) if g is not None else dense_graph(n, es)
+            G = Graph(nodes, edges, R, batch=0)
+            for W in (1, 2, 3, 4):
+                want, _ = rt.tableau_by_updates(n, es, R, W)
+                got = G.window_tableau(W)
+                for i in range(W + 1):
+                    for v in range(n):
+                        assert got[i][v] == want[(i, v)], (es, R, W, i, v)
+                checked += 1
+    assert checked > 300
+    # frames of a recurrence-free network under the sequential rollout do not depend on each other: every frame has the
+    # tableau of frame 1, so a whole window is F(R) update steps (Sec. 4, the GTSRB comparison)
+    g = graphs.dsr(4, classes=43, h1_recurrence=False)
+    G = Graph(g.nodes, g.edges, g.patterns["sequential"], batch=0)
+    T = G.window_tableau(8)
+    assert all(T[i] == T[1] for i in range(1, 9)) and max(T[8]) == G.info["inference_factor"] == 8
+    S = Graph(g.nodes, g.edges, g.patterns["streaming"], batch=0)
+    assert max(S.window_tableau(8)[8]) == 8 and S.window_tableau(8)[3][len(g.nodes) - 1] == 3

@@ -216,7 +216,7 @@ def c3_six_node(batch: int = 256, frames: int = 20, size: int = 32, dtype: str =
     return g
 
 
-def c4_ten_node(batch: int = 128, frames: int = 64, size: int = 32, dtype: str = "bf16") -> GraphSpec:
+def c4_ten_node(batch: int = 128, frames: int = 64, size: int = 32, dtype: str = "bf16", recurrence: bool = True) -> GraphSpec:
     s = size
     chans = [64, 64, 128, 128, 128, 128, 256, 256, 256, 256]
     sizes = [s, s, s // 2, s // 2, s // 2, s // 2, s // 4, s // 4, s // 4, s // 4]
@@ -226,10 +226,11 @@ def c4_ten_node(batch: int = 128, frames: int = 64, size: int = 32, dtype: str =
     for i in range(10):                       # chain in -> n1 -> ... -> n10; n2->n3 and n6->n7 are pooling edges
         pooled = (i + 1) in (3, 7)
         edges.append(Edge(i, i + 1, CONV, 3, 1, 2 if pooled else 0))
-    edges += [Edge(i, i, CONV, 3, 1) for i in (2, 4, 6, 8)]
+    if recurrence:
+        edges += [Edge(i, i, CONV, 3, 1) for i in (2, 4, 6, 8)]
     edges += [Edge(2, 4, CONV, 3, 2), Edge(6, 8, CONV, 3, 2), Edge(2, 8, CONV, 3, 4)]
     edges += [Edge(10, 11, GAP_DENSE)]
-    g = GraphSpec("c4", nodes, edges, batch, frames, dtype, seed=1004)
+    g = GraphSpec("c4" if recurrence else "c4ff", nodes, edges, batch, frames, dtype, seed=1004)
     g.patterns = {"streaming": streaming_pattern(g), "sequential": sequential_pattern(g)}
     return g
 
@@ -289,6 +290,35 @@ def mini_cnn(batch: int = 3, frames: int = 5, dtype: str = "bf16") -> GraphSpec:
     return g
 
 
+def dsr(k: int, batch: int = 4, frames: int = 6, dtype: str = "bf16", classes: int = 10, h1_recurrence: bool = True) -> GraphSpec:
+    """The paper's CIFAR10 networks DSR0 .. DSR6 (Sec. A, paragraph CIFAR10): I 32x32x3; block 1 = H1, H11, H12, H13 at
+    32x32x32; block 2 = H2, H21, H22, H23 at 16x16x64; HD 4x4x512; O 10.  DSR0 is I - H1 - H2 - HD - O with a
+    self-recurrent H1; DSRk adds the first k of H11, H21, H12, H22, H13, H23.  Inside a block every earlier layer
+    feeds every later one, and every layer of a block feeds the head of the next (H2, HD): 3x3 convolutions whose stride
+    is input size / output size; I - H1 has receptive field 5.  The shortest input-output path has 4 edges, the longest
+    4 + k.  DSR4 with 43 classes and without the H1 recurrence is the paper's GTSRB network."""
+    assert 0 <= k <= 6
+    added = ["H11", "H21", "H12", "H22", "H13", "H23"][:k]
+    block1 = ["H1"] + [n for n in ("H11", "H12", "H13") if n in added]
+    block2 = ["H2"] + [n for n in ("H21", "H22", "H23") if n in added]
+    names = ["I"] + block1 + block2 + ["HD", "O"]
+    nodes = [Node("I", 32, 32, 3, IDENTITY)] + [Node(n, 32, 32, 32) for n in block1] + [Node(n, 16, 16, 64) for n in block2]
+    nodes += [Node("HD", 4, 4, 512), Node("O", 1, 1, classes, IDENTITY)]
+    ix = {n: i for i, n in enumerate(names)}
+    edges = [Edge(ix["I"], ix["H1"], CONV, 5, 1)]
+    for blk, head, stride in ((block1, "H2", 2), (block2, "HD", 4)):
+        for i, a in enumerate(blk):
+            for b in blk[i + 1:]:
+                edges.append(Edge(ix[a], ix[b], CONV, 3, 1))
+            edges.append(Edge(ix[a], ix[head], CONV, 3, stride))
+    edges.append(Edge(ix["HD"], ix["O"], DENSE))
+    if h1_recurrence:
+        edges.append(Edge(ix["H1"], ix["H1"], CONV, 3, 1))
+    g = GraphSpec("dsr%d" % k, nodes, edges, batch, frames, dtype, seed=1020 + k)
+    g.patterns = {"streaming": streaming_pattern(g), "sequential": sequential_pattern(g)}
+    return g
+
+
 def conv_sink(batch: int = 3, frames: int = 4, dtype: str = "bf16") -> GraphSpec:
     """A network whose output node is an image: in -> n1 (3x3) -> n2 (3x3, stride 2), recurrence on n1."""
     nodes = [Node("in", 8, 8, 3, IDENTITY), Node("n1", 8, 8, 16), Node("n2", 4, 4, 8, IDENTITY)]
@@ -298,7 +328,9 @@ def conv_sink(batch: int = 3, frames: int = 4, dtype: str = "bf16") -> GraphSpec
     return g
 
 
-BUILDERS = {"mini": mini_cnn, "sink": conv_sink, "c1": c1_mlp, "c2": c2_small_cnn, "c3": c3_six_node, "c4": c4_ten_node, "c5": c5_stress}
+BUILDERS = {"mini": mini_cnn, "sink": conv_sink, "dsr0": lambda **kw: dsr(0, **kw), "dsr2": lambda **kw: dsr(2, **kw),
+            "dsr4": lambda **kw: dsr(4, **kw), "dsr6": lambda **kw: dsr(6, **kw), "c1": c1_mlp, "c2": c2_small_cnn, "c3": c3_six_node, "c4": c4_ten_node, "c5": c5_stress,
+            "c4ff": lambda **kw: c4_ten_node(recurrence=False, **kw)}
 
 
 def build(name: str, **overrides) -> GraphSpec:
