@@ -423,6 +423,48 @@ def measure_workload(torch, args, name, rank, local, dist, pk, flush, steps, war
     return spec, w
 
 
+def measure_window(torch, args, flush, steps, warmup, W=8):
+    """c4 without its recurrent edges under the sequential rollout: T frames as chained windows of size 1
+    (sr_rollout_run) against windows of W frames evaluated at once (sr_rollout_window)."""
+    from paper_1806_04965_b200 import Graph
+    spec = graphs.build("c4ff")
+    X, Wt, Bi = data.make_inputs(spec), data.make_weights(spec), data.make_biases(spec)
+    dev = [torch.from_numpy(np.ascontiguousarray(X[v], dtype=np.float32)).to(torch.bfloat16).cuda().contiguous() for v in spec.input_nodes()]
+    G = Graph(spec.nodes, spec.edges, spec.patterns["sequential"], batch=spec.batch, dtype=spec.dtype, graph_frames=args.graph_frames)
+    G.set_weights(Wt, Bi)
+    G.bind_window(W)
+    T = spec.frames // W * W
+    out = torch.empty((T, spec.batch, spec.nodes[G.output_node].c), dtype=torch.float32, device="cuda")
+    stream = torch.cuda.current_stream()
+
+    def chained():
+        G.run([x[1:T + 1] for x in dev], out)
+
+    def windows():
+        for t in range(0, T, W):
+            G.rollout_window([x[t + 1:t + 1 + W] for x in dev], out[t:t + W])
+
+    res = {}
+    for name, fn in (("w1", chained), ("w%d" % W, windows)):
+        times = []
+        for i in range(warmup + steps):
+            G.reset([x[0] for x in dev])
+            flush.add_(1)
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record(stream)
+            fn()
+            b.record(stream)
+            b.synchronize()
+            if i >= warmup:
+                times.append(a.elapsed_time(b))
+        G.sync_status()
+        res[name] = float(np.mean(times)) * 1e3 / T
+    return {"graph": "c4 without recurrent edges", "pattern": "sequential", "batch": spec.batch, "frames": T, "W": W,
+            "levels_per_frame": G.info["n_groups"], "us_per_frame_w1": res["w1"], "us_per_frame_w%d" % W: res["w%d" % W],
+            "what": "w1 = sr_rollout_run (chained windows of size 1, one launch group per level and frame); "
+                    "w%d = sr_rollout_window (one launch group per level for %d frames at once)" % (W, W)}
+
+
 def run_cuda(args):
     import torch
     rank = int(os.environ.get("RANK", "0"))
@@ -460,6 +502,8 @@ def run_cuda(args):
         main_copy = {k: v for k, v in main.items() if k not in ("e2e_ms_per_step", "h2d_bytes_per_step", "d2h_bytes_per_step")}
         others[spec.name] = main_copy
         line["workloads"] = {k: others[k] for k in sorted(others)}
+        if "c4" in line["workloads"]:
+            line["workloads"]["c4"]["deep_window"] = measure_window(torch, args, flush, max(3, min(args.steps, 10)), 3)
     if rank == 0:
         if world == 1 and not args.no_cpu_baseline:
             cb = time_oracle(spec, args.pattern)

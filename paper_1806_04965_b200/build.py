@@ -8,7 +8,7 @@ import sys
 HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libsr_rollout.so")
-SOURCES = ["sr_compile.cpp", "sr_api.cu", "sr_direct.cu", "sr_tc.cu", "sr_resident.cu"]
+SOURCES = ["sr_compile.cpp", "sr_api.cu", "sr_direct.cu", "sr_tc.cu", "sr_resident.cu", "sr_dense.cu"]
 NVCC_FLAGS = ["-O3", "-std=c++17", "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo",
               "-Xcompiler", "-fPIC", "-cudart", "static"]
 

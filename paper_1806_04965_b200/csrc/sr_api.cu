@@ -11,6 +11,7 @@
 
 #include "sr_internal.h"
 #include "sr_kernels.h"
+#include "sr_dense.h"
 #include "sr_resident.h"
 #include "sr_tc.h"
 
@@ -176,6 +177,8 @@ sr_status plan(sr_graph* g)
     if (st != SR_OK) return st;
     st = sr_rs_plan(g, off);
     if (st != SR_OK) return st;
+    st = sr_dn_plan(g, off);
+    if (st != SR_OK) return st;
     g->ws_bytes = off;
     int n_tc = 0, n_direct = 0;
     for (const SrHostNode& n : g->nodes)
@@ -184,6 +187,10 @@ sr_status plan(sr_graph* g)
     g->info.n_direct_nodes = n_direct;
     int rs_warps = 0;
     sr_rs_describe(g, &g->info.resident_cluster, &rs_warps, &g->info.resident_smem_bytes, &g->info.resident_heads_on_chip);
+    if (sr_dn_available(g)) {
+        sr_dn_describe(g, &g->info.resident_cluster, &g->info.resident_smem_bytes);
+        g->info.resident_heads_on_chip = 1;
+    }
     return SR_OK;
 }
 
@@ -323,6 +330,7 @@ void sr_graph_destroy(sr_graph* g)
     }
     sr_tc_destroy(g);
     sr_rs_destroy(g);
+    sr_dn_destroy(g);
     delete g;
 }
 
@@ -490,6 +498,7 @@ sr_status sr_graph_bind_workspace(sr_graph* g, void* workspace_dev, size_t bytes
     g->ws = ws;
     st = sr_tc_bind(g);
     if (st == SR_OK) st = sr_rs_bind(g);
+    if (st == SR_OK) st = sr_dn_bind(g);
     if (st != SR_OK) {
         g->ws = nullptr;
         return st;
@@ -577,7 +586,8 @@ sr_status sr_graph_set_edge_weights(sr_graph* g, int edge, const float* w, int i
         if (st != SR_OK) return st;
     }
     {
-        const sr_status st = sr_rs_set_weights(g, edge, eff.data());
+        sr_status st = sr_rs_set_weights(g, edge, eff.data());
+        if (st == SR_OK) st = sr_dn_set_weights(g, edge, eff.data());
         if (st != SR_OK) return st;
     }
     he.w_set = true;
@@ -660,6 +670,18 @@ sr_status sr_rollout_run(sr_graph* g, const void* const* in_seq_dev, int T, floa
             g->launches += 1;
             g->t += T;
             g->stage_dirty = true;             // refreshed when the launch path is used next
+            return cuda_ok(cudaGetLastError()) ? SR_OK : SR_ERR_CUDA;
+        }
+    }
+    if (sr_dn_available(g)) {
+        bool aligned = true;                                     // the dense resident kernel fetches input frames in 16-byte words
+        for (size_t i = 0; i < g->input_nodes.size(); ++i)
+            if (reinterpret_cast<uintptr_t>(in_seq_dev[i]) & 15) aligned = false;
+        if (aligned) {
+            st = sr_dn_launch(g, T, make_ctl(g, in_seq_dev, true, out_seq_dev), s);
+            if (st != SR_OK) return st;
+            g->launches += 1;
+            g->t += T;
             return cuda_ok(cudaGetLastError()) ? SR_OK : SR_ERR_CUDA;
         }
     }
@@ -881,8 +903,11 @@ sr_status sr_graph_kernel_time(sr_graph* g, double* ms, int64_t* launches)
     double ms_rs = 0.0;
     sr_status st = sr_tc_timing(g, ms, &n);
     if (st == SR_OK) st = sr_rs_timing(g, &ms_rs, &n_rs);
-    *ms += ms_rs;
-    *launches = n + n_rs;
+    double ms_dn = 0.0;
+    long long n_dn = 0;
+    if (st == SR_OK) st = sr_dn_timing(g, &ms_dn, &n_dn);
+    *ms += ms_rs + ms_dn;
+    *launches = n + n_rs + n_dn;
     return st;
 }
 

@@ -101,6 +101,8 @@ struct sr_graph {
     int64_t launches = 0;
     void* tc = nullptr;                            // tensor-core engine state (opaque here)
     void* rs = nullptr;                            // resident engine state (opaque here)
+    void* dn = nullptr;                            // dense resident engine state (opaque here)
+    std::vector<unsigned char> dn_headers;         // its per-rank table images, uploaded when a workspace is bound
     void* graphs = nullptr;                        // CUDA-graph cache (opaque here)
     void* side = nullptr;                          // side stream and fork / join events (opaque here)
     bool input_feeds_same_frame = false;           // some edge that leaves an input node has R = 0
