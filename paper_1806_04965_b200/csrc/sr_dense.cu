@@ -7,12 +7,13 @@
 //   - every CTA holds a full copy of every node state of its eight sequences (two buffers by frame parity; input
 //     nodes three, because the next input frame is fetched with cp.async while the current update still reads the
 //     previous one);
-//   - a job is eight output rows of one node on one CTA; the warps of a CTA are shared out among the jobs of a tableau
-//     level in proportion to their work.  The warps of a job split its reduction index into chunks of 128: a lane takes
-//     four consecutive indices, loads the state values of all eight sequences (16-byte loads, every byte of a
-//     shared-memory access is used) and runs over the eight rows; shuffles sum over the lanes, shared memory sums over
-//     the warps in a fixed order, and the results (bias, ReLU) are written into the state copies of ALL eight CTAs
-//     through distributed shared memory;
+//   - a work unit is two output rows of one node; a warp takes a unit, its lanes stride over the reduction index with
+//     16-byte loads (one weight vector per row, one state vector per sequence), shuffles sum the lanes (halving the
+//     number of values per step), and the results (bias, ReLU) are written into the state copies of ALL eight CTAs
+//     through distributed shared memory; warps never wait for each other inside a level.  (Measured alternatives:
+//     eight-row jobs whose reduction index is split over warps, with partial sums through shared memory, need two
+//     block-wide barriers per level and came out slower, 5.2 / 10.3 us per frame against 4.6 / 6.4 for the streaming /
+//     sequential rollout of the 784-128-128-10 network.)
 //   - a tableau level (Eq. 4) ends at a cluster barrier; a streaming frame has one.
 // The sums run in a fixed order, so results are reproducible bit for bit.  There is no spin-wait: the only
 // synchronisation is the hardware cluster barrier, reached by every thread the same number of times.
@@ -26,8 +27,7 @@
 
 namespace {
 
-constexpr int kDnMaxNodes = 16, kDnMaxEdges = 32, kDnMaxLevels = 16, kDnMaxJobs = 48, kDnMaxRounds = 32;
-constexpr int kDnRows = 8;             // output rows a job covers (a rank's weight slices are padded with zero rows to a multiple)
+constexpr int kDnMaxNodes = 16, kDnMaxEdges = 32, kDnMaxLevels = 16, kDnMaxUnits = 64;
 constexpr int kDnCluster = 8;          // CTAs per cluster
 constexpr int kDnSamples = 8;          // sequences per cluster
 constexpr int kDnWarps = 16;
@@ -44,22 +44,20 @@ struct DnNode {
 
 struct DnEdge { int32_t src, tgt, R, Kpad; };
 
-// A job: up to kDnRows consecutive rows of one node on one rank, computed by warps [warp0, warp0 + n_warps).
-struct DnJob { int32_t node, row0, nrows, rel_row, warp0, n_warps, pad_[2]; };   // rel_row: row0 relative to the rank's first row
+struct DnUnit { int32_t node, row0, nrows, rel_row; };      // two rows of a node; rel_row: row0 relative to the rank's first row
 
 struct DnBlobHdr {                     // head of a rank's blob; the rank's weight slices follow
-    int32_t n_jobs, pad_[3];
-    int32_t level_round[kDnMaxLevels + 1];                   // rounds of level l: [level_round[l-1], level_round[l])
-    int32_t round_job[kDnMaxRounds + 1];                     // jobs of round k: [round_job[k], round_job[k+1]); their warps partition the CTA
-    int32_t pad2_[2];
+    int32_t n_units, pad_[3];
+    int32_t level_begin[kDnMaxLevels + 1];                   // units of level l: [level_begin[l-1], level_begin[l])
+    int32_t pad2_[3];
     int32_t w_off[kDnMaxEdges];                              // float offset of the rank's slice of every edge's weights
-    DnJob jobs[kDnMaxJobs];
+    DnUnit units[kDnMaxUnits];
 };
 static_assert(sizeof(DnBlobHdr) % 16 == 0, "the weights that follow are read with 16-byte loads");
 
 struct DnParams {
     int32_t n_nodes, n_edges, n_levels, B;
-    int32_t blob_bytes, hdr_floats, total_floats, part_off;  // part_off: float offset of the partial sums [warp][row][sequence]
+    int32_t blob_bytes, hdr_floats, total_floats, pad_;
     const unsigned char* blobs;        // kDnCluster blobs of blob_bytes each
     DnNode nodes[kDnMaxNodes];
     DnEdge edges[kDnMaxEdges];
@@ -73,12 +71,6 @@ __device__ __forceinline__ void dn_cp_async16(void* dst, const void* src)
 __device__ __forceinline__ void dn_cluster_sync()
 {
     asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
-}
-__device__ __forceinline__ void dn_st_cluster4(const float* local, uint32_t rank, float4 v)
-{
-    uint32_t remote;
-    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(remote) : "r"((uint32_t)__cvta_generic_to_shared(local)), "r"(rank));
-    asm volatile("st.shared::cluster.v4.f32 [%0], {%1, %2, %3, %4};" ::"r"(remote), "f"(v.x), "f"(v.y), "f"(v.z), "f"(v.w) : "memory");
 }
 __device__ __forceinline__ void dn_st_cluster(const float* local, uint32_t rank, float v)
 {
@@ -145,113 +137,76 @@ sr_dense_kernel(const DnParams P, SrFrameCtl* __restrict__ ctl_out, const SrFram
         __syncthreads();
         if (f + 1 < T) fetch_inputs(f + 2);
         for (int l = 1; l <= P.n_levels; ++l) {
-            for (int rd = H->level_round[l - 1]; rd < H->level_round[l]; ++rd) {
-                // my job in this round (none if the round leaves this warp idle)
-                int ji = -1;
-                for (int j = H->round_job[rd]; j < H->round_job[rd + 1]; ++j)
-                    if (warp >= H->jobs[j].warp0 && warp < H->jobs[j].warp0 + H->jobs[j].n_warps) ji = j;
-                float* part = dn_smem + P.part_off + warp * (kDnRows * kDnSamples);
-                if (ji >= 0) {
-                    const DnJob jb = H->jobs[ji];
-                    float acc[kDnRows * kDnSamples];                               // [row][sequence]
+            for (int u = H->level_begin[l - 1] + warp; u < H->level_begin[l]; u += kDnWarps) {
+                const DnUnit un = H->units[u];
+                const DnNode& nd = P.nodes[un.node];
+                float acc0[kDnSamples], acc1[kDnSamples];
 #pragma unroll
-                    for (int i = 0; i < kDnRows * kDnSamples; ++i) acc[i] = 0.f;
-                    int first = warp - jb.warp0;                                   // chunks of 128 are dealt out round robin over the job's warps
-                    for (int e = P.first_edge[jb.node]; e < P.first_edge[jb.node + 1]; ++e) {
-                        const DnEdge ed = P.edges[e];
-                        const DnNode& sn = P.nodes[ed.src];
-                        const int sf = f + 1 - ed.R;                               // Eq. 2: the source frame
-                        const float* xs = dn_smem + (sn.is_input ? sn.buf[sf % 3] : sn.buf[sf & 1]) + 4 * lane;
-                        const float* wr = wsm + H->w_off[e] + (size_t)jb.rel_row * ed.Kpad + 4 * lane;
-                        const int n_chunks = (ed.Kpad + 127) >> 7;
-                        int ch = first;
-                        first += ((n_chunks - first + jb.n_warps - 1) / jb.n_warps) * jb.n_warps - n_chunks;   // first chunk of the next edge
-                        for (; ch < n_chunks; ch += jb.n_warps) {
-                            const int k0 = ch << 7;
-                            if (k0 + 4 * lane >= ed.Kpad) continue;                // ragged last chunk
-                            float4 x[kDnSamples];
+                for (int b = 0; b < kDnSamples; ++b) acc0[b] = acc1[b] = 0.f;
+                for (int e = P.first_edge[un.node]; e < P.first_edge[un.node + 1]; ++e) {
+                    const DnEdge ed = P.edges[e];
+                    const DnNode& sn = P.nodes[ed.src];
+                    const int sf = f + 1 - ed.R;                                  // Eq. 2: the source frame
+                    const float* xs = dn_smem + (sn.is_input ? sn.buf[sf % 3] : sn.buf[sf & 1]);
+                    const float* w0 = wsm + H->w_off[e] + (size_t)un.rel_row * ed.Kpad;
+                    const float* w1 = un.nrows > 1 ? w0 + ed.Kpad : w0;
+                    for (int k = lane * 4; k < ed.Kpad; k += 128) {
+                        const float4 a = *reinterpret_cast<const float4*>(w0 + k);
+                        const float4 c = *reinterpret_cast<const float4*>(w1 + k);
 #pragma unroll
-                            for (int b = 0; b < kDnSamples; ++b) x[b] = *reinterpret_cast<const float4*>(xs + b * sn.Cpad + k0);
-#pragma unroll
-                            for (int r = 0; r < kDnRows; ++r) {                    // rows past the job's last are zero rows of the slice
-                                const float4 w = *reinterpret_cast<const float4*>(wr + (size_t)r * ed.Kpad + k0);
-#pragma unroll
-                                for (int b = 0; b < kDnSamples; ++b)
-                                    acc[r * kDnSamples + b] = fmaf(w.w, x[b].w, fmaf(w.z, x[b].z, fmaf(w.y, x[b].y, fmaf(w.x, x[b].x, acc[r * kDnSamples + b]))));
-                            }
+                        for (int b = 0; b < kDnSamples; ++b) {
+                            const float4 x = *reinterpret_cast<const float4*>(xs + b * sn.Cpad + k);
+                            acc0[b] = fmaf(a.w, x.w, fmaf(a.z, x.z, fmaf(a.y, x.y, fmaf(a.x, x.x, acc0[b]))));
+                            acc1[b] = fmaf(c.w, x.w, fmaf(c.z, x.z, fmaf(c.y, x.y, fmaf(c.x, x.x, acc1[b]))));
                         }
                     }
-                    // Sum over the 32 lanes by halving: in the step with distance d a lane keeps the half of its values that
-                    // matches its bit d and adds the partner's; 64 values become 32, 16, 8, 4, 2: lane L ends with
-                    // values 2L, 2L + 1, i.e. row L >> 2, sequences 2 (L & 3) and 2 (L & 3) + 1.
-                    float v32[32], v16[16], v8[8], v4[4], v2[2];
-                    {
-                        const bool up = (lane & 16) != 0;
-#pragma unroll
-                        for (int j = 0; j < 32; ++j) v32[j] = (up ? acc[j + 32] : acc[j]) + __shfl_xor_sync(0xffffffffu, up ? acc[j] : acc[j + 32], 16);
-                    }
-                    {
-                        const bool up = (lane & 8) != 0;
-#pragma unroll
-                        for (int j = 0; j < 16; ++j) v16[j] = (up ? v32[j + 16] : v32[j]) + __shfl_xor_sync(0xffffffffu, up ? v32[j] : v32[j + 16], 8);
-                    }
-                    {
-                        const bool up = (lane & 4) != 0;
-#pragma unroll
-                        for (int j = 0; j < 8; ++j) v8[j] = (up ? v16[j + 8] : v16[j]) + __shfl_xor_sync(0xffffffffu, up ? v16[j] : v16[j + 8], 4);
-                    }
-                    {
-                        const bool up = (lane & 2) != 0;
-#pragma unroll
-                        for (int j = 0; j < 4; ++j) v4[j] = (up ? v8[j + 4] : v8[j]) + __shfl_xor_sync(0xffffffffu, up ? v8[j] : v8[j + 4], 2);
-                    }
-                    {
-                        const bool up = (lane & 1) != 0;
-#pragma unroll
-                        for (int j = 0; j < 2; ++j) v2[j] = (up ? v4[j + 2] : v4[j]) + __shfl_xor_sync(0xffffffffu, up ? v4[j] : v4[j + 2], 1);
-                    }
-                    part[2 * lane] = v2[0];
-                    part[2 * lane + 1] = v2[1];
                 }
-                __syncthreads();
-                if (ji >= 0) {
-                    const DnJob jb = H->jobs[ji];
-                    const DnNode& nd = P.nodes[jb.node];
-                    const float* p0 = dn_smem + P.part_off + jb.warp0 * (kDnRows * kDnSamples);
-                    // Remote stores are the scarce resource here (every value goes to eight CTAs), so four consecutive rows
-                    // of a sequence travel as one 16-byte store where the rows are aligned that way.
-                    if (((jb.row0 | jb.nrows) & 3) == 0) {
-                        for (int o = (warp - jb.warp0) * 32 + lane; o < (jb.nrows >> 2) * kDnSamples; o += jb.n_warps * 32) {
-                            const int rg = o >> 3, b = o & 7, row = jb.row0 + 4 * rg;
-                            float z[4];
+                // Sum over the lanes by halving: in the step with distance d a lane keeps the half of its values that
+                // matches its bit d and adds the partner's; after distances 16, 8, 4, 2 lane L holds value L >> 1
+                // (row (L >> 4), sequence (L >> 1) & 7), and the step with distance 1 completes it in both lanes of a pair.
+                float v8[8], v4[4], v2[2], v1;
+                {
+                    const bool up = (lane & 16) != 0;
 #pragma unroll
-                            for (int i = 0; i < 4; ++i) {
-                                z[i] = dn_smem[nd.bias_off + row + i];
-                                for (int w = 0; w < jb.n_warps; ++w) z[i] += p0[w * (kDnRows * kDnSamples) + (4 * rg + i) * kDnSamples + b];   // fixed order
-                                if (nd.act == 1) z[i] = fmaxf(z[i], 0.f);
-                            }
-                            const float* cell = dn_smem + nd.buf[(f + 1) & 1] + b * nd.Cpad + row;
-                            const float4 zv = make_float4(z[0], z[1], z[2], z[3]);
-#pragma unroll
-                            for (uint32_t k = 0; k < (uint32_t)kDnCluster; ++k) dn_st_cluster4(cell, k, zv);
-                            if (nd.is_output && init.out_base && b < nb)
-                                for (int i = 0; i < 4; ++i)
-                                    init.out_base[(run0 + f) * init.out_stride + (long long)(b0 + b) * nd.C + row + i] = z[i];
-                        }
-                    } else
-                    for (int o = (warp - jb.warp0) * 32 + lane; o < jb.nrows * kDnSamples; o += jb.n_warps * 32) {
-                        const int r = o >> 3, b = o & 7, row = jb.row0 + r;
-                        float z = dn_smem[nd.bias_off + row];
-                        for (int w = 0; w < jb.n_warps; ++w) z += p0[w * (kDnRows * kDnSamples) + o];      // fixed order
-                        if (nd.act == 1) z = fmaxf(z, 0.f);
-                        const float* cell = dn_smem + nd.buf[(f + 1) & 1] + b * nd.Cpad + row;
-#pragma unroll
-                        for (uint32_t k = 0; k < (uint32_t)kDnCluster; ++k) dn_st_cluster(cell, k, z);
-                        if (nd.is_output && init.out_base && b < nb)
-                            init.out_base[(run0 + f) * init.out_stride + (long long)(b0 + b) * nd.C + row] = z;
+                    for (int j = 0; j < 8; ++j) {
+                        const float keep = up ? acc1[j] : acc0[j], send = up ? acc0[j] : acc1[j];
+                        v8[j] = keep + __shfl_xor_sync(0xffffffffu, send, 16);
                     }
                 }
-                __syncthreads();                                 // the partial sums may be overwritten
+                {
+                    const bool up = (lane & 8) != 0;
+#pragma unroll
+                    for (int j = 0; j < 4; ++j) {
+                        const float keep = up ? v8[j + 4] : v8[j], send = up ? v8[j] : v8[j + 4];
+                        v4[j] = keep + __shfl_xor_sync(0xffffffffu, send, 8);
+                    }
+                }
+                {
+                    const bool up = (lane & 4) != 0;
+#pragma unroll
+                    for (int j = 0; j < 2; ++j) {
+                        const float keep = up ? v4[j + 2] : v4[j], send = up ? v4[j] : v4[j + 2];
+                        v2[j] = keep + __shfl_xor_sync(0xffffffffu, send, 4);
+                    }
+                }
+                {
+                    const bool up = (lane & 2) != 0;
+                    const float keep = up ? v2[1] : v2[0], send = up ? v2[0] : v2[1];
+                    v1 = keep + __shfl_xor_sync(0xffffffffu, send, 2);
+                }
+                v1 += __shfl_xor_sync(0xffffffffu, v1, 1);
+                const int r = lane >> 4, b = (lane >> 1) & 7;
+                if (r < un.nrows) {
+                    const int row = un.row0 + r;
+                    float z = v1 + dn_smem[nd.bias_off + row];
+                    if (nd.act == 1) z = fmaxf(z, 0.f);
+                    const float* cell = dn_smem + nd.buf[(f + 1) & 1] + b * nd.Cpad + row;
+                    const uint32_t q = (uint32_t)(lane & 1) * 4u;              // the two lanes of a pair serve four ranks each
+#pragma unroll
+                    for (uint32_t k = 0; k < 4; ++k) dn_st_cluster(cell, q + k, z);
+                    if (nd.is_output && init.out_base && (lane & 1) == 0 && b < nb)
+                        init.out_base[(run0 + f) * init.out_stride + (long long)(b0 + b) * nd.C + row] = z;
+                }
             }
             dn_cluster_sync();                               // the level is complete in every CTA's copy
         }
@@ -347,8 +302,7 @@ sr_status sr_dn_plan(sr_graph* g, size_t& offset)
         }
     }
     P.first_edge[n_nodes] = pos;
-    // row slices and weight offsets per rank; jobs (row blocks of a node) grouped into rounds, the warps of a round shared
-    // out in proportion to the jobs' work (rows x reduction length)
+    // row slices and weight offsets per rank; units (two rows of a node each, longest reduction first inside a level)
     E->row_lo.assign((size_t)n_nodes * (kDnCluster + 1), 0);
     E->w_off.assign(kDnCluster, std::vector<int>(kDnMaxEdges, 0));
     int max_w = 0;
@@ -364,56 +318,28 @@ sr_status sr_dn_plan(sr_graph* g, size_t& offset)
             const int rows = E->row_lo[(size_t)v * (kDnCluster + 1) + r + 1] - E->row_lo[(size_t)v * (kDnCluster + 1) + r];
             E->w_off[r][e] = w;
             h.w_off[e] = w;
-            w += (rows + kDnRows - 1) / kDnRows * kDnRows * P.edges[e].Kpad;       // zero rows up to a whole job
+            w += rows * P.edges[e].Kpad;
         }
         max_w = std::max(max_w, w);
-        int n_jobs = 0, n_rounds = 0;
+        int n_units = 0;
         bool fits = true;
         for (int l = 1; l <= P.n_levels && fits; ++l) {
-            std::vector<std::pair<long long, DnJob>> lv;
+            std::vector<std::pair<long long, DnUnit>> lv;
             for (int v : g->groups[l - 1]) {
                 long long K = 0;
                 for (int e = P.first_edge[v]; e < P.first_edge[v + 1]; ++e) K += P.edges[e].Kpad;
                 const int lo = E->row_lo[(size_t)v * (kDnCluster + 1) + r], hi = E->row_lo[(size_t)v * (kDnCluster + 1) + r + 1];
-                for (int row = lo; row < hi; row += kDnRows) {
-                    const int nr = std::min(kDnRows, hi - row);
-                    lv.push_back({K * nr, DnJob{v, row, nr, row - lo, 0, 0, {0, 0}}});
-                }
+                for (int row = lo; row < hi; row += 2) lv.push_back({K, DnUnit{v, row, std::min(2, hi - row), row - lo}});
             }
             std::stable_sort(lv.begin(), lv.end(), [](const auto& a, const auto& b) { return a.first > b.first; });
-            for (size_t i0 = 0; i0 < lv.size() && fits; i0 += kDnWarps) {
-                const size_t i1 = std::min(lv.size(), i0 + kDnWarps);
-                if (n_rounds >= kDnMaxRounds || n_jobs + (int)(i1 - i0) > kDnMaxJobs) { fits = false; break; }
-                long long total = 0;
-                for (size_t i = i0; i < i1; ++i) total += std::max<long long>(1, lv[i].first);
-                std::vector<int> share(i1 - i0, 1);
-                int left = kDnWarps - (int)(i1 - i0);
-                while (left > 0) {                                   // next warp to the job with the most work per warp
-                    size_t best = 0;
-                    double most = -1.0;
-                    for (size_t i = i0; i < i1; ++i) {
-                        const double per = (double)std::max<long long>(1, lv[i].first) / share[i - i0];
-                        if (per > most) { most = per; best = i - i0; }
-                    }
-                    share[best]++;
-                    --left;
-                }
-                h.round_job[n_rounds] = n_jobs;
-                int w0 = 0;
-                for (size_t i = i0; i < i1; ++i) {
-                    DnJob jb = lv[i].second;
-                    jb.warp0 = w0;
-                    jb.n_warps = share[i - i0];
-                    w0 += jb.n_warps;
-                    h.jobs[n_jobs++] = jb;
-                }
-                ++n_rounds;
-                h.round_job[n_rounds] = n_jobs;
+            for (auto& u : lv) {
+                if (n_units >= kDnMaxUnits) { fits = false; break; }
+                h.units[n_units++] = u.second;
             }
-            h.level_round[l] = n_rounds;
+            h.level_begin[l] = n_units;
         }
-        for (int l = P.n_levels + 1; l <= kDnMaxLevels; ++l) h.level_round[l] = n_rounds;
-        h.n_jobs = n_jobs;
+        for (int l = P.n_levels + 1; l <= kDnMaxLevels; ++l) h.level_begin[l] = n_units;
+        h.n_units = n_units;
         if (!fits) {
             delete E;
             return SR_OK;
@@ -440,8 +366,6 @@ sr_status sr_dn_plan(sr_graph* g, size_t& offset)
         d.bias_off = off;
         if (!n.is_input) off += d.Cpad;
     }
-    P.part_off = off;
-    off += kDnWarps * kDnRows * kDnSamples;
     P.total_floats = off;
     E->smem_bytes = off * 4;
     if (E->smem_bytes > kDnSmemMax) {
