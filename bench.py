@@ -41,6 +41,10 @@ ALL_WORKLOADS = ("c1", "c2", "c3", "c4", "c5")
 # the kernel source it was taken from; the number is reported only while that source is unchanged, else null.
 TRAFFIC = {
     # workload: (bytes per launch, kernel source file, sha256[:12] of that file at capture time, summary under profiles/)
+    "c5": (613.7e6, "sr_tc.cu", "96e6f12e8b16", "profiles/sr_tc_group_kernel_counters.md"),
+    "c3": (263.6e6, "sr_tc.cu", "96e6f12e8b16", "profiles/sr_tc_group_kernel_counters.md"),
+    "c4": (158.7e6, "sr_tc.cu", "96e6f12e8b16", "profiles/sr_tc_group_kernel_counters.md"),
+    "c2": (8.0e6, "sr_resident.cu", "89436108f1ff", "profiles/sr_resident_kernel_c2.md"),     # one launch = all 32 frames
 }
 
 
@@ -359,13 +363,21 @@ def measure_workload(torch, args, name, rank, local, dist, pk, flush, steps, war
         # classification this workload has on a per-frame launch path, not the bound of this kernel (which is the
         # shared-memory pipe; see profiles/).
         ach = by * T / (kernel_us * 1e-6) / 1e9
+        dense = spec.dtype != "bf16"
         roof = {"bound": "hbm", "achieved": ach, "peak": pk["hbm_gbs"], "unit": "GB/s", "frac": ach / pk["hbm_gbs"],
                 "frac_is": "algorithmic bytes / time over measured copy bandwidth; the states never leave the SM, so HBM does not bound this kernel",
-                "kernel": "sr_resident_kernel, mean of %d event-timed launches (%.1f us each = %.2f us per frame, %d frames per launch, "
-                          "%d CTAs per sequence)" % (kernel_n, kernel_us, kernel_us / T, T, res["resident_cluster"]),
-                "tensor": {"achieved_tflops": fl * T / (kernel_us * 1e-6) / 1e12,
-                           "frac_of_burst_peak": fl * T / (kernel_us * 1e-6) / 1e12 / pk["bf16_tflops"],
-                           "note": "mma.sync path; states and weights resident in shared memory"}}
+                "kernel": "%s, mean of %d event-timed launches (%.1f us each = %.2f us per frame, %d frames per launch, %s)"
+                          % ("sr_dense_kernel" if dense else "sr_resident_kernel", kernel_n, kernel_us, kernel_us / T, T,
+                             "one cluster of %d CTAs per 8 sequences" % res["resident_cluster"] if dense
+                             else "%d CTAs per sequence" % res["resident_cluster"])}
+        if dense:
+            roof["alu"] = {"achieved_gflops": fl * T / (kernel_us * 1e-6) / 1e9,
+                           "note": "fp32 FMA on CUDA cores; weights and states resident in the shared memory of a cluster; bound by "
+                                   "cluster-barrier and launch latency"}
+        else:
+            roof["tensor"] = {"achieved_tflops": fl * T / (kernel_us * 1e-6) / 1e12,
+                              "frac_of_burst_peak": fl * T / (kernel_us * 1e-6) / 1e12 / pk["bf16_tflops"],
+                              "note": "mma.sync path; states and weights resident in shared memory"}
     elif tensor_bound:
         if kernel_us:
             ach = cfl / groups / (kernel_us * 1e-6) / 1e12     # average over the group launches of a frame
