@@ -10,6 +10,9 @@ from workloads.graphs import DENSE, GAP_DENSE, IDENTITY, RELU, Edge, GraphSpec, 
 
 pytestmark = pytest.mark.gpu
 
+# CTAs per cluster: sixteen when a frame is one tableau level (streaming), eight otherwise
+CLUSTER = {"streaming": 16, "sequential": 8, "hybrid": 8}
+
 
 def mlp(batch, frames, sizes=(36, 20, 10, 7), seed=31):
     """input -> h1 -> h2 -> out with a skip input -> out, a self-loop on h2 and a back-edge h2 -> h1."""
@@ -24,8 +27,9 @@ def mlp(batch, frames, sizes=(36, 20, 10, 7), seed=31):
 @pytest.mark.parametrize("pattern", ["streaming", "sequential"])
 def test_c1_runs_on_the_dense_resident_engine(pattern):
     g = graphs.build("c1")
-    parity.check_run(g, pattern, expect_resident=8)
-    parity.check_run(g, pattern, frames=1, expect_resident=8)
+    cluster = CLUSTER[pattern]
+    parity.check_run(g, pattern, expect_resident=cluster)
+    parity.check_run(g, pattern, frames=1, expect_resident=cluster)
     parity.check_run(g, pattern, resident=False, expect_resident=0)
 
 
@@ -34,7 +38,7 @@ def test_odd_sizes_and_batches(batch):
     # channel counts that are no multiple of four (padded columns), more sequences than one cluster holds, a ragged last cluster
     g = mlp(batch, 7)
     for p in g.patterns:
-        parity.check_run(g, p, expect_resident=8)
+        parity.check_run(g, p, expect_resident=CLUSTER[p])
 
 
 def test_runs_and_steps_continue_each_other():
@@ -44,7 +48,7 @@ def test_runs_and_steps_continue_each_other():
     X, W, Bi = data.make_inputs(g), data.make_weights(g), data.make_biases(g, zero=False)
     want = fu.rollout_spec(g, "streaming", X, W, Bi)
     G = parity.make_graph(g, "streaming", "auto", 0, W, Bi)
-    assert G.info["resident_cluster"] == 8
+    assert G.info["resident_cluster"] == CLUSTER["streaming"]
     x = parity.to_device(g, X[0])
     G.reset([x[0]])
     out = torch.empty((4, 5, 7), dtype=torch.float32, device="cuda:0")
