@@ -2,8 +2,8 @@
 // whose edges are all dense, in fp32, for all T frames of a run in ONE launch.
 //
 // Such a network (the paper's H2 / O layers, a tiny MLP) moves a few hundred kilobytes of weights per frame and does a
-// million multiply-adds: launched frame by frame it is pure launch latency.  Here a cluster of eight CTAs keeps ALL
-// weights in shared memory, split by output rows, and walks the frames of eight sequences by itself:
+// million multiply-adds: launched frame by frame it is pure launch latency.  Here a cluster of eight or sixteen CTAs
+// keeps ALL weights in shared memory, split by output rows, and walks the frames of eight sequences by itself:
 //   - every CTA holds a full copy of every node state of its eight sequences (two buffers by frame parity; input
 //     nodes three, because the next input frame is fetched with cp.async while the current update still reads the
 //     previous one);
@@ -12,9 +12,11 @@
 //     multiply-adds; what bounds a frame is the shared-memory bandwidth, and two-row units needed 10 loads per 64),
 //     shuffles sum the lanes (halving the number of values per step until a group of four lanes holds the four
 //     rows of one sequence), and the results (bias, ReLU) are written as one 16-byte word into the state copies of
-//     ALL eight CTAs through distributed shared memory; warps never wait for each other inside a level.  (Measured
-//     alternative: eight-row jobs whose reduction index is split over warps, with partial sums through shared memory,
-//     need two block-wide barriers per level and came out slower.)
+//     ALL CTAs of the cluster through distributed shared memory; warps never wait for each other inside a level.
+//     (Measured alternatives, both slower: eight-row jobs whose reduction index is split over warps with two
+//     block-wide barriers per level; four-row units cut along the reduction index into parts on up to fourteen warps
+//     that hand their partial sums to the unit's first part through shared memory and a named barrier, 3.1 against
+//     2.8 us per frame: the shared-memory traffic stays the same and every part pays the reduction over the lanes.)
 //   - units are given to the warps longest first (host side); the warps left without a unit in the first level fetch
 //     the next input frame;
 //   - a tableau level (Eq. 4) ends at a cluster barrier; a streaming frame has one.
