@@ -190,10 +190,14 @@ sr_status sr_graph_set_node_bias(sr_graph* g, int node, const float* bias_host);
  *                  reports SR_ERR_TIMEOUT.  0 is a test hook: every tensor-core launch reports the error at once and
  *                  returns before it touches a barrier, a copy or an MMA.  May be set at any time.
  *           key 11 "tile pairs": the tensor-core kernel's work item is a pair of neighbouring pixel tiles that share every
- *                  weight box (half the weight traffic, twice the work per item).  0 (default) = pairs in launch
- *                  groups with many tiles per SM, 1 = single tiles only, 2 = pairs wherever the geometry allows.
+ *                  weight box (half the weight traffic, twice the work per item).  0 (default) and 1 = single tiles,
+ *                  2 = pairs wherever the geometry allows.
+ *           key 12 "staged boxes in the weight ring": the activation box of a staged few-channel input edge (two MMAs'
+ *                  worth of work) is fetched into the tensor-core kernel's weight ring together with its weights, so
+ *                  that it does not hold one of the few large activation slots.  1 (default) = in launch groups whose
+ *                  weight ring has at least four slots, 2 = wherever the box fits a weight slot, 0 = never.
  * Must be set before sr_graph_workspace_bytes / sr_graph_bind_workspace (engine, weight ring, tile width, tile pairs,
- * resident keys) / before the first run (graphs). */
+ * staged boxes, resident keys) / before the first run (graphs). */
 sr_status sr_graph_set_option(sr_graph* g, int key, int value);
 
 /*

@@ -60,19 +60,30 @@ constexpr int kEpiWarps = 8;                          // warps 4..11
 constexpr int kFifo = 16;                             // burst descriptors in flight between scout and issuer
 constexpr int kMaxA = 4;                              // activation ring depth
 constexpr int kMaxW = 8;                              // weight ring depth (one weight box per slot)
-constexpr int kSmemBudget = 203 * 1024;               // dynamic shared memory; the static part takes the rest of 227 KiB
+// Dynamic shared memory of a CTA.  With the 24 KiB of static shared memory this leaves about 20 KiB of the SM's 228 KiB
+// free: the other kernels of a frame (input staging, dense heads: up to 7.4 KiB per block) run on a second stream beside
+// the persistent CTAs, and measured on B200 they queue behind them, frame after frame, once less than about 10 KiB of
+// the SM's shared-memory partition is left (a 117 us frame then takes 170 us).
+constexpr int kSmemBudget = 184 * 1024;
 constexpr int kMaxNodeKb = 128;                       // K-blocks per node the shared-memory tables hold
 
 // One weight group (consecutive K-blocks of equal channel-block width, fetched by ONE copy) as the weight producer
-// sees it (8 bytes).  A thread that waits for a slot, arms the barrier and starts a copy gets through about one
+// sees it (16 bytes).  A thread that waits for a slot, arms the barrier and starts a copy gets through about one
 // copy per 420 cycles (measured on B200), so copies must be large: a group, not a K-block.
+// The K-block of a staged few-channel edge is two MMAs long, and its activation box would hold one of the two or three
+// large activation slots for that short time only to keep the next filter's box from being requested early.  Such a
+// box travels in the weight ring instead: the group is then the block's weights followed by its activation box.
 struct TcKbWeight {
     uint16_t blk;           // index of the group's first K-block in its tensor map (a run of equally wide blocks)
     uint16_t w_map;         // tensor map of that run: dims (channels of a block, output channels, blocks)
-    uint16_t w_bytes16;     // (bytes of the whole group) / 16
+    uint16_t w_bytes16;     // (bytes of the whole group, the activation box included) / 16
+    uint16_t x_off16;       // (offset of the activation box inside the slot) / 16; 0 = the group has none
+    uint16_t x_map0, x_map1;// tensor map of that box for source frame parity 0 / 1
+    uint8_t c0_16;          // (first channel of the box) / 16
+    uint8_t flags;          // 1: the edge reads frame t (R = 1), else frame t+1
     uint16_t pad_;
 };
-static_assert(sizeof(TcKbWeight) == 8, "copied as one 8-byte word");
+static_assert(sizeof(TcKbWeight) == 16, "copied as one 16-byte word");
 
 // One activation box of a node's reduction as the activation producer sees it (16 bytes); only the K-blocks that
 // open a fresh box have one.
@@ -93,7 +104,8 @@ struct TcBurst {
     uint16_t xa_off16;      // (byte offset of the first block's operand window inside its activation slot) / 16
     uint16_t xb_off16;      // two blocks: the same for the second block; one block: for lane 1's window of that block
     uint8_t flags;          // 1 / 2: the first / second block opens a fresh activation slot; 4 / 8: the first / second
-                            // block is the last reader of its slot; 16: the burst has two blocks
+                            // block is the last reader of its slot; 16: the burst has two blocks; 32: the activation
+                            // box lies in the burst's weight slot (xa_off16 counts from the start of that slot)
     uint8_t state;          // descriptor state of the burst: index into the node's state table
     uint16_t pad_;
 };
@@ -272,7 +284,7 @@ sr_tc_group_kernel(const CUtensorMap* __restrict__ maps, const TcNode* __restric
     __shared__ uint32_t tmem_slot;
     __shared__ int abort_flag;
     __shared__ int epi_stop;
-    __shared__ uint2 w_tab[kMaxNodeKb];                    // K-block records of the weight producer's current node,
+    __shared__ uint4 w_tab[kMaxNodeKb];                    // K-block records of the weight producer's current node,
     __shared__ uint4 a_tab[kMaxNodeKb];                    // of the activation producer's
     __shared__ uint2 m_tab[kMaxNodeKb];                    // and the burst records of the scout's
     __shared__ __align__(16) uint16_t epi_buf[kEpiWarps][32 * 32];   // per epilogue warp: 32 pixels x 32 channels, bf16
@@ -344,7 +356,7 @@ sr_tc_group_kernel(const CUtensorMap* __restrict__ maps, const TcNode* __restric
             const int first_wg = nodes[tl.node].first_wg, n_wg = nodes[tl.node].n_wg;
             if (tl.node != cached_node) {
                 __syncwarp();
-                for (int i = lane; i < n_wg; i += 32) w_tab[i] = reinterpret_cast<const uint2*>(kb_weight)[first_wg + i];
+                for (int i = lane; i < n_wg; i += 32) w_tab[i] = reinterpret_cast<const uint4*>(kb_weight)[first_wg + i];
                 cached_node = tl.node;
                 __syncwarp();
             }
@@ -359,6 +371,11 @@ sr_tc_group_kernel(const CUtensorMap* __restrict__ maps, const TcNode* __restric
                     if (++w_nxt == (uint32_t)n_w) { w_nxt = 0; w_ph ^= 1; }
                     mbar_expect_tx(bar_wfull + 8 * s, (uint32_t)k.w_bytes16 << 4);
                     tma_load_3d(w_ring + s * w_slot, &maps[k.w_map], bar_wfull + 8 * s, 0, tl.m0, (int)k.blk);
+                    if (k.x_off16) {                                      // a staged edge's activation box rides along
+                        const int par = (k.flags & 1) ? prev : cur;
+                        tma_load_4d(w_ring + s * w_slot + ((uint32_t)k.x_off16 << 4), &maps[par ? k.x_map1 : k.x_map0], bar_wfull + 8 * s,
+                                    (int)k.c0_16 << 4, tl.w0, tl.h0, tl.b0);
+                    }
                 }
             }
             ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
@@ -486,7 +503,9 @@ sr_tc_group_kernel(const CUtensorMap* __restrict__ maps, const TcNode* __restric
                             if (++a_nxt == (uint32_t)n_a) { a_nxt = 0; a_ph ^= 1; }
                             a_base16 = (a_ring + a_cur * a_slot) >> 4;
                         }
-                        const uint32_t z = ((a_base16 + (rec.x & 0xFFFFu)) & 0x3FFFu) | 0x10000u;
+                        // the window of the first block: in the activation slot, or (a staged edge) in the weight slot
+                        const uint32_t x_base16 = (fl & 32u) ? (w_ring + w_nxt * w_slot) >> 4 : a_base16;
+                        const uint32_t z = ((x_base16 + (rec.x & 0xFFFFu)) & 0x3FFFu) | 0x10000u;
                         if (fl & 4u) act_mask |= 1u << a_cur;
                         if (fl & 2u) {
                             a_cur = a_nxt;
@@ -784,6 +803,8 @@ struct KbHost {
     int blk = 0;
     bool w_first = false, w_last = false;   // first / last block of a weight group
     int w_off = 0;     // byte offset of this block's weights inside the group's slot
+    bool in_wring = false;   // a staged edge whose activation box travels in the weight ring, behind the block's weights
+    int box_off = 0;         // byte offset of that box inside the slot
 };
 
 // Consecutive K-blocks of equal channel-block width: one 3-D view (channels of a block, output channels, blocks) of
@@ -792,7 +813,7 @@ struct WRun { int bk, first_col, n_blocks; };
 // what the MMAs of one K-block need (host-side; folded into burst records and descriptor states at bind time)
 struct KmHost {
     uint32_t desc_hi = 0, x_off16 = 0, x_l1off16 = 0, x_sbo16 = 0, n_k16 = 0, w_step16 = 0;
-    bool x_load = false, x_release = false;
+    bool x_load = false, x_release = false, in_wring = false;
 };
 struct WGroup { int run, blk, n, bytes; };
 
@@ -801,6 +822,7 @@ struct NodePlan {
     int tw, th, tb, sep, n_cols;
     bool one_box;                   // tw == 8: one activation box per channel block serves all k x k taps
     int pair;                       // 0: single tiles; 1: lane 1 is the tile tw columns to the right; 2: the next tb samples
+    bool stem_ring;                 // boxes of staged edges travel in the weight ring
     int k_total;                    // columns of the concatenated weight matrix
     std::vector<KbHost> kbs;
     std::vector<WRun> runs;
@@ -942,6 +964,13 @@ void build_kblocks(const sr_graph* g, const TcEngine* E, NodePlan& P)
             for (int c0 = 0; c0 < Kp; c0 += bk) {
                 KbHost kb{e, true, si, 0, 0, c0, bk, 0, true, 0, P.lane_w(), true};
                 kb.src_col = c0;
+                // weights, then the box, if both fit the weight slot that full-width groups need anyway (32 KiB)
+                const size_t w_bytes = sr_align_up((size_t)std::min(n.d.c, 128) * bk * 2, 1024);
+                const size_t box_bytes = (size_t)kb.x_width * (P.th + P.sep) * P.box_tb() * bk * 2;
+                if (P.pair == 0 && P.stem_ring && w_bytes + box_bytes <= 32 * 1024) {
+                    kb.in_wring = true;
+                    kb.box_off = (int)w_bytes;
+                }
                 P.kbs.push_back(kb);
             }
         } else {
@@ -994,7 +1023,8 @@ void build_kblocks(const sr_graph* g, const TcEngine* E, NodePlan& P)
         if (P.runs.empty() || P.runs.back().bk != kb.bk) P.runs.push_back(WRun{kb.bk, kb.k_off, 0});
         kb.run = (int)P.runs.size() - 1;
         kb.blk = P.runs.back().n_blocks++;
-        bool open = P.wgroups.empty() || P.wgroups.back().run != kb.run || P.wgroups.back().n >= per_group;
+        bool open = P.wgroups.empty() || P.wgroups.back().run != kb.run || P.wgroups.back().n >= per_group || kb.in_wring ||
+                    (i > 0 && P.kbs[i - 1].in_wring);
         if (!open && kb.x_load) {
             bool had_load = false;
             for (int j = 0; j < P.wgroups.back().n; ++j) had_load |= P.kbs[i - 1 - j].x_load;
@@ -1008,6 +1038,7 @@ void build_kblocks(const sr_graph* g, const TcEngine* E, NodePlan& P)
         kb.w_off = P.wgroups.back().bytes;
         P.wgroups.back().n += 1;
         P.wgroups.back().bytes += rows * kb.bk * 2;
+        if (kb.in_wring) P.wgroups.back().bytes = kb.box_off + kb.x_width * (P.th + P.sep) * P.box_tb() * kb.bk * 2;
     }
     if (!P.kbs.empty()) P.kbs.back().w_last = true;
     P.k_total = k_off;
@@ -1025,6 +1056,7 @@ int act_slot_bytes(const NodePlan& P)
 {
     int a_slot = 1024;
     for (const KbHost& kb : P.kbs) {
+        if (kb.in_wring) continue;
         const size_t box_px = (size_t)kb.x_width * (P.th + P.sep) * P.box_tb();
         // the last 8-pixel group a window reads: shift + (n_cols / 8 - 1) rows of the box + 8 pixels
         const size_t reach_px = (size_t)kb.x_shift + lane1_shift_px(P, kb.x_width) + (size_t)(P.n_cols / 8 - 1) * (kb.x_width * 8 / P.tw) + 8;
@@ -1157,14 +1189,18 @@ sr_status sr_tc_plan(sr_graph* g, size_t& off)
         // geometry allows.
         (void)single_tiles;
         bool pair = g->opt_tc_pair == 2;
+        // The box of a staged edge takes a weight slot for the two MMAs it feeds; that pays where the weight ring is
+        // deep (launch groups of nodes with few output channels: small weight groups), not where it has three slots.
+        bool stem_ring = g->opt_stem_ring != 0;
         int a_slot = 1024, w_slot = 1024, n_a = 2, n_w = 2, per_sm = 1;
-        for (int attempt = 0; attempt < 2; ++attempt) {
+        for (int attempt = 0; attempt < 3; ++attempt) {
             a_slot = 1024;
             w_slot = 1024;
             for (int ni : members) {
                 NodePlan& P = E->nodes[ni];
                 const SrHostNode& n = g->nodes[P.node];
                 P.pair = 0;
+                P.stem_ring = stem_ring;
                 if (pair) {
                     if (P.tw == 8 && n.d.w > P.tw) P.pair = 1;
                     else if (P.th == n.d.h && g->batch > P.tb) P.pair = 2;
@@ -1180,6 +1216,10 @@ sr_status sr_tc_plan(sr_graph* g, size_t& off)
             n_a = 2;
             while (n_a < kMaxA && (n_a + 1) * a_slot + w_max * w_slot <= avail) ++n_a;
             n_w = std::min(w_max, (avail - n_a * a_slot) / w_slot);
+            if (stem_ring && g->opt_stem_ring == 1 && n_w < 4) {
+                stem_ring = false;
+                continue;
+            }
             if (n_w >= 3 || !pair) break;
             pair = false;                                  // the paired boxes do not leave room for a weight ring: single tiles
         }
@@ -1258,6 +1298,10 @@ sr_status sr_tc_bind(sr_graph* g)
     if (!encode) return SR_ERR_CUDA;
     if (cudaFuncSetAttribute(sr_tc_group_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBudget) != cudaSuccess)
         return SR_ERR_CUDA;
+    // Always the largest shared-memory partition: otherwise the SM is configured with the smallest partition that holds
+    // this kernel's CTA, which can leave a few hundred bytes, and the frame's other kernels cannot run beside it.
+    if (cudaFuncSetAttribute(sr_tc_group_kernel, cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxShared) != cudaSuccess)
+        return SR_ERR_CUDA;
     char* ws = g->ws;
     std::vector<CUtensorMap> maps;
     std::map<std::tuple<uintptr_t, int, int, int, int, int, int, int, int>, int> cache;
@@ -1321,6 +1365,7 @@ sr_status sr_tc_bind(sr_graph* g)
             maps.push_back(m);
             run_map[{wg.run, wg.n}] = (int)maps.size() - 1;
         }
+        const size_t first_kw = dw.size();
         for (const WGroup& wg : P.wgroups) {
             TcKbWeight kw{};
             const size_t bytes = (size_t)wg.bytes;
@@ -1331,6 +1376,9 @@ sr_status sr_tc_bind(sr_graph* g)
             kw.w_bytes16 = (uint16_t)(bytes >> 4);
             dw.push_back(kw);
         }
+        std::vector<int> group_of;                    // K-block -> weight group of the node
+        for (size_t gi = 0; gi < P.wgroups.size(); ++gi)
+            for (int j = 0; j < P.wgroups[gi].n; ++j) group_of.push_back((int)gi);
         for (size_t i = 0; i < P.kbs.size(); ++i) {
             const KbHost& kb = P.kbs[i];
             const SrHostEdge& he = g->edges[kb.edge];
@@ -1379,7 +1427,21 @@ sr_status sr_tc_bind(sr_graph* g)
             if (map0 > 65535 || map1 > 65535 || qxv < -128 || qxv > 127 || qyv < -128 || qyv > 127 || kb.c0 / 16 > 255) return SR_ERR_UNSUPPORTED;
             kl.x_map0 = (uint16_t)map0; kl.x_map1 = (uint16_t)map1;
             kl.qx = (int8_t)qxv; kl.qy = (int8_t)qyv;
-            if (kb.x_load) da.push_back(kl);
+            if (kb.in_wring) {
+                // the box belongs to the block's weight group: the weight producer fetches it, no activation slot is used
+                TcKbWeight& kw = dw[first_kw + group_of[i]];
+                if (qxv != 0 || qyv != 0 || (kb.box_off & 1023) != 0 || (kb.box_off >> 4) > 65535) return SR_ERR_UNSUPPORTED;
+                kw.x_off16 = (uint16_t)(kb.box_off >> 4);
+                kw.x_map0 = kl.x_map0;
+                kw.x_map1 = kl.x_map1;
+                kw.c0_16 = kl.c0_16;
+                kw.flags = kl.flags;
+                km.x_load = km.x_release = false;
+                km.x_off16 += (uint32_t)(kb.box_off >> 4);
+                km.in_wring = true;
+            } else if (kb.x_load) {
+                da.push_back(kl);
+            }
             dm.push_back(km);
         }
         d.n_act = (int)da.size() - d.first_act;
@@ -1400,7 +1462,8 @@ sr_status sr_tc_bind(sr_graph* g)
             TcBurst b{};
             b.state = (uint8_t)(si - d.first_state);
             b.xa_off16 = (uint16_t)a.x_off16;
-            b.flags = (uint8_t)((a.x_load ? 1 : 0) | (a.x_release ? 4 : 0));
+            b.flags = (uint8_t)((a.x_load ? 1 : 0) | (a.x_release ? 4 : 0) | (a.in_wring ? 32 : 0));
+            if (a.in_wring && wg.n != 1) return SR_ERR_UNSUPPORTED;
             if (wg.n == 2) {
                 const KmHost& c = dm[i0 + 1];
                 if (c.desc_hi != a.desc_hi || c.x_sbo16 != a.x_sbo16) return SR_ERR_UNSUPPORTED;

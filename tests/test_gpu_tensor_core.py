@@ -46,6 +46,17 @@ def test_few_channel_input_edges_are_staged():
                  [Edge(0, 1, CONV, k, 1), Edge(1, 2, CONV, 3, 1), Edge(0, 2, CONV, k, 1), Edge(1, 1, CONV, 3, 1),
                   Edge(2, 3, GAP_DENSE)], frames=4, R=[1, 1, 0, 1, 0])
         run(g)
+        # the staged edge's activation box in an activation slot (0) / in the weight ring behind its weights (2)
+        for stem_ring in (0, 2):
+            parity.check_stepwise(g, "p", zero_bias=False, stem_ring=stem_ring)
+
+
+def test_a_node_fed_by_a_staged_edge_only():
+    # every K-block of node a travels in the weight ring: the activation ring stays empty for its tiles
+    g = tiny("stem_only", [Node("in", 32, 32, 3, IDENTITY), Node("a", 32, 32, 64), Node("b", 32, 32, 128), Node("o", 1, 1, 4, IDENTITY)],
+             [Edge(0, 1, CONV, 3, 1), Edge(1, 2, CONV, 3, 1), Edge(2, 3, GAP_DENSE)], batch=5, frames=4)
+    for stem_ring in (0, 1, 2):
+        parity.check_stepwise(g, "p", zero_bias=False, stem_ring=stem_ring)
 
 
 def test_pooled_edge_and_recurrence():
