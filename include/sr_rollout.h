@@ -196,8 +196,11 @@ sr_status sr_graph_set_node_bias(sr_graph* g, int node, const float* bias_host);
  *                  worth of work) is fetched into the tensor-core kernel's weight ring together with its weights, so
  *                  that it does not hold one of the few large activation slots.  1 (default) = in launch groups whose
  *                  weight ring has at least four slots, 2 = wherever the box fits a weight slot, 0 = never.
+ *           key 13 "work lists": how the tensor-core kernel's persistent CTAs get their work items.  0 (default) = one
+ *                  list, longest item first, from which the CTAs take as they go (a device-wide counter); 1 = one
+ *                  list per CTA, balanced on the host by estimated cost.
  * Must be set before sr_graph_workspace_bytes / sr_graph_bind_workspace (engine, weight ring, tile width, tile pairs,
- * staged boxes, resident keys) / before the first run (graphs). */
+ * staged boxes, work lists, resident keys) / before the first run (graphs). */
 sr_status sr_graph_set_option(sr_graph* g, int key, int value);
 
 /*

@@ -273,11 +273,40 @@ __device__ __forceinline__ void tc_wait_ld() { asm volatile("tcgen05.wait::ld.sy
 //   y, z (state): upper descriptor words of the weight and of the activation operand; w bits 0-15: the weight step / 16
 constexpr uint32_t kDescState = 1u << 16, kDescStop = 1u << 29;
 
+// Work items.  Either CTA c walks column c of a matrix of items made on the host (sched == nullptr), or the CTAs take
+// the items of ONE list, sorted by decreasing work, from a device-wide counter as they go: the weight producer fetches
+// (one item ahead) into a small queue in shared memory, every other role reads the queue.  The kernel ends when its
+// slowest CTA ends; measured on B200 the static lists left that CTA 2-8 % above the mean (the cost of an item is only
+// an estimate), the shared list ends all CTAs within one small item of each other.
+constexpr int kTileQ = 8;                              // queue entries; no role is ever that many items ahead of the epilogue
+
+// Index of this CTA's it-th item in the tile table, or -1 when there is none (any more).
+__device__ __forceinline__ int tc_item(int it, int n_tiles, const int* sched, const volatile int* tile_q, const volatile int* tile_n,
+                                       volatile int* abort_flag, long long limit)
+{
+    if (!sched) {
+        const long long ti = (long long)blockIdx.x + (long long)it * gridDim.x;
+        return ti < n_tiles ? (int)ti : -1;
+    }
+    if (*tile_n <= it) {
+        const long long t0 = clock64();
+        while (*tile_n <= it) {
+            if (*abort_flag) return -1;
+            if (clock64() - t0 > limit) {
+                *abort_flag = 1;
+                return -1;
+            }
+        }
+    }
+    __threadfence_block();
+    return tile_q[it & (kTileQ - 1)];
+}
+
 __global__ void __launch_bounds__(kThreads, 2)
 sr_tc_group_kernel(const CUtensorMap* __restrict__ maps, const TcNode* __restrict__ nodes,
                    const TcKbWeight* __restrict__ kb_weight, const TcKbAct* __restrict__ kb_act, const TcBurst* __restrict__ bursts, const TcState* __restrict__ states,
                    const TcTile* __restrict__ tiles, int n_tiles, SrFrameCtl* __restrict__ ctl, int t_off, int B,
-                   int n_a, int a_slot, int n_w, int w_slot, int tmem_cols, long long wait_limit)
+                   int n_a, int a_slot, int n_w, int w_slot, int tmem_cols, long long wait_limit, int* sched)
 {
     extern __shared__ uint8_t smem_raw[];
     __shared__ uint64_t bars[2 * kMaxA + 2 * kMaxW + 4];
@@ -291,6 +320,10 @@ sr_tc_group_kernel(const CUtensorMap* __restrict__ maps, const TcNode* __restric
     __shared__ int pix_off[2 * kMaxCols];                  // element offset of every pixel of both lanes, -1 = not stored
     __shared__ __align__(16) uint4 fifo[kFifo];            // burst descriptors, scout -> issuer
     __shared__ volatile uint32_t fifo_read;                // descriptors the issuer has taken
+    __shared__ volatile int tile_q[kTileQ];                // items taken from the shared list (indices into the tile table, -1 = end)
+    __shared__ volatile int tile_n;                        // how many of them so far
+    __shared__ volatile int epi_items;                     // items the epilogue has finished
+    __shared__ volatile int epi_ti;                        // the epilogue's current item
 
     // A wait limit of zero (a host-side test hook) means "every wait has already expired": report it and return
     // before any barrier, tensor memory, copy or MMA is touched.
@@ -312,6 +345,8 @@ sr_tc_group_kernel(const CUtensorMap* __restrict__ maps, const TcNode* __restric
         abort_flag = 0;
         epi_stop = 0;
         fifo_read = 0;
+        tile_n = 0;
+        epi_items = 0;
         for (int s = 0; s < n_a; ++s) {
             mbar_init(bar_afull + 8 * s, 1);
             mbar_init(bar_aempty + 8 * s, 1);
@@ -350,7 +385,29 @@ sr_tc_group_kernel(const CUtensorMap* __restrict__ maps, const TcNode* __restric
         int cached_node = -1;
         uint32_t w_nxt = 0, w_ph = 0, w_used = 0, w_par = 0;  // next slot, phase; slots filled, parity of the latest fill
         bool ok = true;
-        for (int ti = blockIdx.x; ti < n_tiles; ti += gridDim.x) {
+        int n_fetched = 0;
+        bool q_end = false;
+        for (int it = 0;; ++it) {
+            int ti = -1;
+            if (lane == 0) {
+                // take items from the shared list until this one and the next are in the queue
+                while (sched && n_fetched < it + 2 && !q_end && ok) {
+                    if (n_fetched - epi_items >= kTileQ) {
+                        const long long t0 = clock64();
+                        while (n_fetched - epi_items >= kTileQ)
+                            if (abort_flag || clock64() - t0 > wait_limit) { abort_flag = 1; ok = false; break; }
+                        if (!ok) break;
+                    }
+                    const int v = atomicAdd(sched, 1);
+                    tile_q[n_fetched & (kTileQ - 1)] = v < n_tiles ? v : -1;
+                    q_end = v >= n_tiles;
+                    __threadfence_block();
+                    tile_n = ++n_fetched;
+                }
+                if (ok) ti = tc_item(it, n_tiles, sched, tile_q, &tile_n, abortp, wait_limit);
+            }
+            ti = __shfl_sync(0xffffffffu, ti, 0);
+            if (ti < 0) break;
             const TcTile tl = tiles[ti];
             if (tl.node < 0) break;                                   // the rest of this CTA's column of the work list is padding
             const int first_wg = nodes[tl.node].first_wg, n_wg = nodes[tl.node].n_wg;
@@ -389,7 +446,10 @@ sr_tc_group_kernel(const CUtensorMap* __restrict__ maps, const TcNode* __restric
         int cached_node = -1;
         uint32_t a_nxt = 0, a_ph = 0, a_used = 0, a_par = 0;
         bool ok = true;
-        for (int ti = blockIdx.x; ti < n_tiles; ti += gridDim.x) {
+        for (int it = 0;; ++it) {
+            int ti = lane == 0 ? tc_item(it, n_tiles, sched, tile_q, &tile_n, abortp, wait_limit) : 0;
+            ti = __shfl_sync(0xffffffffu, ti, 0);
+            if (ti < 0) break;
             const TcTile tl = tiles[ti];
             if (tl.node < 0) break;
             const int first_act = nodes[tl.node].first_act, n_act = nodes[tl.node].n_act;
@@ -406,7 +466,12 @@ sr_tc_group_kernel(const CUtensorMap* __restrict__ maps, const TcNode* __restric
                 // box two further on (of the next work item when this one ends, if it belongs to the same node).
                 TcTile nx = tl;
                 nx.node = -1;
-                if (ti + (int)gridDim.x < n_tiles) nx = tiles[ti + gridDim.x];
+                if (!sched) {
+                    if (ti + (int)gridDim.x < n_tiles) nx = tiles[ti + gridDim.x];
+                } else if (tile_n > it + 1) {
+                    const int nti = tile_q[(it + 1) & (kTileQ - 1)];
+                    if (nti >= 0) nx = tiles[nti];
+                }
                 for (int i = 0; i < n_act; ++i) {
                     const TcKbAct k = tab[i];
                     {
@@ -457,7 +522,10 @@ sr_tc_group_kernel(const CUtensorMap* __restrict__ maps, const TcNode* __restric
             st_shared_v4(smem_u32(&fifo[n_pub & (kFifo - 1)]), (n_pub & 0xFFFFu) | x, y, z, (w & 0x00FFFFFFu) | (n_pub << 24));
             return true;
         };
-        for (int ti = blockIdx.x; ti < n_tiles; ti += gridDim.x) {
+        for (int it = 0;; ++it) {
+            int ti = lane == 0 ? tc_item(it, n_tiles, sched, tile_q, &tile_n, abortp, wait_limit) : 0;
+            ti = __shfl_sync(0xffffffffu, ti, 0);
+            if (ti < 0) break;
             const TcTile tl = tiles[ti];
             if (tl.node < 0) break;
             const int first_wg = nodes[tl.node].first_wg, n_bursts = nodes[tl.node].n_wg, first_state = nodes[tl.node].first_state;
@@ -660,7 +728,11 @@ sr_tc_group_kernel(const CUtensorMap* __restrict__ maps, const TcNode* __restric
         uint16_t* tbuf = &epi_buf[ew][0];
         uint32_t uses0 = 0, uses1 = 0;
         bool ok = true;
-        for (int ti = blockIdx.x; ti < n_tiles; ti += gridDim.x) {
+        for (int it = 0;; ++it) {
+            if (et == 0) epi_ti = tc_item(it, n_tiles, sched, tile_q, &tile_n, abortp, wait_limit);
+            asm volatile("bar.sync 1, 256;" ::: "memory");           // one answer for all eight warps
+            const int ti = epi_ti;
+            if (ti < 0) break;
             const TcTile tl = tiles[ti];
             if (tl.node < 0) break;
             const TcNode nd = nodes[tl.node];
@@ -721,6 +793,7 @@ sr_tc_group_kernel(const CUtensorMap* __restrict__ maps, const TcNode* __restric
                 if (lane == 0) mbar_arrive(bar_tempty + 8 * acc);
             }
             asm volatile("bar.sync 1, 256;" ::: "memory");           // everybody is done with the offset table
+            if (et == 0) epi_items = it + 1;
             if (tl.lanes == 2) { ++uses0; ++uses1; }
             else if (acc0 == 0) ++uses0;
             else ++uses1;
@@ -730,6 +803,15 @@ sr_tc_group_kernel(const CUtensorMap* __restrict__ maps, const TcNode* __restric
     tc_fence_before();
     __syncthreads();
     if (threadIdx.x == 0 && abort_flag) atomicExch(&ctl->error, 1);
+    if (threadIdx.x == 0 && sched) {
+        // the CTA that leaves last (none takes an item any more) puts the counters back for the next launch
+        __threadfence();
+        if (atomicAdd(sched + 1, 1) == (int)gridDim.x - 1) {
+            sched[0] = 0;
+            sched[1] = 0;
+            __threadfence();
+        }
+    }
     if (warp == 1) {
         tc_fence_after();
         asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(tmem_cols) : "memory");
@@ -845,7 +927,7 @@ struct TcEngine {
     std::vector<int> stem_of_edge;
     std::vector<std::vector<TcTile>> group_tiles;
     std::vector<int> group_tile_offset, group_a_slot, group_n_a, group_n_w, group_w_slot, group_grid, group_ctas_per_sm;
-    SrRegion r_maps, r_nodes, r_kb_weight, r_kb_act, r_bursts, r_states, r_tiles, r_stems;
+    SrRegion r_maps, r_nodes, r_kb_weight, r_kb_act, r_bursts, r_states, r_tiles, r_stems, r_sched;
     int n_maps = 0, n_kbs = 0, n_tiles = 0;
     int sm_count = 148;
     // optional timing of the group launches with CUDA events on the launching stream
@@ -1239,12 +1321,15 @@ sr_status sr_tc_plan(sr_graph* g, size_t& off)
             n_a = 2;
             n_w = std::min(kMaxW, (88 * 1024 - 1024 - 2 * a_slot) / w_slot);
         }
-        // Work lists: the items go, longest first, to the CTA with the least work so far; CTA c then walks column c
-        // of a matrix with one row per round (entries of node -1 pad the shorter columns).
+        // Work lists.  Shared list (default): all items in ONE list, longest first, which the CTAs take from as they
+        // go.  Static lists: the items go, longest first, to the CTA with the least work so far; CTA c then walks
+        // column c of a matrix with one row per round (entries of node -1 pad the shorter columns).
         std::stable_sort(tl.begin(), tl.end(), [](const auto& a, const auto& b) { return a.first > b.first; });
         const int grid = (int)std::min<size_t>(tl.size(), (size_t)E->sm_count * per_sm);
         std::vector<std::vector<TcTile>> lists(std::max(grid, 1));
-        {
+        if (g->opt_tc_lists == 0) {
+            for (auto& it : tl) E->group_tiles[gi].push_back(it.second);
+        } else {
             std::vector<std::pair<long long, int>> heap;     // (-load, cta): the standard heap keeps the largest on top
             for (int c = 0; c < grid; ++c) heap.push_back({0, -c});
             std::make_heap(heap.begin(), heap.end());
@@ -1256,12 +1341,12 @@ sr_status sr_tc_plan(sr_graph* g, size_t& off)
                 heap.back() = top;
                 std::push_heap(heap.begin(), heap.end());
             }
+            size_t n_rows = 0;
+            for (auto& l : lists) n_rows = std::max(n_rows, l.size());
+            for (size_t r = 0; r < n_rows; ++r)
+                for (int c = 0; c < grid; ++c)
+                    E->group_tiles[gi].push_back(r < lists[c].size() ? lists[c][r] : TcTile{-1, 0, 0, 0, 0, 0, {0, 0}});
         }
-        size_t n_rows = 0;
-        for (auto& l : lists) n_rows = std::max(n_rows, l.size());
-        for (size_t r = 0; r < n_rows; ++r)
-            for (int c = 0; c < grid; ++c)
-                E->group_tiles[gi].push_back(r < lists[c].size() ? lists[c][r] : TcTile{-1, 0, 0, 0, 0, 0, {0, 0}});
         E->group_grid.push_back(grid);
         E->group_tile_offset.push_back(n_tiles);
         n_tiles += (int)E->group_tiles[gi].size();
@@ -1287,6 +1372,7 @@ sr_status sr_tc_plan(sr_graph* g, size_t& off)
     E->r_states = take(sizeof(TcState) * (size_t)std::max(1, n_kbs));
     E->r_tiles = take(sizeof(TcTile) * (size_t)std::max(1, n_tiles));
     E->r_stems = take(sizeof(TcStem) * std::max<size_t>(1, E->stems.size()));
+    E->r_sched = take(256);                          // the shared list's counters: next item, CTAs that have left
     return SR_OK;
 }
 
@@ -1556,7 +1642,13 @@ static int launch_stage(sr_graph* g, int t_off, int fixed_parity, cudaStream_t s
 
 int sr_tc_stage_inputs(sr_graph* g, int t_off, cudaStream_t s) { return launch_stage(g, t_off, -1, s); }
 
-int sr_tc_after_state_change(sr_graph* g, cudaStream_t s) { return launch_stage(g, 0, (int)(g->t & 1), s); }
+int sr_tc_after_state_change(sr_graph* g, cudaStream_t s)
+{
+    // the shared work list's counters start from zero (every launch leaves them there; this covers a launch cut short)
+    if (TcEngine* E = eng(g))
+        if (g->ws) cudaMemsetAsync(g->ws + E->r_sched.offset, 0, 256, s);
+    return launch_stage(g, 0, (int)(g->t & 1), s);
+}
 
 int sr_tc_launch_group(sr_graph* g, int group, int t_off, cudaStream_t s)
 {
@@ -1585,7 +1677,8 @@ int sr_tc_launch_group(sr_graph* g, int group, int t_off, cudaStream_t s)
         reinterpret_cast<const TcBurst*>(g->ws + E->r_bursts.offset), reinterpret_cast<const TcState*>(g->ws + E->r_states.offset),
         reinterpret_cast<const TcTile*>(g->ws + E->r_tiles.offset) + E->group_tile_offset[group],
         (int)E->group_tiles[group].size(), reinterpret_cast<SrFrameCtl*>(g->ws + g->r_ctl.offset), t_off, g->batch, n_a, a_slot,
-        n_w, w_slot, E->group_ctas_per_sm[group] > 1 ? 256 : 512, (long long)g->opt_wait_ms * 2000000LL);
+        n_w, w_slot, E->group_ctas_per_sm[group] > 1 ? 256 : 512, (long long)g->opt_wait_ms * 2000000LL,
+        g->opt_tc_lists == 0 ? reinterpret_cast<int*>(g->ws + E->r_sched.offset) : nullptr);
     if (timed) {
         cudaEventRecord(E->ev[E->ev_used + 1], s);
         E->ev_used += 2;

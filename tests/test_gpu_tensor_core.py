@@ -17,12 +17,13 @@ def tiny(name, nodes, edges, batch=3, frames=3, R=None):
 
 
 def run(g):
-    # single tiles, then pairs of tiles that share every weight box (forced: these graphs are too small for the
-    # library to choose pairs by itself)
+    # single tiles (work items from the shared list, then from per-CTA lists), then pairs of tiles that share every
+    # weight box
     from paper_1806_04965_b200 import Graph
     G = Graph(g.nodes, g.edges, g.patterns["p"], batch=g.batch, dtype="bf16")
     assert G.info["n_tensor_core_nodes"] >= 1, G.info
     parity.check_stepwise(g, "p", zero_bias=False, tc_pair=1)
+    parity.check_stepwise(g, "p", zero_bias=False, tc_lists=1)      # a work list per CTA instead of the shared list
     return parity.check_stepwise(g, "p", zero_bias=False, tc_pair=2)
 
 
