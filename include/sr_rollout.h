@@ -199,8 +199,13 @@ sr_status sr_graph_set_node_bias(sr_graph* g, int node, const float* bias_host);
  *           key 13 "work lists": how the tensor-core kernel's persistent CTAs get their work items.  0 (default) = one
  *                  list, longest item first, from which the CTAs take as they go (a device-wide counter); 1 = one
  *                  list per CTA, balanced on the host by estimated cost.
+ *           key 14 "fused nodes": 1 (default) = two convolutional nodes of one launch group that have the same shape,
+ *                  at most 64 channels (a multiple of 32) each and an incoming edge from the same source with the
+ *                  same filter geometry and the same R run as ONE tensor-core work item per pixel tile: the second
+ *                  node's weights fill the otherwise empty rows 64..127 of the M = 128 instruction, and the shared
+ *                  source is read and multiplied once for both.  0 = every node on its own.  Results are identical.
  * Must be set before sr_graph_workspace_bytes / sr_graph_bind_workspace (engine, weight ring, tile width, tile pairs,
- * staged boxes, work lists, resident keys) / before the first run (graphs). */
+ * staged boxes, work lists, fused nodes, resident keys) / before the first run (graphs). */
 sr_status sr_graph_set_option(sr_graph* g, int key, int value);
 
 /*

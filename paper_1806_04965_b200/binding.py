@@ -113,7 +113,7 @@ class Graph:
     def __init__(self, nodes: Sequence, edges: Sequence, R: Sequence[int], batch: int = 0, dtype: str = "bf16",
                  engine: str = "auto", graph_frames: int = 0, device: str = "cuda:0", static_workspace: bool = False, weight_ring_units: int = 0, tile_width: int = 0,
                  resident: bool = True, resident_cluster: int = 0, resident_warps: int = 0, resident_split: int = 0,
-                 wait_limit_ms: Optional[int] = None, tc_pair: int = 0, stem_ring: int = 1, tc_lists: int = 0):
+                 wait_limit_ms: Optional[int] = None, tc_pair: int = 0, stem_ring: int = 1, tc_lists: int = 0, tc_fuse: int = 1):
         self._lib = load_library()
         self._h = ctypes.c_void_p()
         self.nodes, self.edges, self.R = list(nodes), list(edges), [int(r) for r in R]
@@ -146,6 +146,7 @@ class Graph:
             _check(self._lib.sr_graph_set_option(self._h, 11, int(tc_pair)), "sr_graph_set_option")
             _check(self._lib.sr_graph_set_option(self._h, 12, int(stem_ring)), "sr_graph_set_option")
             _check(self._lib.sr_graph_set_option(self._h, 13, int(tc_lists)), "sr_graph_set_option")
+            _check(self._lib.sr_graph_set_option(self._h, 14, int(tc_fuse)), "sr_graph_set_option")
             nbytes = ctypes.c_size_t()
             _check(self._lib.sr_graph_workspace_bytes(self._h, ctypes.byref(nbytes)), "sr_graph_workspace_bytes")
             self.workspace_bytes = nbytes.value

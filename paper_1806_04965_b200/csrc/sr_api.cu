@@ -414,6 +414,12 @@ sr_status sr_graph_set_option(sr_graph* g, int key, int value)
         g->opt_tc_pair = value;
         return SR_OK;
     }
+    if (key == 14) {
+        if (g->ws) return SR_ERR_STATE;
+        if (value < 0 || value > 1) return SR_ERR_INVALID_ARG;
+        g->opt_tc_fuse = value;
+        return SR_OK;
+    }
     if (key == 13) {
         if (g->ws) return SR_ERR_STATE;
         if (value < 0 || value > 1) return SR_ERR_INVALID_ARG;
@@ -798,6 +804,7 @@ sr_status sr_graph_window_workspace_bytes(sr_graph* g, int W, size_t* bytes)
         w->opt_tc_pair = g->opt_tc_pair;
         w->opt_stem_ring = g->opt_stem_ring;
         w->opt_tc_lists = g->opt_tc_lists;
+        w->opt_tc_fuse = g->opt_tc_fuse;
         w->opt_wait_ms = g->opt_wait_ms;
         w->opt_resident = 0;                                     // a window is one update of a large batch: the launch path
         g->window = w;

@@ -85,6 +85,7 @@ struct sr_graph {
     std::vector<std::vector<int>> groups;          // groups[l-1] = nodes of level l
     // options
     int opt_engine = 0, opt_graph_frames = 0, opt_b_units = 0, opt_tile_w = 0, opt_overlap = 1, opt_time_tc = 0;
+    int opt_tc_fuse = 1;                           // two nodes of at most 64 channels that share a source run as one 128-row plan
     int opt_tc_lists = 0;                          // tensor-core work items: 0 = one shared list the CTAs take from, 1 = a list per CTA made on the host
     int opt_stem_ring = 1;                         // activation boxes of staged few-channel edges travel in the weight ring
     int opt_tc_pair = 0;                           // tensor-core work items: 0 = pairs of tiles where it pays, 1 = single tiles, 2 = pairs wherever possible

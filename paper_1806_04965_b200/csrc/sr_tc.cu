@@ -121,9 +121,15 @@ struct TcState {
 };
 static_assert(sizeof(TcState) == 16, "read as one 16-byte word");
 
+// A plan can cover TWO nodes of at most 64 channels each that have the same shape and share a source: an M = 128
+// instruction on a 64-channel node is half empty, so the second node's weights take rows 64..127 and every K-block of
+// a source both read (same filter geometry, same frame) serves both.  TMEM lanes 64..127 then belong to the second node.
 struct TcNode {
     void* state[2];
     const float* bias;
+    void* state2[2];                // the second node of a fused plan (fused != 0)
+    const float* bias2;
+    int32_t act2, fused;
     int32_t H, W, C, act;
     int32_t tw, th, tb, sep;        // geometry of one lane's tile (see the file comment)
     int32_t n_cols;                 // N of the MMA: stacked rows of a lane's tile, rounded up to 32
@@ -752,10 +758,12 @@ sr_tc_group_kernel(const CUtensorMap* __restrict__ maps, const TcNode* __restric
             asm volatile("bar.sync 1, 256;" ::: "memory");           // the offset table is complete
             if (epi_stop) break;
             const uint32_t acc0 = tl.lanes == 2 ? 0u : ((tmem_cols >= 512 && uses0 > uses1) ? 1u : 0u);
-            __nv_bfloat16* out = static_cast<__nv_bfloat16*>(nd.state[cur]);
-            const int co_w = tl.m0 + quarter * 32;                  // first channel of this warp
+            const bool second = nd.fused && quarter >= 2;           // this warp's TMEM lanes belong to the plan's second node
+            __nv_bfloat16* out = static_cast<__nv_bfloat16*>(second ? nd.state2[cur] : nd.state[cur]);
+            const int co_w = nd.fused ? (quarter & 1) * 32 : tl.m0 + quarter * 32;   // first channel of this warp
             const int co = co_w + lane;                             // TMEM lane = output channel
-            const float bias = co < nd.C ? __ldg(nd.bias + co) : 0.f;
+            const float bias = co < nd.C ? __ldg((second ? nd.bias2 : nd.bias) + co) : 0.f;
+            const int act = second ? nd.act2 : nd.act;
             const bool gvalid = co_w + (lane & 3) * 8 < nd.C;       // this thread's group of 8 channels exists
             for (int l = 0; l < tl.lanes && ok; ++l) {
                 const uint32_t acc = l == 0 ? acc0 : 1u;
@@ -772,7 +780,7 @@ sr_tc_group_kernel(const CUtensorMap* __restrict__ maps, const TcNode* __restric
 #pragma unroll
                     for (int j = 0; j < 32; ++j) {
                         float z = __uint_as_float(v[j]) + bias;
-                        if (nd.act == 1) z = fmaxf(z, 0.f);
+                        if (act == 1) z = fmaxf(z, 0.f);
                         const __nv_bfloat16 hz = __float2bfloat16_rn(z);
                         tbuf[j * 32 + lane] = *reinterpret_cast<const uint16_t*>(&hz);
                     }
@@ -887,6 +895,8 @@ struct KbHost {
     int w_off = 0;     // byte offset of this block's weights inside the group's slot
     bool in_wring = false;   // a staged edge whose activation box travels in the weight ring, behind the block's weights
     int box_off = 0;         // byte offset of that box inside the slot
+    int row_off = 0;         // first row of `edge`'s weights in the plan's weight matrix (64: the second node of a fused plan)
+    int edge2 = -1;          // fused plan: the second node's edge that shares this block (its weights take rows 64..127)
 };
 
 // Consecutive K-blocks of equal channel-block width: one 3-D view (channels of a block, output channels, blocks) of
@@ -901,6 +911,8 @@ struct WGroup { int run, blk, n, bytes; };
 
 struct NodePlan {
     int node;
+    int node2 = -1;                 // the second node of a fused plan
+    int rows_total(const sr_graph* g) const { return node2 >= 0 ? 128 : g->nodes[node].d.c; }   // rows of the weight matrix
     int tw, th, tb, sep, n_cols;
     bool one_box;                   // tw == 8: one activation box per channel block serves all k x k taps
     int pair;                       // 0: single tiles; 1: lane 1 is the tile tw columns to the right; 2: the next tb samples
@@ -1007,16 +1019,40 @@ void tap_q(int tap, int pad, int st, int& q, int& r)
     r = a - q * st;
 }
 
-// The K-blocks of a node for its tile geometry and pairing mode (the stems' staging buffers exist already).
+// Do two edges read the same source through the same filter geometry in the same frame?  (Staged edges are not shared.)
+bool same_source(const sr_graph* g, int e1, int e2)
+{
+    const SrHostEdge& a = g->edges[e1];
+    const SrHostEdge& b = g->edges[e2];
+    return a.d.src == b.d.src && a.d.kind == SR_EDGE_CONV && b.d.kind == SR_EDGE_CONV && a.k_eff == b.k_eff &&
+           a.stride_eff == b.stride_eff && a.pad_eff == b.pad_eff && a.d.pool == b.d.pool && a.K == b.K && a.R == b.R &&
+           !is_stem(g, a) && !is_stem(g, b);
+}
+
+// The K-blocks of a plan for its tile geometry and pairing mode (the stems' staging buffers exist already).
 void build_kblocks(const sr_graph* g, const TcEngine* E, NodePlan& P)
 {
     const SrHostNode& n = g->nodes[P.node];
     P.kbs.clear();
     // one_box: every class of an edge gets a box as wide as the widest class of the node needs, so that all
     // K-blocks of equal channel-block width share one activation descriptor state
+    // the incoming edges of the plan: of its node and, fused, of its second node; an edge of the second node that
+    // reads the same source through the same filter geometry in the same frame shares the first node's K-blocks
+    struct Ent { int e, e2, row_off; };
+    std::vector<Ent> ents;
+    for (int e : n.in_edges) ents.push_back(Ent{e, -1, 0});
+    if (P.node2 >= 0)
+        for (int e2 : g->nodes[P.node2].in_edges) {
+            int m = -1;
+            for (size_t i = 0; i < ents.size() && m < 0; ++i)
+                if (ents[i].row_off == 0 && ents[i].e2 < 0 && same_source(g, ents[i].e, e2)) m = (int)i;
+            if (m >= 0) ents[m].e2 = e2;
+            else ents.push_back(Ent{e2, -1, 64});
+        }
     int span = 0;
     if (P.one_box)
-        for (int e : n.in_edges) {
+        for (const Ent& en : ents) {
+            const int e = en.e;
             const SrHostEdge& he = g->edges[e];
             if (is_stem(g, he)) continue;
             for (int r0 = 0; r0 < he.stride_eff; ++r0) {
@@ -1031,13 +1067,14 @@ void build_kblocks(const sr_graph* g, const TcEngine* E, NodePlan& P)
         }
     // The order of the reduction is free (a sum): edges with wider channel blocks come first, so that K-blocks of
     // equal width form one run each and a run's weights are one 3-D tensor.
-    std::vector<int> order(n.in_edges.begin(), n.in_edges.end());
     auto width_of = [&](int e) {
         const SrHostEdge& he = g->edges[e];
         return is_stem(g, he) ? std::min(64, E->stems[E->stem_of_edge[e]].Kp) : block_k(g->nodes[he.d.src].d.c);
     };
-    std::stable_sort(order.begin(), order.end(), [&](int a, int b) { return width_of(a) > width_of(b); });
-    for (int e : order) {
+    std::stable_sort(ents.begin(), ents.end(), [&](const Ent& a, const Ent& b) { return width_of(a.e) > width_of(b.e); });
+    const int rows = std::min(P.rows_total(g), 128);
+    for (const Ent& en : ents) {
+        const int e = en.e;
         const SrHostEdge& he = g->edges[e];
         const SrHostNode& s = g->nodes[he.d.src];
         if (is_stem(g, he)) {
@@ -1046,8 +1083,9 @@ void build_kblocks(const sr_graph* g, const TcEngine* E, NodePlan& P)
             for (int c0 = 0; c0 < Kp; c0 += bk) {
                 KbHost kb{e, true, si, 0, 0, c0, bk, 0, true, 0, P.lane_w(), true};
                 kb.src_col = c0;
+                kb.row_off = en.row_off;
                 // weights, then the box, if both fit the weight slot that full-width groups need anyway (32 KiB)
-                const size_t w_bytes = sr_align_up((size_t)std::min(n.d.c, 128) * bk * 2, 1024);
+                const size_t w_bytes = sr_align_up((size_t)rows * bk * 2, 1024);
                 const size_t box_bytes = (size_t)kb.x_width * (P.th + P.sep) * P.box_tb() * bk * 2;
                 if (P.pair == 0 && P.stem_ring && w_bytes + box_bytes <= 32 * 1024) {
                     kb.in_wring = true;
@@ -1082,6 +1120,8 @@ void build_kblocks(const sr_graph* g, const TcEngine* E, NodePlan& P)
                         KbHost kb{e, false, -1, t.ky, t.kx, c0, bk, 0,
                                   i == 0, (t.qy - qy0) * bw + (t.qx - qx0), bw, i + 1 == taps.size()};
                         kb.src_col = (t.ky * k + t.kx) * s.d.c + c0;
+                        kb.row_off = en.row_off;
+                        kb.edge2 = en.e2;
                         kb.box_qy = qy0;
                         kb.box_qx = qx0;
                         kb.box_ry = std::get<0>(cl.first);
@@ -1096,7 +1136,7 @@ void build_kblocks(const sr_graph* g, const TcEngine* E, NodePlan& P)
     // fresh activation box (the ring may have only two slots)
     P.runs.clear();
     P.wgroups.clear();
-    const int rows = std::min(n.d.c, 128), per_group = P.pair ? 1 : 2;
+    const int per_group = P.pair ? 1 : 2;
     int k_off = 0;
     for (size_t i = 0; i < P.kbs.size(); ++i) {
         KbHost& kb = P.kbs[i];
@@ -1162,7 +1202,7 @@ std::vector<TcTile> node_tiles(const sr_graph* g, const NodePlan& P, int node_in
     for (int b0 = 0; b0 < g->batch; b0 += db)
         for (int h0 = 0; h0 < n.d.h; h0 += P.th)
             for (int w0 = 0; w0 < n.d.w; w0 += dw)
-                for (int m0 = 0; m0 < n.d.c; m0 += 128) {
+                for (int m0 = 0; m0 < P.rows_total(g); m0 += 128) {
                     int lanes = 1;
                     if (P.pair == 1 && w0 + P.tw < n.d.w) lanes = 2;
                     if (P.pair == 2 && b0 + P.tb < g->batch) lanes = 2;
@@ -1216,15 +1256,50 @@ sr_status sr_tc_plan(sr_graph* g, size_t& off)
         off = sr_align_up(off + bytes, 1024);
         return r;
     };
+    // Fused plans: two nodes of one launch group with the same shape and at most 64 channels (a multiple of 32) each,
+    // which share at least one source (see TcNode).
+    std::vector<int> partner(g->nodes.size(), -1), leader(g->nodes.size(), -1);
+    if (g->opt_tc_fuse)
+        for (const std::vector<int>& grp : g->groups)
+            for (size_t i = 0; i < grp.size(); ++i) {
+                const int a = grp[i];
+                const SrHostNode& na = g->nodes[a];
+                if (!na.use_tc || partner[a] >= 0 || leader[a] >= 0 || na.d.c > 64 || na.d.c % 32 != 0) continue;
+                for (size_t j = i + 1; j < grp.size() && partner[a] < 0; ++j) {
+                    const int b = grp[j];
+                    const SrHostNode& nb = g->nodes[b];
+                    if (!nb.use_tc || partner[b] >= 0 || leader[b] >= 0 || nb.d.c != na.d.c || nb.d.h != na.d.h || nb.d.w != na.d.w) continue;
+                    int shared = 0, blocks = 0;
+                    for (int ea : na.in_edges) {
+                        const SrHostEdge& he = g->edges[ea];
+                        blocks += is_stem(g, he) ? 2 : he.k_eff * he.k_eff * (g->nodes[he.d.src].d.c / block_k(g->nodes[he.d.src].d.c));
+                    }
+                    for (int eb : nb.in_edges) {
+                        const SrHostEdge& he = g->edges[eb];
+                        bool sh = false;
+                        for (int ea : na.in_edges) sh |= same_source(g, ea, eb);
+                        if (sh) ++shared;
+                        else blocks += is_stem(g, he) ? 2 : he.k_eff * he.k_eff * (g->nodes[he.d.src].d.c / block_k(g->nodes[he.d.src].d.c));
+                    }
+                    if (shared > 0 && blocks <= kMaxNodeKb) {
+                        partner[a] = b;
+                        leader[b] = a;
+                    }
+                }
+            }
     // tile geometry and staging buffers
     for (size_t v = 0; v < g->nodes.size(); ++v) {
         const SrHostNode& n = g->nodes[v];
         if (!n.use_tc) continue;
+        if (leader[v] >= 0) continue;                     // the second node of a fused plan: its leader's plan covers it
         NodePlan P{};
         P.node = (int)v;
+        P.node2 = partner[v];
         // sep: how many image rows the taps that share one activation box are apart at most
         P.sep = 0;
-        for (int e : n.in_edges) {
+        std::vector<int> in_edges(n.in_edges.begin(), n.in_edges.end());
+        if (P.node2 >= 0) in_edges.insert(in_edges.end(), g->nodes[P.node2].in_edges.begin(), g->nodes[P.node2].in_edges.end());
+        for (int e : in_edges) {
             const SrHostEdge& he = g->edges[e];
             if (is_stem(g, he)) {
                 StemPlan S;
@@ -1253,13 +1328,15 @@ sr_status sr_tc_plan(sr_graph* g, size_t& off)
         E->node_of[v] = (int)E->nodes.size();
         E->nodes.push_back(P);
     }
+    for (size_t v = 0; v < g->nodes.size(); ++v)
+        if (leader[v] >= 0) E->node_of[v] = E->node_of[leader[v]];
     // per launch group: pairing, K-blocks, work list (largest reduction first), ring geometry
     E->group_tiles.assign(g->groups.size(), {});
     int n_tiles = 0;
     for (size_t gi = 0; gi < g->groups.size(); ++gi) {
         std::vector<int> members;
         for (int v : g->groups[gi])
-            if (E->node_of[v] >= 0) members.push_back(E->node_of[v]);
+            if (E->node_of[v] >= 0 && leader[v] < 0) members.push_back(E->node_of[v]);
         size_t single_tiles = 0;
         for (int ni : members) {
             build_kblocks(g, E, E->nodes[ni]);
@@ -1359,7 +1436,7 @@ sr_status sr_tc_plan(sr_graph* g, size_t& off)
     int n_kbs = 0;
     for (NodePlan& P : E->nodes) {
         n_kbs += (int)P.kbs.size();
-        P.wcat = take((size_t)g->nodes[P.node].d.c * P.k_total * 2);
+        P.wcat = take((size_t)P.rows_total(g) * P.k_total * 2);
     }
     E->n_tiles = n_tiles;
     E->n_kbs = n_kbs;
@@ -1422,6 +1499,14 @@ sr_status sr_tc_bind(sr_graph* g)
         d.state[1] = ws + n.state[1].offset;
         d.bias = reinterpret_cast<const float*>(ws + n.bias.offset);
         d.H = n.d.h; d.W = n.d.w; d.C = n.d.c; d.act = n.d.act;
+        if (P.node2 >= 0) {
+            const SrHostNode& n2 = g->nodes[P.node2];
+            d.state2[0] = ws + n2.state[0].offset;
+            d.state2[1] = ws + n2.state[1].offset;
+            d.bias2 = reinterpret_cast<const float*>(ws + n2.bias.offset);
+            d.act2 = n2.d.act;
+            d.fused = 1;
+        }
         d.tw = P.tw; d.th = P.th; d.tb = P.tb; d.sep = P.sep;
         d.n_cols = P.n_cols;
         d.l1_dw = P.pair == 1 ? P.tw : 0;
@@ -1440,9 +1525,9 @@ sr_status sr_tc_bind(sr_graph* g)
             if (run_map.count({wg.run, wg.n})) continue;
             const WRun& R = P.runs[wg.run];
             CUtensorMap m;
-            cuuint64_t dims[3] = {(cuuint64_t)R.bk, (cuuint64_t)n.d.c, (cuuint64_t)R.n_blocks};
+            cuuint64_t dims[3] = {(cuuint64_t)R.bk, (cuuint64_t)P.rows_total(g), (cuuint64_t)R.n_blocks};
             cuuint64_t strides[2] = {(cuuint64_t)P.k_total * 2, (cuuint64_t)R.bk * 2};
-            cuuint32_t box[3] = {(cuuint32_t)R.bk, (cuuint32_t)std::min(n.d.c, 128), (cuuint32_t)wg.n};
+            cuuint32_t box[3] = {(cuuint32_t)R.bk, (cuuint32_t)std::min(P.rows_total(g), 128), (cuuint32_t)wg.n};
             cuuint32_t es[3] = {1, 1, 1};
             if (encode(&m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, ws + P.wcat.offset + (size_t)R.first_col * 2, dims, strides, box, es,
                        CU_TENSOR_MAP_INTERLEAVE_NONE, swizzle_of(R.bk), CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
@@ -1475,7 +1560,7 @@ sr_status sr_tc_bind(sr_graph* g)
             kl.flags = (uint8_t)(he.R ? 1 : 0);
             km.x_load = kb.x_load;
             km.x_release = kb.x_release;
-            km.w_step16 = (uint32_t)((std::min(n.d.c, 128) * kb.bk * 2) >> 4);
+            km.w_step16 = (uint32_t)((std::min(P.rows_total(g), 128) * kb.bk * 2) >> 4);
             km.n_k16 = (uint32_t)(kb.bk / 16);
             km.desc_hi = desc_hi_of(kb.bk);
             const size_t x_bytes = (size_t)kb.bk * 2 * kb.x_width * rows * box_tb;
@@ -1606,7 +1691,8 @@ sr_status sr_tc_set_weights(sr_graph* g, int edge, const float* w_eff)
     // takes its slice [C_out][block width] of the edge's own matrix (a staged edge: all of it, zero-padded)
     bool any = false;
     for (const KbHost& kb : P.kbs) {
-        if (kb.edge != edge) continue;
+        if (kb.edge != edge && kb.edge2 != edge) continue;
+        const int row_off = kb.edge == edge ? kb.row_off : 64;
         any = true;
         const int n_src = kb.stem ? std::max(0, std::min(kb.bk, he.K - kb.src_col)) : kb.bk;
         std::vector<uint16_t> h((size_t)t.d.c * kb.bk, 0);
@@ -1615,7 +1701,7 @@ sr_status sr_tc_set_weights(sr_graph* g, int edge, const float* w_eff)
                 const __nv_bfloat16 b = __float2bfloat16_rn(w_eff[(size_t)co * he.K + kb.src_col + k]);
                 std::memcpy(&h[(size_t)co * kb.bk + k], &b, 2);
             }
-        char* dst = g->ws + P.wcat.offset + (size_t)kb.k_off * 2;
+        char* dst = g->ws + P.wcat.offset + ((size_t)row_off * P.k_total + kb.k_off) * 2;
         if (cudaMemcpy2D(dst, (size_t)P.k_total * 2, h.data(), (size_t)kb.bk * 2, (size_t)kb.bk * 2, t.d.c,
                          cudaMemcpyHostToDevice) != cudaSuccess)
             return SR_ERR_CUDA;

@@ -60,6 +60,22 @@ def test_a_node_fed_by_a_staged_edge_only():
         parity.check_stepwise(g, "p", zero_bias=False, stem_ring=stem_ring)
 
 
+@pytest.mark.parametrize("c,act_b", [(64, RELU), (32, IDENTITY)])
+def test_two_narrow_nodes_that_share_a_source_run_as_one_plan(c, act_b):
+    # a <- {in (staged), a}, b <- {a, b, in (1x1, staged)}, d <- {a, b}: a and b have the same shape, at most 64 channels
+    # and both read a through a 3x3 filter from the previous frame, so b's weights take rows 64..127 of a's tiles
+    g = tiny("fused", [Node("in", 24, 16, 3, IDENTITY), Node("a", 24, 16, c), Node("b", 24, 16, c, act_b), Node("d", 12, 8, 128),
+                       Node("o", 1, 1, 4, IDENTITY)],
+             [Edge(0, 1, CONV, 3, 1), Edge(1, 1, CONV, 3, 1), Edge(1, 2, CONV, 3, 1), Edge(2, 2, CONV, 3, 1), Edge(0, 2, CONV, 1, 1),
+              Edge(1, 3, CONV, 3, 2), Edge(2, 3, CONV, 1, 2), Edge(3, 4, GAP_DENSE)], batch=5, frames=4)
+    for fuse in (1, 0):
+        parity.check_stepwise(g, "p", zero_bias=False, tc_fuse=fuse)
+    parity.check_stepwise(g, "p", zero_bias=False, tc_fuse=1, tc_lists=1, stem_ring=2)
+    # with a -> b inside the frame (R = 0) the two nodes are in different launch groups: nothing to fuse, same results
+    g.patterns["q"] = [1, 1, 0, 1, 1, 1, 1, 1]
+    parity.check_stepwise(g, "q", zero_bias=False)
+
+
 def test_pooled_edge_and_recurrence():
     g = tiny("pool", [Node("in", 16, 16, 64, IDENTITY), Node("a", 8, 8, 128), Node("b", 8, 8, 128), Node("o", 1, 1, 4, IDENTITY)],
              [Edge(0, 1, CONV, 3, 1, 2), Edge(1, 1, CONV, 3, 1), Edge(1, 2, CONV, 3, 1), Edge(0, 2, CONV, 3, 2),
