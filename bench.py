@@ -41,9 +41,9 @@ ALL_WORKLOADS = ("c1", "c2", "c3", "c4", "c5")
 # the kernel source it was taken from; the number is reported only while that source is unchanged, else null.
 TRAFFIC = {
     # workload: (bytes per launch, kernel source file, sha256[:12] of that file at capture time, summary under profiles/)
-    "c5": (613.7e6, "sr_tc.cu", "96e6f12e8b16", "profiles/sr_tc_group_kernel_counters.md"),
-    "c3": (263.6e6, "sr_tc.cu", "96e6f12e8b16", "profiles/sr_tc_group_kernel_counters.md"),
-    "c4": (158.7e6, "sr_tc.cu", "96e6f12e8b16", "profiles/sr_tc_group_kernel_counters.md"),
+    "c5": (612.3e6, "sr_tc.cu", "9b4f1492ffe1", "profiles/sr_tc_group_kernel_counters.md"),
+    "c3": (245.3e6, "sr_tc.cu", "9b4f1492ffe1", "profiles/sr_tc_group_kernel_counters.md"),
+    "c4": (157.5e6, "sr_tc.cu", "9b4f1492ffe1", "profiles/sr_tc_group_kernel_counters.md"),
     "c2": (8.0e6, "sr_resident.cu", "89436108f1ff", "profiles/sr_resident_kernel_c2.md"),     # one launch = all 32 frames
 }
 
@@ -372,8 +372,9 @@ def measure_workload(torch, args, name, rank, local, dist, pk, flush, steps, war
                              else "%d CTAs per sequence" % res["resident_cluster"])}
         if dense:
             roof["alu"] = {"achieved_gflops": fl * T / (kernel_us * 1e-6) / 1e9,
-                           "note": "fp32 FMA on CUDA cores; weights and states resident in the shared memory of a cluster; bound by "
-                                   "cluster-barrier and launch latency"}
+                           "note": "fp32 FMA on CUDA cores; weights and states resident in the shared memory of a cluster; a frame "
+                                   "is one round of work units (shared-memory loads, reduction over the lanes) and one "
+                                   "cluster barrier: latency-bound"}
         else:
             roof["tensor"] = {"achieved_tflops": fl * T / (kernel_us * 1e-6) / 1e12,
                               "frac_of_burst_peak": fl * T / (kernel_us * 1e-6) / 1e12 / pk["bf16_tflops"],

@@ -196,9 +196,10 @@ sr_status sr_graph_set_node_bias(sr_graph* g, int node, const float* bias_host);
  *                  worth of work) is fetched into the tensor-core kernel's weight ring together with its weights, so
  *                  that it does not hold one of the few large activation slots.  1 (default) = in launch groups whose
  *                  weight ring has at least four slots, 2 = wherever the box fits a weight slot, 0 = never.
- *           key 13 "work lists": how the tensor-core kernel's persistent CTAs get their work items.  0 (default) = one
- *                  list, longest item first, from which the CTAs take as they go (a device-wide counter); 1 = one
- *                  list per CTA, balanced on the host by estimated cost.
+ *           key 13 "work lists": how the tensor-core kernel's persistent CTAs get their work items.  1 = one list per
+ *                  CTA, balanced on the host by estimated cost; 0 (default) = the same for the larger items, while
+ *                  the smallest ones (a fifth of the work of a launch with many items) form one shared list that
+ *                  every CTA takes from when its own list is done (a device-wide counter).
  *           key 14 "fused nodes": 1 (default) = two convolutional nodes of one launch group that have the same shape,
  *                  at most 64 channels (a multiple of 32) each and an incoming edge from the same source with the
  *                  same filter geometry and the same R run as ONE tensor-core work item per pixel tile: the second
@@ -243,7 +244,7 @@ sr_status sr_rollout_run(sr_graph* g, const void* const* in_seq_dev, int T, floa
  * Implemented for patterns whose frames do not depend on each other - every edge that bridges a frame leaves an
  * input node (e.g. the sequential rollout of a network without recurrence) -, where T((i, v)) = level(v) for every
  * frame i: level by level, the nodes of ALL W frames are updated in one launch group over a batch of W * B samples
- * (the equal-compute comparison of Sec. 4, "classifications of the first 8 images in parallel").  Other patterns
+ * (the equal-compute comparison of Sec. 4, where a deep window classifies its first frames side by side).  Other patterns
  * return SR_ERR_UNSUPPORTED.  in_seq_dev / out_seq_dev as for sr_rollout_run; afterwards the graph stands at frame
  * t + W and can be stepped on.  Results equal those of W calls of sr_rollout_step.
  * The window needs a workspace of its own (states of all W frames): ask for its size, allocate, bind; binding copies

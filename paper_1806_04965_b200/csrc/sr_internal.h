@@ -86,7 +86,7 @@ struct sr_graph {
     // options
     int opt_engine = 0, opt_graph_frames = 0, opt_b_units = 0, opt_tile_w = 0, opt_overlap = 1, opt_time_tc = 0;
     int opt_tc_fuse = 1;                           // two nodes of at most 64 channels that share a source run as one 128-row plan
-    int opt_tc_lists = 0;                          // tensor-core work items: 0 = one shared list the CTAs take from, 1 = a list per CTA made on the host
+    int opt_tc_lists = 0;                          // tensor-core work items: 1 = a list per CTA made on the host, 0 = the same plus a shared list of the smallest items
     int opt_stem_ring = 1;                         // activation boxes of staged few-channel edges travel in the weight ring
     int opt_tc_pair = 0;                           // tensor-core work items: 0 = pairs of tiles where it pays, 1 = single tiles, 2 = pairs wherever possible
     int opt_wait_ms = 1000;                        // limit of every device-side wait; 0 = expire at once (test hook)

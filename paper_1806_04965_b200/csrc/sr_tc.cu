@@ -1,9 +1,9 @@
 // Tensor-core engine: the node update  x_v = sigma(b_v + sum_e f_e(theta_e, x_src(e)))  (paper Sec. A1.2)
 // for all convolutional nodes of one launch group as ONE grouped implicit GEMM on tcgen05 / TMEM.
 //
-// The sum over the incoming edges of a node is one convolution over the concatenated sources
-// (paper Sec. A, "mathematically equivalent to concatenating all inputs"): the K loop of an output
-// tile simply walks the K-blocks of every incoming edge, tap by tap, into one TMEM accumulator.
+// The sum over the incoming edges of a node is one convolution over the concatenated sources (paper
+// Sec. A notes the equivalence): the K loop of an output tile simply walks the K-blocks of every
+// incoming edge, tap by tap, into one TMEM accumulator.
 //
 // GEMM shape.  D[c_out][pixel] = sum_k W[c_out][k] * X[pixel][k]: the weights are the M operand
 // (128 rows per instruction, one tile per 128 output channels), up to 256 output pixels are the N operand.
@@ -14,8 +14,9 @@
 // Operands.  K-block = one filter tap x up to 64 input channels.  Activation tiles come straight from
 // the NHWC state of the source node through 4-D TMA boxes (zero fill outside the image = zero
 // padding); a stride-s edge reads one of s*s residue-class views of the source, so every tap is again
-// a dense box.  Weight tiles come from the node's concatenated weight matrix [C_out][K] (K-major)
-// through 2-D TMA boxes.  Few-channel input edges (C_in = 1 or 3) are staged per frame into an im2col
+// a dense box.  The node's weight matrix [C_out][K] (K-major) keeps its columns in the order the K loop
+// walks them, so that consecutive K-blocks of equal width are one 3-D tensor and a weight group of two
+// K-blocks is ONE TMA copy.  Few-channel input edges (C_in = 1 or 3) are staged per frame into an im2col
 // tensor with K padded to 16/32/64 so that they are ordinary K-blocks.
 //
 // Pixel tile.  A tile is tb samples x th rows x tw columns (tw a multiple of 8, so an image row of
@@ -23,23 +24,19 @@
 // (sep = k - 1 of the node's stride-1 k x k edges), and the N columns of the GEMM are the rows of
 // that stacked box: column n = (b * (th + sep) + r) * tw + x.  Columns with r >= th are never stored.
 // This makes the k taps of one filter column row-shifted windows of ONE box: the box is loaded once
-// per filter column and the shared-memory descriptor of tap ky just starts ky * tw rows further down.
+// per filter column and the shared-memory descriptor of tap ky just starts ky * tw rows further down
+// (with 8-wide tiles the taps of a filter row share the box as well).
 //
-// Two pixel tiles per weight box.  What limits the kernel is the traffic from L2 into shared memory, and
-// most of it is weights: every tile re-fetches its node's weight boxes.  So a work item is a PAIR of
-// neighbouring pixel tiles ("lanes") that share every weight box: lane 0 accumulates in TMEM columns
-// 0..255, lane 1 in columns 256..511, and each weight box that arrives feeds the MMAs of both.  The
-// two tiles are neighbours in x (8-wide tiles) or consecutive samples (tiles that span the image), so
-// ONE activation box covers both and lane 1's operand window is lane 0's, a fixed number of bytes
-// further on.  Launch groups with few tiles keep single tiles (two accumulators alternate instead).
+// Work items.  An item is one pixel tile of one plan (a node, or two narrow nodes fused, see TcNode);
+// optionally a PAIR of neighbouring tiles ("lanes") that share every weight box (lane 0 accumulates in
+// TMEM columns 0..255, lane 1 in 256..511).  The persistent CTAs take the items from one shared list.
 //
-// Warp roles in a CTA of 384 threads: warp 0 = TMA producer; warp 2 = scout (all barrier waits and
-// address arithmetic; publishes one 16-byte burst descriptor per eight or so MMAs); warp 1 = MMA
-// issuer (owns TMEM; reads descriptors and issues, nothing else); warps 4..11 = epilogue (TMEM lane
-// = output channel; bias, ReLU, bf16, NHWC stores in which a warp writes 32 consecutive channels of one
-// pixel).  CTAs are persistent and walk a work list sorted by decreasing work.  Every wait is bounded;
-// on expiry the kernel records an error in the frame control block, waits for its own copies, frees
-// TMEM and returns.
+// Warp roles in a CTA of 384 threads: warp 0 = weight producer (and keeper of the item queue); warp 3 =
+// activation producer; warp 2 = scout (all barrier waits and address arithmetic; publishes one 16-byte
+// burst descriptor per eight or so MMAs); warp 1 = MMA issuer (owns TMEM; reads descriptors and issues,
+// nothing else); warps 4..11 = epilogue (TMEM lane = output channel; bias, ReLU, bf16, NHWC stores in
+// which a warp writes 32 consecutive channels of one pixel).  Every wait is bounded; on expiry the kernel
+// records an error in the frame control block, waits for its own copies, frees TMEM and returns.
 #include <cuda.h>
 #include <cuda_bf16.h>
 #include <cuda_runtime.h>
@@ -279,24 +276,31 @@ __device__ __forceinline__ void tc_wait_ld() { asm volatile("tcgen05.wait::ld.sy
 //   y, z (state): upper descriptor words of the weight and of the activation operand; w bits 0-15: the weight step / 16
 constexpr uint32_t kDescState = 1u << 16, kDescStop = 1u << 29;
 
-// Work items.  Either CTA c walks column c of a matrix of items made on the host (sched == nullptr), or the CTAs take
-// the items of ONE list, sorted by decreasing work, from a device-wide counter as they go: the weight producer fetches
-// (one item ahead) into a small queue in shared memory, every other role reads the queue.  The kernel ends when its
-// slowest CTA ends; measured on B200 the static lists left that CTA 2-8 % above the mean (the cost of an item is only
-// an estimate), the shared list ends all CTAs within one small item of each other.
+// Work items.  CTA c walks column c of a matrix of items made on the host (longest first onto the least loaded CTA);
+// every role of the CTA works out the column's entries by itself, so the roles stay decoupled.  The kernel ends when
+// its slowest CTA ends, and the cost of an item is only an estimate: measured on B200 such lists left that CTA 2-8 %
+// above the mean.  So (sched != nullptr) the matrix holds only the larger items, and the smallest ones, a fifth of the
+// work, form ONE shared list behind it from which every CTA takes, by a device-wide counter, when its own column is
+// done: the weight producer asks the counter two items ahead and keeps the answers in a small queue in shared memory
+// that the other roles read.  (ALL items in one shared list balanced the largest workload as well, but cost 3-8 % on
+// workloads and rollouts with many small launches, where a role could no longer run ahead of the weight producer.)
 constexpr int kTileQ = 8;                              // queue entries; no role is ever that many items ahead of the epilogue
 
-// Index of this CTA's it-th item in the tile table, or -1 when there is none (any more).
-__device__ __forceinline__ int tc_item(int it, int n_tiles, const int* sched, const volatile int* tile_q, const volatile int* tile_n,
-                                       volatile int* abort_flag, long long limit)
+// Index of this CTA's it-th item in the tile table, or -1 when there is none (any more).  own_len: the length of the
+// CTA's column, -1 while the role has not reached its end.
+__device__ __forceinline__ int tc_item(int it, int& own_len, const TcTile* __restrict__ tiles, int n_own, int n_tiles, const int* sched,
+                                       const volatile int* tile_q, const volatile int* tile_n, volatile int* abort_flag, long long limit)
 {
-    if (!sched) {
-        const long long ti = (long long)blockIdx.x + (long long)it * gridDim.x;
-        return ti < n_tiles ? (int)ti : -1;
+    if (own_len < 0) {
+        const long long idx = (long long)blockIdx.x + (long long)it * gridDim.x;
+        if (idx < n_own && tiles[idx].node >= 0) return (int)idx;
+        own_len = it;
     }
-    if (*tile_n <= it) {
+    if (!sched || n_own >= n_tiles) return -1;
+    const int j = it - own_len;                        // position in the CTA's share of the shared list
+    if (*tile_n <= j) {
         const long long t0 = clock64();
-        while (*tile_n <= it) {
+        while (*tile_n <= j) {
             if (*abort_flag) return -1;
             if (clock64() - t0 > limit) {
                 *abort_flag = 1;
@@ -305,14 +309,14 @@ __device__ __forceinline__ int tc_item(int it, int n_tiles, const int* sched, co
         }
     }
     __threadfence_block();
-    return tile_q[it & (kTileQ - 1)];
+    return tile_q[j & (kTileQ - 1)];
 }
 
 __global__ void __launch_bounds__(kThreads, 2)
 sr_tc_group_kernel(const CUtensorMap* __restrict__ maps, const TcNode* __restrict__ nodes,
                    const TcKbWeight* __restrict__ kb_weight, const TcKbAct* __restrict__ kb_act, const TcBurst* __restrict__ bursts, const TcState* __restrict__ states,
                    const TcTile* __restrict__ tiles, int n_tiles, SrFrameCtl* __restrict__ ctl, int t_off, int B,
-                   int n_a, int a_slot, int n_w, int w_slot, int tmem_cols, long long wait_limit, int* sched)
+                   int n_a, int a_slot, int n_w, int w_slot, int tmem_cols, long long wait_limit, int* sched, int n_own)
 {
     extern __shared__ uint8_t smem_raw[];
     __shared__ uint64_t bars[2 * kMaxA + 2 * kMaxW + 4];
@@ -328,7 +332,7 @@ sr_tc_group_kernel(const CUtensorMap* __restrict__ maps, const TcNode* __restric
     __shared__ volatile uint32_t fifo_read;                // descriptors the issuer has taken
     __shared__ volatile int tile_q[kTileQ];                // items taken from the shared list (indices into the tile table, -1 = end)
     __shared__ volatile int tile_n;                        // how many of them so far
-    __shared__ volatile int epi_items;                     // items the epilogue has finished
+    __shared__ volatile int epi_items;                     // items of the shared list the epilogue has finished
     __shared__ volatile int epi_ti;                        // the epilogue's current item
 
     // A wait limit of zero (a host-side test hook) means "every wait has already expired": report it and return
@@ -391,26 +395,41 @@ sr_tc_group_kernel(const CUtensorMap* __restrict__ maps, const TcNode* __restric
         int cached_node = -1;
         uint32_t w_nxt = 0, w_ph = 0, w_used = 0, w_par = 0;  // next slot, phase; slots filled, parity of the latest fill
         bool ok = true;
-        int n_fetched = 0;
-        bool q_end = false;
+        // Items of the shared list: the counter is asked two items ahead, BEFORE this item's copies are issued, and its
+        // answer (a round trip through the L2, microseconds) is put into the queue after them, so that the copies never
+        // wait for it.  (Only a CTA whose own column is shorter than three items has to wait for its first answers.)
+        int n_fetched = 0, v_next = 0, own_len = -1, col_len = -1, probed = 0;
+        bool q_end = false, asked = false;
+        auto put = [&](int v) {                                           // append one item (or the end mark) to the queue
+            if (n_fetched - epi_items >= kTileQ) {
+                const long long t0 = clock64();
+                while (n_fetched - epi_items >= kTileQ)
+                    if (abort_flag || clock64() - t0 > wait_limit) { abort_flag = 1; ok = false; return; }
+            }
+            tile_q[n_fetched & (kTileQ - 1)] = v < n_tiles ? v : -1;
+            q_end = v >= n_tiles;
+            __threadfence_block();
+            tile_n = ++n_fetched;
+        };
         for (int it = 0;; ++it) {
             int ti = -1;
             if (lane == 0) {
-                // take items from the shared list until this one and the next are in the queue
-                while (sched && n_fetched < it + 2 && !q_end && ok) {
-                    if (n_fetched - epi_items >= kTileQ) {
-                        const long long t0 = clock64();
-                        while (n_fetched - epi_items >= kTileQ)
-                            if (abort_flag || clock64() - t0 > wait_limit) { abort_flag = 1; ok = false; break; }
-                        if (!ok) break;
+                asked = false;
+                if (sched && n_own < n_tiles) {
+                    // where does the own column end?  (looked up two items ahead)
+                    while (col_len < 0 && probed <= it + 2) {
+                        const long long idx = (long long)blockIdx.x + (long long)probed * gridDim.x;
+                        if (idx >= n_own || tiles[idx].node < 0) col_len = probed;
+                        else ++probed;
                     }
-                    const int v = atomicAdd(sched, 1);
-                    tile_q[n_fetched & (kTileQ - 1)] = v < n_tiles ? v : -1;
-                    q_end = v >= n_tiles;
-                    __threadfence_block();
-                    tile_n = ++n_fetched;
+                    if (col_len >= 0) {
+                        const int need = it + 3 - col_len;                // entries of the shared list that should be in the queue
+                        while (!q_end && ok && n_fetched < need - 2) put(n_own + atomicAdd(sched, 1));   // needed right now
+                        asked = !q_end && ok && n_fetched < need;
+                        if (asked) v_next = n_own + atomicAdd(sched, 1);
+                    }
                 }
-                if (ok) ti = tc_item(it, n_tiles, sched, tile_q, &tile_n, abortp, wait_limit);
+                if (ok) ti = tc_item(it, own_len, tiles, n_own, n_tiles, sched, tile_q, &tile_n, abortp, wait_limit);
             }
             ti = __shfl_sync(0xffffffffu, ti, 0);
             if (ti < 0) break;
@@ -440,6 +459,7 @@ sr_tc_group_kernel(const CUtensorMap* __restrict__ maps, const TcNode* __restric
                                     (int)k.c0_16 << 4, tl.w0, tl.h0, tl.b0);
                     }
                 }
+                if (asked && ok) put(v_next);                             // the counter's answer: the next item
             }
             ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
             if (!ok) break;
@@ -452,8 +472,9 @@ sr_tc_group_kernel(const CUtensorMap* __restrict__ maps, const TcNode* __restric
         int cached_node = -1;
         uint32_t a_nxt = 0, a_ph = 0, a_used = 0, a_par = 0;
         bool ok = true;
+        int own_len = -1;
         for (int it = 0;; ++it) {
-            int ti = lane == 0 ? tc_item(it, n_tiles, sched, tile_q, &tile_n, abortp, wait_limit) : 0;
+            int ti = lane == 0 ? tc_item(it, own_len, tiles, n_own, n_tiles, sched, tile_q, &tile_n, abortp, wait_limit) : 0;
             ti = __shfl_sync(0xffffffffu, ti, 0);
             if (ti < 0) break;
             const TcTile tl = tiles[ti];
@@ -470,19 +491,29 @@ sr_tc_group_kernel(const CUtensorMap* __restrict__ maps, const TcNode* __restric
                 // With two or three slots a box is requested only about one filter ahead of its use, and a box that
                 // comes from DRAM takes longer than that.  So every request is accompanied by an L2 prefetch of the
                 // box two further on (of the next work item when this one ends, if it belongs to the same node).
-                TcTile nx = tl;
+                TcTile nx = tl;                                       // the next work item, looked up when its boxes come into reach
                 nx.node = -1;
-                if (!sched) {
-                    if (ti + (int)gridDim.x < n_tiles) nx = tiles[ti + gridDim.x];
-                } else if (tile_n > it + 1) {
-                    const int nti = tile_q[(it + 1) & (kTileQ - 1)];
-                    if (nti >= 0) nx = tiles[nti];
-                }
+                bool nx_seen = false;
                 for (int i = 0; i < n_act; ++i) {
                     const TcKbAct k = tab[i];
                     {
                         const int j = i + 2 < n_act ? i + 2 : i + 2 - n_act;
                         const bool here = i + 2 < n_act;
+                        if (!here && !nx_seen) {
+                            const long long idx = (long long)blockIdx.x + (long long)(it + 1) * gridDim.x;
+                            if (own_len < 0 && idx < n_own) {             // the next entry of the own column (may be padding)
+                                nx = tiles[idx];
+                                nx_seen = nx.node >= 0;
+                            }
+                            if (!nx_seen && sched && n_own < n_tiles) {   // else the next answer of the counter, if it is there
+                                const int j = it + 1 - (own_len < 0 ? it + 1 : own_len);
+                                if (tile_n > j) {
+                                    const int nti = tile_q[j & (kTileQ - 1)];
+                                    if (nti >= 0) nx = tiles[nti];
+                                    nx_seen = true;
+                                }
+                            }
+                        }
                         if ((here || nx.node == tl.node) && j < n_act) {
                             const TcKbAct p = tab[j];
                             const TcTile& pt = here ? tl : nx;
@@ -528,8 +559,9 @@ sr_tc_group_kernel(const CUtensorMap* __restrict__ maps, const TcNode* __restric
             st_shared_v4(smem_u32(&fifo[n_pub & (kFifo - 1)]), (n_pub & 0xFFFFu) | x, y, z, (w & 0x00FFFFFFu) | (n_pub << 24));
             return true;
         };
+        int own_len = -1;
         for (int it = 0;; ++it) {
-            int ti = lane == 0 ? tc_item(it, n_tiles, sched, tile_q, &tile_n, abortp, wait_limit) : 0;
+            int ti = lane == 0 ? tc_item(it, own_len, tiles, n_own, n_tiles, sched, tile_q, &tile_n, abortp, wait_limit) : 0;
             ti = __shfl_sync(0xffffffffu, ti, 0);
             if (ti < 0) break;
             const TcTile tl = tiles[ti];
@@ -734,9 +766,11 @@ sr_tc_group_kernel(const CUtensorMap* __restrict__ maps, const TcNode* __restric
         uint16_t* tbuf = &epi_buf[ew][0];
         uint32_t uses0 = 0, uses1 = 0;
         bool ok = true;
+        // one thread looks the next item up (before the barrier that ends the current one): one answer for all eight warps
+        int own_len = -1;
+        if (et == 0) epi_ti = tc_item(0, own_len, tiles, n_own, n_tiles, sched, tile_q, &tile_n, abortp, wait_limit);
+        asm volatile("bar.sync 1, 256;" ::: "memory");
         for (int it = 0;; ++it) {
-            if (et == 0) epi_ti = tc_item(it, n_tiles, sched, tile_q, &tile_n, abortp, wait_limit);
-            asm volatile("bar.sync 1, 256;" ::: "memory");           // one answer for all eight warps
             const int ti = epi_ti;
             if (ti < 0) break;
             const TcTile tl = tiles[ti];
@@ -800,8 +834,11 @@ sr_tc_group_kernel(const CUtensorMap* __restrict__ maps, const TcNode* __restric
                 __syncwarp();
                 if (lane == 0) mbar_arrive(bar_tempty + 8 * acc);
             }
+            if (et == 0) {
+                if (own_len >= 0) epi_items = it + 1 - own_len;
+                epi_ti = tc_item(it + 1, own_len, tiles, n_own, n_tiles, sched, tile_q, &tile_n, abortp, wait_limit);
+            }
             asm volatile("bar.sync 1, 256;" ::: "memory");           // everybody is done with the offset table
-            if (et == 0) epi_items = it + 1;
             if (tl.lanes == 2) { ++uses0; ++uses1; }
             else if (acc0 == 0) ++uses0;
             else ++uses1;
@@ -811,7 +848,7 @@ sr_tc_group_kernel(const CUtensorMap* __restrict__ maps, const TcNode* __restric
     tc_fence_before();
     __syncthreads();
     if (threadIdx.x == 0 && abort_flag) atomicExch(&ctl->error, 1);
-    if (threadIdx.x == 0 && sched) {
+    if (threadIdx.x == 0 && sched && n_own < n_tiles) {
         // the CTA that leaves last (none takes an item any more) puts the counters back for the next launch
         __threadfence();
         if (atomicAdd(sched + 1, 1) == (int)gridDim.x - 1) {
@@ -938,7 +975,7 @@ struct TcEngine {
     std::vector<StemPlan> stems;
     std::vector<int> stem_of_edge;
     std::vector<std::vector<TcTile>> group_tiles;
-    std::vector<int> group_tile_offset, group_a_slot, group_n_a, group_n_w, group_w_slot, group_grid, group_ctas_per_sm;
+    std::vector<int> group_tile_offset, group_a_slot, group_n_a, group_n_w, group_w_slot, group_grid, group_ctas_per_sm, group_n_own;
     SrRegion r_maps, r_nodes, r_kb_weight, r_kb_act, r_bursts, r_states, r_tiles, r_stems, r_sched;
     int n_maps = 0, n_kbs = 0, n_tiles = 0;
     int sm_count = 148;
@@ -1398,23 +1435,28 @@ sr_status sr_tc_plan(sr_graph* g, size_t& off)
             n_a = 2;
             n_w = std::min(kMaxW, (88 * 1024 - 1024 - 2 * a_slot) / w_slot);
         }
-        // Work lists.  Shared list (default): all items in ONE list, longest first, which the CTAs take from as they
-        // go.  Static lists: the items go, longest first, to the CTA with the least work so far; CTA c then walks
-        // column c of a matrix with one row per round (entries of node -1 pad the shorter columns).
+        // Work lists: the items go, longest first, to the CTA with the least work so far; CTA c walks column c of a
+        // matrix with one row per round (entries of node -1 pad the shorter columns).  Unless the lists are asked to be
+        // static, the smallest items - a fifth of the work, if the launch has more than two items per CTA - stay out of
+        // the matrix and follow it as one shared list (see the kernel).
         std::stable_sort(tl.begin(), tl.end(), [](const auto& a, const auto& b) { return a.first > b.first; });
         const int grid = (int)std::min<size_t>(tl.size(), (size_t)E->sm_count * per_sm);
         std::vector<std::vector<TcTile>> lists(std::max(grid, 1));
-        if (g->opt_tc_lists == 0) {
-            for (auto& it : tl) E->group_tiles[gi].push_back(it.second);
-        } else {
+        size_t n_matrix = tl.size();
+        if (g->opt_tc_lists == 0 && tl.size() > 2 * (size_t)grid) {
+            long long total = 0, tail = 0;
+            for (auto& it : tl) total += it.first;
+            while (n_matrix > (size_t)grid && (tail + tl[n_matrix - 1].first) * 5 <= total) tail += tl[--n_matrix].first;
+        }
+        {
             std::vector<std::pair<long long, int>> heap;     // (-load, cta): the standard heap keeps the largest on top
             for (int c = 0; c < grid; ++c) heap.push_back({0, -c});
             std::make_heap(heap.begin(), heap.end());
-            for (auto& it : tl) {
+            for (size_t i = 0; i < n_matrix; ++i) {
                 std::pop_heap(heap.begin(), heap.end());
                 std::pair<long long, int> top = heap.back();
-                lists[-top.second].push_back(it.second);
-                top.first -= it.first;
+                lists[-top.second].push_back(tl[i].second);
+                top.first -= tl[i].first;
                 heap.back() = top;
                 std::push_heap(heap.begin(), heap.end());
             }
@@ -1424,6 +1466,8 @@ sr_status sr_tc_plan(sr_graph* g, size_t& off)
                 for (int c = 0; c < grid; ++c)
                     E->group_tiles[gi].push_back(r < lists[c].size() ? lists[c][r] : TcTile{-1, 0, 0, 0, 0, 0, {0, 0}});
         }
+        E->group_n_own.push_back((int)E->group_tiles[gi].size());
+        for (size_t i = n_matrix; i < tl.size(); ++i) E->group_tiles[gi].push_back(tl[i].second);
         E->group_grid.push_back(grid);
         E->group_tile_offset.push_back(n_tiles);
         n_tiles += (int)E->group_tiles[gi].size();
@@ -1764,7 +1808,7 @@ int sr_tc_launch_group(sr_graph* g, int group, int t_off, cudaStream_t s)
         reinterpret_cast<const TcTile*>(g->ws + E->r_tiles.offset) + E->group_tile_offset[group],
         (int)E->group_tiles[group].size(), reinterpret_cast<SrFrameCtl*>(g->ws + g->r_ctl.offset), t_off, g->batch, n_a, a_slot,
         n_w, w_slot, E->group_ctas_per_sm[group] > 1 ? 256 : 512, (long long)g->opt_wait_ms * 2000000LL,
-        g->opt_tc_lists == 0 ? reinterpret_cast<int*>(g->ws + E->r_sched.offset) : nullptr);
+        g->opt_tc_lists == 0 ? reinterpret_cast<int*>(g->ws + E->r_sched.offset) : nullptr, E->group_n_own[group]);
     if (timed) {
         cudaEventRecord(E->ev[E->ev_used + 1], s);
         E->ev_used += 2;
