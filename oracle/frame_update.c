@@ -12,6 +12,9 @@
  * tableau level inside a frame (the caller passes that order).  Input nodes
  * are given at all frames 0..T; every other state is zero at frame 0 (Sec. A,
  * "Training details": states of all but the input layers start at zero).
+ * R(e) may exceed 1 (Sec. 6: an edge that bridges d > 1 frames stands for a chain of
+ * d - 1 copy-nodes); where t + 1 - R(e) < 0 the edge contributes nothing, because
+ * the copy-nodes it stands for start at zero like every other non-input node.
  * sigma is ReLU or the identity; b is a channel-wise bias; f_e is
  *   kind 0  a k x k cross-correlation with stride s and symmetric zero padding
  *           (k-1)/2, output size floor((n + 2p - k)/s) + 1; with pool = 2 it is
@@ -136,6 +139,7 @@ int sro_rollout(int n_nodes, const sro_node* nodes, int n_edges, const sro_edge*
                     const sro_node* s = &nodes[e->src];
                     const size_t sper = (size_t)s->h * s->w * s->c;
                     const int frame = t + 1 - (int)R[ei];
+                    if (frame < 0) continue;                     /* before frame 0: the copy-nodes of a long edge hold zeros */
                     const double* x = states[e->src] + ((size_t)frame * B + b) * sper;
                     edge_transform(s, v, e, x, weights[ei], acc, oy);
                 }

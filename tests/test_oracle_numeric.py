@@ -215,6 +215,35 @@ def test_resume_from_saved_states():
         assert not np.array_equal(cold[3][1], full[3][4])
 
 
+def test_edges_that_bridge_several_frames_equal_chains_of_copy_nodes():
+    # Sec. 6: R(e) > 1 is covered by the theory through copy-nodes.  An edge with R(e) = d evaluated directly
+    # (x_u of d frames earlier, nothing before frame 0) gives, bit for bit, what the chain u -> c_1 -> ... -> c_{d-1} -> v
+    # of one-frame edges with identity copies gives; and the delay really shifts the response (a hand-checked case).
+    g = graphs.mnist_net("SR", batch=2, frames=7)
+    W, B = data.make_weights(g), data.make_biases(g, zero=False)
+    X = {0: np.abs(randn(121, (8, 2, 28, 28, 1)))}
+    delays = list(g.patterns["streaming"])
+    skip = [i for i, e in enumerate(g.edges) if (e.src, e.tgt) == (1, 3)][0]          # H1 -> O
+    rec = [i for i, e in enumerate(g.edges) if e.src == e.tgt][0]                    # H1 -> H1
+    delays[skip], delays[rec] = 3, 2
+    g.patterns["delayed"] = delays
+    direct = fu.rollout_spec(g, "delayed", X, W, B)
+    ex, ident = graphs.with_copy_nodes(g, delays)
+    assert set(ex.patterns["p"]) <= {0, 1} and len(ex.nodes) == len(g.nodes) + 3 and len(ex.edges) == len(g.edges) + 3
+    assert rt.is_valid(len(ex.nodes), [(e.src, e.tgt) for e in ex.edges], ex.patterns["p"])
+    W_ex = list(W) + [np.eye(c).reshape(c, 1, 1, c) for c in ident]
+    B_ex = list(B) + [np.zeros(n.c) for n in ex.nodes[len(g.nodes):]]
+    chain = fu.rollout_spec(ex, "p", X, W_ex, B_ex)
+    for v in range(len(g.nodes)):
+        assert np.array_equal(direct[v], chain[v]), g.nodes[v].name
+    assert not np.array_equal(direct[len(g.nodes) - 1], fu.rollout_spec(g, "streaming", X, W, B)[len(g.nodes) - 1])
+    # hand-checked: in -> out, a dense identity edge that bridges 3 frames: out^t = in^(t-3), zero before
+    nodes = [node(1, 1, 2, 0), node(1, 1, 2, 0)]
+    x = np.arange(12, dtype=np.float64).reshape(6, 1, 1, 1, 2) + 1.0
+    s = fu.rollout(nodes, [edge(0, 1, DENSE)], [3], 1, 5, {0: x}, [np.eye(2).reshape(2, 1, 1, 2)], [np.zeros(2), np.zeros(2)])
+    assert s[1].reshape(6, 2).tolist() == [[0, 0], [0, 0], [0, 0], [1, 2], [3, 4], [5, 6]]
+
+
 def test_bf16_rounding_switch():
     v = np.array([1.0, 1.00390625, 1.005859375, 1.0078125, -3.14159], dtype=np.float32)
     want = rng.round_to_bf16(v)

@@ -333,6 +333,31 @@ BUILDERS = {"mini": mini_cnn, "sink": conv_sink, "dsr0": lambda **kw: dsr(0, **k
             "c4ff": lambda **kw: c4_ten_node(recurrence=False, **kw)}
 
 
+def with_copy_nodes(spec: GraphSpec, delays: List[int]):
+    """Edges that bridge more than one frame, R(e) = d > 1, written with copy-nodes (paper Sec. 6: longer forward
+    connections are covered by the theory through copy-nodes): edge e = (u, v) becomes the chain
+    u -> c_1 -> ... -> c_{d-1} -> v, every link bridging one frame; a copy-node has the shape of u, the identity as its
+    activation, no bias, and its one incoming edge is a 1x1 convolution whose weight is the identity matrix.
+    Returns the expanded GraphSpec (pattern "p" with values in {0, 1}; edge i of spec is still edge i) and, per added
+    edge, the channel count of its identity weight."""
+    nodes, edges, R = list(spec.nodes), list(spec.edges), [min(int(d), 1) for d in delays]
+    identity_channels = []
+    for ei, d in enumerate(delays):
+        e = spec.edges[ei]
+        src = e.src
+        for j in range(int(d) - 1):
+            u = spec.nodes[e.src]
+            nodes.append(Node("copy%d_%d" % (ei, j + 1), u.h, u.w, u.c, IDENTITY))
+            edges.append(Edge(src, len(nodes) - 1, CONV, 1, 1))
+            R.append(1)
+            identity_channels.append(u.c)
+            src = len(nodes) - 1
+        edges[ei] = Edge(src, e.tgt, e.kind, e.k, e.stride, e.pool)
+    g = GraphSpec(spec.name + "_copy", nodes, edges, spec.batch, spec.frames, spec.dtype, spec.seed, spec.weight_gain)
+    g.patterns = {"p": R}
+    return g, identity_channels
+
+
 def build(name: str, **overrides) -> GraphSpec:
     g = BUILDERS[name](**overrides)
     check_shapes(g)
