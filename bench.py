@@ -510,6 +510,8 @@ def run_cuda(args):
         # the other configurations, fewer steps each; same measurement, reported beside the headline
         others = {}
         for name in [n for n in args.also.split(",") if n and n != args.workload]:
+            torch.cuda.synchronize()
+            time.sleep(3.0)          # let the clocks recover from the power-capped headline run before the next workload
             _, w = measure_workload(torch, args, name, rank, local, None, pk, flush, max(3, min(args.steps, 10)), max(3, args.warmup), False)
             others[name] = w
         main_copy = {k: v for k, v in main.items() if k not in ("e2e_ms_per_step", "h2d_bytes_per_step", "d2h_bytes_per_step")}

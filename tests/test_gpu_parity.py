@@ -186,3 +186,34 @@ def test_deep_window_refuses_patterns_with_recurrence():
     with pytest.raises(SrError) as e:
         G.bind_window(4)
     assert e.value.status == "SR_ERR_UNSUPPORTED"
+
+
+@pytest.mark.parametrize("dtype", ["fp32", "bf16"])
+def test_edges_that_bridge_several_frames_run_as_chains_of_copy_nodes(dtype):
+    # Sec. 6: R(e) > 1 is covered through copy-nodes.  The library takes patterns with values in {0, 1}; the expanded
+    # graph (identity 1x1 copies, one frame per link) must reproduce the oracle's direct evaluation of the delays, on the
+    # tensor cores (64-channel nodes, bf16) as on the CUDA cores (fp32).
+    from oracle import frame_update as fu
+    from workloads.graphs import CONV, GAP_DENSE, IDENTITY, Edge, GraphSpec, Node
+    g = GraphSpec("delays", [Node("in", 16, 16, 3, IDENTITY), Node("a", 16, 16, 64), Node("b", 8, 8, 64), Node("o", 1, 1, 5, IDENTITY)],
+                  [Edge(0, 1, CONV, 3, 1), Edge(1, 2, CONV, 3, 2), Edge(2, 2, CONV, 3, 1), Edge(1, 1, CONV, 3, 1), Edge(0, 2, CONV, 1, 2),
+                   Edge(2, 3, GAP_DENSE)], batch=3, frames=7, dtype=dtype, seed=77)
+    delays = [1, 1, 2, 3, 2, 1]                        # b's recurrence bridges 2 frames, a's 3, the skip from the input 2
+    g.patterns["delayed"] = delays
+    X, W, Bi = data.make_inputs(g), data.make_weights(g), data.make_biases(g, zero=False)
+    want = fu.rollout_spec(g, "delayed", X, W, Bi)
+    ex, ident = graphs.with_copy_nodes(g, delays)
+    assert len(ex.nodes) == len(g.nodes) + 4
+    W_ex = list(W) + [np.eye(c, dtype=np.float32).reshape(c, 1, 1, c) for c in ident]
+    B_ex = list(Bi) + [np.zeros(n.c, dtype=np.float32) for n in ex.nodes[len(g.nodes):]]
+    G = parity.make_graph(ex, "p", "auto", 0, W_ex, B_ex)
+    if dtype == "bf16":
+        assert G.info["n_tensor_core_nodes"] >= 2, G.info
+    out = G.rollout([parity.to_device(ex, X[0])])
+    G.sync_status()
+    o = G.output_node
+    assert o == 3
+    tol = parity.TOL[dtype]
+    assert parity.rel_err(out.cpu().numpy().reshape(want[o][1:].shape), want[o][1:]) <= tol
+    for v in range(len(g.nodes)):
+        assert parity.rel_err(G.get_state(v).float().cpu().numpy(), want[v][g.frames]) <= tol, g.nodes[v].name
