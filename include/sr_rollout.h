@@ -202,7 +202,8 @@ sr_status sr_graph_set_node_bias(sr_graph* g, int node, const float* bias_host);
  *                  every CTA takes from when its own list is done (a device-wide counter).
  *           key 14 "fused nodes": 1 (default) = two convolutional nodes of one launch group that have the same shape,
  *                  at most 64 channels (a multiple of 32) each and an incoming edge from the same source with the
- *                  same filter geometry and the same R run as ONE tensor-core work item per pixel tile: the second
+ *                  same filter geometry and the same R (or of which one has two K-blocks of reduction at most)
+ *                  run as ONE tensor-core work item per pixel tile: the second
  *                  node's weights fill the otherwise empty rows 64..127 of the M = 128 instruction, and the shared
  *                  source is read and multiplied once for both.  0 = every node on its own.  Results are identical.
  * Must be set before sr_graph_workspace_bytes / sr_graph_bind_workspace (engine, weight ring, tile width, tile pairs,

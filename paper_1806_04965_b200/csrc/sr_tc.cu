@@ -118,9 +118,10 @@ struct TcState {
 };
 static_assert(sizeof(TcState) == 16, "read as one 16-byte word");
 
-// A plan can cover TWO nodes of at most 64 channels each that have the same shape and share a source: an M = 128
-// instruction on a 64-channel node is half empty, so the second node's weights take rows 64..127 and every K-block of
-// a source both read (same filter geometry, same frame) serves both.  TMEM lanes 64..127 then belong to the second node.
+// A plan can cover TWO nodes of at most 64 channels each that have the same shape: an M = 128 instruction on a
+// 64-channel node is half empty, so the second node's weights take rows 64..127 and every K-block of a source both
+// read (same filter geometry, same frame) serves both.  TMEM lanes 64..127 then belong to the second node.  Nodes are
+// paired if they share a source, or if one of them has next to no reduction of its own.
 struct TcNode {
     void* state[2];
     const float* bias;
@@ -1294,7 +1295,7 @@ sr_status sr_tc_plan(sr_graph* g, size_t& off)
         return r;
     };
     // Fused plans: two nodes of one launch group with the same shape and at most 64 channels (a multiple of 32) each,
-    // which share at least one source (see TcNode).
+    // which share at least one source or of which one is fed by next to nothing (see TcNode).
     std::vector<int> partner(g->nodes.size(), -1), leader(g->nodes.size(), -1);
     if (g->opt_tc_fuse)
         for (const std::vector<int>& grp : g->groups)
@@ -1306,19 +1307,26 @@ sr_status sr_tc_plan(sr_graph* g, size_t& off)
                     const int b = grp[j];
                     const SrHostNode& nb = g->nodes[b];
                     if (!nb.use_tc || partner[b] >= 0 || leader[b] >= 0 || nb.d.c != na.d.c || nb.d.h != na.d.h || nb.d.w != na.d.w) continue;
-                    int shared = 0, blocks = 0;
+                    int shared = 0, blocks = 0, blocks_a = 0, blocks_b = 0;
                     for (int ea : na.in_edges) {
                         const SrHostEdge& he = g->edges[ea];
-                        blocks += is_stem(g, he) ? 2 : he.k_eff * he.k_eff * (g->nodes[he.d.src].d.c / block_k(g->nodes[he.d.src].d.c));
+                        blocks_a += is_stem(g, he) ? 2 : he.k_eff * he.k_eff * (g->nodes[he.d.src].d.c / block_k(g->nodes[he.d.src].d.c));
                     }
+                    blocks = blocks_a;
                     for (int eb : nb.in_edges) {
                         const SrHostEdge& he = g->edges[eb];
                         bool sh = false;
                         for (int ea : na.in_edges) sh |= same_source(g, ea, eb);
+                        const int nb_e = is_stem(g, he) ? 2 : he.k_eff * he.k_eff * (g->nodes[he.d.src].d.c / block_k(g->nodes[he.d.src].d.c));
+                        blocks_b += nb_e;
                         if (sh) ++shared;
-                        else blocks += is_stem(g, he) ? 2 : he.k_eff * he.k_eff * (g->nodes[he.d.src].d.c / block_k(g->nodes[he.d.src].d.c));
+                        else blocks += nb_e;
                     }
-                    if (shared > 0 && blocks <= kMaxNodeKb) {
+                    // without a shared source the fused plan issues as many MMAs as the two nodes; it still pays when one
+                    // of them has next to no reduction (a node fed by a staged edge only): its tiles are all epilogue,
+                    // which then runs beside the other node's MMAs
+                    const bool tiny = std::min(blocks_a, blocks_b) <= 2;
+                    if ((shared > 0 || tiny) && blocks <= kMaxNodeKb) {
                         partner[a] = b;
                         leader[b] = a;
                     }
