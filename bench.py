@@ -41,9 +41,9 @@ ALL_WORKLOADS = ("c1", "c2", "c3", "c4", "c5")
 # the kernel source it was taken from; the number is reported only while that source is unchanged, else null.
 TRAFFIC = {
     # workload: (bytes per launch, kernel source file, sha256[:12] of that file at capture time, summary under profiles/)
-    "c5": (617.1e6, "sr_tc.cu", "f907f9065e14", "profiles/sr_tc_group_kernel_counters.md"),
-    "c3": (246.1e6, "sr_tc.cu", "f907f9065e14", "profiles/sr_tc_group_kernel_counters.md"),
-    "c4": (164.8e6, "sr_tc.cu", "f907f9065e14", "profiles/sr_tc_group_kernel_counters.md"),
+    "c5": (615.7e6, "sr_tc.cu", "6985e1c55246", "profiles/sr_tc_group_kernel_counters.md"),
+    "c3": (245.2e6, "sr_tc.cu", "6985e1c55246", "profiles/sr_tc_group_kernel_counters.md"),
+    "c4": (165.1e6, "sr_tc.cu", "6985e1c55246", "profiles/sr_tc_group_kernel_counters.md"),
     "c2": (8.0e6, "sr_resident.cu", "89436108f1ff", "profiles/sr_resident_kernel_c2.md"),     # one launch = all 32 frames
 }
 

@@ -88,7 +88,7 @@ struct sr_graph {
     int opt_tc_fuse = 1;                           // two nodes of at most 64 channels that share a source run as one 128-row plan
     int opt_tc_lists = 0;                          // tensor-core work items: 1 = a list per CTA made on the host, 0 = the same plus a shared list of the smallest items
     int opt_stem_ring = 1;                         // activation boxes of staged few-channel edges travel in the weight ring
-    int opt_tc_pair = 0;                           // tensor-core work items: 0 = pairs of tiles where it pays, 1 = single tiles, 2 = pairs wherever possible
+    int opt_tc_pair = 0;                           // tensor-core work items: 0 / 1 = single pixel tiles, 2 = pairs of tiles wherever the geometry allows
     int opt_wait_ms = 1000;                        // limit of every device-side wait; 0 = expire at once (test hook)
     int opt_resident = 1, opt_rs_cluster = 0, opt_rs_warps = 0, opt_rs_split = 0;   // 16-channel work units: 0 never, 1 always, 2 by cost
     // workspace

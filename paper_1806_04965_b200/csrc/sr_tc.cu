@@ -56,7 +56,7 @@ constexpr int kThreads = 384;
 constexpr int kEpiWarps = 8;                          // warps 4..11
 constexpr int kFifo = 16;                             // burst descriptors in flight between scout and issuer
 constexpr int kMaxA = 4;                              // activation ring depth
-constexpr int kMaxW = 8;                              // weight ring depth (one weight box per slot)
+constexpr int kMaxW = 8;                              // weight ring depth (one weight group per slot)
 // Dynamic shared memory of a CTA.  With the 24 KiB of static shared memory this leaves about 20 KiB of the SM's 228 KiB
 // free: the other kernels of a frame (input staging, dense heads: up to 7.4 KiB per block) run on a second stream beside
 // the persistent CTAs, and measured on B200 they queue behind them, frame after frame, once less than about 10 KiB of
@@ -1382,16 +1382,10 @@ sr_status sr_tc_plan(sr_graph* g, size_t& off)
         std::vector<int> members;
         for (int v : g->groups[gi])
             if (E->node_of[v] >= 0 && leader[v] < 0) members.push_back(E->node_of[v]);
-        size_t single_tiles = 0;
-        for (int ni : members) {
-            build_kblocks(g, E, E->nodes[ni]);
-            single_tiles += node_tiles(g, E->nodes[ni], ni).size();
-        }
         // Pairs halve the weight traffic but double the size of a work item, expose the epilogue (both accumulators
         // are busy) and leave room for fewer weight slots; with copies issued group-wise the L2 keeps single tiles
         // fed, so pairs are used on request only.  Option "pair": 0 / 1 = single tiles, 2 = pairs wherever the
         // geometry allows.
-        (void)single_tiles;
         bool pair = g->opt_tc_pair == 2;
         // The box of a staged edge takes a weight slot for the two MMAs it feeds; that pays where the weight ring is
         // deep (launch groups of nodes with few output channels: small weight groups), not where it has three slots.
