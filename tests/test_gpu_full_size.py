@@ -55,3 +55,11 @@ def test_c5_all_128_frames_reduced_images():
     g = graphs.build("c5", size=16, batch=8)
     for p in ("streaming", "hybrid1"):
         parity.check_run(g, p, graph_frames=16, samples=[0, 7])
+
+
+@pytest.mark.parametrize("name,options", [("c3", dict(tc_fuse=0, tc_lists=1)), ("c4", dict(tc_fuse=0, tc_lists=1, stem_ring=0)),
+                                          ("c4", dict(stem_ring=2))])
+def test_full_size_with_the_optional_paths_switched(name, options):
+    # every node on its own, per-CTA work lists only, staged boxes in / out of the weight ring: same results
+    g = graphs.build(name, frames=6)
+    parity.check_run(g, "streaming", graph_frames=0, samples=[1], **options)
