@@ -35,6 +35,8 @@ from workloads import data, graphs  # noqa: E402
 METRIC = "streaming_rollout_frames_per_sec"
 UNIT = "frames/s"
 ALL_WORKLOADS = ("c1", "c2", "c3", "c4", "c5")
+# The paper's own CIFAR10 networks (Sec. A): shallowest and deepest of DSR0..DSR6, at a batch the paper does not fix.
+PAPER_NETS = {"dsr0": dict(batch=128, frames=16), "dsr6": dict(batch=128, frames=16)}
 
 # DRAM traffic (dram__bytes_read.sum + dram__bytes_write.sum) of ONE launch of the dominant kernel, from the ncu
 # captures summarised under profiles/.  Every entry names its capture and the first 12 hex digits of the SHA-256 of
@@ -125,7 +127,10 @@ def build_spec(args, name=None):
             kw["batch"] = args.batch
         if args.frames:
             kw["frames"] = args.frames
-    return graphs.build(name or args.workload, **kw)
+    n = name or args.workload
+    if n in PAPER_NETS:
+        kw = dict(PAPER_NETS[n], **kw)
+    return graphs.build(n, **kw)
 
 
 def replica_spec(args, rank: int, name=None):
@@ -517,6 +522,14 @@ def run_cuda(args):
         main_copy = {k: v for k, v in main.items() if k not in ("e2e_ms_per_step", "h2d_bytes_per_step", "d2h_bytes_per_step")}
         others[spec.name] = main_copy
         line["workloads"] = {k: others[k] for k in sorted(others)}
+        paper = {}
+        for name in [n for n in args.paper_nets.split(",") if n]:
+            torch.cuda.synchronize()
+            time.sleep(1.0)
+            _, w = measure_workload(torch, args, name, rank, local, None, pk, flush, max(3, min(args.steps, 5)), max(3, args.warmup), False)
+            paper[name] = w
+        if paper:
+            line["paper_networks"] = paper
         if "c4" in line["workloads"]:
             line["workloads"]["c4"]["deep_window"] = measure_window(torch, args, flush, max(3, min(args.steps, 10)), 3)
     if rank == 0:
@@ -563,6 +576,7 @@ def main():
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="cuda", choices=["cuda", "reference"])
     ap.add_argument("--workload", default="c5", choices=list(graphs.BUILDERS))
+    ap.add_argument("--paper-nets", default=",".join(PAPER_NETS), help="the paper's own networks reported beside the configs (one GPU)")
     ap.add_argument("--also", default=",".join(ALL_WORKLOADS), help="workloads reported beside the headline at one GPU")
     ap.add_argument("--pattern", default="streaming")
     ap.add_argument("--batch", type=int, default=0)

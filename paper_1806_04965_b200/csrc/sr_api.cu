@@ -157,9 +157,13 @@ sr_status plan(sr_graph* g)
                     if (g->edges[e].d.kind == SR_EDGE_MEAN_DENSE && g->nodes[g->edges[e].d.src].d.c > sr_direct_head_max_channels())
                         fast = false;
                 if (fast) {
-                    const int hco = sr_direct_head_outputs_per_block();
+                    // a block takes up to 16 outputs of one sample; with a long reduction (thousands of inputs per
+                    // output) only 4, so that a small batch still gives every SM several blocks' worth of loads in flight
+                    long long k_in = 0;
+                    for (int e : n.in_edges) k_in += g->edges[e].K;
+                    const int hco = k_in >= 4096 ? 4 : sr_direct_head_outputs_per_block();
                     for (int b0 = 0; b0 < g->batch; ++b0)
-                        for (int c0 = 0; c0 < n.d.c; c0 += hco) g->items.push_back(SrDirectItem{v, b0, c0, 1});
+                        for (int c0 = 0; c0 < n.d.c; c0 += hco) g->items.push_back(SrDirectItem{v, b0, c0, 1 | (hco << 8)});
                 } else {
                     for (int b0 = 0; b0 < g->batch; b0 += dsb)
                         for (int c0 = 0; c0 < n.d.c; c0 += dco) g->items.push_back(SrDirectItem{v, b0, c0, 0});

@@ -184,7 +184,7 @@ __device__ void head_item(const SrDevNode& nd, const SrDevEdge* edges, const SrD
     __shared__ float red[kWarps][kHeadCo];
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, tid = threadIdx.x;
     const int b = it.b0, co0 = it.p0;
-    const int nco = min(kHeadCo, nd.C - co0);
+    const int nco = min(it.pad_ >> 8, nd.C - co0);      // outputs of this block (at most kHeadCo)
     float acc[kHeadCo];
 #pragma unroll
     for (int o = 0; o < kHeadCo; ++o) acc[o] = 0.f;
@@ -234,7 +234,12 @@ __device__ void head_item(const SrDevNode& nd, const SrDevEdge* edges, const SrD
                     if (o < nco) acc[o] = fmaf(w0[(size_t)o * e.K + c], m, acc[o]);
             }
         } else if ((Kx & 3) == 0) {
-            for (int k = 4 * tid; k < Kx; k += 4 * (int)blockDim.x) {
+            // all blocks of a launch walk the same weight rows: every block starts at another step (its sample index),
+            // so that they do not all ask the same L2 lines at the same moment
+            const int stride = 4 * (int)blockDim.x, steps = (Kx + stride - 1) / stride;
+            for (int s = 0; s < steps; ++s) {
+                const int k = 4 * tid + ((s + b) % steps) * stride;
+                if (k >= Kx) continue;
                 float x[4];
                 load4(src + k, x);
 #pragma unroll
@@ -285,7 +290,7 @@ sr_direct_group_kernel(const SrDevNode* __restrict__ nodes, const SrDevEdge* __r
     float* out = nullptr;
     if (nd.is_output && ctl->out_base) out = ctl->out_base + (ctl->run_t + t_off) * ctl->out_stride;
     if (nd.H == 1 && nd.W == 1 && edges[nd.first_edge].kind != SR_EDGE_CONV) {
-        if (it.pad_ == 1) head_item<T>(nd, edges, it, prev, cur, out);
+        if ((it.pad_ & 0xFF) == 1) head_item<T>(nd, edges, it, prev, cur, out);
         else dense_item<T>(nd, edges, it, prev, cur, B, out);
     }
     else
