@@ -47,6 +47,7 @@ TRAFFIC = {
     "c3": (245.2e6, "sr_tc.cu", "6985e1c55246", "profiles/sr_tc_group_kernel_counters.md"),
     "c4": (165.1e6, "sr_tc.cu", "6985e1c55246", "profiles/sr_tc_group_kernel_counters.md"),
     "c2": (8.0e6, "sr_resident.cu", "89436108f1ff", "profiles/sr_resident_kernel_c2.md"),     # one launch = all 32 frames
+    "c1": (1.30e6, "sr_dense.cu", "9f15eb3bde12", "profiles/sr_dense_kernel_c1.md"),           # one launch = all 16 frames
 }
 
 
